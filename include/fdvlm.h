@@ -1,0 +1,193 @@
+/*
+ * fdvlm.h -- C ABI of the B200 (sm_100a) block-diffusion denoise-step library.
+ *
+ * One handle = one request at batch size one of a Qwen2.5-shaped decoder run as a block-diffusion
+ * language model (Fast-dVLM, Sec. 3.4 "Inference" and Appendix B, Alg. 1):
+ *
+ *   fdvlm_prefill       causal forward over the prefix (vision embeddings, then text tokens) that
+ *                       fills the KV cache                               (Alg. 1, "Prefill")
+ *   fdvlm_block_begin   start a block of B positions, all [MASK] unless tokens are given (Sec. 3.4)
+ *   fdvlm_block_step    one denoise step: forward of the B block rows -- bidirectional inside the
+ *                       block, full over the cache, cache NOT updated (Alg. 1 draft step; Sec. 3.3
+ *                       M_N2N, M_N2C) -- then softmax max-probability confidence and
+ *                       threshold / top-k parallel unmasking (Sec. 3.4; Sec. 4.5)
+ *   fdvlm_commit_block  causal forward of the finished block WITH cache update (Alg. 1 verify step;
+ *                       Sec. 3.3 M_C2C: clean context is token-causal)
+ *
+ * Conventions
+ *   - All `device` pointers are CUDA device memory of the handle's GPU; `host` pointers are ordinary
+ *     host memory.  No pointer is retained beyond a call except the weight pointers given to
+ *     fdvlm_create, which are BORROWED and must stay valid and unchanged until fdvlm_destroy.
+ *   - Matrices are row-major [out_features, in_features] (K contiguous); vectors are dense.
+ *   - The KV cache, workspace and block state belong to the handle (allocated in fdvlm_create with
+ *     cudaMalloc, freed in fdvlm_destroy).
+ *   - All work is issued on the CUDA stream given at create time.  Calls that return data to the host
+ *     (info / *_host variants) synchronise that stream before returning; others are asynchronous.
+ *   - Every function returns FDVLM_OK (0) or a negative fdvlm_status; argument and state errors are
+ *     detected on the host before anything is launched.  fdvlm_last_error gives a message.
+ *   - A handle is not thread-safe; distinct handles are independent.  There is no CPU fallback: with
+ *     no usable GPU fdvlm_create fails with FDVLM_ERR_CUDA.
+ */
+#ifndef FDVLM_H_
+#define FDVLM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct fdvlm fdvlm_t; /* opaque */
+
+typedef enum {
+  FDVLM_OK = 0,
+  FDVLM_ERR_INVALID_ARG = -1, /* NULL / out-of-range argument, unsupported shape relation          */
+  FDVLM_ERR_STATE = -2,       /* step without begin, commit with masks left, begin inside a block  */
+  FDVLM_ERR_CAPACITY = -3,    /* cache_len + rows > max_seq, or block_size > max_block             */
+  FDVLM_ERR_UNSUPPORTED = -4, /* shape or dtype the kernels do not cover                           */
+  FDVLM_ERR_CUDA = -5,        /* a CUDA runtime call failed (message has the CUDA error string)    */
+  FDVLM_ERR_TIMEOUT = -6,     /* a bounded device-side wait gave up; outputs of that call invalid  */
+  FDVLM_ERR_OOM = -7          /* device allocation failed in fdvlm_create                          */
+} fdvlm_status;
+
+/* Storage type of the linear weights.  Activations, KV cache and the embedding table are fp32 for
+ * FDVLM_F32 and bf16 otherwise; accumulation, residual stream, norms and softmax are always fp32. */
+typedef enum {
+  FDVLM_F32 = 0,
+  FDVLM_BF16 = 1,
+  FDVLM_W_FP8E4M3 = 2 /* OCP e4m3fn bytes + fp32 per-output-channel scale: w = e4m3(byte) * scale[out] */
+} fdvlm_dtype;
+
+typedef struct {
+  int n_layers, hidden, n_q_heads, n_kv_heads, head_dim, intermediate, vocab;
+  int mask_id;        /* id of [MASK]; never predicted (its logit is excluded from softmax/argmax) */
+  float rms_eps;      /* RMSNorm epsilon */
+  float rope_theta;   /* rotary base; rotate-half pairing (j, j + head_dim/2), position = index in the
+                         committed sequence (vision rows included) */
+  int tie_embeddings; /* 1: LM head = embedding table (lm_head must be NULL) */
+  fdvlm_dtype dtype;
+  int max_seq;        /* KV-cache capacity in positions; every call needs cache_len + rows <= max_seq */
+  int max_block;      /* largest block size (1..64) */
+} fdvlm_config;
+
+typedef struct {
+  const void *wq, *wk, *wv, *wo, *w_gate, *w_up, *w_down; /* device, [out,in], storage per dtype */
+  const float *bq, *bk, *bv;                              /* device fp32 [out], all NULL or all set */
+  const float *s_q, *s_k, *s_v, *s_o, *s_gate, *s_up, *s_down; /* device fp32 [out]; fp8 only    */
+  const float *g_attn, *g_mlp;                            /* device fp32 [hidden] RMSNorm gains     */
+} fdvlm_layer_weights;
+
+typedef struct {
+  const void *embed;      /* device [vocab, hidden], fp32 (F32) or bf16 (BF16 / FP8); never fp8      */
+  const void *lm_head;    /* device [vocab, hidden] in dtype storage; NULL iff tie_embeddings        */
+  const float *s_lm_head; /* device fp32 [vocab]; fp8 untied only                                   */
+  const float *g_final;   /* device fp32 [hidden]                                                   */
+  const fdvlm_layer_weights *layers; /* HOST array of n_layers entries (copied by fdvlm_create)     */
+} fdvlm_weights;
+
+/* Unmasking rule of one step (Sec. 3.4 / Sec. 4.5).
+ *  THRESHOLD: reveal every masked position whose confidence is strictly above `threshold`; if none
+ *             is, reveal the single masked position of highest confidence (so tau = 1.0 gives one
+ *             token per step).
+ *  TOPK:      reveal the min(k, #masked) masked positions of highest confidence.
+ *  Ties go to the lowest position index; the vocabulary argmax takes the lowest token id. */
+typedef enum { FDVLM_RULE_THRESHOLD = 0, FDVLM_RULE_TOPK = 1 } fdvlm_rule;
+typedef struct { fdvlm_rule rule; float threshold; int k; } fdvlm_step_params;
+typedef struct { int n_unmasked, n_remaining, step_index; } fdvlm_step_info;
+
+/* Create a handle on the current CUDA device.  `cuda_stream` is a cudaStream_t (NULL = default
+ * stream).  Allocates the KV cache (n_layers * 2 * n_kv_heads * max_seq * head_dim elements) and a
+ * workspace.  Requires: head_dim in {64, 128}; n_q_heads % n_kv_heads == 0; hidden, intermediate,
+ * q/kv widths multiples of 8 (bf16/fp8: hidden and intermediate multiples of 16); 1 <= max_block <= 64. */
+int fdvlm_create(const fdvlm_config *cfg, const fdvlm_weights *w, void *cuda_stream, fdvlm_t **out);
+void fdvlm_destroy(fdvlm_t *h);
+
+/* Forget the cache and any open block (cache_len = 0). */
+int fdvlm_reset(fdvlm_t *h);
+
+/* Append `n_embeds` embedding rows (device, [n_embeds, hidden], fp32 for F32 else bf16; may be NULL
+ * when n_embeds = 0) and then `n_tokens` token ids (device int32; may be NULL when 0) to the cache
+ * with a causal forward (Alg. 1 "Prefill (causal attention)").  May be called repeatedly; not inside
+ * an open block.  last_logits (device fp32 [vocab], nullable) receives the logits of the last row
+ * appended -- the AR seed of Sec. 3.4 "causal context decoding". */
+int fdvlm_prefill(fdvlm_t *h, const void *embeds, int n_embeds, const int32_t *tokens, int n_tokens,
+                  float *last_logits);
+
+/* Open a block of `block_size` positions at cache_len .. cache_len + block_size - 1.
+ * init_tokens (device int32 [block_size], nullable): positions holding mask_id are masked, any other
+ * id is an already revealed token; NULL = all masked.  fdvlm_block_begin_host takes a host pointer. */
+int fdvlm_block_begin(fdvlm_t *h, int block_size, const int32_t *init_tokens);
+int fdvlm_block_begin_host(fdvlm_t *h, int block_size, const int32_t *init_tokens_host);
+
+/* One denoise step over the open block (B = block_size rows).  All outputs nullable:
+ *   logits       device fp32 [B, vocab]   raw logits (mask_id column not suppressed)
+ *   conf         device fp32 [B]          max softmax probability with mask_id excluded, every row
+ *   pred         device int32 [B]         argmax token with mask_id excluded, every row
+ *   unmask       device uint8 [B]         1 where a masked position was revealed by this step
+ *   block_tokens device int32 [B]         block tokens after the update
+ *   info         HOST                     counts after the step; passing it makes the call synchronous
+ * Errors: STATE if no block is open or no masked position is left.  The KV cache contents at
+ * positions < cache_len are never written by this call. */
+int fdvlm_block_step(fdvlm_t *h, const fdvlm_step_params *p, float *logits, float *conf,
+                     int32_t *pred, uint8_t *unmask, int32_t *block_tokens, fdvlm_step_info *info);
+
+/* Same step, results copied to HOST buffers (any may be NULL); always synchronous. */
+int fdvlm_block_step_host(fdvlm_t *h, const fdvlm_step_params *p, float *conf_host,
+                          int32_t *pred_host, uint8_t *unmask_host, int32_t *block_tokens_host,
+                          fdvlm_step_info *info);
+
+/* Replace the open block's tokens / masked flags (device int32 [B]; mask_id = masked) without
+ * touching the step counter: lets a test replay another implementation's block state. */
+int fdvlm_block_set_tokens(fdvlm_t *h, const int32_t *tokens);
+
+/* Commit the open, fully unmasked block: causal forward with cache update, cache_len += B.
+ * next_logits (device fp32 [vocab], nullable) = logits of the block's last row.
+ * Errors: STATE if no block is open or masked positions remain. */
+int fdvlm_commit_block(fdvlm_t *h, float *next_logits);
+
+/* Committed positions, or a negative status for a NULL handle. */
+int fdvlm_cache_len(const fdvlm_t *h);
+
+/* Copy cached K (which = 0, post-rotary) or V (which = 1) of `layer`, positions [pos0, pos0 + n), to
+ * dst (device, [n, n_kv_heads, head_dim], fp32 for F32 else bf16).  For tests and checkpointing. */
+int fdvlm_cache_read(const fdvlm_t *h, int layer, int which, int pos0, int n, void *dst);
+
+/* Number of kernel launches issued by the last prefill / step / commit call of this handle. */
+int fdvlm_last_launch_count(const fdvlm_t *h);
+
+/* Message of the last error on this handle ("" if none); valid until the next call on it.
+ * With h = NULL returns the message of the last failed fdvlm_create on this thread. */
+const char *fdvlm_last_error(const fdvlm_t *h);
+
+/* ---- single operators of the path, for kernel-level tests and timing -------------------------------- */
+
+/* y[m, n] = sum_k x[m, k] * w[n, k] (* scale[n]) (+ bias[n]): the small-M weight-streaming GEMM that
+ * every projection of the decoder is (QKV, O, gate/up, down, LM head; M = block size <= 64).
+ * x: device [m, k], fp32 for F32 else bf16; w: device [n, k] in `dtype` storage; scale: device fp32
+ * [n] (fp8) or NULL; bias: device fp32 [n] or NULL; y: device fp32 [m, n].
+ * workspace: device scratch of at least fdvlm_op_linear_workspace_bytes(m, n, k, dtype) bytes (used
+ * for split-K partial sums; may be NULL when that size is 0). */
+int fdvlm_op_linear(const void *x, const void *w, const float *scale, const float *bias, float *y,
+                    int m, int n, int k, fdvlm_dtype dtype, void *workspace, void *cuda_stream);
+size_t fdvlm_op_linear_workspace_bytes(int m, int n, int k, fdvlm_dtype dtype);
+
+/* Block-masked GQA attention of n_rows new rows at positions cache_len .. cache_len + n_rows - 1
+ * (Sec. 3.3 masks; Alg. 1 draft / verify).  q: device [n_rows, n_q_heads, head_dim] (post-rotary);
+ * k_cache / v_cache: device [n_kv_heads, max_seq, head_dim] holding cache_len committed positions
+ * followed by the n_rows new positions; causal = 0: every row reads all cache_len + n_rows keys,
+ * causal = 1: row i reads keys 0 .. cache_len + i.  out: device [n_rows, n_q_heads * head_dim].
+ * Element type fp32 for F32, bf16 otherwise.  workspace: device scratch of at least
+ * fdvlm_op_attention_workspace_bytes(...) bytes for the split-KV partial results. */
+int fdvlm_op_attention(const void *q, const void *k_cache, const void *v_cache, void *out,
+                       int n_rows, int cache_len, int max_seq, int n_q_heads, int n_kv_heads,
+                       int head_dim, int causal, fdvlm_dtype dtype, void *workspace, void *cuda_stream);
+size_t fdvlm_op_attention_workspace_bytes(int n_rows, int n_q_heads, int n_kv_heads, int head_dim);
+
+/* Version string of the library. */
+const char *fdvlm_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FDVLM_H_ */

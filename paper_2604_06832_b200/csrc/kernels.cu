@@ -1,0 +1,458 @@
+// CUDA-core (SIMT) kernels of the denoise step: the exact-fp32 path of the fp32 configuration and
+// the small fused glue of every configuration (embedding gather, RMSNorm, rotary + KV staging,
+// SwiGLU, softmax-max confidence / argmax, unmask selection).
+#include "common.cuh"
+#include "kernels.h"
+
+namespace fdk {
+
+// ================================================================================================
+// small-M linear, CUDA-core version.  Register-tiled: CTA tile BM x 64 outputs, BK = 32 deep.
+// Used for fp32 weights (TF32 tensor cores would miss the 1e-4 parity bound of that path) and for
+// shapes the tensor-core kernel does not take.
+// ================================================================================================
+template <typename T> struct Vec8;
+template <> struct Vec8<float> {
+  static __device__ __forceinline__ void load(const float* p, float* o) {
+    float4 a = *reinterpret_cast<const float4*>(p), b = *reinterpret_cast<const float4*>(p + 4);
+    o[0] = a.x; o[1] = a.y; o[2] = a.z; o[3] = a.w; o[4] = b.x; o[5] = b.y; o[6] = b.z; o[7] = b.w;
+  }
+};
+template <> struct Vec8<bf16> {
+  static __device__ __forceinline__ void load(const bf16* p, float* o) {
+    uint4 v = *reinterpret_cast<const uint4*>(p);
+    const unsigned u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      o[2 * i] = __uint_as_float(u[i] << 16);
+      o[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u);
+    }
+  }
+};
+template <> struct Vec8<fp8e4m3> {
+  static __device__ __forceinline__ void load(const fp8e4m3* p, float* o) {
+    uint2 v = *reinterpret_cast<const uint2*>(p);
+    const unsigned u[2] = {v.x, v.y};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      fp8e4m3 e;
+      e.b = (uint8_t)((u[i >> 2] >> (8 * (i & 3))) & 0xffu);
+      o[i] = to_f32(e);
+    }
+  }
+};
+
+constexpr int SBN = 64, SBK = 32;
+
+template <typename WT, typename XT, int BM>
+__global__ void __launch_bounds__((BM / 4) * 16)
+linear_simt_kernel(const XT* __restrict__ x, const WT* __restrict__ w, float* __restrict__ part,
+                   int m, int N, int K, int k_per_split) {
+  constexpr int NT = (BM / 4) * 16;
+  __shared__ __align__(16) float xs[SBK][BM + 4];
+  __shared__ __align__(16) float ws[SBK][SBN + 4];
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int n0 = blockIdx.x * SBN;
+  const int kb = blockIdx.y * k_per_split;
+  const int ke = min(K, kb + k_per_split);
+  float acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+  for (int k0 = kb; k0 < ke; k0 += SBK) {
+    // W tile: 64 rows x 32 k as 256 vectors of 8; vector v -> row v % 64, k-quarter v / 64
+    for (int v = tid; v < SBN * (SBK / 8); v += NT) {
+      int r = v % SBN, kq = v / SBN;
+      int n = n0 + r, k = k0 + kq * 8;
+      float f[8];
+      if (n < N && k < ke) Vec8<WT>::load(w + (size_t)n * K + k, f);
+      else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) f[i] = 0.f;
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) ws[kq * 8 + i][r] = f[i];
+    }
+    for (int v = tid; v < BM * (SBK / 8); v += NT) {
+      int r = v % BM, kq = v / BM;
+      int k = k0 + kq * 8;
+      float f[8];
+      if (r < m && k < ke) Vec8<XT>::load(x + (size_t)r * K + k, f);
+      else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) f[i] = 0.f;
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) xs[kq * 8 + i][r] = f[i];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < SBK; ++kk) {
+      float4 xv = *reinterpret_cast<const float4*>(&xs[kk][ty * 4]);
+      float4 wv = *reinterpret_cast<const float4*>(&ws[kk][tx * 4]);
+      const float xa[4] = {xv.x, xv.y, xv.z, xv.w}, wa[4] = {wv.x, wv.y, wv.z, wv.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(xa[i], wa[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+  float* dst = part + (size_t)blockIdx.y * m * N;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    int r = ty * 4 + i;
+    if (r >= m) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      int n = n0 + tx * 4 + j;
+      if (n < N) dst[(size_t)r * N + n] = acc[i][j];
+    }
+  }
+}
+
+// y[r, n] = (accumulate ? y : 0) + (sum_s part[s][r][n]) * scale[n] + bias[n]; fixed summation order.
+__global__ void splitk_epilogue_kernel(const float* __restrict__ part, int S, int m, int N,
+                                       const float* __restrict__ scale, const float* __restrict__ bias,
+                                       float* __restrict__ y, int ldy, int accumulate) {
+  size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  size_t total = (size_t)m * N;
+  if (idx >= total) return;
+  int r = (int)(idx / N), n = (int)(idx % N);
+  float s = 0.f;
+  for (int i = 0; i < S; ++i) s += part[(size_t)i * total + idx];
+  if (scale) s *= scale[n];
+  if (bias) s += bias[n];
+  float* o = y + (size_t)r * ldy + n;
+  *o = accumulate ? (*o + s) : s;
+}
+
+static void simt_plan(int m, int n, int k, int* bm, int* splits, int* kps) {
+  *bm = m <= 16 ? 16 : (m <= 32 ? 32 : 64);
+  int tiles = ceil_div(n, SBN);
+  int kblocks = ceil_div(k, SBK);
+  int want = ceil_div(2 * 148, tiles);                 // at least ~2 CTAs per SM when K allows
+  int s = want < 1 ? 1 : want;
+  int max_s = kblocks / 8 > 0 ? kblocks / 8 : 1;       // >= 256 deep per split
+  if (s > max_s) s = max_s;
+  if (s > 16) s = 16;
+  int per = ceil_div(kblocks, s) * SBK;
+  *kps = per;
+  *splits = ceil_div(k, per);
+}
+
+size_t simt_workspace_bytes(int m, int n, int k) {
+  int bm, s, kps;
+  simt_plan(m, n, k, &bm, &s, &kps);
+  return (size_t)s * m * n * sizeof(float);
+}
+
+template <typename WT, typename XT>
+static void simt_dispatch(const LinearArgs& a, int bm, dim3 grid, float* part, int kps, cudaStream_t st) {
+  const XT* x = (const XT*)a.x;
+  const WT* w = (const WT*)a.w;
+  if (bm == 16) linear_simt_kernel<WT, XT, 16><<<grid, 64, 0, st>>>(x, w, part, a.m, a.n, a.k, kps);
+  else if (bm == 32) linear_simt_kernel<WT, XT, 32><<<grid, 128, 0, st>>>(x, w, part, a.m, a.n, a.k, kps);
+  else linear_simt_kernel<WT, XT, 64><<<grid, 256, 0, st>>>(x, w, part, a.m, a.n, a.k, kps);
+}
+
+int launch_linear_simt(const LinearArgs& a, cudaStream_t st, cudaError_t* err) {
+  int bm, s, kps;
+  simt_plan(a.m, a.n, a.k, &bm, &s, &kps);
+  size_t need = (size_t)s * a.m * a.n * sizeof(float);
+  if (need > a.workspace_bytes || a.workspace == nullptr) { *err = cudaErrorInvalidValue; return -1; }
+  float* part = (float*)a.workspace;
+  dim3 grid(ceil_div(a.n, SBN), s);
+  if (a.dtype == DT_F32) simt_dispatch<float, float>(a, bm, grid, part, kps, st);
+  else if (a.dtype == DT_BF16) simt_dispatch<bf16, bf16>(a, bm, grid, part, kps, st);
+  else simt_dispatch<fp8e4m3, bf16>(a, bm, grid, part, kps, st);
+  size_t total = (size_t)a.m * a.n;
+  splitk_epilogue_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(part, s, a.m, a.n, a.scale, a.bias, a.y,
+                                                                         a.ldy, a.accumulate);
+  *err = cudaGetLastError();
+  return *err == cudaSuccess ? 2 : -1;
+}
+
+// ================================================================================================
+// embedding gather / row conversion
+// ================================================================================================
+template <typename ET>
+__global__ void embed_kernel(const ET* __restrict__ table, const int32_t* __restrict__ tokens,
+                             float* __restrict__ h, int hidden) {
+  int r = blockIdx.x;
+  const ET* src = table + (size_t)(tokens ? tokens[r] : r) * hidden;
+  for (int c = threadIdx.x; c < hidden; c += blockDim.x) h[(size_t)r * hidden + c] = to_f32(src[c]);
+}
+void launch_embed(const void* table, const int32_t* tokens, float* h, int n, int hidden, int dtype, cudaStream_t st) {
+  if (dtype == DT_F32) embed_kernel<float><<<n, 256, 0, st>>>((const float*)table, tokens, h, hidden);
+  else embed_kernel<bf16><<<n, 256, 0, st>>>((const bf16*)table, tokens, h, hidden);
+}
+void launch_rows_to_f32(const void* rows, float* h, int n, int hidden, int dtype, cudaStream_t st) {
+  launch_embed(rows, nullptr, h, n, hidden, dtype, st);
+}
+
+// ================================================================================================
+// RMSNorm: out = x * rsqrt(mean(x^2) + eps) * g, fp32 math, output in the activation type
+// ================================================================================================
+template <typename AT>
+__global__ void rmsnorm_kernel(const float* __restrict__ h, const float* __restrict__ g, AT* __restrict__ out,
+                               int hidden, float eps) {
+  __shared__ float red[32];
+  const float* x = h + (size_t)blockIdx.x * hidden;
+  float ss = 0.f;
+  for (int c = threadIdx.x; c < hidden; c += blockDim.x) { float v = x[c]; ss = fmaf(v, v, ss); }
+  ss = block_sum(ss, red);
+  float r = rsqrtf(ss / (float)hidden + eps);
+  AT* o = out + (size_t)blockIdx.x * hidden;
+  for (int c = threadIdx.x; c < hidden; c += blockDim.x) o[c] = from_f32<AT>(x[c] * r * g[c]);
+}
+void launch_rmsnorm(const float* h, const float* g, void* out, int n, int hidden, float eps, int dtype, cudaStream_t st) {
+  if (dtype == DT_F32) rmsnorm_kernel<float><<<n, 256, 0, st>>>(h, g, (float*)out, hidden, eps);
+  else rmsnorm_kernel<bf16><<<n, 256, 0, st>>>(h, g, (bf16*)out, hidden, eps);
+}
+
+// ================================================================================================
+// rotary table: cs[r][j] = (cos, sin)(pos * theta^(-2j/d)), angles formed in fp64
+// ================================================================================================
+__global__ void rope_table_kernel(float2* __restrict__ cs, int n, int pos0, int half, double theta) {
+  int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= n * half) return;
+  int r = idx / half, j = idx % half;
+  double inv = pow(theta, -(double)j / (double)half);
+  double ang = (double)(pos0 + r) * inv, s, c;
+  sincos(ang, &s, &c);
+  cs[idx] = make_float2((float)c, (float)s);
+}
+void launch_rope_table(float* cs, int n, int pos0, int head_dim, float theta, cudaStream_t st) {
+  int half = head_dim / 2, total = n * half;
+  rope_table_kernel<<<(total + 127) / 128, 128, 0, st>>>((float2*)cs, n, pos0, half, (double)theta);
+}
+
+// rotate-half pairing (j, j + d/2); q -> q buffer, k -> cache K plane, v -> cache V plane
+template <typename AT>
+__global__ void qkv_post_kernel(const float* __restrict__ qkv, const float2* __restrict__ cs, AT* __restrict__ q,
+                                AT* __restrict__ kc, AT* __restrict__ vc, int pos0, int hq, int hkv, int d, int max_seq) {
+  int r = blockIdx.x, half = d >> 1;
+  int width = (hq + 2 * hkv) * d;
+  const float* row = qkv + (size_t)r * width;
+  int pairs = (hq + hkv) * half;
+  for (int t = threadIdx.x; t < pairs; t += blockDim.x) {
+    int head = t / half, j = t % half;
+    float2 c = cs[r * half + j];
+    float a = row[head * d + j], b = row[head * d + j + half];
+    float ra = a * c.x - b * c.y, rb = b * c.x + a * c.y;
+    if (head < hq) {
+      AT* o = q + ((size_t)r * hq + head) * d;
+      o[j] = from_f32<AT>(ra); o[j + half] = from_f32<AT>(rb);
+    } else {
+      AT* o = kc + ((size_t)(head - hq) * max_seq + pos0 + r) * d;
+      o[j] = from_f32<AT>(ra); o[j + half] = from_f32<AT>(rb);
+    }
+  }
+  const float* vrow = row + (hq + hkv) * d;
+  for (int t = threadIdx.x; t < hkv * d; t += blockDim.x) {
+    int head = t / d, j = t % d;
+    vc[((size_t)head * max_seq + pos0 + r) * d + j] = from_f32<AT>(vrow[t]);
+  }
+}
+void launch_qkv_post(const float* qkv, const float* cs, void* q, void* kc, void* vc, int n, int pos0, int hq, int hkv,
+                     int d, int max_seq, int dtype, cudaStream_t st) {
+  if (dtype == DT_F32)
+    qkv_post_kernel<float><<<n, 256, 0, st>>>(qkv, (const float2*)cs, (float*)q, (float*)kc, (float*)vc, pos0, hq, hkv, d, max_seq);
+  else
+    qkv_post_kernel<bf16><<<n, 256, 0, st>>>(qkv, (const float2*)cs, (bf16*)q, (bf16*)kc, (bf16*)vc, pos0, hq, hkv, d, max_seq);
+}
+
+// ================================================================================================
+// SwiGLU: act = silu(gate) * up, gu = [n, 2*inter] with gate in the first half of each row
+// ================================================================================================
+template <typename AT>
+__global__ void swiglu_kernel(const float* __restrict__ gu, AT* __restrict__ act, int n, int inter) {
+  size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (size_t)n * inter) return;
+  int r = (int)(idx / inter), c = (int)(idx % inter);
+  float g = gu[(size_t)r * 2 * inter + c], u = gu[(size_t)r * 2 * inter + inter + c];
+  act[idx] = from_f32<AT>(g / (1.f + expf(-g)) * u);
+}
+void launch_swiglu(const float* gu, void* act, int n, int inter, int dtype, cudaStream_t st) {
+  size_t total = (size_t)n * inter;
+  unsigned blocks = (unsigned)((total + 255) / 256);
+  if (dtype == DT_F32) swiglu_kernel<float><<<blocks, 256, 0, st>>>(gu, (float*)act, n, inter);
+  else swiglu_kernel<bf16><<<blocks, 256, 0, st>>>(gu, (bf16*)act, n, inter);
+}
+
+// ================================================================================================
+// confidence and prediction of a row: pred = argmax_{v != mask_id} l_v (lowest id on a tie),
+// conf = 1 / sum_{v != mask_id} exp(l_v - l_pred)
+// ================================================================================================
+__global__ void __launch_bounds__(1024) row_stats_kernel(const float* __restrict__ logits, int vocab, int mask_id,
+                                                       float* __restrict__ conf, int32_t* __restrict__ pred) {
+  __shared__ float red[32];
+  __shared__ float smax[32];
+  __shared__ int sidx[32];
+  const float* l = logits + (size_t)blockIdx.x * vocab;
+  float best = -INFINITY;
+  int bi = 0x7fffffff;
+  for (int v = threadIdx.x; v < vocab; v += blockDim.x) {
+    if (v == mask_id) continue;
+    float x = l[v];
+    if (x > best) { best = x; bi = v; }
+  }
+  int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    float ob = __shfl_xor_sync(0xffffffffu, best, o);
+    int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+    if (ob > best || (ob == best && oi < bi)) { best = ob; bi = oi; }
+  }
+  if (lane == 0) { smax[w] = best; sidx[w] = bi; }
+  __syncthreads();
+  if (w == 0) {
+    best = lane < nw ? smax[lane] : -INFINITY;
+    bi = lane < nw ? sidx[lane] : 0x7fffffff;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      float ob = __shfl_xor_sync(0xffffffffu, best, o);
+      int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+      if (ob > best || (ob == best && oi < bi)) { best = ob; bi = oi; }
+    }
+    if (lane == 0) { smax[0] = best; sidx[0] = bi; }
+  }
+  __syncthreads();
+  best = smax[0];
+  float s = 0.f;
+  for (int v = threadIdx.x; v < vocab; v += blockDim.x)
+    if (v != mask_id) s += __expf(l[v] - best);
+  s = block_sum(s, red);
+  if (threadIdx.x == 0) { conf[blockIdx.x] = 1.f / s; pred[blockIdx.x] = sidx[0]; }
+}
+void launch_row_stats(const float* logits, int n, int vocab, int mask_id, float* conf, int32_t* pred, cudaStream_t st) {
+  row_stats_kernel<<<n, 1024, 0, st>>>(logits, vocab, mask_id, conf, pred);
+}
+
+// ================================================================================================
+// unmask selection (one CTA of 64 threads; n <= 64)
+// ================================================================================================
+__global__ void select_kernel(const float* __restrict__ conf, const int32_t* __restrict__ pred,
+                              int32_t* __restrict__ tokens, uint8_t* __restrict__ masked,
+                              uint8_t* __restrict__ unmask, int32_t* __restrict__ info, int n, int rule,
+                              float threshold, int k) {
+  __shared__ float c[64];
+  __shared__ int mk[64];
+  int i = threadIdx.x;
+  c[i] = i < n ? conf[i] : -1.f;
+  mk[i] = i < n ? (int)masked[i] : 0;
+  __syncthreads();
+  int is_m = mk[i];
+  int rank = 0, n_masked = 0;
+  for (int j = 0; j < n; ++j) {
+    if (!mk[j]) continue;
+    ++n_masked;
+    if (c[j] > c[i] || (c[j] == c[i] && j < i)) ++rank;
+  }
+  int sel;
+  if (rule == 0) {
+    int hit = is_m && (c[i] > threshold);
+    int any = __syncthreads_or(hit);
+    sel = any ? hit : (is_m && rank == 0);
+  } else {
+    sel = is_m && rank < k;
+  }
+  int n_sel = __syncthreads_count(sel);
+  if (i < n) {
+    unmask[i] = (uint8_t)sel;
+    if (sel) { tokens[i] = pred[i]; masked[i] = 0; }
+  }
+  if (i == 0) { info[0] = n_sel; info[1] = n_masked - n_sel; info[2] = info[2] + 1; }
+}
+void launch_select(const float* conf, const int32_t* pred, int32_t* tokens, uint8_t* masked, uint8_t* unmask,
+                   int32_t* info, int n, int rule, float threshold, int k, cudaStream_t st) {
+  select_kernel<<<1, 64, 0, st>>>(conf, pred, tokens, masked, unmask, info, n, rule, threshold, k);
+}
+
+__global__ void init_block_kernel(int32_t* tokens, uint8_t* masked, int32_t* info, const int32_t* init, int n, int mask_id,
+                                  int step) {
+  int i = threadIdx.x;
+  int t = (i < n && init) ? init[i] : mask_id;
+  int m = (i < n) && (t == mask_id);
+  if (i < n) { tokens[i] = t; masked[i] = (uint8_t)m; }
+  int cnt = __syncthreads_count(m);
+  if (i == 0) { info[0] = 0; info[1] = cnt; info[2] = step; }
+}
+void launch_init_block(int32_t* tokens, uint8_t* masked, int32_t* info, const int32_t* init, int n, int mask_id, int step,
+                       cudaStream_t st) {
+  init_block_kernel<<<1, 64, 0, st>>>(tokens, masked, info, init, n, mask_id, step);
+}
+
+// ================================================================================================
+// attention, CUDA-core version: one CTA per (query head, row).  Exact-fp32 path of the fp32
+// configuration and the fallback where the tensor-core kernel does not apply.
+// ================================================================================================
+template <typename AT>
+__global__ void __launch_bounds__(128) attn_simt_kernel(const AT* __restrict__ q, const AT* __restrict__ kc,
+                                                        const AT* __restrict__ vc, AT* __restrict__ out, int n,
+                                                        int L, int max_seq, int hq, int hkv, int d, int causal) {
+  extern __shared__ float smem[];
+  float* qs = smem;          // [d]
+  float* red = smem + d;     // [32]
+  float* ov = red + 32;      // [128]
+  float* sc = ov + 128;      // [T]
+  const int hqi = blockIdx.x, r = blockIdx.y;
+  const int hk = hqi / (hq / hkv);
+  const int T = causal ? (L + r + 1) : (L + n);
+  const float scale = rsqrtf((float)d);
+  const AT* qrow = q + ((size_t)r * hq + hqi) * d;
+  for (int t = threadIdx.x; t < d; t += blockDim.x) qs[t] = to_f32(qrow[t]) * scale;
+  __syncthreads();
+  const AT* kbase = kc + (size_t)hk * max_seq * d;
+  const AT* vbase = vc + (size_t)hk * max_seq * d;
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  const int epl = d / 32;
+  for (int j = w; j < T; j += nw) {
+    const AT* kr = kbase + (size_t)j * d + lane * epl;
+    float p = 0.f;
+    for (int e = 0; e < epl; ++e) p = fmaf(qs[lane * epl + e], to_f32(kr[e]), p);
+    p = warp_sum(p);
+    if (lane == 0) sc[j] = p;
+  }
+  __syncthreads();
+  float mx = -INFINITY;
+  for (int j = threadIdx.x; j < T; j += blockDim.x) mx = fmaxf(mx, sc[j]);
+  mx = block_max(mx, red);
+  float sum = 0.f;
+  for (int j = threadIdx.x; j < T; j += blockDim.x) { float e = expf(sc[j] - mx); sc[j] = e; sum += e; }
+  sum = block_sum(sum, red);
+  __syncthreads();
+  const int dd = threadIdx.x % d, part = threadIdx.x / d, nparts = blockDim.x / d;
+  float acc = 0.f;
+  for (int j = part; j < T; j += nparts) acc = fmaf(sc[j], to_f32(vbase[(size_t)j * d + dd]), acc);
+  ov[threadIdx.x] = acc;
+  __syncthreads();
+  if (part == 0) {
+    for (int p2 = 1; p2 < nparts; ++p2) acc += ov[p2 * d + dd];
+    out[((size_t)r * hq + hqi) * d + dd] = from_f32<AT>(acc / sum);
+  }
+}
+
+int launch_attention_simt(const AttnArgs& a, cudaStream_t st, cudaError_t* err) {
+  size_t smem = (size_t)(a.d + 32 + 128 + a.cache_len + a.n) * sizeof(float);
+  dim3 grid(a.hq, a.n);
+  *err = cudaSuccess;
+  if (a.dtype == DT_F32) {
+    if (smem > 48 * 1024) *err = cudaFuncSetAttribute(attn_simt_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (*err != cudaSuccess) return -1;
+    attn_simt_kernel<float><<<grid, 128, smem, st>>>((const float*)a.q, (const float*)a.kc, (const float*)a.vc,
+                                                     (float*)a.out, a.n, a.cache_len, a.max_seq, a.hq, a.hkv, a.d, a.causal);
+  } else {
+    if (smem > 48 * 1024) *err = cudaFuncSetAttribute(attn_simt_kernel<bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (*err != cudaSuccess) return -1;
+    attn_simt_kernel<bf16><<<grid, 128, smem, st>>>((const bf16*)a.q, (const bf16*)a.kc, (const bf16*)a.vc, (bf16*)a.out,
+                                                    a.n, a.cache_len, a.max_seq, a.hq, a.hkv, a.d, a.causal);
+  }
+  *err = cudaGetLastError();
+  return *err == cudaSuccess ? 1 : -1;
+}
+
+}  // namespace fdk

@@ -1,0 +1,55 @@
+// Launchers of the fdvlm kernels (host-callable; all asynchronous on `st`).
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace fdk {
+
+// ---- small-M linear: y[m,n] = sum_k x[m,k] w[n,k] (* scale[n]) (+ bias[n]) ---------------------
+struct LinearArgs {
+  const void* x;        // [m, k]   fp32 (DT_F32) or bf16
+  const void* w;        // [n, k]   per dtype
+  const float* scale;   // [n] or null
+  const float* bias;    // [n] or null
+  float* y;             // [m, ldy] fp32 result (written, or accumulated into when `accumulate`)
+  int m, n, k, ldy;
+  int accumulate;       // 1: y += result (residual add)
+  int dtype;            // DT_*
+  void* workspace;      // split-K partial sums
+  size_t workspace_bytes;
+};
+size_t linear_workspace_bytes(int m, int n, int k, int dtype);
+// Returns the number of kernels launched, or -1 with *err set.
+int launch_linear(const LinearArgs& a, cudaStream_t st, cudaError_t* err);
+
+// ---- elementwise / reduction kernels -----------------------------------------------------------
+void launch_embed(const void* table, const int32_t* tokens, float* h, int n, int hidden, int dtype, cudaStream_t st);
+void launch_rows_to_f32(const void* rows, float* h, int n, int hidden, int dtype, cudaStream_t st);
+void launch_rmsnorm(const float* h, const float* g, void* out, int n, int hidden, float eps, int dtype, cudaStream_t st);
+void launch_rope_table(float* cs, int n, int pos0, int head_dim, float theta, cudaStream_t st);
+// qkv fp32 [n, (Hq + 2 Hkv) d] -> q (act type) [n, Hq, d] rotated; K (rotated) and V written into the
+// layer's cache planes [Hkv, max_seq, d] at positions pos0 .. pos0 + n - 1.
+void launch_qkv_post(const float* qkv, const float* cs, void* q, void* kc, void* vc, int n, int pos0,
+                     int hq, int hkv, int d, int max_seq, int dtype, cudaStream_t st);
+void launch_swiglu(const float* gu, void* act, int n, int inter, int dtype, cudaStream_t st);
+void launch_row_stats(const float* logits, int n, int vocab, int mask_id, float* conf, int32_t* pred, cudaStream_t st);
+// Unmask selection + block-state update.  info = {n_unmasked, n_remaining, step_index}.
+void launch_select(const float* conf, const int32_t* pred, int32_t* tokens, uint8_t* masked, uint8_t* unmask,
+                   int32_t* info, int n, int rule, float threshold, int k, cudaStream_t st);
+void launch_init_block(int32_t* tokens, uint8_t* masked, int32_t* info, const int32_t* init, int n, int mask_id,
+                       int step, cudaStream_t st);
+
+// ---- attention -----------------------------------------------------------------------------------
+struct AttnArgs {
+  const void* q;   // [n, Hq, d]
+  const void* kc;  // [Hkv, max_seq, d]
+  const void* vc;
+  void* out;       // [n, Hq*d]
+  int n, cache_len, max_seq, hq, hkv, d, causal, dtype;
+  void* workspace;
+};
+size_t attention_workspace_bytes(int n, int hq, int hkv, int d);
+int launch_attention(const AttnArgs& a, cudaStream_t st, cudaError_t* err);
+
+}  // namespace fdk
