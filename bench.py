@@ -1,0 +1,339 @@
+#!/usr/bin/env python
+"""Benchmark of the block-diffusion decode hot path (one JSON line on stdout).
+
+A "step" of this bench is one whole pass of the hot path over one block: block_begin, the denoise
+steps of the workload's schedule (each = decoder forward in denoise mode + LM head + confidence +
+unmask selection) and commit_block (causal forward with KV-cache update).  The metric is batch-1
+decode tokens/s = block tokens / time, whole job over all GPUs (independent replicas, one request
+per GPU: the path has no data-path collective).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+`--impl reference` times the CPU oracle (as it stands) on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2604_06832_b200 import inputs as I  # noqa: E402
+
+DEFAULT_WORKLOAD = "cfg2_3b_bf16_p1024_b32_top8"
+METRIC = "batch-1 decode tok/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.t.join(timeout=2)
+        sm = [float(r[0]) for r in self.rows if len(r) >= 7 and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) >= 7 and r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(len(r) >= 7 and r[3 + i].lower().startswith("active") for r in self.rows)]
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(sm)}
+
+
+def schedule(wl: I.Workload, block: int):
+    """Denoise steps per block on a random-init model: top-k gives ceil(B/k) steps; threshold 0.9 never
+    fires on near-uniform confidences, so the at-least-one rule gives B steps."""
+    return (block + wl.k - 1) // wl.k if wl.rule == "topk" else block
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle timing (the reported cpu_baseline, and the whole of --impl reference)
+# ------------------------------------------------------------------------------------------------
+def oracle_sample(wl: I.Workload, block: int, weights_cpu: dict, reps: int = 1):
+    """Time the oracle on a bounded sample: after an (untimed) 32-row prefill, one denoise step and one
+    commit of a block; tokens/s extrapolated with the workload's schedule."""
+    import numpy as np
+    from oracle import fdvlm_oracle as orc
+    shape = wl.shape
+    o = orc.Oracle(shape, I.weights_to_numpy(weights_cpu))
+    emb, toks = I.make_prefix(shape, 16, 16, wl.prefix_seed)
+    o.prefill(I.as_numpy_storage(emb), toks.numpy(), want_logits=False)
+    rule = orc.TOPK if wl.rule == "topk" else orc.THRESHOLD
+    t_steps, t_commits = [], []
+    for _ in range(reps):
+        o.block_begin(block)
+        t0 = time.perf_counter()
+        o.block_step(rule, wl.threshold, wl.k)
+        t_steps.append(time.perf_counter() - t0)
+        o.block_tokens[:] = np.arange(block) % (shape.vocab - 1)
+        o.masked[:] = False
+        t0 = time.perf_counter()
+        o.commit_block(want_logits=True)
+        t_commits.append(time.perf_counter() - t0)
+    ts, tc = statistics.median(t_steps), statistics.median(t_commits)
+    n_steps = schedule(wl, block)
+    tok_s = block / (n_steps * ts + tc)
+    return tok_s, ts, tc
+
+
+def run_reference(args, wl, block):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    shape = wl.shape
+    weights = I.make_weights(shape, wl.weight_seed)
+    cores = torch.get_num_threads()
+    vals = []
+    for _ in range(args.warmup):
+        pass   # nothing to warm on the CPU path beyond the first BLAS call inside the first sample
+    t_all0 = time.perf_counter()
+    for _ in range(max(1, args.steps)):
+        v, ts, tc = oracle_sample(wl, block, weights)
+        vals.append(v)
+        if time.perf_counter() - t_all0 > 150.0:     # keep the whole arm within a few minutes
+            break
+    wall = time.perf_counter() - t_all0
+    value = statistics.median(vals)
+    sample = (f"per step: one denoise forward + one commit forward of a {block}-token block at cache length 32, "
+              f"tokens/s extrapolated over the schedule ({schedule(wl, block)} denoise steps + 1 commit per block)")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "tok/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1000.0 * block / value, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "block": block},
+            "cpu_baseline": {"value": value, "unit": "tok/s", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "tok/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "wall_s": wall}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------
+# the CUDA path
+# ------------------------------------------------------------------------------------------------
+def run_ours(args, wl, block):
+    from paper_2604_06832_b200 import binding as B
+    from paper_2604_06832_b200 import build as build_mod
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the CUDA path has no fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        build_mod.build()
+    if dist is not None:
+        dist.barrier()
+    shape = wl.shape
+    n_steps = schedule(wl, block)
+    K, W = args.steps, args.warmup
+    L0 = wl.n_embeds + wl.n_tokens
+    max_seq = L0 + (2 * (K + W) + 2) * block + 64
+    weights = I.make_weights(shape, wl.weight_seed, device="cuda")
+    stream = torch.cuda.Stream()
+    handle = B.Handle(shape, weights, max_seq=max_seq, max_block=max(block, 32), stream=stream)
+    emb, toks = I.make_prefix(shape, wl.n_embeds, wl.n_tokens, wl.prefix_seed)
+    emb_d, toks_d = emb.cuda(), toks.cuda()
+    rule = B.RULE_TOPK if wl.rule == "topk" else B.RULE_THRESHOLD
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    with torch.cuda.stream(stream):
+        t0, t1 = ev(), ev()
+        t0.record(stream)
+        handle.prefill(emb_d, toks_d)
+        t1.record(stream)
+        stream.synchronize()
+        prefill_ms = t0.elapsed_time(t1)
+
+        launches = [0]
+
+        def one_block_device():
+            handle.block_begin(block)
+            n = 0
+            while True:
+                info = handle.block_step(rule, wl.threshold, wl.k)
+                launches[0] += handle.last_launch_count()
+                n += 1
+                if info.n_remaining == 0:
+                    break
+            handle.commit_block()
+            launches[0] += handle.last_launch_count()
+            return n
+
+        conf_h = torch.empty(block, dtype=torch.float32).pin_memory()
+        pred_h = torch.empty(block, dtype=torch.int32).pin_memory()
+        um_h = torch.empty(block, dtype=torch.uint8).pin_memory()
+        tok_h = torch.empty(block, dtype=torch.int32).pin_memory()
+        init_h = torch.full((block,), shape.mask_id, dtype=torch.int32).pin_memory()
+
+        def one_block_host():
+            handle.block_begin_host(block, init_h)
+            while True:
+                info = handle.block_step_host(rule, wl.threshold, wl.k, conf=conf_h, pred=pred_h, unmask=um_h, block_tokens=tok_h)
+                if info.n_remaining == 0:
+                    break
+            handle.commit_block()
+
+        def timed(fn, k):
+            if dist is not None:
+                dist.barrier()
+            torch.cuda.synchronize()
+            a, b = ev(), ev()
+            a.record(stream)
+            for _ in range(k):
+                fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            ms = a.elapsed_time(b)
+            if dist is not None:
+                t = torch.tensor([ms], device="cuda")
+                dist.all_reduce(t, op=dist.ReduceOp.MAX)
+                ms = float(t.item())
+            return ms
+
+        for _ in range(W):
+            steps_seen = one_block_device()
+        sampler = ClockSampler(local)
+        sampler.start()
+        launches[0] = 0
+        ms_dev = timed(one_block_device, K)
+        n_launch = launches[0]
+        clocks = sampler.stop()
+        # end to end: host buffers through the C ABI (H2D of the block's init tokens, D2H of every step's results)
+        one_block_host()
+        ms_e2e = timed(one_block_host, K)
+
+        # per-step latency and roofline of the dominant kernel family (projection GEMMs), profiled repeat
+        handle.profile_enable(True)
+        step_ms = []
+        handle.block_begin(block)
+        L_step = handle.cache_len()
+        for _ in range(n_steps):
+            a, b = ev(), ev()
+            a.record(stream)
+            handle.block_step(rule, wl.threshold, wl.k)
+            b.record(stream)
+            stream.synchronize()
+            step_ms.append(a.elapsed_time(b))
+        prof = handle.profile_read()
+        handle.profile_enable(False)
+        # unprofiled per-step latency
+        handle.commit_block()
+        handle.block_begin(block)
+        L_step = handle.cache_len()
+        lat = []
+        for _ in range(n_steps):
+            a, b = ev(), ev()
+            a.record(stream)
+            handle.block_step(rule, wl.threshold, wl.k)
+            b.record(stream)
+            stream.synchronize()
+            lat.append(a.elapsed_time(b))
+        handle.commit_block()
+
+    tokens = K * block * world
+    value = tokens / (ms_dev / 1000.0)
+    e2e_value = tokens / (ms_e2e / 1000.0)
+    peak, peak_kind = measured_peaks()
+    wbytes = shape.weight_bytes()
+    gemm_ms_per_fwd = prof["ms_linear"] / n_steps
+    gemm_gbs = wbytes / (gemm_ms_per_fwd / 1000.0) / 1e9
+    step_bytes = wbytes + shape.kv_bytes_per_token() * L_step
+    step_med = statistics.median(lat)
+    line = {
+        "metric": METRIC, "value": value, "unit": "tok/s", "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms_dev / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": {"f32": "f32", "bf16": "bf16", "fp8": "bf16 x e4m3 weights"}[shape.dtype], "data": "synthetic",
+        "config": {"workload": wl.name, "block": block, "prefix": L0, "denoise_steps_per_block": n_steps,
+                   "rule": wl.rule, "cache_flush": "inputs (6.2 GB of weights per forward) larger than L2",
+                   "parallelism": f"replicas x{world}"},
+        "e2e": {"value": e2e_value, "unit": "tok/s", "h2d_bytes_per_step": block * 4,
+                "d2h_bytes_per_step": n_steps * (block * 13 + 16)},
+        "gpu_launches": n_launch,
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "achieved": gemm_gbs, "peak": peak, "unit": "GB/s", "frac": gemm_gbs / peak,
+                     "traffic": None, "peak_kind": peak_kind, "kernel": "projection GEMMs (all linear weights of one forward)",
+                     "algorithmic_bytes_per_forward": wbytes, "ms_per_forward": gemm_ms_per_fwd},
+        "step": {"latency_ms_median": step_med, "latency_ms_all": lat, "cache_len": L_step, "bytes": step_bytes,
+                 "gbs": step_bytes / (step_med / 1000.0) / 1e9, "frac_of_peak": step_bytes / (step_med / 1000.0) / 1e9 / peak,
+                 "frac_of_8tbs": step_bytes / (step_med / 1000.0) / 1e9 / 8000.0},
+        "prefill_ms": prefill_ms,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        wcpu = {k: (v.cpu() if isinstance(v, torch.Tensor) else v) for k, v in weights.items() if k != "layers"}
+        wcpu["layers"] = [{k: (v.cpu() if isinstance(v, torch.Tensor) else v) for k, v in lw.items()} for lw in weights["layers"]]
+        v, ts, tc = oracle_sample(wl, block, wcpu)
+        line["cpu_baseline"] = {"value": v, "unit": "tok/s", "cores": torch.get_num_threads(), "kind": "oracle",
+                                "sample": f"one denoise forward ({ts:.1f} s) + one commit forward ({tc:.1f} s) of a {block}-token block "
+                                          f"at cache length 32, extrapolated over {n_steps} denoise steps + 1 commit per block"}
+    handle.close()
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=8)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(I.WORKLOADS))
+    ap.add_argument("--block", type=int, default=0, help="block size (default: the workload's last listed size)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    wl = I.WORKLOADS[args.workload]
+    block = args.block or (32 if 32 in wl.block_sizes else wl.block_sizes[-1])
+    if args.impl == "reference":
+        run_reference(args, wl, block)
+    else:
+        run_ours(args, wl, block)
+
+
+if __name__ == "__main__":
+    main()

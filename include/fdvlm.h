@@ -156,6 +156,13 @@ int fdvlm_cache_read(const fdvlm_t *h, int layer, int which, int pos0, int n, vo
 /* Number of kernel launches issued by the last prefill / step / commit call of this handle. */
 int fdvlm_last_launch_count(const fdvlm_t *h);
 
+/* Instrumentation: while enabled, every projection (GEMM) launch group and every attention launch of
+ * this handle is bracketed by CUDA events on the handle's stream.  fdvlm_profile_read synchronises
+ * the stream, returns the summed device time (milliseconds) and the number of bracketed groups per
+ * family since the last enable / read, and clears the counters.  Any output pointer may be NULL. */
+int fdvlm_profile_enable(fdvlm_t *h, int on);
+int fdvlm_profile_read(fdvlm_t *h, double *ms_linear, int *n_linear, double *ms_attention, int *n_attention);
+
 /* Message of the last error on this handle ("" if none); valid until the next call on it.
  * With h = NULL returns the message of the last failed fdvlm_create on this thread. */
 const char *fdvlm_last_error(const fdvlm_t *h);

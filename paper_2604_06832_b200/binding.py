@@ -70,6 +70,9 @@ EXPORTS = {
     "fdvlm_cache_read": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p]),
     "fdvlm_last_launch_count": (C.c_int, [C.c_void_p]),
     "fdvlm_last_error": (C.c_char_p, [C.c_void_p]),
+    "fdvlm_profile_enable": (C.c_int, [C.c_void_p, C.c_int]),
+    "fdvlm_profile_read": (C.c_int, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int), C.POINTER(C.c_double),
+                                     C.POINTER(C.c_int)]),
     "fdvlm_op_linear": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                                   C.c_int, C.c_void_p, C.c_void_p]),
     "fdvlm_op_linear_workspace_bytes": (C.c_size_t, [C.c_int, C.c_int, C.c_int, C.c_int]),
@@ -201,6 +204,14 @@ class Handle:
 
     def last_launch_count(self) -> int:
         return lib().fdvlm_last_launch_count(self._h)
+
+    def profile_enable(self, on: bool):
+        self._check(lib().fdvlm_profile_enable(self._h, int(on)))
+
+    def profile_read(self) -> dict:
+        ml, ma, nl, na = C.c_double(), C.c_double(), C.c_int(), C.c_int()
+        self._check(lib().fdvlm_profile_read(self._h, C.byref(ml), C.byref(nl), C.byref(ma), C.byref(na)))
+        return dict(ms_linear=ml.value, n_linear=nl.value, ms_attention=ma.value, n_attention=na.value)
 
 
 def op_linear(x: torch.Tensor, w: torch.Tensor, scale=None, bias=None, dtype: int = DT_BF16,

@@ -64,8 +64,29 @@ struct fdvlm {
   // state
   int cache_len, block_size, n_remaining, step_index, block_open;
   int launches;
+  // optional per-kernel-family timing (events around each launch group), see fdvlm_profile_*
+  int prof_on;
+  std::vector<cudaEvent_t> prof_ev;   // pairs (start, stop)
+  std::vector<int> prof_kind;         // per pair: 0 = linear, 1 = attention
+  size_t prof_used;
   char err[512];
 };
+
+static void prof_begin(fdvlm_t* h, int kind) {
+  if (!h->prof_on) return;
+  if (h->prof_used * 2 + 2 > h->prof_ev.size()) {
+    cudaEvent_t a, b;
+    if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { h->prof_on = 0; return; }
+    h->prof_ev.push_back(a); h->prof_ev.push_back(b); h->prof_kind.push_back(kind);
+  }
+  h->prof_kind[h->prof_used] = kind;
+  cudaEventRecord(h->prof_ev[h->prof_used * 2], h->st);
+}
+static void prof_end(fdvlm_t* h) {
+  if (!h->prof_on) return;
+  cudaEventRecord(h->prof_ev[h->prof_used * 2 + 1], h->st);
+  h->prof_used++;
+}
 
 static int fail(fdvlm_t* h, int code, const char* fmt, ...) {
   va_list ap;
@@ -109,6 +130,7 @@ extern "C" void fdvlm_destroy(fdvlm_t* h) {
   void* bufs[] = {h->kv, h->h, h->a, h->act, h->q, h->y, h->cs, h->logits, h->conf, h->pred, h->unmask,
                   h->blk_tokens, h->blk_masked, h->info, h->init_stage, h->ws};
   for (void* p : bufs) if (p) cudaFree(p);
+  for (cudaEvent_t ev : h->prof_ev) cudaEventDestroy(ev);
   if (h->info_host) cudaFreeHost(h->info_host);
   if (h->host_stage) cudaFreeHost(h->host_stage);
   delete h;
@@ -151,6 +173,8 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
   h->err[0] = 0;
   h->cache_len = h->block_size = h->n_remaining = h->step_index = h->block_open = 0;
   h->launches = 0;
+  h->prof_on = 0;
+  h->prof_used = 0;
   h->kv = nullptr; h->h = nullptr; h->a = h->act = h->q = nullptr; h->y = nullptr; h->cs = nullptr; h->logits = nullptr;
   h->conf = nullptr; h->pred = nullptr; h->unmask = nullptr; h->blk_tokens = nullptr; h->blk_masked = nullptr;
   h->info = nullptr; h->init_stage = nullptr; h->ws = nullptr; h->info_host = nullptr; h->host_stage = nullptr;
@@ -233,7 +257,9 @@ static int forward_rows(fdvlm_t* h, int n, int mode, int logits_rows) {
     LinearArgs a;
     a.x = x; a.w = w; a.scale = scale; a.bias = bias; a.y = y; a.m = m; a.n = nn; a.k = kk; a.ldy = ldy;
     a.accumulate = accumulate; a.dtype = h->dt; a.workspace = h->ws; a.workspace_bytes = h->ws_bytes;
+    prof_begin(h, 0);
     int r = launch_linear(a, h->st, &e);
+    prof_end(h);
     if (r < 0) return -1;
     h->launches += r;
     return 0;
@@ -252,7 +278,9 @@ static int forward_rows(fdvlm_t* h, int n, int mode, int logits_rows) {
     at.q = h->q; at.kc = kv_ptr(h, l, 0); at.vc = kv_ptr(h, l, 1); at.out = h->a; at.n = n; at.cache_len = h->cache_len;
     at.max_seq = c.max_seq; at.hq = c.n_q_heads; at.hkv = c.n_kv_heads; at.d = d; at.causal = (mode == MODE_CAUSAL);
     at.dtype = h->dt; at.workspace = h->ws;
+    prof_begin(h, 1);
     int r = launch_attention(at, h->st, &e);
+    prof_end(h);
     if (r < 0) return fail(h, FDVLM_ERR_CUDA, "attention launch: %s", cudaGetErrorString(e));
     h->launches += r + 2;
     if (lin(h->a, lw.wo, lw.s_o, nullptr, h->h, H, NQ, H, 1, n))
@@ -462,6 +490,33 @@ extern "C" int fdvlm_cache_read(const fdvlm_t* hc, int layer, int which, int pos
     const char* src = kv_ptr(h, layer, which) + ((size_t)hk * h->cfg.max_seq + pos0) * rowb;
     CU(h, cudaMemcpy2DAsync((char*)dst + hk * rowb, (size_t)hkv * rowb, src, rowb, rowb, (size_t)n, cudaMemcpyDeviceToDevice, h->st));
   }
+  return FDVLM_OK;
+}
+
+// ---- instrumentation --------------------------------------------------------------------------------
+extern "C" int fdvlm_profile_enable(fdvlm_t* h, int on) {
+  if (!h) return FDVLM_ERR_INVALID_ARG;
+  h->prof_on = on ? 1 : 0;
+  h->prof_used = 0;
+  return FDVLM_OK;
+}
+
+extern "C" int fdvlm_profile_read(fdvlm_t* h, double* ms_linear, int* n_linear, double* ms_attention, int* n_attention) {
+  if (!h) return FDVLM_ERR_INVALID_ARG;
+  CU(h, cudaStreamSynchronize(h->st));
+  double ms[2] = {0, 0};
+  int cnt[2] = {0, 0};
+  for (size_t i = 0; i < h->prof_used; ++i) {
+    float t = 0.f;
+    CU(h, cudaEventElapsedTime(&t, h->prof_ev[2 * i], h->prof_ev[2 * i + 1]));
+    ms[h->prof_kind[i]] += t;
+    cnt[h->prof_kind[i]]++;
+  }
+  if (ms_linear) *ms_linear = ms[0];
+  if (n_linear) *n_linear = cnt[0];
+  if (ms_attention) *ms_attention = ms[1];
+  if (n_attention) *n_attention = cnt[1];
+  h->prof_used = 0;
   return FDVLM_OK;
 }
 

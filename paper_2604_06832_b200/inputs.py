@@ -102,7 +102,7 @@ def _storage_dtype(dtype: str) -> torch.dtype:
 
 
 def _normal(gen: torch.Generator, rows: int, cols: int, std: float = 0.02) -> torch.Tensor:
-    return torch.empty(rows, cols, dtype=torch.float32).normal_(0.0, std, generator=gen)
+    return torch.empty(rows, cols, dtype=torch.float32, device=gen.device).normal_(0.0, std, generator=gen)
 
 
 def quantize_e4m3_rows(w: torch.Tensor):
@@ -135,7 +135,7 @@ def linear_dims(shape: ModelShape) -> Dict[str, tuple]:
 
 
 def make_weights(shape: ModelShape, seed: int, *, qkv_bias: bool = False, final_gain: float = 1.0,
-                 std: float = 0.02) -> dict:
+                 std: float = 0.02, device: str = "cpu") -> dict:
     """All model weights as CPU tensors in storage dtype.
 
     Layout of the returned dict: 'embed' [vocab, hidden] (fp32 for an fp32 model, else bf16; never
@@ -143,8 +143,10 @@ def make_weights(shape: ModelShape, seed: int, *, qkv_bias: bool = False, final_
     dicts with wq, wk, wv, wo, w_gate, w_up, w_down ([out, in] row-major), s_* fp32 [out] scales
     (fp8 only), optional fp32 biases bq, bk, bv, and fp32 gains g_attn, g_mlp.
     The draw order is fixed: embed, (lm_head), then per layer q, k, v, o, gate, up, down, (biases).
+    `device` selects where the generator runs (the CPU stream is the one the parity tests use; a CUDA
+    generator gives a different, equally seeded stream and is used by the bench for speed).
     """
-    gen = torch.Generator(device="cpu").manual_seed(seed)
+    gen = torch.Generator(device=device).manual_seed(seed)
     H = shape.hidden
     out = {"shape": shape}
     out["embed"] = _normal(gen, shape.vocab, H, std).to(_storage_dtype(shape.dtype))
@@ -152,7 +154,7 @@ def make_weights(shape: ModelShape, seed: int, *, qkv_bias: bool = False, final_
         out["lm_head"], out["s_lm_head"] = None, None
     else:
         out["lm_head"], out["s_lm_head"] = _store_linear(_normal(gen, shape.vocab, H, std), shape.dtype)
-    out["g_final"] = torch.full((H,), float(final_gain), dtype=torch.float32)
+    out["g_final"] = torch.full((H,), float(final_gain), dtype=torch.float32, device=device)
     dims = linear_dims(shape)
     layers: List[dict] = []
     for _ in range(shape.n_layers):
@@ -163,8 +165,8 @@ def make_weights(shape: ModelShape, seed: int, *, qkv_bias: bool = False, final_
             lw[_SCALE_NAMES[name]] = sc
         for bname, wname in (("bq", "wq"), ("bk", "wk"), ("bv", "wv")):
             lw[bname] = (_normal(gen, 1, dims[wname][0], std).reshape(-1) if qkv_bias else None)
-        lw["g_attn"] = torch.ones(H, dtype=torch.float32)
-        lw["g_mlp"] = torch.ones(H, dtype=torch.float32)
+        lw["g_attn"] = torch.ones(H, dtype=torch.float32, device=device)
+        lw["g_mlp"] = torch.ones(H, dtype=torch.float32, device=device)
         layers.append(lw)
     out["layers"] = layers
     return out
@@ -193,6 +195,7 @@ def as_numpy_storage(t: Optional[torch.Tensor]):
     patterns, fp8 bytes (already uint8) -> uint8.  No value conversion happens here."""
     if t is None:
         return None
+    t = t.detach().cpu()
     if t.dtype == torch.bfloat16:
         return t.contiguous().view(torch.int16).numpy().view("uint16")
     return t.contiguous().numpy()
