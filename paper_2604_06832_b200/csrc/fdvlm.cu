@@ -18,11 +18,40 @@ int launch_linear_simt(const LinearArgs& a, cudaStream_t st, cudaError_t* err);
 size_t simt_workspace_bytes(int m, int n, int k);
 int launch_attention_simt(const AttnArgs& a, cudaStream_t st, cudaError_t* err);
 
-size_t linear_workspace_bytes(int m, int n, int k, int dtype) {
-  (void)dtype;
-  return simt_workspace_bytes(m, n, k);
+void launch_splitk_epilogue(const float* part, int S, int m, int n, const float* scale, const float* bias, float* y, int ldy,
+                            int accumulate, cudaStream_t st);
+
+// Device word shared by the stand-alone operator entry points for the kernels' timeout reports.
+static int* op_status_word() {
+  static int* w = nullptr;
+  if (!w) {
+    if (cudaMalloc((void**)&w, sizeof(int)) != cudaSuccess) return nullptr;
+    cudaMemset(w, 0, sizeof(int));
+  }
+  return w;
 }
-int launch_linear(const LinearArgs& a, cudaStream_t st, cudaError_t* err) { return launch_linear_simt(a, st, err); }
+
+size_t linear_workspace_bytes(int m, int n, int k, int dtype) {
+  size_t a = simt_workspace_bytes(m, n, k);
+  size_t b = tc_linear_supported(m, n, k, dtype) ? tc_workspace_bytes(m, n, (n + 127) / 128, k) : 0;
+  return a > b ? a : b;
+}
+// One projection y = x w^T (* scale) (+ bias) (+ y): bf16 weights go to the tensor-core kernel
+// (split-K partial sums + fixed-order reduction), everything else to the CUDA-core kernel.
+int launch_linear(const LinearArgs& a, cudaStream_t st, cudaError_t* err) {
+  if (!tc_linear_supported(a.m, a.n, a.k, a.dtype)) return launch_linear_simt(a, st, err);
+  TcGroup g;
+  memset(&g, 0, sizeof(g));
+  g.x = a.x; g.m = a.m; g.k = a.k; g.w[0] = a.w; g.n[0] = a.n; g.n_mats = 1;
+  int splits = 0;
+  int* status = op_status_word();
+  if (!status || !a.workspace) { *err = cudaErrorInvalidValue; return -1; }
+  *err = tc_group_launch(g, TC_MODE_PARTIAL, (float*)a.workspace, a.workspace_bytes, &splits, nullptr, a.n, 0, nullptr, status, st);
+  if (*err != cudaSuccess) return -1;
+  launch_splitk_epilogue((const float*)a.workspace, splits, a.m, a.n, a.scale, a.bias, a.y, a.ldy, a.accumulate, st);
+  *err = cudaGetLastError();
+  return *err == cudaSuccess ? 2 : -1;
+}
 size_t attention_workspace_bytes(int n, int hq, int hkv, int d) {
   (void)n; (void)hq; (void)hkv; (void)d;
   return 0;
@@ -64,6 +93,7 @@ struct fdvlm {
   // state
   int cache_len, block_size, n_remaining, step_index, block_open;
   int launches;
+  int use_tc;      // bf16 weights on the tcgen05 + TMA kernels
   // optional per-kernel-family timing (events around each launch group), see fdvlm_profile_*
   int prof_on;
   std::vector<cudaEvent_t> prof_ev;   // pairs (start, stop)
@@ -187,6 +217,12 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
   for (auto& s : shapes) { size_t b = linear_workspace_bytes(R, s[0], s[1], h->dt); if (b > ws) ws = b; }
   size_t wa = attention_workspace_bytes(R, cfg->n_q_heads, cfg->n_kv_heads, d);
   if (wa > ws) ws = wa;
+  h->use_tc = (h->dt == DT_BF16) && tc_linear_supported(R, NQ, H, DT_BF16);
+  if (h->use_tc) {
+    const size_t g3[] = {tc_workspace_bytes(R, NQKV, (NQ + 127) / 128 + 2 * ((NKV + 127) / 128), H),
+                         tc_workspace_bytes(R, H, (H + 127) / 128, NQ), tc_workspace_bytes(R, H, (H + 127) / 128, I)};
+    for (size_t b : g3) if (b > ws) ws = b;
+  }
   h->ws_bytes = ws;
   struct { void** p; size_t bytes; } allocs[] = {
       {(void**)&h->kv, (size_t)cfg->n_layers * 2 * kv_plane(h)},
@@ -242,6 +278,8 @@ extern "C" int fdvlm_reset(fdvlm_t* h) {
 extern "C" int fdvlm_cache_len(const fdvlm_t* h) { return h ? h->cache_len : (int)FDVLM_ERR_INVALID_ARG; }
 extern "C" int fdvlm_last_launch_count(const fdvlm_t* h) { return h ? h->launches : (int)FDVLM_ERR_INVALID_ARG; }
 
+static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows);
+
 // ---- one forward over n rows already gathered into h->h -------------------------------------------
 // mode: MODE_BIDIR (denoise; Alg. 1 draft mask) or MODE_CAUSAL (prefill / commit; Alg. 1 verify mask).
 // K/V of the n rows are always staged at cache positions cache_len .. cache_len + n - 1; only the
@@ -252,6 +290,7 @@ static int forward_rows(fdvlm_t* h, int n, int mode, int logits_rows) {
   const int H = c.hidden, I = c.intermediate, d = c.head_dim;
   const int NQ = c.n_q_heads * d, NKV = c.n_kv_heads * d, NQKV = NQ + 2 * NKV;
   cudaError_t e = cudaSuccess;
+  if (h->use_tc) return forward_rows_tc(h, n, mode, logits_rows);
   auto lin = [&](const void* x, const void* w, const float* scale, const float* bias, float* y, int nn, int kk, int ldy,
                  int accumulate, int m) -> int {
     LinearArgs a;
@@ -312,6 +351,83 @@ static int forward_rows(fdvlm_t* h, int n, int mode, int logits_rows) {
   return FDVLM_OK;
 }
 
+// The same forward on the tensor-core path (bf16 weights): per layer
+//   [QKV GEMM -> split-K partials] [reduce + bias + rotary + K/V staging] [attention]
+//   [O GEMM -> partials] [reduce + residual + RMSNorm] [gate/up GEMM with SwiGLU epilogue]
+//   [down GEMM -> partials] [reduce + residual + next RMSNorm]
+// and the LM head as one GEMM writing fp32 logits.
+static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows) {
+  const fdvlm_config& c = h->cfg;
+  const int H = c.hidden, I = c.intermediate, d = c.head_dim;
+  const int NQ = c.n_q_heads * d, NKV = c.n_kv_heads * d, NQKV = NQ + 2 * NKV;
+  int* status = h->info + 3;
+  float* part = (float*)h->ws;
+  cudaError_t e = cudaSuccess;
+  auto group = [&](const void* x, int k, int nm, const void* w0, int n0, const void* w1, int n1, const void* w2, int n2) {
+    TcGroup g;
+    memset(&g, 0, sizeof(g));
+    g.x = x; g.m = n; g.k = k; g.n_mats = nm;
+    g.w[0] = w0; g.n[0] = n0; g.w[1] = w1; g.n[1] = n1; g.w[2] = w2; g.n[2] = n2;
+    return g;
+  };
+  launch_rope_table(h->cs, n, h->cache_len, d, c.rope_theta, h->st);
+  launch_reduce_residual_rmsnorm(nullptr, 0, n, H, nullptr, h->h, h->layers[0].g_attn, h->a, c.rms_eps, h->st);
+  h->launches += 2;
+  for (int l = 0; l < c.n_layers; ++l) {
+    const fdvlm_layer_weights& lw = h->layers[l];
+    int S = 0;
+    TcGroup g = group(h->a, H, 3, lw.wq, NQ, lw.wk, NKV, lw.wv, NKV);
+    prof_begin(h, 0);
+    e = tc_group_launch(g, TC_MODE_PARTIAL, part, h->ws_bytes, &S, nullptr, NQKV, 0, nullptr, status, h->st);
+    prof_end(h);
+    if (e != cudaSuccess) return fail(h, FDVLM_ERR_CUDA, "qkv projection launch: %s", cudaGetErrorString(e));
+    launch_qkv_reduce_rope(part, S, n, h->cs, nullptr, nullptr, nullptr, lw.bq, lw.bk, lw.bv, h->q, kv_ptr(h, l, 0),
+                           kv_ptr(h, l, 1), h->cache_len, c.n_q_heads, c.n_kv_heads, d, c.max_seq, h->st);
+    AttnArgs at;
+    at.q = h->q; at.kc = kv_ptr(h, l, 0); at.vc = kv_ptr(h, l, 1); at.out = h->a; at.n = n; at.cache_len = h->cache_len;
+    at.max_seq = c.max_seq; at.hq = c.n_q_heads; at.hkv = c.n_kv_heads; at.d = d; at.causal = (mode == MODE_CAUSAL);
+    at.dtype = h->dt; at.workspace = h->ws;
+    prof_begin(h, 1);
+    int r = launch_attention(at, h->st, &e);
+    prof_end(h);
+    if (r < 0) return fail(h, FDVLM_ERR_CUDA, "attention launch: %s", cudaGetErrorString(e));
+    h->launches += r + 2;
+    g = group(h->a, NQ, 1, lw.wo, H, nullptr, 0, nullptr, 0);
+    prof_begin(h, 0);
+    e = tc_group_launch(g, TC_MODE_PARTIAL, part, h->ws_bytes, &S, nullptr, H, 0, nullptr, status, h->st);
+    prof_end(h);
+    if (e != cudaSuccess) return fail(h, FDVLM_ERR_CUDA, "o projection launch: %s", cudaGetErrorString(e));
+    launch_reduce_residual_rmsnorm(part, S, n, H, nullptr, h->h, lw.g_mlp, h->a, c.rms_eps, h->st);
+    g = group(h->a, H, 2, lw.w_gate, I, lw.w_up, I, nullptr, 0);
+    prof_begin(h, 0);
+    e = tc_group_launch(g, TC_MODE_SWIGLU, nullptr, 0, nullptr, nullptr, 0, 0, h->act, status, h->st);
+    prof_end(h);
+    if (e != cudaSuccess) return fail(h, FDVLM_ERR_CUDA, "gate/up projection launch: %s", cudaGetErrorString(e));
+    g = group(h->act, I, 1, lw.w_down, H, nullptr, 0, nullptr, 0);
+    prof_begin(h, 0);
+    e = tc_group_launch(g, TC_MODE_PARTIAL, part, h->ws_bytes, &S, nullptr, H, 0, nullptr, status, h->st);
+    prof_end(h);
+    if (e != cudaSuccess) return fail(h, FDVLM_ERR_CUDA, "down projection launch: %s", cudaGetErrorString(e));
+    const float* g_next = (l + 1 < c.n_layers) ? h->layers[l + 1].g_attn : h->w.g_final;
+    launch_reduce_residual_rmsnorm(part, S, n, H, nullptr, h->h, g_next, h->a, c.rms_eps, h->st);
+    h->launches += 5;
+  }
+  if (logits_rows > 0) {
+    const int first = (logits_rows == n) ? 0 : n - 1;
+    const void* table = c.tie_embeddings ? h->w.embed : h->w.lm_head;
+    TcGroup g = group((const char*)h->a + (size_t)first * H * 2, H, 1, table, c.vocab, nullptr, 0, nullptr, 0);
+    g.m = n - first;
+    prof_begin(h, 0);
+    e = tc_group_launch(g, TC_MODE_DIRECT, nullptr, 0, nullptr, h->logits, c.vocab, 0, nullptr, status, h->st);
+    prof_end(h);
+    if (e != cudaSuccess) return fail(h, FDVLM_ERR_CUDA, "lm head launch: %s", cudaGetErrorString(e));
+    h->launches++;
+  }
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(h, FDVLM_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
+  return FDVLM_OK;
+}
+
 extern "C" int fdvlm_prefill(fdvlm_t* h, const void* embeds, int n_embeds, const int32_t* tokens, int n_tokens,
                              float* last_logits) {
   if (!h) return FDVLM_ERR_INVALID_ARG;
@@ -363,6 +479,11 @@ static int sync_info(fdvlm_t* h) {
   CU(h, cudaMemcpyAsync(h->info_host, h->info, 16, cudaMemcpyDeviceToHost, h->st));
   CU(h, cudaStreamSynchronize(h->st));
   h->n_remaining = h->info_host[1];
+  if (h->info_host[3] != 0) {
+    int code = h->info_host[3];
+    cudaMemsetAsync(h->info + 3, 0, 4, h->st);
+    return fail(h, FDVLM_ERR_TIMEOUT, "a bounded device-side wait gave up (kernel role %d); results of this call are invalid", code);
+  }
   return FDVLM_OK;
 }
 

@@ -1,0 +1,480 @@
+// Small-M weight-streaming GEMM for sm_100a: y[m, n] = sum_k x[m, k] w[n, k], m <= 64.
+//
+// The weight matrix is the MMA "A" operand (128 output features per tile fill the tensor-core M
+// dimension), the m activation rows are the MMA "N" dimension (padded to 16/32/48/64), so a CTA
+// streams 128 x K weights once while the tiny activation tile comes from L2.  Weights and
+// activations are staged by TMA (128-byte swizzle, K-major) into a ring of shared-memory stages;
+// one elected thread issues tcgen05.mma with fp32 accumulators in tensor memory (two accumulator
+// buffers, so the epilogue of one work item overlaps the mainloop of the next); four epilogue warps
+// read the accumulators with tcgen05.ld.  CTAs are persistent over a static round-robin list of
+// work items (tile, K-split).  Every mbarrier wait is bounded: on a timeout the CTA records an
+// error code in a status word, drains its own bulk copies, frees its tensor memory and returns.
+#include <cuda.h>
+
+#include <map>
+#include <mutex>
+#include <tuple>
+
+#include "common.cuh"
+#include "kernels.h"
+
+namespace fdk {
+
+constexpr int TC_BM = 128;       // weight rows per tile (MMA M)
+constexpr int TC_BK = 64;        // bf16 elements per k-block: 128 bytes = one swizzle atom row
+constexpr int TC_STAGES = 4;
+constexpr int TC_THREADS = 192;  // warp 0 TMA producer, warp 1 MMA issuer, warps 2..5 epilogue
+constexpr long long TC_TIMEOUT = 1ll << 28;  // clock cycles (~0.14 s) before a wait gives up
+constexpr int TC_A_BYTES = TC_BM * TC_BK * 2;
+
+enum { TC_ERR_PRODUCER = 1, TC_ERR_MMA = 2, TC_ERR_EPILOGUE = 3 };
+
+struct TcParams {
+  CUtensorMap tm_w[3];  // weight matrices, box {64 k, 64 rows}
+  CUtensorMap tm_x;     // activations, box {64 k, m_pad rows}
+  int n_out[3];         // rows (output features) of each matrix
+  int tile_begin[4];    // first tile of each matrix; [n_mats] = total tiles
+  int out_col[3];       // column of each matrix's first feature in the output row
+  const float* scale[3];
+  const float* bias[3];
+  int n_mats, kblocks, splits, kb_per_split, m, mode;
+  float* part;          // [splits][m][ldp]     (PARTIAL)
+  int ldp;
+  float* y;             // [m][ldy]             (DIRECT)
+  int ldy, accumulate;
+  bf16* act;            // [m][inter]           (SWIGLU)
+  int inter;
+  int* status;          // device word, set non-zero when a wait timed out
+};
+
+// ---- PTX wrappers -------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the wait gave up (timeout here, or another thread's abort).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > TC_TIMEOUT) { *abort_flag = 1; return false; }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+      ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "l"(pol)
+      : "memory");
+}
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows 128 bytes apart, groups
+// of 8 rows 1024 bytes apart (stride-dimension byte offset), descriptor version 1 (sm_100).
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)1 << 16;                 // leading-dimension offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;       // stride-dimension offset
+  d |= (uint64_t)1 << 46;                 // version
+  d |= (uint64_t)2 << 61;                 // SWIZZLE_128B
+  return d;
+}
+// Instruction descriptor, kind::f16: D = f32, A = B = bf16, both K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t umma_idesc_bf16(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\ttcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
+  uint32_t r[16];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+template <int M_PAD>
+struct TcSmem {
+  static constexpr int B_BYTES = M_PAD * TC_BK * 2;
+  static constexpr int STAGE_BYTES = TC_A_BYTES + B_BYTES;
+  static constexpr int BAR_OFF = TC_STAGES * STAGE_BYTES;
+  static constexpr int TOTAL = BAR_OFF + 256 + 1024;  // barriers + alignment slack
+};
+
+template <int M_PAD>
+__global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_constant__ TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  using L = TcSmem<M_PAD>;
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* sm = smem_raw + (base - raw);
+  const uint32_t bar0 = base + L::BAR_OFF;
+  // barrier slots (8 bytes each): full[S], empty[S], tmem_full[2], tmem_empty[2]
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (TC_STAGES + s); };
+  auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * TC_STAGES + a); };
+  auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * TC_STAGES + 2 + a); };
+  volatile uint32_t* tmem_slot = (volatile uint32_t*)(sm + L::BAR_OFF + 8 * (2 * TC_STAGES + 4));
+  volatile int* abort_flag = (volatile int*)(sm + L::BAR_OFF + 8 * (2 * TC_STAGES + 4) + 8);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr int TMEM_COLS = (2 * M_PAD <= 32) ? 32 : ((2 * M_PAD <= 64) ? 64 : 128);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int total_tiles = p.tile_begin[p.n_mats];
+  const int n_items = total_tiles * p.splits;
+
+  if (warp == 0) {
+    // ------------------------------------------------ TMA producer ------------------------------------------------
+    if (lane == 0) {
+      const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
+      int stage = 0;
+      uint32_t phase = 0;
+      uint32_t armed = 0;           // bit s: full[s] armed and not yet known complete
+      uint32_t armed_parity = 0;    // bit s: parity of that arming
+      bool ok = true;
+      for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+        const int tile = it % total_tiles, split = it / total_tiles;
+        int mi = 0, r0 = 0;
+        if (p.mode != TC_MODE_SWIGLU) {
+          while (mi + 1 < p.n_mats && tile >= p.tile_begin[mi + 1]) ++mi;
+          r0 = (tile - p.tile_begin[mi]) * TC_BM;
+        }
+        const int kb0 = split * p.kb_per_split;
+        const int kb1 = min(p.kblocks, kb0 + p.kb_per_split);
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t a_dst = base + stage * L::STAGE_BYTES;
+          mbar_expect_tx(full_bar(stage), L::STAGE_BYTES);
+          armed |= 1u << stage;
+          armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
+          if (p.mode == TC_MODE_SWIGLU) {
+            // 64 features per tile; TMEM lane quarter qq holds gate rows of features 16qq..16qq+15 in its lanes
+            // 0..15 and the matching up rows in lanes 16..31, so the epilogue pairs them with one shuffle
+#pragma unroll
+            for (int qq = 0; qq < 4; ++qq) {
+              tma_load_2d(a_dst + (32 * qq) * 128, &p.tm_w[0], full_bar(stage), kb * TC_BK, tile * 64 + 16 * qq, pol_w);
+              tma_load_2d(a_dst + (32 * qq + 16) * 128, &p.tm_w[1], full_bar(stage), kb * TC_BK, tile * 64 + 16 * qq, pol_w);
+            }
+          } else {
+            tma_load_2d(a_dst, &p.tm_w[mi], full_bar(stage), kb * TC_BK, r0, pol_w);
+            tma_load_2d(a_dst + TC_A_BYTES / 2, &p.tm_w[mi], full_bar(stage), kb * TC_BK, r0 + 64, pol_w);
+          }
+          tma_load_2d(a_dst + TC_A_BYTES, &p.tm_x, full_bar(stage), kb * TC_BK, 0, pol_x);
+          if (++stage == TC_STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        atomicCAS(p.status, 0, TC_ERR_PRODUCER);
+        // drain: wait (bounded) for every bulk copy this thread has in flight
+        for (int s = 0; s < TC_STAGES; ++s) {
+          if (!(armed & (1u << s))) continue;
+          const uint32_t par = (armed_parity >> s) & 1u;
+          const long long t0 = clock64();
+          while (!mbar_try_wait(full_bar(s), par) && clock64() - t0 < TC_TIMEOUT) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------ MMA issuer --------------------------------------------------
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc_bf16(M_PAD);
+      int stage = 0;
+      uint32_t phase = 0;
+      int local = 0;
+      bool ok = true;
+      for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++local) {
+        const int split = it / total_tiles;
+        const int acc = local & 1;
+        const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * M_PAD);
+        const int kb0 = split * p.kb_per_split;
+        const int kb1 = min(p.kblocks, kb0 + p.kb_per_split);
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t a_addr = base + stage * L::STAGE_BYTES;
+          const uint64_t adesc = umma_desc_sw128(a_addr);
+          const uint64_t bdesc = umma_desc_sw128(a_addr + TC_A_BYTES);
+#pragma unroll
+          for (int kk = 0; kk < TC_BK / 16; ++kk)
+            umma_bf16(d_tmem, adesc + 2u * kk, bdesc + 2u * kk, idesc, (kb > kb0 || kk > 0) ? 1u : 0u);
+          umma_commit(empty_bar(stage));
+          if (++stage == TC_STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) umma_commit(tfull_bar(acc));
+      }
+      if (!ok) atomicCAS(p.status, 0, TC_ERR_MMA);
+    }
+  } else {
+    // ------------------------------------------------ epilogue warps ----------------------------------------------
+    const int q = warp & 3;  // TMEM lane quarter this warp may read
+    int local = 0;
+    bool ok = true;
+    for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++local) {
+      const int tile = it % total_tiles, split = it / total_tiles;
+      const int acc = local & 1;
+      const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
+      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      float v[M_PAD];
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * M_PAD);
+#pragma unroll
+      for (int c = 0; c < M_PAD; c += 16) tmem_ld16(taddr + c, v + c);
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
+
+      if (p.mode == TC_MODE_SWIGLU) {
+        const int col = tile * 64 + q * 16 + (lane & 15);
+        const bool live = lane < 16 && col < p.inter;
+        const float sg = (live && p.scale[0]) ? p.scale[0][col] : 1.f;
+        const float su = (live && p.scale[1]) ? p.scale[1][col] : 1.f;
+#pragma unroll
+        for (int b = 0; b < M_PAD; ++b) {
+          const float other = __shfl_xor_sync(0xffffffffu, v[b], 16);   // lanes 0..15: the matching "up" value
+          if (live && b < p.m) {
+            const float g = v[b] * sg;
+            p.act[(size_t)b * p.inter + col] = __float2bfloat16_rn(g / (1.f + __expf(-g)) * (other * su));
+          }
+        }
+      } else {
+        int mi = 0;
+        while (mi + 1 < p.n_mats && tile >= p.tile_begin[mi + 1]) ++mi;
+        const int n = (tile - p.tile_begin[mi]) * TC_BM + q * 32 + lane;
+        if (n < p.n_out[mi]) {
+          const int col = p.out_col[mi] + n;
+          if (p.mode == TC_MODE_PARTIAL) {
+            float* dst = p.part + (size_t)split * p.m * p.ldp + col;
+#pragma unroll
+            for (int b = 0; b < M_PAD; ++b)
+              if (b < p.m) dst[(size_t)b * p.ldp] = v[b];
+          } else {
+            const float sc = p.scale[mi] ? p.scale[mi][n] : 1.f;
+            const float bi = p.bias[mi] ? p.bias[mi][n] : 0.f;
+            float* dst = p.y + col;
+#pragma unroll
+            for (int b = 0; b < M_PAD; ++b) {
+              if (b < p.m) {
+                float r = v[b] * sc + bi;
+                if (p.accumulate) r += dst[(size_t)b * p.ldy];
+                dst[(size_t)b * p.ldy] = r;
+              }
+            }
+          }
+        }
+      }
+    }
+    if (!ok && lane == 0) atomicCAS(p.status, 0, TC_ERR_EPILOGUE);
+  }
+
+  // ---- teardown: every thread arrives here, whatever happened ----
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// ================================================================================================
+// host side
+// ================================================================================================
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qr) == cudaSuccess &&
+        qr == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)ptr;
+  });
+  return fn;
+}
+
+// 2-D bf16 row-major [rows, cols] tensor, box {64 columns, box_rows}, 128-byte swizzle, zero OOB fill.
+static bool make_tmap(CUtensorMap* tm, const void* ptr, int rows, int cols, int box_rows) {
+  typedef std::tuple<const void*, int, int, int> Key;
+  static std::map<Key, CUtensorMap> cache;
+  static std::mutex mu;
+  std::lock_guard<std::mutex> lock(mu);
+  Key key(ptr, rows, cols, box_rows);
+  auto it = cache.find(key);
+  if (it != cache.end()) { *tm = it->second; return true; }
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return false;
+  if (cache.size() > 4096) cache.clear();
+  cache[key] = *tm;
+  return true;
+}
+
+static int sm_count() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (n <= 0) n = 148;
+  }
+  return n;
+}
+
+static int pad_m(int m) { return m <= 16 ? 16 : (m <= 32 ? 32 : (m <= 48 ? 48 : 64)); }
+
+// Split-K plan: enough (tile, split) items to occupy every SM about twice, each split at least 2
+// k-blocks deep, never more splits than k-blocks.
+static void tc_plan(int tiles, int kblocks, int* splits, int* kbps) {
+  int s = (2 * sm_count()) / tiles;
+  if (s < 1) s = 1;
+  int max_s = kblocks / 2 > 0 ? kblocks / 2 : 1;
+  if (s > max_s) s = max_s;
+  if (s > 32) s = 32;
+  int per = ceil_div(kblocks, s);
+  *kbps = per;
+  *splits = ceil_div(kblocks, per);
+}
+
+bool tc_linear_supported(int m, int n, int k, int dtype) {
+  return dtype == DT_BF16 && m >= 1 && m <= 64 && n >= 1 && k >= 8 && (k % 8) == 0 && encode_fn() != nullptr;
+}
+
+size_t tc_workspace_bytes(int m, int ld, int tiles, int k) {
+  int s, kbps;
+  tc_plan(tiles, ceil_div(k, TC_BK), &s, &kbps);
+  return (size_t)s * m * ld * sizeof(float);
+}
+
+template <int M_PAD>
+static cudaError_t tc_launch_t(const TcParams& p, int grid, cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<M_PAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<M_PAD>::TOTAL);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  gemm_tc_kernel<M_PAD><<<grid, TC_THREADS, TcSmem<M_PAD>::TOTAL, st>>>(p);
+  return cudaGetLastError();
+}
+
+static cudaError_t tc_launch(const TcParams& p, cudaStream_t st) {
+  const int items = p.tile_begin[p.n_mats] * p.splits;
+  const int grid = items < 2 * sm_count() ? items : 2 * sm_count();
+  switch (pad_m(p.m)) {
+    case 16: return tc_launch_t<16>(p, grid, st);
+    case 32: return tc_launch_t<32>(p, grid, st);
+    case 48: return tc_launch_t<48>(p, grid, st);
+    default: return tc_launch_t<64>(p, grid, st);
+  }
+}
+
+// A group of up to three bf16 matrices that share x and K, outputs side by side in one row of width ld.
+//   mode PARTIAL: part[split][m][ld] (split-K sums left to the caller's reduce kernel); *splits_out tells how many
+//   mode DIRECT : y[m][ld] = x w^T * scale + bias (+ y)   (forces one split)
+//   mode SWIGLU : act[m][inter] = silu(x wg^T * sg) * (x wu^T * su)  (w[0] = gate, w[1] = up; one split)
+
+cudaError_t tc_group_launch(const TcGroup& g, int mode, float* part, size_t part_bytes, int* splits_out, float* y, int ld,
+                            int accumulate, void* act, int* status, cudaStream_t st) {
+  TcParams p;
+  memset(&p, 0, sizeof(p));
+  const int mp = pad_m(g.m);
+  if (!make_tmap(&p.tm_x, g.x, g.m, g.k, mp)) return cudaErrorInvalidValue;
+  int tiles = 0, col = 0;
+  for (int i = 0; i < g.n_mats; ++i) {
+    if (!make_tmap(&p.tm_w[i], g.w[i], g.n[i], g.k, mode == TC_MODE_SWIGLU ? 16 : 64)) return cudaErrorInvalidValue;
+    p.n_out[i] = g.n[i];
+    p.tile_begin[i] = tiles;
+    p.out_col[i] = col;
+    p.scale[i] = g.scale[i];
+    p.bias[i] = g.bias[i];
+    tiles += ceil_div(g.n[i], TC_BM);
+    col += g.n[i];
+  }
+  p.n_mats = g.n_mats;
+  p.kblocks = ceil_div(g.k, TC_BK);
+  p.m = g.m;
+  p.mode = mode;
+  p.status = status;
+  if (mode == TC_MODE_SWIGLU) {
+    tiles = ceil_div(g.n[0], 64);      // one combined list of 64-feature tiles (gate + up rows interleaved)
+    p.n_mats = 1;
+    p.tile_begin[0] = 0; p.tile_begin[1] = tiles;
+    p.splits = 1; p.kb_per_split = p.kblocks;
+    p.act = (bf16*)act; p.inter = g.n[0];
+  } else {
+    p.tile_begin[g.n_mats] = tiles;
+    if (mode == TC_MODE_DIRECT) { p.splits = 1; p.kb_per_split = p.kblocks; }
+    else tc_plan(tiles, p.kblocks, &p.splits, &p.kb_per_split);
+    p.part = part; p.ldp = ld; p.y = y; p.ldy = ld; p.accumulate = accumulate;
+    if (mode == TC_MODE_PARTIAL && (size_t)p.splits * g.m * ld * sizeof(float) > part_bytes) return cudaErrorInvalidValue;
+  }
+  if (splits_out) *splits_out = p.splits;
+  return tc_launch(p, st);
+}
+
+}  // namespace fdk

@@ -129,6 +129,12 @@ __global__ void splitk_epilogue_kernel(const float* __restrict__ part, int S, in
   *o = accumulate ? (*o + s) : s;
 }
 
+void launch_splitk_epilogue(const float* part, int S, int m, int n, const float* scale, const float* bias, float* y, int ldy,
+                            int accumulate, cudaStream_t st) {
+  size_t total = (size_t)m * n;
+  splitk_epilogue_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(part, S, m, n, scale, bias, y, ldy, accumulate);
+}
+
 static void simt_plan(int m, int n, int k, int* bm, int* splits, int* kps) {
   *bm = m <= 16 ? 16 : (m <= 32 ? 32 : 64);
   int tiles = ceil_div(n, SBN);
@@ -263,6 +269,83 @@ void launch_qkv_post(const float* qkv, const float* cs, void* q, void* kc, void*
     qkv_post_kernel<float><<<n, 256, 0, st>>>(qkv, (const float2*)cs, (float*)q, (float*)kc, (float*)vc, pos0, hq, hkv, d, max_seq);
   else
     qkv_post_kernel<bf16><<<n, 256, 0, st>>>(qkv, (const float2*)cs, (bf16*)q, (bf16*)kc, (bf16*)vc, pos0, hq, hkv, d, max_seq);
+}
+
+// ================================================================================================
+// Fused split-K reductions of the tensor-core path (fixed summation order => deterministic).
+// ================================================================================================
+// part[S][m][(hq + 2 hkv) d] -> sum over S, * scale, + bias, rotary on q and k, q to its buffer, k and v
+// straight into the layer's cache planes at positions pos0 + row.
+template <typename AT>
+__global__ void qkv_reduce_rope_kernel(const float* __restrict__ part, int S, int m, const float2* __restrict__ cs,
+                                       const float* __restrict__ sq, const float* __restrict__ sk,
+                                       const float* __restrict__ sv, const float* __restrict__ bq,
+                                       const float* __restrict__ bk, const float* __restrict__ bv, AT* __restrict__ q,
+                                       AT* __restrict__ kc, AT* __restrict__ vc, int pos0, int hq, int hkv, int d,
+                                       int max_seq) {
+  const int r = blockIdx.x, half = d >> 1;
+  const int nq = hq * d, nkv = hkv * d, width = nq + 2 * nkv;
+  const size_t sstride = (size_t)m * width;
+  const float* row = part + (size_t)r * width;
+  auto val = [&](int col) {
+    float s = 0.f;
+    for (int i = 0; i < S; ++i) s += row[i * sstride + col];
+    if (col < nq) { if (sq) s *= sq[col]; if (bq) s += bq[col]; }
+    else if (col < nq + nkv) { int c = col - nq; if (sk) s *= sk[c]; if (bk) s += bk[c]; }
+    else { int c = col - nq - nkv; if (sv) s *= sv[c]; if (bv) s += bv[c]; }
+    return s;
+  };
+  const int pairs = (hq + hkv) * half;
+  for (int t = threadIdx.x; t < pairs; t += blockDim.x) {
+    const int head = t / half, j = t % half;
+    const float2 c = cs[r * half + j];
+    const float a = val(head * d + j), b = val(head * d + j + half);
+    const float ra = a * c.x - b * c.y, rb = b * c.x + a * c.y;
+    AT* o = head < hq ? q + ((size_t)r * hq + head) * d : kc + ((size_t)(head - hq) * max_seq + pos0 + r) * d;
+    o[j] = from_f32<AT>(ra);
+    o[j + half] = from_f32<AT>(rb);
+  }
+  for (int t = threadIdx.x; t < nkv; t += blockDim.x) {
+    const int head = t / d, j = t % d;
+    vc[((size_t)head * max_seq + pos0 + r) * d + j] = from_f32<AT>(val(nq + nkv + t));
+  }
+}
+void launch_qkv_reduce_rope(const float* part, int S, int m, const float* cs, const float* sq, const float* sk,
+                            const float* sv, const float* bq, const float* bk, const float* bv, void* q, void* kc, void* vc,
+                            int pos0, int hq, int hkv, int d, int max_seq, cudaStream_t st) {
+  qkv_reduce_rope_kernel<bf16><<<m, 256, 0, st>>>(part, S, m, (const float2*)cs, sq, sk, sv, bq, bk, bv, (bf16*)q,
+                                                  (bf16*)kc, (bf16*)vc, pos0, hq, hkv, d, max_seq);
+}
+
+// h[r] += (sum_s part[s][r]) * scale (S may be 0: nothing added); out[r] = RMSNorm(h[r]; g) in the activation type.
+template <typename AT>
+__global__ void reduce_residual_rmsnorm_kernel(const float* __restrict__ part, int S, int m, int H,
+                                               const float* __restrict__ scale, float* __restrict__ h,
+                                               const float* __restrict__ g, AT* __restrict__ out, float eps) {
+  __shared__ float red[32];
+  const int r = blockIdx.x;
+  const size_t sstride = (size_t)m * H;
+  float* hr = h + (size_t)r * H;
+  float ss = 0.f;
+  for (int c = threadIdx.x; c < H; c += blockDim.x) {
+    float v = hr[c];
+    if (S > 0) {
+      float s = 0.f;
+      for (int i = 0; i < S; ++i) s += part[i * sstride + (size_t)r * H + c];
+      if (scale) s *= scale[c];
+      v += s;
+      hr[c] = v;
+    }
+    ss = fmaf(v, v, ss);
+  }
+  ss = block_sum(ss, red);
+  const float rs = rsqrtf(ss / (float)H + eps);
+  AT* o = out + (size_t)r * H;
+  for (int c = threadIdx.x; c < H; c += blockDim.x) o[c] = from_f32<AT>(hr[c] * rs * g[c]);
+}
+void launch_reduce_residual_rmsnorm(const float* part, int S, int m, int H, const float* scale, float* h, const float* g,
+                                    void* out, float eps, cudaStream_t st) {
+  reduce_residual_rmsnorm_kernel<bf16><<<m, 256, 0, st>>>(part, S, m, H, scale, h, g, (bf16*)out, eps);
 }
 
 // ================================================================================================

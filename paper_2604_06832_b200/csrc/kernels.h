@@ -40,6 +40,29 @@ void launch_select(const float* conf, const int32_t* pred, int32_t* tokens, uint
 void launch_init_block(int32_t* tokens, uint8_t* masked, int32_t* info, const int32_t* init, int n, int mask_id,
                        int step, cudaStream_t st);
 
+// ---- tensor-core (tcgen05 + TMA) small-M GEMM, bf16 ---------------------------------------------------
+enum { TC_MODE_PARTIAL = 0, TC_MODE_DIRECT = 1, TC_MODE_SWIGLU = 2 };
+// Up to three bf16 matrices that share x and K; their outputs sit side by side in one row of width ld.
+struct TcGroup {
+  const void* x; int m, k;
+  const void* w[3]; int n[3]; int n_mats;
+  const float* scale[3]; const float* bias[3];
+};
+bool tc_linear_supported(int m, int n, int k, int dtype);
+// Split-K workspace of a group with m rows, output width ld, `tiles` 128-row weight tiles and depth k.
+size_t tc_workspace_bytes(int m, int ld, int tiles, int k);
+//   PARTIAL: part[split][m][ld] holds the split-K partial sums (*splits_out of them), summed by the caller's
+//            reduce kernel;  DIRECT: y[m][ld] = x w^T * scale + bias (+ y when accumulate);
+//   SWIGLU : act[m][n0] = silu(x w0^T * s0) * (x w1^T * s1)  (w[0] = gate, w[1] = up)
+// status: device word set non-zero if a bounded wait inside the kernel gave up.
+cudaError_t tc_group_launch(const TcGroup& g, int mode, float* part, size_t part_bytes, int* splits_out, float* y, int ld,
+                            int accumulate, void* act, int* status, cudaStream_t st);
+void launch_qkv_reduce_rope(const float* part, int S, int m, const float* cs, const float* sq, const float* sk,
+                            const float* sv, const float* bq, const float* bk, const float* bv, void* q, void* kc, void* vc,
+                            int pos0, int hq, int hkv, int d, int max_seq, cudaStream_t st);
+void launch_reduce_residual_rmsnorm(const float* part, int S, int m, int H, const float* scale, float* h, const float* g,
+                                    void* out, float eps, cudaStream_t st);
+
 // ---- attention -----------------------------------------------------------------------------------
 struct AttnArgs {
   const void* q;   // [n, Hq, d]
