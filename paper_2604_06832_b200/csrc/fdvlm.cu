@@ -52,11 +52,13 @@ int launch_linear(const LinearArgs& a, cudaStream_t st, cudaError_t* err) {
   *err = cudaGetLastError();
   return *err == cudaSuccess ? 2 : -1;
 }
-size_t attention_workspace_bytes(int n, int hq, int hkv, int d) {
-  (void)n; (void)hq; (void)hkv; (void)d;
-  return 0;
+size_t attention_mma_workspace_bytes(int n, int hq, int hkv, int d);
+int launch_attention_mma(const AttnArgs& a, cudaStream_t st, cudaError_t* err);
+size_t attention_workspace_bytes(int n, int hq, int hkv, int d) { return attention_mma_workspace_bytes(n, hq, hkv, d); }
+// bf16 rows go to the split-KV tensor-core kernel, fp32 rows to the exact CUDA-core kernel.
+int launch_attention(const AttnArgs& a, cudaStream_t st, cudaError_t* err) {
+  return a.dtype == DT_F32 ? launch_attention_simt(a, st, err) : launch_attention_mma(a, st, err);
 }
-int launch_attention(const AttnArgs& a, cudaStream_t st, cudaError_t* err) { return launch_attention_simt(a, st, err); }
 }  // namespace fdk
 
 static thread_local char g_create_error[512] = "";
