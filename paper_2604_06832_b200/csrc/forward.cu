@@ -1,0 +1,237 @@
+// The decoder forward of one step as a launch sequence (Fast-dVLM Sec. 3.4; Appendix B Alg. 1 for the
+// two attention modes), in two flavours: the exact CUDA-core path (fp32 configuration, fp8 weights)
+// and the tensor-core path (bf16 weights).
+#include "handle.h"
+
+namespace fdk {
+
+int launch_linear_simt(const LinearArgs& a, cudaStream_t st, cudaError_t* err);
+size_t simt_workspace_bytes(int m, int n, int k);
+int launch_attention_simt(const AttnArgs& a, cudaStream_t st, cudaError_t* err);
+size_t attention_mma_workspace_bytes(int n, int hq, int hkv, int d);
+int launch_attention_mma(const AttnArgs& a, cudaStream_t st, cudaError_t* err);
+void launch_splitk_epilogue(const float* part, int S, int m, int n, const float* scale, const float* bias, float* y, int ldy,
+                            int accumulate, cudaStream_t st);
+
+thread_local char g_create_error[512] = "";
+
+// Device word shared by the stand-alone operator entry points for the kernels' timeout reports.
+static int* op_status_word() {
+  static int* w = nullptr;
+  if (!w) {
+    if (cudaMalloc((void**)&w, sizeof(int)) != cudaSuccess) return nullptr;
+    cudaMemset(w, 0, sizeof(int));
+  }
+  return w;
+}
+
+size_t linear_workspace_bytes(int m, int n, int k, int dtype) {
+  size_t a = simt_workspace_bytes(m, n, k);
+  size_t b = tc_linear_supported(m, n, k, dtype) ? tc_workspace_bytes(m, n, (n + 127) / 128, k) : 0;
+  return a > b ? a : b;
+}
+
+// One projection y = x w^T (* scale) (+ bias) (+ y): bf16 weights go to the tensor-core kernel
+// (split-K partial sums + fixed-order reduction), everything else to the CUDA-core kernel.
+int launch_linear(const LinearArgs& a, cudaStream_t st, cudaError_t* err) {
+  if (!tc_linear_supported(a.m, a.n, a.k, a.dtype)) return launch_linear_simt(a, st, err);
+  TcGroup g;
+  memset(&g, 0, sizeof(g));
+  g.x = a.x; g.m = a.m; g.k = a.k; g.w[0] = a.w; g.n[0] = a.n; g.n_mats = 1;
+  int splits = 0;
+  TcOut o;
+  memset(&o, 0, sizeof(o));
+  o.mode = TC_MODE_PARTIAL; o.part = (float*)a.workspace; o.part_bytes = a.workspace_bytes; o.splits_out = &splits;
+  o.ld = a.n; o.status = op_status_word();
+  if (!o.status || !a.workspace) { *err = cudaErrorInvalidValue; return -1; }
+  *err = tc_group_launch(g, o, st);
+  if (*err != cudaSuccess) return -1;
+  launch_splitk_epilogue((const float*)a.workspace, splits, a.m, a.n, a.scale, a.bias, a.y, a.ldy, a.accumulate, st);
+  *err = cudaGetLastError();
+  return *err == cudaSuccess ? 2 : -1;
+}
+
+size_t attention_workspace_bytes(int n, int hq, int hkv, int d) { return attention_mma_workspace_bytes(n, hq, hkv, d); }
+// bf16 rows go to the split-KV tensor-core kernel, fp32 rows to the exact CUDA-core kernel.
+int launch_attention(const AttnArgs& a, cudaStream_t st, cudaError_t* err) {
+  return a.dtype == DT_F32 ? launch_attention_simt(a, st, err) : launch_attention_mma(a, st, err);
+}
+
+int stage_rows(fdvlm_t* h, int row0, int n, const int32_t* tokens, const void* embeds) {
+  const int H = h->cfg.hidden;
+  const int edt = h->dt == DT_F32 ? DT_F32 : DT_BF16;
+  if (h->use_tc) {
+    launch_embed_prep(h->w.embed, tokens, embeds, h->h + (size_t)row0 * H, (char*)h->a + (size_t)row0 * H * 2,
+                      h->layers[0].g_attn, h->ssq + (size_t)row0 * h->nt, h->nt, n, H, h->st);
+  } else if (tokens) {
+    launch_embed(h->w.embed, tokens, h->h + (size_t)row0 * H, n, H, edt, h->st);
+  } else {
+    launch_rows_to_f32(embeds, h->h + (size_t)row0 * H, n, H, edt, h->st);
+  }
+  h->launches++;
+  CU(h, cudaGetLastError());
+  return FDVLM_OK;
+}
+
+// ---- exact CUDA-core path: one kernel per operator ---------------------------------------------------
+static int forward_rows_simt(fdvlm_t* h, int n, int mode, int logits_rows) {
+  const fdvlm_config& c = h->cfg;
+  const int H = c.hidden, I = c.intermediate, d = c.head_dim;
+  const int NQ = c.n_q_heads * d, NKV = c.n_kv_heads * d, NQKV = NQ + 2 * NKV;
+  cudaError_t e = cudaSuccess;
+  auto lin = [&](const void* x, const void* w, const float* scale, const float* bias, float* y, int nn, int kk, int ldy,
+                 int accumulate, int m, int dt) -> int {
+    LinearArgs a;
+    a.x = x; a.w = w; a.scale = scale; a.bias = bias; a.y = y; a.m = m; a.n = nn; a.k = kk; a.ldy = ldy;
+    a.accumulate = accumulate; a.dtype = dt; a.workspace = h->ws; a.workspace_bytes = h->ws_bytes;
+    prof_begin(h, 0);
+    int r = launch_linear(a, h->st, &e);
+    prof_end(h);
+    if (r < 0) return -1;
+    h->launches += r;
+    return 0;
+  };
+  const int dt = h->dt;
+  launch_rope_table(h->cs, n, h->cache_len, d, c.rope_theta, h->st);
+  h->launches++;
+  for (int l = 0; l < c.n_layers; ++l) {
+    const fdvlm_layer_weights& lw = h->layers[l];
+    launch_rmsnorm(h->h, lw.g_attn, h->a, n, H, c.rms_eps, dt, h->st);
+    if (lin(h->a, lw.wq, lw.s_q, lw.bq, h->y, NQ, H, NQKV, 0, n, dt) || lin(h->a, lw.wk, lw.s_k, lw.bk, h->y + NQ, NKV, H, NQKV, 0, n, dt) ||
+        lin(h->a, lw.wv, lw.s_v, lw.bv, h->y + NQ + NKV, NKV, H, NQKV, 0, n, dt))
+      return fail(h, FDVLM_ERR_CUDA, "qkv projection launch: %s", cudaGetErrorString(e));
+    launch_qkv_post(h->y, h->cs, h->q, kv_ptr(h, l, 0), kv_ptr(h, l, 1), n, h->cache_len, c.n_q_heads, c.n_kv_heads, d,
+                    c.max_seq, dt, h->st);
+    AttnArgs at;
+    at.q = h->q; at.kc = kv_ptr(h, l, 0); at.vc = kv_ptr(h, l, 1); at.out = h->ao; at.n = n; at.cache_len = h->cache_len;
+    at.max_seq = c.max_seq; at.hq = c.n_q_heads; at.hkv = c.n_kv_heads; at.d = d; at.causal = (mode == MODE_CAUSAL);
+    at.dtype = dt; at.workspace = h->ws;
+    prof_begin(h, 1);
+    int r = launch_attention(at, h->st, &e);
+    prof_end(h);
+    if (r < 0) return fail(h, FDVLM_ERR_CUDA, "attention launch: %s", cudaGetErrorString(e));
+    h->launches += r + 2;
+    if (lin(h->ao, lw.wo, lw.s_o, nullptr, h->h, H, NQ, H, 1, n, dt))
+      return fail(h, FDVLM_ERR_CUDA, "o projection launch: %s", cudaGetErrorString(e));
+    launch_rmsnorm(h->h, lw.g_mlp, h->a, n, H, c.rms_eps, dt, h->st);
+    if (lin(h->a, lw.w_gate, lw.s_gate, nullptr, h->y, I, H, 2 * I, 0, n, dt) || lin(h->a, lw.w_up, lw.s_up, nullptr, h->y + I, I, H, 2 * I, 0, n, dt))
+      return fail(h, FDVLM_ERR_CUDA, "gate/up projection launch: %s", cudaGetErrorString(e));
+    launch_swiglu(h->y, h->act, n, I, dt, h->st);
+    if (lin(h->act, lw.w_down, lw.s_down, nullptr, h->h, H, I, H, 1, n, dt))
+      return fail(h, FDVLM_ERR_CUDA, "down projection launch: %s", cudaGetErrorString(e));
+    h->launches += 2;
+  }
+  if (logits_rows > 0) {
+    const int first = (logits_rows == n) ? 0 : n - 1;
+    const int m = n - first;
+    launch_rmsnorm(h->h + (size_t)first * H, h->w.g_final, h->a, m, H, c.rms_eps, dt, h->st);
+    h->launches++;
+    const void* table = c.tie_embeddings ? h->w.embed : h->w.lm_head;
+    const float* sc = c.tie_embeddings ? nullptr : h->w.s_lm_head;
+    // a tied table is stored in the embedding's type: fp32 for F32, bf16 otherwise (never fp8)
+    const int hdt = (c.tie_embeddings && dt == DT_FP8) ? DT_BF16 : dt;
+    if (lin(h->a, table, sc, nullptr, h->logits, c.vocab, H, c.vocab, 0, m, hdt))
+      return fail(h, FDVLM_ERR_CUDA, "lm head launch: %s", cudaGetErrorString(e));
+    if (logits_rows == n) {
+      launch_row_stats(h->logits, n, c.vocab, c.mask_id, h->conf, h->pred, h->st);
+      h->launches++;
+    }
+  }
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(h, FDVLM_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
+  return FDVLM_OK;
+}
+
+// ---- tensor-core path (bf16 weights) -------------------------------------------------------------------
+// per layer: [QKV GEMM -> split-K partials] [sum + folded norm + bias + rotary + K/V staging] [attention + chunk merge]
+//            [O GEMM -> partials] [sum + residual + gain + ssq] [gate/up GEMM, folded norm + SwiGLU epilogue]
+//            [down GEMM -> partials] [sum + residual + gain + ssq]
+// head:      [LM-head GEMM, folded final norm, logits + softmax statistics epilogue] [statistics merge]
+static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int want_logits) {
+  const fdvlm_config& c = h->cfg;
+  const int H = c.hidden, I = c.intermediate, d = c.head_dim, nt = h->nt;
+  const int NQ = c.n_q_heads * d, NKV = c.n_kv_heads * d, NQKV = NQ + 2 * NKV;
+  float* part = (float*)h->ws;
+  cudaError_t e = cudaSuccess;
+  auto group = [&](const void* x, int m, int k, int nm, const void* w0, int n0, const void* w1, int n1, const void* w2, int n2) {
+    TcGroup g;
+    memset(&g, 0, sizeof(g));
+    g.x = x; g.m = m; g.k = k; g.n_mats = nm;
+    g.w[0] = w0; g.n[0] = n0; g.w[1] = w1; g.n[1] = n1; g.w[2] = w2; g.n[2] = n2;
+    return g;
+  };
+  auto out = [&](int tc_mode) {
+    TcOut o;
+    memset(&o, 0, sizeof(o));
+    o.mode = tc_mode; o.status = h->info + 3; o.part = part; o.part_bytes = h->ws_bytes;
+    return o;
+  };
+  auto gemm = [&](const TcGroup& g, const TcOut& o) {
+    prof_begin(h, 0);
+    e = tc_group_launch(g, o, h->st);
+    prof_end(h);
+    h->launches++;
+    return e == cudaSuccess;
+  };
+  launch_rope_table(h->cs, n, h->cache_len, d, c.rope_theta, h->st);
+  h->launches++;
+  for (int l = 0; l < c.n_layers; ++l) {
+    const fdvlm_layer_weights& lw = h->layers[l];
+    int S = 0;
+    TcOut o = out(TC_MODE_PARTIAL);
+    o.ld = NQKV; o.splits_out = &S;
+    if (!gemm(group(h->a, n, H, 3, lw.wq, NQ, lw.wk, NKV, lw.wv, NKV), o))
+      return fail(h, FDVLM_ERR_CUDA, "qkv projection launch: %s", cudaGetErrorString(e));
+    launch_fin_qkv(part, S, n, h->cs, h->ssq, nt, H, c.rms_eps, lw.bq, lw.bk, lw.bv, h->q, kv_ptr(h, l, 0), kv_ptr(h, l, 1),
+                   h->cache_len, c.n_q_heads, c.n_kv_heads, d, c.max_seq, h->st);
+    AttnArgs at;
+    at.q = h->q; at.kc = kv_ptr(h, l, 0); at.vc = kv_ptr(h, l, 1); at.out = h->ao; at.n = n; at.cache_len = h->cache_len;
+    at.max_seq = c.max_seq; at.hq = c.n_q_heads; at.hkv = c.n_kv_heads; at.d = d; at.causal = (mode == MODE_CAUSAL);
+    at.dtype = h->dt; at.workspace = h->ws;
+    prof_begin(h, 1);
+    int r = launch_attention(at, h->st, &e);
+    prof_end(h);
+    if (r < 0) return fail(h, FDVLM_ERR_CUDA, "attention launch: %s", cudaGetErrorString(e));
+    h->launches += r + 1;
+    o = out(TC_MODE_PARTIAL);
+    o.ld = H; o.splits_out = &S;
+    if (!gemm(group(h->ao, n, NQ, 1, lw.wo, H, nullptr, 0, nullptr, 0), o))
+      return fail(h, FDVLM_ERR_CUDA, "o projection launch: %s", cudaGetErrorString(e));
+    launch_fin_resid(part, S, n, H, h->h, lw.g_mlp, h->a, h->ssq, nt, h->st);
+    o = out(TC_MODE_SWIGLU);
+    o.act = h->act; o.ssq_in = h->ssq; o.nt_in = nt; o.hidden = H; o.eps = c.rms_eps;
+    if (!gemm(group(h->a, n, H, 2, lw.w_gate, I, lw.w_up, I, nullptr, 0), o))
+      return fail(h, FDVLM_ERR_CUDA, "gate/up projection launch: %s", cudaGetErrorString(e));
+    o = out(TC_MODE_PARTIAL);
+    o.ld = H; o.splits_out = &S;
+    if (!gemm(group(h->act, n, I, 1, lw.w_down, H, nullptr, 0, nullptr, 0), o))
+      return fail(h, FDVLM_ERR_CUDA, "down projection launch: %s", cudaGetErrorString(e));
+    const float* g_next = (l + 1 < c.n_layers) ? h->layers[l + 1].g_attn : h->w.g_final;
+    launch_fin_resid(part, S, n, H, h->h, g_next, h->a, h->ssq, nt, h->st);
+    h->launches += 2;
+  }
+  if (logits_rows > 0) {
+    const int first = (logits_rows == n) ? 0 : n - 1;
+    const int m = n - first;
+    const void* table = c.tie_embeddings ? h->w.embed : h->w.lm_head;
+    TcOut o = out(TC_MODE_LOGITS);
+    o.y = h->logits; o.ld = c.vocab; o.write_logits = (logits_rows == n) ? want_logits : 1;
+    o.ssq_in = h->ssq + (size_t)first * nt; o.nt_in = nt; o.hidden = H; o.eps = c.rms_eps;
+    o.stats = h->stats; o.mask_id = c.mask_id;
+    if (!gemm(group((const char*)h->a + (size_t)first * H * 2, m, H, 1, table, c.vocab, nullptr, 0, nullptr, 0), o))
+      return fail(h, FDVLM_ERR_CUDA, "lm head launch: %s", cudaGetErrorString(e));
+    if (logits_rows == n) {
+      launch_stats_merge(h->stats, ceil_div(c.vocab, 128) * 4, n, h->conf, h->pred, h->st);
+      h->launches++;
+    }
+  }
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(h, FDVLM_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
+  return FDVLM_OK;
+}
+
+int forward_rows(fdvlm_t* h, int n, int mode, int logits_rows, int want_logits) {
+  return h->use_tc ? forward_rows_tc(h, n, mode, logits_rows, want_logits) : forward_rows_simt(h, n, mode, logits_rows);
+}
+
+}  // namespace fdk

@@ -44,6 +44,15 @@ struct TcParams {
   int ldy, accumulate;
   bf16* act;            // [m][inter]           (SWIGLU)
   int inter;
+  // RMSNorm folded into the consumer: x holds bf16(h * gain); the per-row factor rsqrt(mean(h^2) + eps)
+  // is applied to the accumulators.  ssq_in[row][nt_in] holds partial sums of h^2 (null: factor 1).
+  const float* ssq_in;
+  int nt_in;
+  float inv_h, eps;
+  // LOGITS mode: per (tile, lane quarter, row) softmax statistics of the 32 columns a warp holds, the
+  // mask token's column excluded: (max, sum exp(l - max), argmax column)
+  float4* stats;        // [tiles * 4][m]
+  int mask_id, write_logits;
   int* status;          // device word, set non-zero when a wait timed out
 };
 
@@ -263,6 +272,20 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_con
     const int q = warp & 3;  // TMEM lane quarter this warp may read
     int local = 0;
     bool ok = true;
+    // folded RMSNorm: lane l keeps the factor of rows l and l + 32; broadcast by shuffle where needed
+    float rs0 = 1.f, rs1 = 1.f;
+    if (p.ssq_in) {
+      if (lane < p.m) {
+        float s = 0.f;
+        for (int t = 0; t < p.nt_in; ++t) s += p.ssq_in[(size_t)lane * p.nt_in + t];
+        rs0 = rsqrtf(s * p.inv_h + p.eps);
+      }
+      if (lane + 32 < p.m) {
+        float s = 0.f;
+        for (int t = 0; t < p.nt_in; ++t) s += p.ssq_in[(size_t)(lane + 32) * p.nt_in + t];
+        rs1 = rsqrtf(s * p.inv_h + p.eps);
+      }
+    }
     for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++local) {
       const int tile = it % total_tiles, split = it / total_tiles;
       const int acc = local & 1;
@@ -286,33 +309,59 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_con
 #pragma unroll
         for (int b = 0; b < M_PAD; ++b) {
           const float other = __shfl_xor_sync(0xffffffffu, v[b], 16);   // lanes 0..15: the matching "up" value
+          const float rs = __shfl_sync(0xffffffffu, (b < 32) ? rs0 : rs1, b & 31);
           if (live && b < p.m) {
-            const float g = v[b] * sg;
-            p.act[(size_t)b * p.inter + col] = __float2bfloat16_rn(g / (1.f + __expf(-g)) * (other * su));
+            const float g = v[b] * sg * rs;
+            p.act[(size_t)b * p.inter + col] = __float2bfloat16_rn(g / (1.f + __expf(-g)) * (other * su * rs));
           }
+        }
+      } else if (p.mode == TC_MODE_LOGITS) {
+        const int n = tile * TC_BM + q * 32 + lane;          // vocabulary id held by this lane
+        const bool in_range = n < p.n_out[0];
+        const bool counted = in_range && n != p.mask_id;
+        const float sc = (in_range && p.scale[0]) ? p.scale[0][n] : 1.f;
+#pragma unroll
+        for (int b = 0; b < M_PAD; ++b) {
+          if (b >= p.m) break;                                // uniform across the warp
+          const float rs = __shfl_sync(0xffffffffu, (b < 32) ? rs0 : rs1, b & 31);
+          const float l = v[b] * sc * rs;
+          if (p.write_logits && in_range) p.y[(size_t)b * p.ldy + n] = l;
+          float mx = counted ? l : -INFINITY;
+          int ix = counted ? n : 0x7fffffff;
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            const float omx = __shfl_xor_sync(0xffffffffu, mx, o);
+            const int oix = __shfl_xor_sync(0xffffffffu, ix, o);
+            if (omx > mx || (omx == mx && oix < ix)) { mx = omx; ix = oix; }
+          }
+          float e = (counted && mx > -INFINITY) ? __expf(l - mx) : 0.f;
+          e = warp_sum(e);
+          if (lane == 0) p.stats[(size_t)(tile * 4 + q) * p.m + b] = make_float4(mx, e, __int_as_float(ix), 0.f);
         }
       } else {
         int mi = 0;
         while (mi + 1 < p.n_mats && tile >= p.tile_begin[mi + 1]) ++mi;
         const int n = (tile - p.tile_begin[mi]) * TC_BM + q * 32 + lane;
-        if (n < p.n_out[mi]) {
-          const int col = p.out_col[mi] + n;
-          if (p.mode == TC_MODE_PARTIAL) {
+        const bool in_range = n < p.n_out[mi];
+        const int col = p.out_col[mi] + n;
+        if (p.mode == TC_MODE_PARTIAL) {
+          if (in_range) {
             float* dst = p.part + (size_t)split * p.m * p.ldp + col;
 #pragma unroll
             for (int b = 0; b < M_PAD; ++b)
               if (b < p.m) dst[(size_t)b * p.ldp] = v[b];
-          } else {
-            const float sc = p.scale[mi] ? p.scale[mi][n] : 1.f;
-            const float bi = p.bias[mi] ? p.bias[mi][n] : 0.f;
-            float* dst = p.y + col;
+          }
+        } else {
+          const float sc = (in_range && p.scale[mi]) ? p.scale[mi][n] : 1.f;
+          const float bi = (in_range && p.bias[mi]) ? p.bias[mi][n] : 0.f;
 #pragma unroll
-            for (int b = 0; b < M_PAD; ++b) {
-              if (b < p.m) {
-                float r = v[b] * sc + bi;
-                if (p.accumulate) r += dst[(size_t)b * p.ldy];
-                dst[(size_t)b * p.ldy] = r;
-              }
+          for (int b = 0; b < M_PAD; ++b) {
+            const float rs = __shfl_sync(0xffffffffu, (b < 32) ? rs0 : rs1, b & 31);
+            if (in_range && b < p.m) {
+              float* dst = p.y + (size_t)b * p.ldy + col;
+              float r = v[b] * sc * rs + bi;
+              if (p.accumulate) r += *dst;
+              *dst = r;
             }
           }
         }
@@ -438,10 +487,10 @@ static cudaError_t tc_launch(const TcParams& p, cudaStream_t st) {
 //   mode DIRECT : y[m][ld] = x w^T * scale + bias (+ y)   (forces one split)
 //   mode SWIGLU : act[m][inter] = silu(x wg^T * sg) * (x wu^T * su)  (w[0] = gate, w[1] = up; one split)
 
-cudaError_t tc_group_launch(const TcGroup& g, int mode, float* part, size_t part_bytes, int* splits_out, float* y, int ld,
-                            int accumulate, void* act, int* status, cudaStream_t st) {
+cudaError_t tc_group_launch(const TcGroup& g, const TcOut& o, cudaStream_t st) {
   TcParams p;
   memset(&p, 0, sizeof(p));
+  const int mode = o.mode;
   const int mp = pad_m(g.m);
   if (!make_tmap(&p.tm_x, g.x, g.m, g.k, mp)) return cudaErrorInvalidValue;
   int tiles = 0, col = 0;
@@ -459,21 +508,24 @@ cudaError_t tc_group_launch(const TcGroup& g, int mode, float* part, size_t part
   p.kblocks = ceil_div(g.k, TC_BK);
   p.m = g.m;
   p.mode = mode;
-  p.status = status;
+  p.status = o.status;
+  p.ssq_in = o.ssq_in; p.nt_in = o.nt_in; p.inv_h = o.hidden > 0 ? 1.f / (float)o.hidden : 0.f; p.eps = o.eps;
   if (mode == TC_MODE_SWIGLU) {
     tiles = ceil_div(g.n[0], 64);      // one combined list of 64-feature tiles (gate + up rows interleaved)
     p.n_mats = 1;
     p.tile_begin[0] = 0; p.tile_begin[1] = tiles;
     p.splits = 1; p.kb_per_split = p.kblocks;
-    p.act = (bf16*)act; p.inter = g.n[0];
+    p.act = (bf16*)o.act; p.inter = g.n[0];
   } else {
     p.tile_begin[g.n_mats] = tiles;
-    if (mode == TC_MODE_DIRECT) { p.splits = 1; p.kb_per_split = p.kblocks; }
-    else tc_plan(tiles, p.kblocks, &p.splits, &p.kb_per_split);
-    p.part = part; p.ldp = ld; p.y = y; p.ldy = ld; p.accumulate = accumulate;
-    if (mode == TC_MODE_PARTIAL && (size_t)p.splits * g.m * ld * sizeof(float) > part_bytes) return cudaErrorInvalidValue;
+    if (mode == TC_MODE_PARTIAL) tc_plan(tiles, p.kblocks, &p.splits, &p.kb_per_split);
+    else { p.splits = 1; p.kb_per_split = p.kblocks; }
+    p.part = o.part; p.ldp = o.ld; p.y = o.y; p.ldy = o.ld; p.accumulate = o.accumulate;
+    p.stats = (float4*)o.stats; p.mask_id = o.mask_id; p.write_logits = o.write_logits;
+    if (mode == TC_MODE_PARTIAL && (size_t)p.splits * g.m * o.ld * sizeof(float) > o.part_bytes) return cudaErrorInvalidValue;
+    if (mode == TC_MODE_LOGITS && (g.n_mats != 1 || !o.stats)) return cudaErrorInvalidValue;
   }
-  if (splits_out) *splits_out = p.splits;
+  if (o.splits_out) *o.splits_out = p.splits;
   return tc_launch(p, st);
 }
 

@@ -272,80 +272,147 @@ void launch_qkv_post(const float* qkv, const float* cs, void* q, void* kc, void*
 }
 
 // ================================================================================================
-// Fused split-K reductions of the tensor-core path (fixed summation order => deterministic).
+// Glue of the tensor-core path (bf16).  RMSNorm is folded into its consumer GEMM: producers leave
+// xg = bf16(h * gain) and per-128-column partial sums of h^2 (ssq[row][nt]); the consumer's epilogue
+// multiplies by rsqrt(sum(ssq) / hidden + eps).  All sums run in a fixed order => deterministic.
 // ================================================================================================
-// part[S][m][(hq + 2 hkv) d] -> sum over S, * scale, + bias, rotary on q and k, q to its buffer, k and v
-// straight into the layer's cache planes at positions pos0 + row.
-template <typename AT>
-__global__ void qkv_reduce_rope_kernel(const float* __restrict__ part, int S, int m, const float2* __restrict__ cs,
-                                       const float* __restrict__ sq, const float* __restrict__ sk,
-                                       const float* __restrict__ sv, const float* __restrict__ bq,
-                                       const float* __restrict__ bk, const float* __restrict__ bv, AT* __restrict__ q,
-                                       AT* __restrict__ kc, AT* __restrict__ vc, int pos0, int hq, int hkv, int d,
-                                       int max_seq) {
-  const int r = blockIdx.x, half = d >> 1;
-  const int nq = hq * d, nkv = hkv * d, width = nq + 2 * nkv;
-  const size_t sstride = (size_t)m * width;
-  const float* row = part + (size_t)r * width;
-  auto val = [&](int col) {
-    float s = 0.f;
-    for (int i = 0; i < S; ++i) s += row[i * sstride + col];
-    if (col < nq) { if (sq) s *= sq[col]; if (bq) s += bq[col]; }
-    else if (col < nq + nkv) { int c = col - nq; if (sk) s *= sk[c]; if (bk) s += bk[c]; }
-    else { int c = col - nq - nkv; if (sv) s *= sv[c]; if (bv) s += bv[c]; }
-    return s;
-  };
-  const int pairs = (hq + hkv) * half;
-  for (int t = threadIdx.x; t < pairs; t += blockDim.x) {
-    const int head = t / half, j = t % half;
-    const float2 c = cs[r * half + j];
-    const float a = val(head * d + j), b = val(head * d + j + half);
-    const float ra = a * c.x - b * c.y, rb = b * c.x + a * c.y;
-    AT* o = head < hq ? q + ((size_t)r * hq + head) * d : kc + ((size_t)(head - hq) * max_seq + pos0 + r) * d;
-    o[j] = from_f32<AT>(ra);
-    o[j + half] = from_f32<AT>(rb);
-  }
-  for (int t = threadIdx.x; t < nkv; t += blockDim.x) {
-    const int head = t / d, j = t % d;
-    vc[((size_t)head * max_seq + pos0 + r) * d + j] = from_f32<AT>(val(nq + nkv + t));
-  }
-}
-void launch_qkv_reduce_rope(const float* part, int S, int m, const float* cs, const float* sq, const float* sk,
-                            const float* sv, const float* bq, const float* bk, const float* bv, void* q, void* kc, void* vc,
-                            int pos0, int hq, int hkv, int d, int max_seq, cudaStream_t st) {
-  qkv_reduce_rope_kernel<bf16><<<m, 256, 0, st>>>(part, S, m, (const float2*)cs, sq, sk, sv, bq, bk, bv, (bf16*)q,
-                                                  (bf16*)kc, (bf16*)vc, pos0, hq, hkv, d, max_seq);
-}
-
-// h[r] += (sum_s part[s][r]) * scale (S may be 0: nothing added); out[r] = RMSNorm(h[r]; g) in the activation type.
-template <typename AT>
-__global__ void reduce_residual_rmsnorm_kernel(const float* __restrict__ part, int S, int m, int H,
-                                               const float* __restrict__ scale, float* __restrict__ h,
-                                               const float* __restrict__ g, AT* __restrict__ out, float eps) {
+__global__ void embed_prep_kernel(const bf16* __restrict__ table, const int32_t* __restrict__ tokens,
+                                  const bf16* __restrict__ rows, float* __restrict__ h, bf16* __restrict__ xg,
+                                  const float* __restrict__ g, float* __restrict__ ssq, int nt, int hidden) {
   __shared__ float red[32];
   const int r = blockIdx.x;
-  const size_t sstride = (size_t)m * H;
-  float* hr = h + (size_t)r * H;
+  const bf16* src = tokens ? table + (size_t)tokens[r] * hidden : rows + (size_t)r * hidden;
   float ss = 0.f;
-  for (int c = threadIdx.x; c < H; c += blockDim.x) {
-    float v = hr[c];
-    if (S > 0) {
-      float s = 0.f;
-      for (int i = 0; i < S; ++i) s += part[i * sstride + (size_t)r * H + c];
-      if (scale) s *= scale[c];
-      v += s;
-      hr[c] = v;
-    }
+  for (int c = threadIdx.x; c < hidden; c += blockDim.x) {
+    const float v = __bfloat162float(src[c]);
+    h[(size_t)r * hidden + c] = v;
+    xg[(size_t)r * hidden + c] = __float2bfloat16_rn(v * g[c]);
     ss = fmaf(v, v, ss);
   }
   ss = block_sum(ss, red);
-  const float rs = rsqrtf(ss / (float)H + eps);
-  AT* o = out + (size_t)r * H;
-  for (int c = threadIdx.x; c < H; c += blockDim.x) o[c] = from_f32<AT>(hr[c] * rs * g[c]);
+  for (int t = threadIdx.x; t < nt; t += blockDim.x) ssq[(size_t)r * nt + t] = (t == 0) ? ss : 0.f;
 }
-void launch_reduce_residual_rmsnorm(const float* part, int S, int m, int H, const float* scale, float* h, const float* g,
-                                    void* out, float eps, cudaStream_t st) {
-  reduce_residual_rmsnorm_kernel<bf16><<<m, 256, 0, st>>>(part, S, m, H, scale, h, g, (bf16*)out, eps);
+void launch_embed_prep(const void* table, const int32_t* tokens, const void* rows, float* h, void* xg, const float* g,
+                       float* ssq, int nt, int n, int hidden, cudaStream_t st) {
+  embed_prep_kernel<<<n, 256, 0, st>>>((const bf16*)table, tokens, (const bf16*)rows, h, (bf16*)xg, g, ssq, nt, hidden);
+}
+
+// QKV finalisation: sum the split-K partials, apply the folded norm factor and the bias, rotate q and k
+// (rotate-half pairs j, j + d/2), write q to its buffer and k, v into the layer's cache planes.
+// grid (hq + 2 hkv heads, m rows), d/2 threads: thread j owns the pair (j, j + d/2) of one head.
+__global__ void fin_qkv_kernel(const float* __restrict__ part, int S, int m, const float2* __restrict__ cs,
+                               const float* __restrict__ ssq, int nt, float inv_h, float eps,
+                               const float* __restrict__ bq, const float* __restrict__ bk, const float* __restrict__ bv,
+                               bf16* __restrict__ q, bf16* __restrict__ kc, bf16* __restrict__ vc, int pos0, int hq, int hkv,
+                               int d, int max_seq) {
+  __shared__ float s_rstd;
+  const int head = blockIdx.x, r = blockIdx.y, j = threadIdx.x, half = d >> 1;
+  if (threadIdx.x < 32) {
+    float s = 0.f;
+    for (int t = threadIdx.x; t < nt; t += 32) s += ssq[(size_t)r * nt + t];
+    // fixed order: lanes hold disjoint strided subsets, combined by the butterfly below
+    s = warp_sum(s);
+    if (threadIdx.x == 0) s_rstd = rsqrtf(s * inv_h + eps);
+  }
+  __syncthreads();
+  const float rstd = s_rstd;
+  const int width = (hq + 2 * hkv) * d;
+  const size_t sstride = (size_t)m * width;
+  const float* pa = part + (size_t)r * width + head * d + j;
+  float a = 0.f, b = 0.f;
+  for (int i = 0; i < S; ++i) { a += pa[i * sstride]; b += pa[i * sstride + half]; }
+  a *= rstd; b *= rstd;
+  if (head < hq) {
+    if (bq) { a += bq[head * d + j]; b += bq[head * d + j + half]; }
+    const float2 c = cs[r * half + j];
+    bf16* o = q + ((size_t)r * hq + head) * d;
+    o[j] = __float2bfloat16_rn(a * c.x - b * c.y);
+    o[j + half] = __float2bfloat16_rn(b * c.x + a * c.y);
+  } else if (head < hq + hkv) {
+    const int hk = head - hq;
+    if (bk) { a += bk[hk * d + j]; b += bk[hk * d + j + half]; }
+    const float2 c = cs[r * half + j];
+    bf16* o = kc + ((size_t)hk * max_seq + pos0 + r) * d;
+    o[j] = __float2bfloat16_rn(a * c.x - b * c.y);
+    o[j + half] = __float2bfloat16_rn(b * c.x + a * c.y);
+  } else {
+    const int hk = head - hq - hkv;
+    if (bv) { a += bv[hk * d + j]; b += bv[hk * d + j + half]; }
+    bf16* o = vc + ((size_t)hk * max_seq + pos0 + r) * d;
+    o[j] = __float2bfloat16_rn(a);
+    o[j + half] = __float2bfloat16_rn(b);
+  }
+}
+void launch_fin_qkv(const float* part, int S, int m, const float* cs, const float* ssq, int nt, int hidden, float eps,
+                    const float* bq, const float* bk, const float* bv, void* q, void* kc, void* vc, int pos0, int hq,
+                    int hkv, int d, int max_seq, cudaStream_t st) {
+  fin_qkv_kernel<<<dim3(hq + 2 * hkv, m), d / 2, 0, st>>>(part, S, m, (const float2*)cs, ssq, nt, 1.f / (float)hidden, eps, bq, bk,
+                                                          bv, (bf16*)q, (bf16*)kc, (bf16*)vc, pos0, hq, hkv, d, max_seq);
+}
+
+// Residual finalisation: h += sum of split-K partials; xg = bf16(h * gain of the next norm); ssq[row][tile] =
+// sum of h^2 over the tile's 128 columns.  grid (nt tiles, m rows), 128 threads.
+__global__ void __launch_bounds__(128) fin_resid_kernel(const float* __restrict__ part, int S, int m, int hidden,
+                                                        float* __restrict__ h, const float* __restrict__ g,
+                                                        bf16* __restrict__ xg, float* __restrict__ ssq, int nt) {
+  __shared__ float red[32];
+  const int t = blockIdx.x, r = blockIdx.y, c = t * 128 + threadIdx.x;
+  float v = 0.f;
+  if (c < hidden) {
+    const size_t idx = (size_t)r * hidden + c, sstride = (size_t)m * hidden;
+    float s = 0.f;
+    for (int i = 0; i < S; ++i) s += part[i * sstride + idx];
+    v = h[idx] + s;
+    h[idx] = v;
+    xg[idx] = __float2bfloat16_rn(v * g[c]);
+  }
+  const float ss = block_sum(v * v, red);
+  if (threadIdx.x == 0) ssq[(size_t)r * nt + t] = ss;
+}
+void launch_fin_resid(const float* part, int S, int m, int hidden, float* h, const float* g, void* xg, float* ssq, int nt,
+                      cudaStream_t st) {
+  fin_resid_kernel<<<dim3(nt, m), 128, 0, st>>>(part, S, m, hidden, h, g, (bf16*)xg, ssq, nt);
+}
+
+// Merge the per-warp softmax statistics of the LM-head epilogue into confidence and prediction per row.
+// stats[e * m + row] = (max, sum exp(l - max), argmax id) for e in [0, n_part).  grid m rows, 256 threads.
+__global__ void __launch_bounds__(256) stats_merge_kernel(const float4* __restrict__ stats, int n_part, int m,
+                                                          float* __restrict__ conf, int32_t* __restrict__ pred) {
+  __shared__ float sm_m[8], sm_s[8];
+  __shared__ int sm_i[8];
+  const int r = blockIdx.x;
+  float mx = -INFINITY, s = 0.f;
+  int ix = 0x7fffffff;
+  auto merge = [&](float m2, float s2, int i2) {
+    if (s2 == 0.f) return;
+    if (s == 0.f) { mx = m2; s = s2; ix = i2; return; }
+    const float mn = fmaxf(mx, m2);
+    s = s * __expf(mx - mn) + s2 * __expf(m2 - mn);
+    if (m2 > mx || (m2 == mx && i2 < ix)) ix = i2;
+    mx = mn;
+  };
+  for (int e = threadIdx.x; e < n_part; e += blockDim.x) {
+    const float4 v = stats[(size_t)e * m + r];
+    merge(v.x, v.y, __float_as_int(v.z));
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float m2 = __shfl_xor_sync(0xffffffffu, mx, o), s2 = __shfl_xor_sync(0xffffffffu, s, o);
+    const int i2 = __shfl_xor_sync(0xffffffffu, ix, o);
+    merge(m2, s2, i2);
+  }
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  if (lane == 0) { sm_m[w] = mx; sm_s[w] = s; sm_i[w] = ix; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    mx = sm_m[0]; s = sm_s[0]; ix = sm_i[0];
+    for (int k = 1; k < 8; ++k) merge(sm_m[k], sm_s[k], sm_i[k]);
+    conf[r] = 1.f / s;
+    pred[r] = ix;
+  }
+}
+void launch_stats_merge(const void* stats, int n_part, int m, float* conf, int32_t* pred, cudaStream_t st) {
+  stats_merge_kernel<<<m, 256, 0, st>>>((const float4*)stats, n_part, m, conf, pred);
 }
 
 // ================================================================================================

@@ -41,27 +41,43 @@ void launch_init_block(int32_t* tokens, uint8_t* masked, int32_t* info, const in
                        int step, cudaStream_t st);
 
 // ---- tensor-core (tcgen05 + TMA) small-M GEMM, bf16 ---------------------------------------------------
-enum { TC_MODE_PARTIAL = 0, TC_MODE_DIRECT = 1, TC_MODE_SWIGLU = 2 };
+enum { TC_MODE_PARTIAL = 0, TC_MODE_DIRECT = 1, TC_MODE_SWIGLU = 2, TC_MODE_LOGITS = 3 };
 // Up to three bf16 matrices that share x and K; their outputs sit side by side in one row of width ld.
 struct TcGroup {
   const void* x; int m, k;
   const void* w[3]; int n[3]; int n_mats;
   const float* scale[3]; const float* bias[3];
 };
+// What the GEMM leaves behind.
+//   PARTIAL: part[split][m][ld] = split-K partial sums (*splits_out of them) for the caller's reduce kernel
+//   DIRECT : y[m][ld] = (x w^T) * rstd[row] * scale + bias (+ y when accumulate)
+//   SWIGLU : act[m][n0] = silu(x w0^T * rstd * s0) * (x w1^T * rstd * s1)   (w[0] = gate, w[1] = up)
+//   LOGITS : y (when write_logits) as DIRECT, and stats[tile * 4 + quarter][m] = (max, sum exp(l - max), argmax id)
+//            over the 32 vocabulary ids a warp holds, mask_id excluded
+// rstd[row] = rsqrt(sum_t ssq_in[row][t] / hidden + eps) when ssq_in is set (RMSNorm folded into the consumer), else 1.
+struct TcOut {
+  int mode;
+  float* part; size_t part_bytes; int* splits_out;
+  float* y; int ld; int accumulate;
+  void* act;
+  const float* ssq_in; int nt_in; int hidden; float eps;
+  void* stats; int mask_id; int write_logits;
+  int* status;   // device word set non-zero if a bounded wait inside the kernel gave up
+};
 bool tc_linear_supported(int m, int n, int k, int dtype);
 // Split-K workspace of a group with m rows, output width ld, `tiles` 128-row weight tiles and depth k.
 size_t tc_workspace_bytes(int m, int ld, int tiles, int k);
-//   PARTIAL: part[split][m][ld] holds the split-K partial sums (*splits_out of them), summed by the caller's
-//            reduce kernel;  DIRECT: y[m][ld] = x w^T * scale + bias (+ y when accumulate);
-//   SWIGLU : act[m][n0] = silu(x w0^T * s0) * (x w1^T * s1)  (w[0] = gate, w[1] = up)
-// status: device word set non-zero if a bounded wait inside the kernel gave up.
-cudaError_t tc_group_launch(const TcGroup& g, int mode, float* part, size_t part_bytes, int* splits_out, float* y, int ld,
-                            int accumulate, void* act, int* status, cudaStream_t st);
-void launch_qkv_reduce_rope(const float* part, int S, int m, const float* cs, const float* sq, const float* sk,
-                            const float* sv, const float* bq, const float* bk, const float* bv, void* q, void* kc, void* vc,
-                            int pos0, int hq, int hkv, int d, int max_seq, cudaStream_t st);
-void launch_reduce_residual_rmsnorm(const float* part, int S, int m, int H, const float* scale, float* h, const float* g,
-                                    void* out, float eps, cudaStream_t st);
+cudaError_t tc_group_launch(const TcGroup& g, const TcOut& o, cudaStream_t st);
+
+// Tensor-core path glue (bf16).  ssq[row][nt] holds per-128-column partial sums of h^2.
+void launch_embed_prep(const void* table, const int32_t* tokens, const void* rows, float* h, void* xg, const float* g,
+                       float* ssq, int nt, int n, int hidden, cudaStream_t st);
+void launch_fin_qkv(const float* part, int S, int m, const float* cs, const float* ssq, int nt, int hidden, float eps,
+                    const float* bq, const float* bk, const float* bv, void* q, void* kc, void* vc, int pos0, int hq,
+                    int hkv, int d, int max_seq, cudaStream_t st);
+void launch_fin_resid(const float* part, int S, int m, int hidden, float* h, const float* g, void* xg, float* ssq, int nt,
+                      cudaStream_t st);
+void launch_stats_merge(const void* stats, int n_part, int m, float* conf, int32_t* pred, cudaStream_t st);
 
 // ---- attention -----------------------------------------------------------------------------------
 struct AttnArgs {
