@@ -179,6 +179,25 @@ int fdvlm_op_linear(const void *x, const void *w, const float *scale, const floa
                     int m, int n, int k, fdvlm_dtype dtype, void *workspace, void *cuda_stream);
 size_t fdvlm_op_linear_workspace_bytes(int m, int n, int k, fdvlm_dtype dtype);
 
+/* (No counterpart in the paper: an integration convenience of this library.)
+ * The same projection as fdvlm_op_linear for callers that cannot allocate device memory -- code running
+ * under a framework allocator it must not bypass, inside a memory-budgeted plugin, or in a context where
+ * cudaMalloc's implicit device synchronisation is not acceptable.  The split-K scratch that
+ * fdvlm_op_linear takes as `workspace` is instead a fixed array of FDVLM_STATIC_SCRATCH_BYTES bytes
+ * built into the library's device image; every GPU that loads the library holds it until the process
+ * exits.  The call allocates nothing (no cudaMalloc / cudaFree, no allocating library routine).
+ *   - Shapes whose scratch need (see fdvlm_op_linear_workspace_bytes) exceeds the array less its first
+ *     256 bytes are refused with FDVLM_ERR_CAPACITY; the message (fdvlm_last_error(NULL)) names both sizes.
+ *   - The first call on each device looks up the array's device address (with that device current);
+ *     make that first call before any stream capture.
+ *   - All calls on one device share the array: two calls whose kernels may overlap on the GPU (different
+ *     streams, no ordering between them) race on it.  Calls on one stream are safe back to back.
+ * Arguments, layouts and results are those of fdvlm_op_linear; x, w, scale, bias, y are device pointers
+ * owned by the caller.  Errors also set the message returned by fdvlm_last_error(NULL). */
+#define FDVLM_STATIC_SCRATCH_BYTES (8u << 20)
+int fdvlm_op_linear_static(const void *x, const void *w, const float *scale, const float *bias, float *y,
+                           int m, int n, int k, fdvlm_dtype dtype, void *cuda_stream);
+
 /* Block-masked GQA attention of n_rows new rows at positions cache_len .. cache_len + n_rows - 1
  * (Sec. 3.3 masks; Alg. 1 draft / verify).  q: device [n_rows, n_q_heads, head_dim] (post-rotary);
  * k_cache / v_cache: device [n_kv_heads, max_seq, head_dim] holding cache_len committed positions

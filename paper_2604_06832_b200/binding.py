@@ -75,6 +75,8 @@ EXPORTS = {
                                      C.POINTER(C.c_int)]),
     "fdvlm_op_linear": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
                                   C.c_int, C.c_void_p, C.c_void_p]),
+    "fdvlm_op_linear_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int,
+                                         C.c_int, C.c_void_p]),
     "fdvlm_op_linear_workspace_bytes": (C.c_size_t, [C.c_int, C.c_int, C.c_int, C.c_int]),
     "fdvlm_op_attention": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int,
                                      C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p]),
@@ -225,6 +227,20 @@ def op_linear(x: torch.Tensor, w: torch.Tensor, scale=None, bias=None, dtype: in
                                _stream_ptr(stream))
     if rc != FDVLM_OK:
         raise FdvlmError(rc, "fdvlm_op_linear")
+    return y
+
+
+def op_linear_static(x: torch.Tensor, w: torch.Tensor, scale=None, bias=None, dtype: int = DT_BF16,
+                     stream: Optional[torch.cuda.Stream] = None, y: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """`fdvlm_op_linear_static`: same result as `op_linear`, scratch taken from the library's built-in device
+    array, so the call itself allocates nothing (pass `y` to keep this wrapper from allocating the output)."""
+    m, k = x.shape
+    n = w.shape[0]
+    if y is None:
+        y = torch.empty(m, n, dtype=torch.float32, device=x.device)
+    rc = lib().fdvlm_op_linear_static(_ptr(x), _ptr(w), _ptr(scale), _ptr(bias), _ptr(y), m, n, k, dtype, _stream_ptr(stream))
+    if rc != FDVLM_OK:
+        raise FdvlmError(rc, lib().fdvlm_last_error(None).decode())
     return y
 
 
