@@ -7,203 +7,19 @@
 // each CTA leaves an unnormalised partial (O, running max, running sum) and a small second kernel
 // merges the chunks.  The in-block mask is applied by key index: denoise rows see all L + n keys,
 // commit / prefill rows see keys <= L + i.
-#include "common.cuh"
+#include "attn_core.cuh"
 #include "kernels.h"
 
 namespace fdk {
-
-constexpr int AT_ROWS = 64;    // query rows per CTA (4 warps x 16)
-constexpr int AT_KEYS = 64;    // keys per shared-memory tile
-constexpr float LOG2E = 1.4426950408889634f;
-
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
-__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
-}
-__device__ __forceinline__ void mma_bf16(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
-               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&v);
-}
-
-// byte offset of 16-byte chunk `chunk` of row `row` in a swizzled [rows][D] bf16 tile
-template <int D>
-__device__ __forceinline__ uint32_t swz(int row, int chunk) {
-  return (uint32_t)(row * (D * 2) + ((chunk ^ (row & 7)) << 4));
-}
 
 template <int D>
 __global__ void __launch_bounds__(128) attn_mma_kernel(const bf16* __restrict__ q, const bf16* __restrict__ kc,
                                                        const bf16* __restrict__ vc, float* __restrict__ part_o,
                                                        float2* __restrict__ part_ml, int n, int L, int max_seq, int hq,
                                                        int hkv, int qh, int chunk_keys, int n_chunks, int causal) {
-  constexpr int CH = D / 8;                 // 16-byte chunks per row
-  constexpr int TILE_BYTES = AT_KEYS * D * 2;
   extern __shared__ __align__(128) uint8_t smem[];
-  const uint32_t sQ = (uint32_t)__cvta_generic_to_shared(smem);
-  const uint32_t sK = sQ + AT_ROWS * D * 2;            // 2 buffers
-  const uint32_t sV = sK + 2 * TILE_BYTES;             // 2 buffers
-  const int chunk = blockIdx.x, grp = blockIdx.y, hk = blockIdx.z;
-  const int G = hq / hkv;
-  const int head0 = hk * G + grp * qh;                 // first query head of this CTA
-  const int heads_here = min(qh, G - grp * qh);
-  const int m_valid = heads_here * n;
-  const int T = L + n;
-  const int key_begin = chunk * chunk_keys;
-  const int key_end = min(T, key_begin + chunk_keys);
-  const int n_tiles = (key_end - key_begin + AT_KEYS - 1) / AT_KEYS;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const bf16* kbase = kc + (size_t)hk * max_seq * D;
-  const bf16* vbase = vc + (size_t)hk * max_seq * D;
-
-  // ---- stage Q (rows = heads_here x n; row r -> head r / n, token r % n) ----
-  for (int v = tid; v < AT_ROWS * CH; v += 128) {
-    const int r = v / CH, c = v % CH;
-    const bool ok = r < m_valid;
-    const int hl = ok ? r / n : 0, i = ok ? r % n : 0;
-    const bf16* src = q + ((size_t)i * hq + head0 + hl) * D + c * 8;
-    cp_async16(sQ + swz<D>(r, c), src, ok ? 16 : 0);
-  }
-  auto load_tile = [&](int t, int buf) {
-    const int j0 = key_begin + t * AT_KEYS;
-    for (int v = tid; v < AT_KEYS * CH; v += 128) {
-      const int r = v / CH, c = v % CH;
-      const int j = j0 + r;
-      const bool ok = j < key_end;
-      const size_t off = (size_t)(ok ? j : 0) * D + c * 8;
-      cp_async16(sK + buf * TILE_BYTES + swz<D>(r, c), kbase + off, ok ? 16 : 0);
-      cp_async16(sV + buf * TILE_BYTES + swz<D>(r, c), vbase + off, ok ? 16 : 0);
-    }
-  };
-  if (n_tiles > 0) load_tile(0, 0);
-  cp_async_commit();
-
-  const int row0 = warp * 16;                       // this warp's rows of the CTA tile
-  const bool warp_live = row0 < m_valid;
-  const int g = lane >> 2, tq = lane & 3;
-  const int r_lo = row0 + g, r_hi = r_lo + 8;       // the two rows this thread owns
-  // last visible key (exclusive) of each row
-  const int lim_lo = (r_lo < m_valid) ? (causal ? L + (r_lo % n) + 1 : T) : 0;
-  const int lim_hi = (r_hi < m_valid) ? (causal ? L + (r_hi % n) + 1 : T) : 0;
-  const float sl2 = rsqrtf((float)D) * LOG2E;       // scores kept in the log2 domain
-
-  uint32_t qf[D / 16][4];
-  float o[D / 8][4];
-#pragma unroll
-  for (int i = 0; i < D / 8; ++i) { o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f; }
-  float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
-
-  for (int t = 0; t < n_tiles; ++t) {
-    const int buf = t & 1;
-    if (t + 1 < n_tiles) load_tile(t + 1, buf ^ 1);
-    cp_async_commit();
-    cp_async_wait<1>();
-    __syncthreads();
-    if (t == 0) {
-#pragma unroll
-      for (int kk = 0; kk < D / 16; ++kk)
-        ldsm_x4(sQ + swz<D>(row0 + (lane & 15), kk * 2 + (lane >> 4)), qf[kk][0], qf[kk][1], qf[kk][2], qf[kk][3]);
-    }
-    if (warp_live) {
-      float s[AT_KEYS / 8][4];
-#pragma unroll
-      for (int i = 0; i < AT_KEYS / 8; ++i) { s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f; }
-      const uint32_t kt = sK + buf * TILE_BYTES;
-#pragma unroll
-      for (int kk = 0; kk < D / 16; ++kk) {
-#pragma unroll
-        for (int np = 0; np < AT_KEYS / 16; ++np) {
-          uint32_t b0, b1, b2, b3;
-          ldsm_x4(kt + swz<D>(np * 16 + (lane & 7) + ((lane >> 4) << 3), kk * 2 + ((lane >> 3) & 1)), b0, b1, b2, b3);
-          mma_bf16(s[2 * np], qf[kk], b0, b1);
-          mma_bf16(s[2 * np + 1], qf[kk], b2, b3);
-        }
-      }
-      // mask + running max
-      const int j0 = key_begin + t * AT_KEYS;
-      float mx_lo = -INFINITY, mx_hi = -INFINITY;
-#pragma unroll
-      for (int nt = 0; nt < AT_KEYS / 8; ++nt) {
-        const int j = j0 + nt * 8 + tq * 2;
-        s[nt][0] = (j < lim_lo) ? s[nt][0] * sl2 : -INFINITY;
-        s[nt][1] = (j + 1 < lim_lo) ? s[nt][1] * sl2 : -INFINITY;
-        s[nt][2] = (j < lim_hi) ? s[nt][2] * sl2 : -INFINITY;
-        s[nt][3] = (j + 1 < lim_hi) ? s[nt][3] * sl2 : -INFINITY;
-        mx_lo = fmaxf(mx_lo, fmaxf(s[nt][0], s[nt][1]));
-        mx_hi = fmaxf(mx_hi, fmaxf(s[nt][2], s[nt][3]));
-      }
-      mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
-      mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
-      mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
-      mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
-      const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
-      const float ref_lo = (mn_lo == -INFINITY) ? 0.f : mn_lo, ref_hi = (mn_hi == -INFINITY) ? 0.f : mn_hi;
-      const float al_lo = exp2f(m_lo - ref_lo), al_hi = exp2f(m_hi - ref_hi);   // exp2(-inf) = 0 on the first tile
-      m_lo = mn_lo; m_hi = mn_hi;
-      float sum_lo = 0.f, sum_hi = 0.f;
-#pragma unroll
-      for (int nt = 0; nt < AT_KEYS / 8; ++nt) {
-        s[nt][0] = exp2f(s[nt][0] - ref_lo); s[nt][1] = exp2f(s[nt][1] - ref_lo);
-        s[nt][2] = exp2f(s[nt][2] - ref_hi); s[nt][3] = exp2f(s[nt][3] - ref_hi);
-        sum_lo += s[nt][0] + s[nt][1];
-        sum_hi += s[nt][2] + s[nt][3];
-      }
-      l_lo = l_lo * al_lo + sum_lo;
-      l_hi = l_hi * al_hi + sum_hi;
-#pragma unroll
-      for (int i = 0; i < D / 8; ++i) { o[i][0] *= al_lo; o[i][1] *= al_lo; o[i][2] *= al_hi; o[i][3] *= al_hi; }
-      const uint32_t vt = sV + buf * TILE_BYTES;
-#pragma unroll
-      for (int kk = 0; kk < AT_KEYS / 16; ++kk) {
-        uint32_t pa[4];
-        pa[0] = pack_bf16(s[2 * kk][0], s[2 * kk][1]);
-        pa[1] = pack_bf16(s[2 * kk][2], s[2 * kk][3]);
-        pa[2] = pack_bf16(s[2 * kk + 1][0], s[2 * kk + 1][1]);
-        pa[3] = pack_bf16(s[2 * kk + 1][2], s[2 * kk + 1][3]);
-#pragma unroll
-        for (int dp = 0; dp < D / 16; ++dp) {
-          uint32_t b0, b1, b2, b3;
-          ldsm_x4_t(vt + swz<D>(kk * 16 + (lane & 7) + (((lane >> 3) & 1) << 3), dp * 2 + (lane >> 4)), b0, b1, b2, b3);
-          mma_bf16(o[2 * dp], pa, b0, b1);
-          mma_bf16(o[2 * dp + 1], pa, b2, b3);
-        }
-      }
-    }
-    __syncthreads();
-  }
-  cp_async_wait<0>();
-
-  // ---- partial results: the quad's four lanes hold the row sums in pieces ----
-  l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
-  l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
-  l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
-  l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
-#pragma unroll
-  for (int half = 0; half < 2; ++half) {
-    const int r = half ? r_hi : r_lo;
-    if (r >= m_valid) continue;
-    const int head = head0 + r / n, i = r % n;
-    const size_t slot = ((size_t)head * n + i) * n_chunks + chunk;
-    float* dst = part_o + slot * D;
-#pragma unroll
-    for (int dt = 0; dt < D / 8; ++dt) {
-      float2 v = half ? make_float2(o[dt][2], o[dt][3]) : make_float2(o[dt][0], o[dt][1]);
-      *reinterpret_cast<float2*>(dst + dt * 8 + tq * 2) = v;
-    }
-    if (tq == 0) part_ml[slot] = half ? make_float2(m_hi, l_hi) : make_float2(m_lo, l_lo);
-  }
+  attn_item<D>(q, kc, vc, part_o, part_ml, n, L, max_seq, hq, hkv, qh, chunk_keys, n_chunks, causal, blockIdx.x, blockIdx.y,
+               blockIdx.z, (uint32_t)__cvta_generic_to_shared(smem), threadIdx.x);
 }
 
 // out[i][head] = sum_c w_c O_c / sum_c w_c l_c, w_c = 2^(m_c - max_c m_c)
