@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfdvlm.so")
-SOURCES = ["fdvlm.cu", "forward.cu", "kernels.cu", "gemm_tc.cu", "attention.cu", "op_static.cu"]
+SOURCES = ["fdvlm.cu", "forward.cu", "kernels.cu", "gemm_tc.cu", "attention.cu", "op_static.cu", "mega.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-cudart", "static", "--expt-relaxed-constexpr"]
 

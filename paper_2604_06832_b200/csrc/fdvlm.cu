@@ -1,5 +1,7 @@
 // The C ABI: handle life cycle, argument and state checks, and the request-level operations
 // (Fast-dVLM Sec. 3.4 decode loop: prefill, block begin / step / commit).
+#include <stdlib.h>
+
 #include <new>
 
 #include "handle.h"
@@ -29,6 +31,7 @@ extern "C" const char* fdvlm_last_error(const fdvlm_t* h) { return h ? h->err : 
 
 extern "C" void fdvlm_destroy(fdvlm_t* h) {
   if (!h) return;
+  mega_destroy(h);
   void* bufs[] = {h->kv, h->h, h->a, h->ao, h->act, h->q, h->y, h->cs, h->ssq, h->stats, h->logits, h->conf, h->pred,
                   h->unmask, h->blk_tokens, h->blk_masked, h->info, h->init_stage, h->ws};
   for (void* p : bufs) if (p) cudaFree(p);
@@ -80,6 +83,7 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
   h->stats = nullptr; h->logits = nullptr; h->conf = nullptr; h->pred = nullptr; h->unmask = nullptr; h->blk_tokens = nullptr;
   h->blk_masked = nullptr; h->info = nullptr; h->init_stage = nullptr; h->ws = nullptr; h->info_host = nullptr;
   h->host_stage = nullptr;
+  h->mega = nullptr;
   cudaGetDevice(&h->device);
 
   const int R = cfg->max_block, H = cfg->hidden, I = cfg->intermediate, d = cfg->head_dim;
@@ -139,6 +143,9 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
     fdvlm_destroy(h);
     return FDVLM_ERR_CUDA;
   }
+  // bf16 weights: the persistent forward kernel, for now only on request (FDVLM_MEGA=1)
+  const char* want_mega = getenv("FDVLM_MEGA");
+  if (h->use_tc && want_mega && want_mega[0] == '1') mega_create(h);
   *out = h;
   return FDVLM_OK;
 }

@@ -231,6 +231,7 @@ static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int wan
 }
 
 int forward_rows(fdvlm_t* h, int n, int mode, int logits_rows, int want_logits) {
+  if (h->mega) return mega_forward(h, n, mode, logits_rows, want_logits);
   return h->use_tc ? forward_rows_tc(h, n, mode, logits_rows, want_logits) : forward_rows_simt(h, n, mode, logits_rows);
 }
 

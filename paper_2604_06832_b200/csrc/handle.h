@@ -19,6 +19,7 @@ struct fdvlm {
   int dt;          // DT_*
   size_t act_sz;   // bytes per activation / KV element
   int use_tc;      // bf16 weights: tcgen05 + TMA GEMMs, tensor-core attention, folded norms
+  void* mega;      // persistent forward kernel context (null: kernel-per-operator path)
   // device buffers (R = max_block rows)
   char* kv;        // [n_layers][2][Hkv][max_seq][d]
   float* h;        // [R, H] residual stream, fp32
@@ -105,5 +106,10 @@ int forward_rows(fdvlm_t* h, int n, int mode, int logits_rows, int want_logits);
 
 size_t linear_workspace_bytes(int m, int n, int k, int dtype);
 size_t attention_workspace_bytes(int n, int hq, int hkv, int d);
+
+// mega.cu: the persistent whole-forward kernel of the bf16 path
+bool mega_create(fdvlm_t* h);
+void mega_destroy(fdvlm_t* h);
+int mega_forward(fdvlm_t* h, int n, int mode, int logits_rows, int want_logits);
 
 }  // namespace fdk

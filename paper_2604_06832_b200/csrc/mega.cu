@@ -1,0 +1,867 @@
+// Persistent forward kernel of the bf16 path (sm_100a): one cooperative launch runs every layer of one
+// denoise / commit / prefill pass (Fast-dVLM Sec. 3.4; Appendix B Alg. 1 draft and verify passes).
+//
+// One CTA per SM.  Roles inside a CTA:
+//   warp 0   weight producer: walks the whole forward's list of weight tiles owned by this CTA and keeps a
+//            ring of 16 KB shared-memory stages full by TMA.  Weights do not depend on activations, so this
+//            warp runs ahead across operator boundaries: while the CTA waits for other SMs, the next
+//            operator's weights are already arriving.
+//   warp 6   activation producer: waits (bounded) for the global counter that says the operator's input rows
+//            are complete, then streams the matching activation k-blocks by TMA into a small second ring.
+//   warp 1   MMA issuer: tcgen05.mma, weights = A operand (128 rows), block rows = N, fp32 accumulators in
+//            tensor memory (two buffers).
+//   warps 2-5 epilogue group: tcgen05.ld, split-K bookkeeping and the fused operator epilogues; the same four
+//            warps run the attention items and the split-KV merge between the QKV and O projections.
+//
+// Work split ("stream-K"): an operator with T weight tiles of KB k-blocks is a line of T*KB units cut into
+// gridDim.x equal contiguous shares, so every SM streams the same number of bytes.  A share that does not
+// cover a whole tile leaves an fp32 partial in a per-CTA slot and bumps the tile's arrival counter; the CTA
+// that arrives last sums the partials in CTA order (deterministic) and runs the epilogue:
+//   QKV   folded RMSNorm factor, bias, rotary, q -> buffer, k / v -> cache rows L .. L + m - 1
+//   O, D  residual add, next norm's gain folded into the bf16 copy, per-tile sum of squares
+//   GU    SwiGLU -> bf16 activations
+//   LM    logits (optional) and per-warp softmax statistics with the mask token excluded
+// Operators are chained by monotonic global counters (release: fence + atomic add; acquire: ld.acquire).
+// Every wait has an iteration / clock bound; a wait that gives up records a code in the status word, the CTA
+// drains its bulk copies, frees its tensor memory and returns.
+//
+// The role loops are written with small iterator structs rather than lambdas: closures that captured the
+// kernel parameter by reference were compiled into reads past the end of the parameter block.
+#include <cuda.h>
+#include <stdlib.h>
+
+#include <mutex>
+
+#include "attn_core.cuh"
+#include "handle.h"
+#include "tc_ptx.cuh"
+
+namespace fdk {
+
+constexpr int MG_THREADS = 224;
+constexpr int MG_NX = 4;                 // activation ring stages
+constexpr int MG_W_BYTES = 16384;        // one weight stage: 128 rows x 64 k bf16
+constexpr long long MG_TIMEOUT = 1ll << 29;  // clock cycles (~0.3 s) before a global wait gives up
+constexpr int MG_SMEM_LIMIT = 232448;    // 227 KB
+
+enum { OP_QKV = 0, OP_O = 1, OP_GU = 2, OP_D = 3, OP_LM = 4 };
+enum { MG_ERR_WPROD = 1, MG_ERR_XPROD = 2, MG_ERR_MMA = 3, MG_ERR_EPI = 4 };
+// per-layer counter slots
+enum { C_QKV = 0, C_ATT = 1, C_AO = 2, C_H2 = 3, C_ACT = 4, C_HOUT = 5, C_TILES = 8 };
+
+// (tensor maps read from global memory by the TMA unit sit on 128-byte boundaries)
+struct alignas(128) MgLayer {
+  CUtensorMap tm_q, tm_k, tm_v, tm_o, tm_d;  // box {64 k, 128 rows}
+  CUtensorMap tm_g, tm_u;                     // box {64 k, 16 rows}: gate / up rows interleaved per 16
+  const float *bq, *bk, *bv, *g_attn, *g_mlp;
+  bf16 *kc, *vc;                              // cache planes [Hkv][max_seq][d]
+};
+
+struct alignas(128) MgModel {
+  CUtensorMap tm_lm;
+  CUtensorMap tm_xg[4], tm_ao[4], tm_act[4];  // activation maps, box {64 k, 16 / 32 / 48 / 64 rows}
+  const MgLayer* layers;
+  int n_layers, H, I, NQ, NKV, hq, hkv, d, vocab, mask_id, max_seq, nt;
+  float eps, inv_h;
+  const float* g_final;
+  float* h;            // [R][H] residual stream
+  bf16 *xg, *q, *ao, *act;
+  float* ssq;          // [R][nt]
+  const float2* cs;    // [R][d/2]
+  float* part;         // [grid * 2][64][128] stream-K partial slots
+  float* att_o;
+  float2* att_ml;
+  float* logits;
+  float4* stats;
+  int* sync;
+  int* status;
+  int* trace;          // optional host-mapped words, one per role of CTA 0: (operator index << 8) | step last reached
+  int tq_begin[4];     // first tile of q, k, v; [3] = T_qkv
+  int T_o, T_g, T_l, KB_h, KB_q, KB_i;
+  int layer_stride, off_to, off_tg, off_td, off_lm;
+};
+static_assert(sizeof(MgLayer) % 128 == 0 && sizeof(CUtensorMap) == 128, "tensor maps must stay 128-byte aligned");
+
+struct MgRun {
+  const MgModel* M;
+  int m, L, causal;
+  int lm_rows;         // 0: no LM head; 1: last row only; m: every row
+  int write_logits;
+  int qh, att_groups, chunk_keys, n_chunks;
+};
+
+// ---- stream-K partition --------------------------------------------------------------------------
+__host__ __device__ inline long long sk_start(int c, long long U, int G) { return ((long long)c * U) / G; }
+__host__ __device__ inline int sk_owner(long long u, long long U, int G) { return (int)(((u + 1) * G - 1) / U); }
+
+// The segments (tile, k-blocks [kb0, kb1)) of CTA c's share of an operator with T tiles of KB k-blocks.
+struct SegIter {
+  long long u, ue;
+  int KB;
+  __device__ __forceinline__ SegIter(int T, int KB_, int c, int G) : KB(KB_) {
+    const long long U = (long long)T * KB_;
+    u = sk_start(c, U, G);
+    ue = sk_start(c + 1, U, G);
+  }
+  __device__ __forceinline__ bool next(int& tile, int& kb0, int& kb1) {
+    if (u >= ue) return false;
+    tile = (int)(u / KB);
+    kb0 = (int)(u - (long long)tile * KB);
+    const long long left = ue - u;
+    kb1 = (left < (long long)(KB - kb0)) ? kb0 + (int)left : KB;
+    u += kb1 - kb0;
+    return true;
+  }
+};
+
+// The operators of one forward in launch order: per layer QKV, O, GU, D; then the LM head (layer index n_layers).
+struct OpIter {
+  int l, kind, n_layers, lm;
+  __device__ __forceinline__ OpIter(int n_layers_, int lm_rows) : l(0), kind(-1), n_layers(n_layers_), lm(lm_rows > 0) {}
+  __device__ __forceinline__ bool next() {
+    if (l >= n_layers) return false;          // the LM head was the last one
+    if (++kind > OP_D) { kind = OP_QKV; ++l; }
+    if (l < n_layers) return true;
+    if (!lm) return false;
+    kind = OP_LM;
+    return true;
+  }
+};
+
+// ---- global-memory synchronisation ------------------------------------------------------------------
+__device__ __forceinline__ int ld_acquire(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ int ld_relaxed(const int* p) {
+  int v;
+  asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void red_release_add(int* p, int v) {
+  asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+// Bounded wait until *p >= target.  False when the wait gave up or the CTA / grid is aborting.
+__device__ __forceinline__ bool wait_count(const int* p, int target, volatile int* abort_flag, const int* status) {
+  if (target <= 0) return true;
+  if (ld_acquire(p) >= target) return true;
+  const long long t0 = clock64();
+  for (int it = 1;; ++it) {
+    if (ld_acquire(p) >= target) return true;
+    if (*abort_flag) return false;
+    if ((it & 127) == 0 && (ld_relaxed(status) != 0 || clock64() - t0 > MG_TIMEOUT)) { *abort_flag = 1; return false; }
+  }
+}
+__device__ __forceinline__ void epi_bar() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+// A tensor map kept in global memory (written there by a host copy) has to be acquired by the thread that
+// hands it to the TMA unit, which reads it through its own proxy.
+__device__ __forceinline__ void tensormap_acquire(const CUtensorMap* tm) {
+  asm volatile("fence.proxy.tensormap::generic.acquire.sys [%0], 128;" ::"l"(tm) : "memory");
+}
+__device__ __forceinline__ void trace_mark(const int* trace, int cta, int role, int op, int step) {
+  if (trace && cta == 0) ((volatile int*)trace)[role] = (op << 8) | step;
+}
+
+template <int M_PAD, int D>
+struct MgSmem {
+  static constexpr int X_BYTES = M_PAD * 128;
+  static constexpr int ATT_BYTES = attn_smem_bytes<D>() > M_PAD * 128 * 4 ? attn_smem_bytes<D>() : M_PAD * 128 * 4;
+  static constexpr int BAR_BYTES = 2048;
+  static constexpr int NW_RAW = (MG_SMEM_LIMIT - 1024 - BAR_BYTES - ATT_BYTES - MG_NX * X_BYTES) / MG_W_BYTES;
+  static constexpr int NW = NW_RAW > 12 ? 12 : NW_RAW;
+  static constexpr int W_OFF = 0;
+  static constexpr int X_OFF = NW * MG_W_BYTES;
+  static constexpr int ATT_OFF = X_OFF + MG_NX * X_BYTES;
+  static constexpr int BAR_OFF = ATT_OFF + ATT_BYTES;
+  static constexpr int TOTAL = BAR_OFF + BAR_BYTES + 1024;
+};
+
+struct OpGeom { int T, KB; };
+__device__ __forceinline__ OpGeom op_geom(const MgModel& M, int kind) {
+  OpGeom g;
+  switch (kind) {
+    case OP_QKV: g.T = M.tq_begin[3]; g.KB = M.KB_h; break;
+    case OP_O: g.T = M.T_o; g.KB = M.KB_q; break;
+    case OP_GU: g.T = M.T_g; g.KB = M.KB_h; break;
+    case OP_D: g.T = M.T_o; g.KB = M.KB_i; break;
+    default: g.T = M.T_l; g.KB = M.KB_h; break;
+  }
+  return g;
+}
+
+// ---- helpers of the epilogue group (128 threads, etid = index inside the group) ----------------------------
+// group-wide bounded wait on a global counter: one thread polls, the result is broadcast
+__device__ __forceinline__ bool group_wait(const int* flag, int target, int etid, volatile int* s_flag, volatile int* abort_flag,
+                                           const int* status) {
+  if (etid == 0) *s_flag = wait_count(flag, target, abort_flag, status) ? 1 : 0;
+  epi_bar();
+  const bool r = *s_flag != 0;
+  epi_bar();
+  return r;
+}
+// release: every thread's stores, then one counter increment
+__device__ __forceinline__ void group_signal(int* flag, int etid) {
+  __threadfence();
+  fence_proxy_async_all();
+  epi_bar();
+  if (etid == 0) red_release_add(flag, 1);
+}
+// s_rstd[i] = rsqrt(mean(h[row0 + i]^2) + eps) from the per-tile sums of squares
+__device__ __forceinline__ void load_rstd(const float* ssq, int nt, float inv_h, float eps, float* s_rstd, int row0, int rows,
+                                          int etid) {
+  if (etid < rows) {
+    float s = 0.f;
+    for (int t = 0; t < nt; ++t) s += __ldcg(&ssq[(size_t)(row0 + etid) * nt + t]);
+    s_rstd[etid] = rsqrtf(s * inv_h + eps);
+  }
+  epi_bar();
+}
+
+template <int M_PAD, int D>
+__global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun Rp) {
+  using S = MgSmem<M_PAD, D>;
+  constexpr int NW = S::NW;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* sm = smem_raw + (base - raw);
+  const uint32_t bar0 = base + S::BAR_OFF;
+  // barrier slots (8 bytes each)
+  const uint32_t w_full0 = bar0, w_empty0 = bar0 + 8u * NW, x_full0 = bar0 + 8u * (2 * NW), x_empty0 = bar0 + 8u * (2 * NW + MG_NX);
+  const uint32_t t_full0 = bar0 + 8u * (2 * NW + 2 * MG_NX), t_empty0 = t_full0 + 16u;
+  constexpr int MISC = 8 * (2 * 12 + 2 * MG_NX + 4);   // 288
+  volatile uint32_t* tmem_slot = (volatile uint32_t*)(sm + S::BAR_OFF + MISC);
+  volatile int* abort_flag = (volatile int*)(sm + S::BAR_OFF + MISC + 8);
+  volatile int* s_flag = (volatile int*)(sm + S::BAR_OFF + MISC + 16);     // epilogue group broadcast word
+  float* s_rstd = (float*)(sm + S::BAR_OFF + MISC + 32);                    // [64]
+  float* s_red = s_rstd + 64;                                               // [4][M_PAD <= 64]
+  float* s_xch = (float*)(sm + S::ATT_OFF);                                 // [M_PAD][128] exchange (GEMM epilogues only)
+
+  // the run description in registers
+  const MgModel* const Mp = Rp.M;
+  const int r_m = Rp.m, r_L = Rp.L, r_causal = Rp.causal, r_lm_rows = Rp.lm_rows, r_write_logits = Rp.write_logits;
+  const int r_qh = Rp.qh, r_groups = Rp.att_groups, r_chunk_keys = Rp.chunk_keys, r_n_chunks = Rp.n_chunks;
+  const MgModel& M = *Mp;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int cta = blockIdx.x, G = gridDim.x;
+  constexpr int TMEM_COLS = (2 * M_PAD <= 32) ? 32 : ((2 * M_PAD <= 64) ? 64 : 128);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < NW; ++s) { mbar_init(w_full0 + 8u * s, 1); mbar_init(w_empty0 + 8u * s, 1); }
+    for (int s = 0; s < MG_NX; ++s) { mbar_init(x_full0 + 8u * s, 1); mbar_init(x_empty0 + 8u * s, 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(t_full0 + 8u * a, 1); mbar_init(t_empty0 + 8u * a, 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+  int* const sync = M.sync;
+  const int* const status = M.status;
+  const int* const trace = M.trace;
+  const int n_layers = M.n_layers, layer_stride = M.layer_stride, T_o = M.T_o, T_g = M.T_g;
+  const int mpi = M_PAD / 16 - 1;
+
+  if (warp == 0) {
+    // =========================================== weight producer ===========================================
+    if (lane == 0) {
+      const uint64_t pol_w = policy_evict_first();
+      int stage = 0;
+      uint32_t phase = 0, armed = 0, armed_parity = 0;
+      bool ok = true;
+      OpIter ops(n_layers, r_lm_rows);
+      while (ok && ops.next()) {
+        const int kind = ops.kind, l = ops.l;
+        const OpGeom g = op_geom(M, kind);
+        const MgLayer* Ly = &M.layers[kind == OP_LM ? 0 : l];
+        trace_mark(trace, cta, 0, l * 4 + kind, 1);
+        switch (kind) {
+          case OP_QKV: tensormap_acquire(&Ly->tm_q); tensormap_acquire(&Ly->tm_k); tensormap_acquire(&Ly->tm_v); break;
+          case OP_O: tensormap_acquire(&Ly->tm_o); break;
+          case OP_GU: tensormap_acquire(&Ly->tm_g); tensormap_acquire(&Ly->tm_u); break;
+          case OP_D: tensormap_acquire(&Ly->tm_d); break;
+          default: tensormap_acquire(&M.tm_lm); break;
+        }
+        SegIter seg(g.T, g.KB, cta, G);
+        int tile, kb0, kb1;
+        while (ok && seg.next(tile, kb0, kb1)) {
+          const CUtensorMap* tm = &M.tm_lm;
+          int r0 = tile * TC_BM;
+          if (kind == OP_QKV) {
+            int mi = 0;
+            while (mi < 2 && tile >= M.tq_begin[mi + 1]) ++mi;
+            tm = mi == 0 ? &Ly->tm_q : (mi == 1 ? &Ly->tm_k : &Ly->tm_v);
+            r0 = (tile - M.tq_begin[mi]) * TC_BM;
+          } else if (kind == OP_O) tm = &Ly->tm_o;
+          else if (kind == OP_D) tm = &Ly->tm_d;
+          for (int kb = kb0; kb < kb1; ++kb) {
+            if (!mbar_wait(w_empty0 + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+            const uint32_t dst = base + S::W_OFF + stage * MG_W_BYTES;
+            const uint32_t fb = w_full0 + 8u * stage;
+            mbar_expect_tx(fb, MG_W_BYTES);
+            armed |= 1u << stage;
+            armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
+            if (kind == OP_GU) {
+              // 64 features per tile: lane quarter qq of the accumulator holds gate rows of features 16qq .. 16qq+15
+              // in its lanes 0..15 and the matching up rows in lanes 16..31
+#pragma unroll
+              for (int qq = 0; qq < 4; ++qq) {
+                tma_load_2d(dst + (32 * qq) * 128, &Ly->tm_g, fb, kb * TC_BK, tile * 64 + 16 * qq, pol_w);
+                tma_load_2d(dst + (32 * qq + 16) * 128, &Ly->tm_u, fb, kb * TC_BK, tile * 64 + 16 * qq, pol_w);
+              }
+            } else {
+              tma_load_2d(dst, tm, fb, kb * TC_BK, r0, pol_w);
+            }
+            if (++stage == NW) { stage = 0; phase ^= 1u; }
+          }
+        }
+      }
+      if (!ok) {
+        atomicCAS(M.status, 0, MG_ERR_WPROD);
+        for (int s = 0; s < NW; ++s) {
+          if (!(armed & (1u << s))) continue;
+          const uint32_t par = (armed_parity >> s) & 1u;
+          const long long t0 = clock64();
+          while (!mbar_try_wait(w_full0 + 8u * s, par) && clock64() - t0 < TC_TIMEOUT) {}
+        }
+      }
+    }
+  } else if (warp == 6) {
+    // ========================================= activation producer =========================================
+    if (lane == 0) {
+      const uint64_t pol_x = policy_evict_last();
+      tensormap_acquire(&M.tm_xg[mpi]);
+      tensormap_acquire(&M.tm_ao[mpi]);
+      tensormap_acquire(&M.tm_act[mpi]);
+      int stage = 0;
+      uint32_t phase = 0, armed = 0, armed_parity = 0;
+      bool ok = true;
+      OpIter ops(n_layers, r_lm_rows);
+      while (ok && ops.next()) {
+        const int kind = ops.kind, l = ops.l;
+        const OpGeom g = op_geom(M, kind);
+        const int* lc = sync + (size_t)(kind == OP_LM ? l - 1 : l) * layer_stride;
+        const CUtensorMap* tm = &M.tm_xg[mpi];
+        const int* flag = lc;
+        int target = 0, row0 = 0;
+        switch (kind) {
+          case OP_QKV: if (l > 0) { flag = lc - layer_stride + C_HOUT; target = T_o; } break;
+          case OP_O: tm = &M.tm_ao[mpi]; flag = lc + C_AO; target = G; break;
+          case OP_GU: flag = lc + C_H2; target = T_o; break;
+          case OP_D: tm = &M.tm_act[mpi]; flag = lc + C_ACT; target = T_g; break;
+          default: flag = lc + C_HOUT; target = T_o; row0 = r_m - r_lm_rows; break;
+        }
+        trace_mark(trace, cta, 1, l * 4 + kind, 1);
+        if (!wait_count(flag, target, abort_flag, status)) { ok = false; break; }
+        trace_mark(trace, cta, 1, l * 4 + kind, 2);
+        fence_proxy_async_all();   // rows written by other SMs' generic stores are read by the async proxy below
+        SegIter seg(g.T, g.KB, cta, G);
+        int tile, kb0, kb1;
+        while (ok && seg.next(tile, kb0, kb1)) {
+          for (int kb = kb0; kb < kb1; ++kb) {
+            if (!mbar_wait(x_empty0 + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+            const uint32_t fb = x_full0 + 8u * stage;
+            mbar_expect_tx(fb, S::X_BYTES);
+            armed |= 1u << stage;
+            armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
+            tma_load_2d(base + S::X_OFF + stage * S::X_BYTES, tm, fb, kb * TC_BK, row0, pol_x);
+            if (++stage == MG_NX) { stage = 0; phase ^= 1u; }
+          }
+        }
+      }
+      if (!ok) {
+        atomicCAS(M.status, 0, MG_ERR_XPROD);
+        for (int s = 0; s < MG_NX; ++s) {
+          if (!(armed & (1u << s))) continue;
+          const uint32_t par = (armed_parity >> s) & 1u;
+          const long long t0 = clock64();
+          while (!mbar_try_wait(x_full0 + 8u * s, par) && clock64() - t0 < TC_TIMEOUT) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ============================================== MMA issuer ==============================================
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc_bf16(M_PAD);
+      int ws = 0, xs = 0, nseg = 0;
+      uint32_t wph = 0, xph = 0;
+      bool ok = true;
+      OpIter ops(n_layers, r_lm_rows);
+      while (ok && ops.next()) {
+        const int kind = ops.kind, l = ops.l;
+        trace_mark(trace, cta, 2, l * 4 + kind, 1);
+        const OpGeom g = op_geom(M, kind);
+        SegIter seg(g.T, g.KB, cta, G);
+        int tile, kb0, kb1;
+        while (ok && seg.next(tile, kb0, kb1)) {
+          const int acc = nseg & 1;
+          const uint32_t acc_phase = (uint32_t)(nseg >> 1) & 1u;
+          ++nseg;
+          if (!mbar_wait(t_empty0 + 8u * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t d_tmem = tmem_base + (uint32_t)(acc * M_PAD);
+          for (int kb = kb0; kb < kb1; ++kb) {
+            if (!mbar_wait(w_full0 + 8u * ws, wph, abort_flag) || !mbar_wait(x_full0 + 8u * xs, xph, abort_flag)) { ok = false; break; }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint64_t adesc = umma_desc_sw128(base + S::W_OFF + ws * MG_W_BYTES);
+            const uint64_t bdesc = umma_desc_sw128(base + S::X_OFF + xs * S::X_BYTES);
+#pragma unroll
+            for (int kk = 0; kk < TC_BK / 16; ++kk)
+              umma_bf16(d_tmem, adesc + 2u * kk, bdesc + 2u * kk, idesc, (kb > kb0 || kk > 0) ? 1u : 0u);
+            umma_commit(w_empty0 + 8u * ws);
+            umma_commit(x_empty0 + 8u * xs);
+            if (++ws == NW) { ws = 0; wph ^= 1u; }
+            if (++xs == MG_NX) { xs = 0; xph ^= 1u; }
+          }
+          if (ok) umma_commit(t_full0 + 8u * acc);
+        }
+      }
+      if (!ok) atomicCAS(M.status, 0, MG_ERR_MMA);
+    }
+  } else {
+    // ================================ epilogue group (warps 2..5, 128 threads) ================================
+    const int q = warp & 3;                       // tensor-memory lane quarter this warp may read
+    const int et = q * 32 + lane;                 // accumulator row held by this thread (0..127)
+    const int etid = (warp - 2) * 32 + lane;      // index inside the group
+    const int nt = M.nt, hq = M.hq, hkv = M.hkv, max_seq = M.max_seq, H = M.H, I = M.I, vocab = M.vocab, mask_id = M.mask_id;
+    const float inv_h = M.inv_h, eps = M.eps;
+    int nseg = 0;
+    bool ok = true;
+    OpIter ops(n_layers, r_lm_rows);
+    while (ok && ops.next()) {
+      const int kind = ops.kind, l = ops.l;
+      const OpGeom g = op_geom(M, kind);
+      int* lc = sync + (size_t)(kind == OP_LM ? l - 1 : l) * layer_stride;
+      const MgLayer* Ly = &M.layers[kind == OP_LM ? 0 : l];
+      const int m = (kind == OP_LM) ? r_lm_rows : r_m;
+      const int xrow0 = (kind == OP_LM) ? r_m - r_lm_rows : 0;
+      if (etid == 0) trace_mark(trace, cta, 3, l * 4 + kind, 1);
+
+      if (kind == OP_O) {
+        // ---------------- attention of this layer: split-KV items, then the merge of the key chunks ----------------
+        if (!group_wait(lc + C_QKV, M.tq_begin[3], etid, s_flag, abort_flag, status)) { ok = false; break; }
+        const int n_items = hkv * r_groups * r_n_chunks;
+        for (int item = cta; item < n_items; item += G) {
+          const int chunk = item % r_n_chunks, rest = item / r_n_chunks;
+          const int grp = rest % r_groups, hk = rest / r_groups;
+          attn_item<D>(M.q, Ly->kc, Ly->vc, M.att_o, M.att_ml, r_m, r_L, max_seq, hq, hkv, r_qh, r_chunk_keys, r_n_chunks,
+                       r_causal, chunk, grp, hk, base + S::ATT_OFF, etid);
+        }
+        if (etid == 0) trace_mark(trace, cta, 3, l * 4 + kind, 2);
+        group_signal(lc + C_ATT, etid);
+        if (!group_wait(lc + C_ATT, G, etid, s_flag, abort_flag, status)) { ok = false; break; }
+        if (etid == 0) trace_mark(trace, cta, 3, l * 4 + kind, 3);
+        for (int p = cta; p < r_m * hq; p += G) {
+          const int i = p / hq, head = p % hq;
+          if (etid < D) {
+            const size_t slot0 = ((size_t)head * r_m + i) * r_n_chunks;
+            float mx = -INFINITY;
+            for (int c = 0; c < r_n_chunks; ++c) mx = fmaxf(mx, __ldcg(&M.att_ml[slot0 + c]).x);
+            float den = 0.f, acc = 0.f;
+            for (int c = 0; c < r_n_chunks; ++c) {
+              const float2 ml = __ldcg(&M.att_ml[slot0 + c]);
+              if (ml.y == 0.f) continue;
+              const float w = exp2f(ml.x - mx);
+              den = fmaf(w, ml.y, den);
+              acc = fmaf(w, __ldcg(&M.att_o[(slot0 + c) * D + etid]), acc);
+            }
+            M.ao[((size_t)i * hq + head) * D + etid] = __float2bfloat16_rn(acc / den);
+          }
+        }
+        group_signal(lc + C_AO, etid);
+        if (etid == 0) trace_mark(trace, cta, 3, l * 4 + kind, 4);
+      }
+
+      // the folded RMSNorm factor of this operator's input rows (QKV, GU, LM) is loaded before the first epilogue
+      bool have_rstd = false;
+      const int* rstd_flag = (kind == OP_QKV) ? lc - layer_stride + C_HOUT : (kind == OP_GU ? lc + C_H2 : lc + C_HOUT);
+      const int rstd_target = (kind == OP_QKV && l == 0) ? 0 : T_o;
+      const bool wants_rstd = (kind == OP_QKV || kind == OP_GU || kind == OP_LM);
+
+      SegIter seg(g.T, g.KB, cta, G);
+      int tile, kb0, kb1;
+      while (ok && seg.next(tile, kb0, kb1)) {
+        const int acc = nseg & 1;
+        const uint32_t acc_phase = (uint32_t)(nseg >> 1) & 1u;
+        ++nseg;
+        if (etid == 0) *s_flag = mbar_wait(t_full0 + 8u * acc, acc_phase, abort_flag) ? 1 : 0;
+        epi_bar();
+        if (*s_flag == 0) { ok = false; break; }
+        if (etid == 0) trace_mark(trace, cta, 3, l * 4 + kind, 5);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        float v[M_PAD];
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * M_PAD);
+#pragma unroll
+        for (int c = 0; c < M_PAD; c += 16) tmem_ld16(taddr + c, v + c);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(t_empty0 + 8u * acc);
+
+        // ---- split tile: leave a partial; the last CTA to arrive sums all partials in CTA order ----
+        if (!(kb0 == 0 && kb1 == g.KB)) {
+          const long long U = (long long)g.T * g.KB;
+          const int first_tile = (int)(sk_start(cta, U, G) / g.KB);
+          float* mine = M.part + ((size_t)(cta * 2 + (tile == first_tile ? 0 : 1)) * 64) * 128;
+#pragma unroll
+          for (int b = 0; b < M_PAD; ++b)
+            if (b < m) mine[b * 128 + et] = v[b];
+          __threadfence();
+          epi_bar();
+          const int cf = sk_owner((long long)tile * g.KB, U, G), cl = sk_owner((long long)tile * g.KB + g.KB - 1, U, G);
+          int* tcnt = lc + (kind == OP_LM ? M.off_lm : (kind == OP_QKV ? (int)C_TILES : (kind == OP_O ? M.off_to : (kind == OP_GU ? M.off_tg : M.off_td)))) + tile;
+          if (etid == 0) *s_flag = (atomicAdd(tcnt, 1) == cl - cf) ? 1 : 0;
+          epi_bar();
+          const bool last = *s_flag != 0;
+          epi_bar();
+          if (!last) continue;
+          __threadfence();
+#pragma unroll
+          for (int b = 0; b < M_PAD; ++b) v[b] = 0.f;
+          for (int c2 = cf; c2 <= cl; ++c2) {
+            const int ft = (int)(sk_start(c2, U, G) / g.KB);
+            const float* src = M.part + ((size_t)(c2 * 2 + (tile == ft ? 0 : 1)) * 64) * 128;
+#pragma unroll
+            for (int b = 0; b < M_PAD; ++b)
+              if (b < m) v[b] += __ldcg(&src[b * 128 + et]);
+          }
+        }
+
+        if (wants_rstd && !have_rstd) {
+          if (!group_wait(rstd_flag, rstd_target, etid, s_flag, abort_flag, status)) { ok = false; break; }
+          load_rstd(M.ssq, nt, inv_h, eps, s_rstd, xrow0, m, etid);
+          have_rstd = true;
+        }
+
+        // ---- operator epilogue on a complete tile: v[b] = sum_k w[row et of the tile][k] x[b][k] ----
+        if (kind == OP_QKV) {
+          int mi = 0;
+          while (mi < 2 && tile >= M.tq_begin[mi + 1]) ++mi;
+          const int n = (tile - M.tq_begin[mi]) * TC_BM + et;          // feature inside its matrix
+          const int n_out = (mi == 0) ? M.NQ : M.NKV;
+          const bool in_range = n < n_out;
+          const float* bias = (mi == 0) ? Ly->bq : (mi == 1 ? Ly->bk : Ly->bv);
+          const float bi = (in_range && bias) ? bias[n] : 0.f;
+          const int head = n / D, j = n % D;
+          constexpr int half = D / 2;
+          const bool lo = j < half;
+          const int jj = lo ? j : j - half;
+#pragma unroll
+          for (int b = 0; b < M_PAD; ++b) v[b] = v[b] * s_rstd[b < m ? b : 0] + bi;
+          if (mi < 2) {
+            // rotary: the partner feature j +- d/2 sits in another warp's rows -> exchange through shared memory
+#pragma unroll
+            for (int b = 0; b < M_PAD; ++b) s_xch[b * 128 + et] = v[b];
+            epi_bar();
+            const int pt = lo ? et + half : et - half;
+#pragma unroll
+            for (int b = 0; b < M_PAD; ++b) {
+              if (b < m) {
+                const float other = s_xch[b * 128 + pt];
+                const float2 c = M.cs[b * half + jj];
+                v[b] = lo ? v[b] * c.x - other * c.y : v[b] * c.x + other * c.y;
+              }
+            }
+            epi_bar();
+          }
+          if (in_range) {
+            bf16* dst;
+            size_t stride;
+            if (mi == 0) { dst = M.q + (size_t)head * D + j; stride = (size_t)hq * D; }
+            else { dst = (mi == 1 ? Ly->kc : Ly->vc) + ((size_t)head * max_seq + r_L) * D + j; stride = D; }
+#pragma unroll
+            for (int b = 0; b < M_PAD; ++b)
+              if (b < m) dst[(size_t)b * stride] = __float2bfloat16_rn(v[b]);
+          }
+          group_signal(lc + C_QKV, etid);
+        } else if (kind == OP_O || kind == OP_D) {
+          const int c = tile * TC_BM + et;
+          const bool in_range = c < H;
+          const float* gain = (kind == OP_O) ? Ly->g_mlp : (l + 1 < n_layers ? M.layers[l + 1].g_attn : M.g_final);
+          const float gn = in_range ? gain[c] : 0.f;
+#pragma unroll
+          for (int b = 0; b < M_PAD; ++b) {
+            if (b < m) {                                   // uniform across the group
+              float hv = 0.f;
+              if (in_range) {
+                const size_t idx = (size_t)b * H + c;
+                hv = __ldcg(&M.h[idx]) + v[b];
+                M.h[idx] = hv;
+                M.xg[idx] = __float2bfloat16_rn(hv * gn);
+              }
+              const float ss = warp_sum(hv * hv);
+              if (lane == 0) s_red[(warp - 2) * M_PAD + b] = ss;
+            }
+          }
+          epi_bar();
+          if (etid < m) M.ssq[(size_t)etid * nt + tile] = s_red[etid] + s_red[M_PAD + etid] + s_red[2 * M_PAD + etid] + s_red[3 * M_PAD + etid];
+          group_signal(lc + (kind == OP_O ? C_H2 : C_HOUT), etid);
+        } else if (kind == OP_GU) {
+          const int col = tile * 64 + q * 16 + (lane & 15);
+          const bool live = lane < 16 && col < I;
+#pragma unroll
+          for (int b = 0; b < M_PAD; ++b) {
+            const float other = __shfl_xor_sync(0xffffffffu, v[b], 16);   // lanes 0..15: the matching "up" value
+            if (live && b < m) {
+              const float rs = s_rstd[b];
+              const float gt = v[b] * rs;
+              M.act[(size_t)b * I + col] = __float2bfloat16_rn(gt / (1.f + __expf(-gt)) * (other * rs));
+            }
+          }
+          group_signal(lc + C_ACT, etid);
+        } else {
+          const int n = tile * TC_BM + et;                    // vocabulary id held by this thread
+          const bool in_range = n < vocab;
+          const bool counted = in_range && n != mask_id;
+#pragma unroll
+          for (int b = 0; b < M_PAD; ++b) {
+            if (b >= m) break;                                // uniform across the group
+            const float lg = v[b] * s_rstd[b];
+            if (r_write_logits && in_range) M.logits[(size_t)b * vocab + n] = lg;
+            float mx = counted ? lg : -INFINITY;
+            int ix = counted ? n : 0x7fffffff;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+              const float omx = __shfl_xor_sync(0xffffffffu, mx, o);
+              const int oix = __shfl_xor_sync(0xffffffffu, ix, o);
+              if (omx > mx || (omx == mx && oix < ix)) { mx = omx; ix = oix; }
+            }
+            float e = (counted && mx > -INFINITY) ? __expf(lg - mx) : 0.f;
+            e = warp_sum(e);
+            if (lane == 0) M.stats[(size_t)(tile * 4 + q) * m + b] = make_float4(mx, e, __int_as_float(ix), 0.f);
+          }
+        }
+      }
+    }
+    if (!ok && etid == 0) atomicCAS(M.status, 0, MG_ERR_EPI);
+  }
+
+  // ---- teardown: every thread arrives here, whatever happened ----
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// ================================================================================================
+// host side
+// ================================================================================================
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn mg_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qr) == cudaSuccess &&
+        qr == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)ptr;
+  });
+  return fn;
+}
+// 2-D bf16 row-major [rows, cols], box {64 columns, box_rows}, 128-byte swizzle, zero fill outside.
+static bool mg_tmap(CUtensorMap* tm, const void* ptr, int rows, int cols, int box_rows) {
+  EncodeTiledFn fn = mg_encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct MegaCtx {
+  MgModel* d_model = nullptr;
+  MgLayer* d_layers = nullptr;
+  int* d_sync = nullptr;
+  float* d_part = nullptr;
+  float* d_att_o = nullptr;
+  float2* d_att_ml = nullptr;
+  size_t sync_bytes = 0;
+  int* h_trace = nullptr;   // host-mapped, only with FDVLM_MEGA_TRACE=1
+  int grid = 0;
+};
+
+struct MgAttPlan { int qh, groups, chunk_keys, n_chunks; };
+static MgAttPlan mg_att_plan(int n, int T, int hq, int hkv, int G) {
+  const int Gh = hq / hkv;
+  MgAttPlan p;
+  p.qh = 1;
+  for (int c = Gh; c >= 1; --c)
+    if (c * n <= AT_ROWS) { p.qh = c; break; }
+  p.groups = ceil_div(Gh, p.qh);
+  const int per_chunk = hkv * p.groups;
+  const int tiles = ceil_div(T, AT_KEYS);
+  int want = G / per_chunk;
+  if (want > tiles) want = tiles;
+  if (want < 1) want = 1;
+  p.chunk_keys = ceil_div(tiles, want) * AT_KEYS;
+  p.n_chunks = ceil_div(T, p.chunk_keys);
+  return p;
+}
+
+template <int M_PAD, int D>
+static cudaError_t mg_launch_t(const MgRun& run, int grid, cudaStream_t st) {
+  using S = MgSmem<M_PAD, D>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(forward_mega_kernel<M_PAD, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, S::TOTAL);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  void* args[] = {(void*)&run};
+  return cudaLaunchCooperativeKernel((const void*)forward_mega_kernel<M_PAD, D>, dim3(grid), dim3(MG_THREADS), args, S::TOTAL, st);
+}
+
+template <int D>
+static cudaError_t mg_launch_d(const MgRun& run, int grid, cudaStream_t st) {
+  const int mp = run.m <= 16 ? 16 : (run.m <= 32 ? 32 : (run.m <= 48 ? 48 : 64));
+  switch (mp) {
+    case 16: return mg_launch_t<16, D>(run, grid, st);
+    case 32: return mg_launch_t<32, D>(run, grid, st);
+    case 48: return mg_launch_t<48, D>(run, grid, st);
+    default: return mg_launch_t<64, D>(run, grid, st);
+  }
+}
+
+void mega_destroy(fdvlm_t* h) {
+  MegaCtx* c = (MegaCtx*)h->mega;
+  if (!c) return;
+  if (c->h_trace) {
+    fprintf(stderr, "fdvlm persistent kernel trace (CTA 0; op<<8|step): wprod %x  xprod %x  mma %x  epi %x\n", c->h_trace[0],
+            c->h_trace[1], c->h_trace[2], c->h_trace[3]);
+    cudaFreeHost(c->h_trace);
+  }
+  void* bufs[] = {c->d_model, c->d_layers, c->d_sync, c->d_part, c->d_att_o, c->d_att_ml};
+  for (void* p : bufs) if (p) cudaFree(p);
+  delete c;
+  h->mega = nullptr;
+}
+
+// Builds the device-side model description.  Returns false (and leaves h->mega null) when the shape or the
+// device does not fit the persistent kernel; the caller then keeps the kernel-per-operator path.
+bool mega_create(fdvlm_t* h) {
+  const fdvlm_config& cf = h->cfg;
+  h->mega = nullptr;
+  if (h->dt != DT_BF16 || !mg_encode_fn()) return false;
+  const int d = cf.head_dim, H = cf.hidden, I = cf.intermediate;
+  const int NQ = cf.n_q_heads * d, NKV = cf.n_kv_heads * d;
+  if ((H % 8) || (I % 16) || (NQ % 8)) return false;
+  int dev = 0, coop = 0, sms = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (!coop || sms < 1) return false;
+
+  MegaCtx* c = new MegaCtx;
+  c->grid = sms;
+  MgModel mm;
+  memset(&mm, 0, sizeof(mm));
+  std::vector<MgLayer> layers(cf.n_layers);
+  bool ok = true;
+  for (int l = 0; l < cf.n_layers && ok; ++l) {
+    const fdvlm_layer_weights& lw = h->layers[l];
+    MgLayer& L = layers[l];
+    memset(&L, 0, sizeof(L));
+    ok = mg_tmap(&L.tm_q, lw.wq, NQ, H, 128) && mg_tmap(&L.tm_k, lw.wk, NKV, H, 128) && mg_tmap(&L.tm_v, lw.wv, NKV, H, 128) &&
+         mg_tmap(&L.tm_o, lw.wo, H, NQ, 128) && mg_tmap(&L.tm_d, lw.w_down, H, I, 128) && mg_tmap(&L.tm_g, lw.w_gate, I, H, 16) &&
+         mg_tmap(&L.tm_u, lw.w_up, I, H, 16);
+    L.bq = lw.bq; L.bk = lw.bk; L.bv = lw.bv; L.g_attn = lw.g_attn; L.g_mlp = lw.g_mlp;
+    L.kc = (bf16*)kv_ptr(h, l, 0); L.vc = (bf16*)kv_ptr(h, l, 1);
+  }
+  const void* table = cf.tie_embeddings ? h->w.embed : h->w.lm_head;
+  const int R = cf.max_block;
+  ok = ok && mg_tmap(&mm.tm_lm, table, cf.vocab, H, 128);
+  for (int i = 0; i < 4 && ok; ++i)
+    ok = mg_tmap(&mm.tm_xg[i], h->a, R, H, 16 * (i + 1)) && mg_tmap(&mm.tm_ao[i], h->ao, R, NQ, 16 * (i + 1)) &&
+         mg_tmap(&mm.tm_act[i], h->act, R, I, 16 * (i + 1));
+  if (!ok) { delete c; return false; }
+
+  mm.n_layers = cf.n_layers; mm.H = H; mm.I = I; mm.NQ = NQ; mm.NKV = NKV; mm.hq = cf.n_q_heads; mm.hkv = cf.n_kv_heads;
+  mm.d = d; mm.vocab = cf.vocab; mm.mask_id = cf.mask_id; mm.max_seq = cf.max_seq; mm.nt = h->nt;
+  mm.eps = cf.rms_eps; mm.inv_h = 1.f / (float)H; mm.g_final = h->w.g_final;
+  mm.h = h->h; mm.xg = (bf16*)h->a; mm.q = (bf16*)h->q; mm.ao = (bf16*)h->ao; mm.act = (bf16*)h->act; mm.ssq = h->ssq;
+  mm.cs = (const float2*)h->cs; mm.logits = h->logits; mm.stats = (float4*)h->stats; mm.status = h->info + 3;
+  mm.tq_begin[0] = 0; mm.tq_begin[1] = ceil_div(NQ, 128); mm.tq_begin[2] = mm.tq_begin[1] + ceil_div(NKV, 128);
+  mm.tq_begin[3] = mm.tq_begin[2] + ceil_div(NKV, 128);
+  mm.T_o = ceil_div(H, 128); mm.T_g = ceil_div(I, 64); mm.T_l = ceil_div(cf.vocab, 128);
+  mm.KB_h = ceil_div(H, 64); mm.KB_q = ceil_div(NQ, 64); mm.KB_i = ceil_div(I, 64);
+  mm.off_to = C_TILES + mm.tq_begin[3]; mm.off_tg = mm.off_to + mm.T_o; mm.off_td = mm.off_tg + mm.T_g;
+  mm.layer_stride = ((mm.off_td + mm.T_o + 31) / 32) * 32;
+  mm.off_lm = mm.layer_stride + 32;   // relative to the last layer's counters
+  c->sync_bytes = ((size_t)cf.n_layers * mm.layer_stride + 32 + mm.T_l + 32) * sizeof(int);
+
+  // attention partials: worst case over the block sizes this handle may see
+  size_t worst = 0;
+  for (int n = 1; n <= R; ++n) {
+    const MgAttPlan p = mg_att_plan(n, cf.max_seq, cf.n_q_heads, cf.n_kv_heads, c->grid);
+    const size_t slots = (size_t)cf.n_q_heads * n * p.n_chunks;
+    if (slots > worst) worst = slots;
+  }
+  bool alloc_ok = cudaMalloc((void**)&c->d_model, sizeof(MgModel)) == cudaSuccess &&
+                  cudaMalloc((void**)&c->d_layers, sizeof(MgLayer) * cf.n_layers) == cudaSuccess &&
+                  cudaMalloc((void**)&c->d_sync, c->sync_bytes) == cudaSuccess &&
+                  cudaMalloc((void**)&c->d_part, (size_t)c->grid * 2 * 64 * 128 * sizeof(float)) == cudaSuccess &&
+                  cudaMalloc((void**)&c->d_att_o, worst * d * sizeof(float)) == cudaSuccess &&
+                  cudaMalloc((void**)&c->d_att_ml, worst * sizeof(float2)) == cudaSuccess;
+  const char* tr = getenv("FDVLM_MEGA_TRACE");
+  if (alloc_ok && tr && tr[0] == '1' && cudaHostAlloc((void**)&c->h_trace, 64, cudaHostAllocMapped) == cudaSuccess) {
+    memset(c->h_trace, 0, 64);
+    void* dp = nullptr;
+    if (cudaHostGetDevicePointer(&dp, c->h_trace, 0) == cudaSuccess) mm.trace = (int*)dp;
+  }
+  if (alloc_ok) {
+    mm.layers = c->d_layers; mm.sync = c->d_sync; mm.part = c->d_part; mm.att_o = c->d_att_o; mm.att_ml = c->d_att_ml;
+    alloc_ok = cudaMemcpy(c->d_layers, layers.data(), sizeof(MgLayer) * cf.n_layers, cudaMemcpyHostToDevice) == cudaSuccess &&
+               cudaMemcpy(c->d_model, &mm, sizeof(MgModel), cudaMemcpyHostToDevice) == cudaSuccess;
+  }
+  h->mega = c;
+  if (!alloc_ok) {
+    cudaGetLastError();
+    mega_destroy(h);
+    return false;
+  }
+  return true;
+}
+
+// One forward over the n rows staged in the residual stream (see forward_rows for the arguments).
+int mega_forward(fdvlm_t* h, int n, int mode, int logits_rows, int want_logits) {
+  MegaCtx* c = (MegaCtx*)h->mega;
+  const fdvlm_config& cf = h->cfg;
+  launch_rope_table(h->cs, n, h->cache_len, cf.head_dim, cf.rope_theta, h->st);
+  CU(h, cudaMemsetAsync(c->d_sync, 0, c->sync_bytes, h->st));
+  const MgAttPlan p = mg_att_plan(n, h->cache_len + n, cf.n_q_heads, cf.n_kv_heads, c->grid);
+  MgRun run;
+  run.M = c->d_model; run.m = n; run.L = h->cache_len; run.causal = (mode == MODE_CAUSAL);
+  run.lm_rows = (logits_rows == 0) ? 0 : (logits_rows == n ? n : 1);
+  run.write_logits = (logits_rows == n) ? want_logits : 1;
+  run.qh = p.qh; run.att_groups = p.groups; run.chunk_keys = p.chunk_keys; run.n_chunks = p.n_chunks;
+  prof_begin(h, 0);
+  cudaError_t e = (cf.head_dim == 128) ? mg_launch_d<128>(run, c->grid, h->st) : mg_launch_d<64>(run, c->grid, h->st);
+  prof_end(h);
+  if (e != cudaSuccess) return fail(h, FDVLM_ERR_CUDA, "persistent forward launch: %s", cudaGetErrorString(e));
+  h->launches += 2;
+  if (logits_rows == n) {
+    launch_stats_merge(h->stats, ceil_div(cf.vocab, 128) * 4, n, h->conf, h->pred, h->st);
+    h->launches++;
+  }
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(h, FDVLM_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
+  return FDVLM_OK;
+}
+
+}  // namespace fdk
