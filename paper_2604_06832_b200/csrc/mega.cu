@@ -95,13 +95,18 @@ __host__ __device__ inline long long sk_start(int c, long long U, int G) { retur
 __host__ __device__ inline int sk_owner(long long u, long long U, int G) { return (int)(((u + 1) * G - 1) / U); }
 
 // The segments (tile, k-blocks [kb0, kb1)) of CTA c's share of an operator with T tiles of KB k-blocks.
+// An operator with fewer units than CTAs is shared by the first `units` CTAs only, so that every CTA inside a
+// tile's owner range really holds a share (the last-arriver count relies on it).
+__host__ __device__ inline int sk_grid(long long U, int G) { return U < (long long)G ? (int)U : G; }
+
 struct SegIter {
   long long u, ue;
   int KB;
   __device__ __forceinline__ SegIter(int T, int KB_, int c, int G) : KB(KB_) {
     const long long U = (long long)T * KB_;
-    u = sk_start(c, U, G);
-    ue = sk_start(c + 1, U, G);
+    const int Ge = sk_grid(U, G);
+    if (c < Ge) { u = sk_start(c, U, Ge); ue = sk_start(c + 1, U, Ge); }
+    else { u = 0; ue = 0; }
   }
   __device__ __forceinline__ bool next(int& tile, int& kb0, int& kb1) {
     if (u >= ue) return false;
@@ -509,14 +514,15 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
         // ---- split tile: leave a partial; the last CTA to arrive sums all partials in CTA order ----
         if (!(kb0 == 0 && kb1 == g.KB)) {
           const long long U = (long long)g.T * g.KB;
-          const int first_tile = (int)(sk_start(cta, U, G) / g.KB);
+          const int Ge = sk_grid(U, G);
+          const int first_tile = (int)(sk_start(cta, U, Ge) / g.KB);
           float* mine = M.part + ((size_t)(cta * 2 + (tile == first_tile ? 0 : 1)) * 64) * 128;
 #pragma unroll
           for (int b = 0; b < M_PAD; ++b)
             if (b < m) mine[b * 128 + et] = v[b];
           __threadfence();
           epi_bar();
-          const int cf = sk_owner((long long)tile * g.KB, U, G), cl = sk_owner((long long)tile * g.KB + g.KB - 1, U, G);
+          const int cf = sk_owner((long long)tile * g.KB, U, Ge), cl = sk_owner((long long)tile * g.KB + g.KB - 1, U, Ge);
           int* tcnt = lc + (kind == OP_LM ? M.off_lm : (kind == OP_QKV ? (int)C_TILES : (kind == OP_O ? M.off_to : (kind == OP_GU ? M.off_tg : M.off_td)))) + tile;
           if (etid == 0) *s_flag = (atomicAdd(tcnt, 1) == cl - cf) ? 1 : 0;
           epi_bar();
@@ -527,7 +533,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
 #pragma unroll
           for (int b = 0; b < M_PAD; ++b) v[b] = 0.f;
           for (int c2 = cf; c2 <= cl; ++c2) {
-            const int ft = (int)(sk_start(c2, U, G) / g.KB);
+            const int ft = (int)(sk_start(c2, U, Ge) / g.KB);
             const float* src = M.part + ((size_t)(c2 * 2 + (tile == ft ? 0 : 1)) * 64) * 128;
 #pragma unroll
             for (int b = 0; b < M_PAD; ++b)
