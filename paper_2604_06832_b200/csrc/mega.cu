@@ -76,9 +76,12 @@ struct alignas(128) MgModel {
   int* sync;
   int* status;
   int* trace;          // optional host-mapped words, one per role of CTA 0: (operator index << 8) | step last reached
+  long long* tline;    // optional host-mapped timeline of one traced CTA: [operator][8] globaltimer stamps
+  int trace_cta;
   int tq_begin[4];     // first tile of q, k, v; [3] = T_qkv
   int T_o, T_g, T_l, KB_h, KB_q, KB_i;
   int layer_stride, off_to, off_tg, off_td, off_lm;
+  int op_sk[5], op_ge[5], op_off[5];   // per operator kind: K-splits per tile, participating CTAs, first CTA
 };
 static_assert(sizeof(MgLayer) % 128 == 0 && sizeof(CUtensorMap) == 128, "tensor maps must stay 128-byte aligned");
 
@@ -90,31 +93,44 @@ struct MgRun {
   int qh, att_groups, chunk_keys, n_chunks;
 };
 
-// ---- stream-K partition --------------------------------------------------------------------------
-__host__ __device__ inline long long sk_start(int c, long long U, int G) { return ((long long)c * U) / G; }
-__host__ __device__ inline int sk_owner(long long u, long long U, int G) { return (int)(((u + 1) * G - 1) / U); }
+// ---- work partition ----------------------------------------------------------------------------------
+// An operator with T weight tiles of KB k-blocks is cut into W = T * SK units (unit j of a tile = k-blocks
+// [j KB / SK, (j + 1) KB / SK)); the units form a line cut into Ge equal contiguous shares, one per participating
+// CTA.  SK = 1 gives whole tiles (direct epilogue), SK = KB is stream-K (every SM streams the same bytes), a small
+// SK is a classic split-K.  The Ge logical CTAs are spread over the grid: logical p runs on CTA (p G / Ge + off) % G.
+struct Part {
+  int T, KB, SK, Ge, off, G;
+  __host__ __device__ long long W() const { return (long long)T * SK; }
+  __host__ __device__ long long start(int p) const { return ((long long)p * W()) / Ge; }
+  __host__ __device__ int owner(long long w) const { return (int)(((w + 1) * Ge - 1) / W()); }
+  __host__ __device__ int kb_of(int j) const { return (int)(((long long)j * KB) / SK); }
+  __host__ __device__ int phys(int p) const { return (int)((((long long)p * G) / Ge + off) % G); }
+  // logical index of physical CTA c, or -1
+  __host__ __device__ int logical(int c) const {
+    const int cr = (c - off % G + G) % G;
+    const int p = (int)(((long long)cr * Ge + G - 1) / G);
+    return (p < Ge && (int)(((long long)p * G) / Ge) == cr) ? p : -1;
+  }
+};
 
-// The segments (tile, k-blocks [kb0, kb1)) of CTA c's share of an operator with T tiles of KB k-blocks.
-// An operator with fewer units than CTAs is shared by the first `units` CTAs only, so that every CTA inside a
-// tile's owner range really holds a share (the last-arriver count relies on it).
-__host__ __device__ inline int sk_grid(long long U, int G) { return U < (long long)G ? (int)U : G; }
-
+// The segments (tile, k-blocks [kb0, kb1)) of one CTA's share.
 struct SegIter {
-  long long u, ue;
-  int KB;
-  __device__ __forceinline__ SegIter(int T, int KB_, int c, int G) : KB(KB_) {
-    const long long U = (long long)T * KB_;
-    const int Ge = sk_grid(U, G);
-    if (c < Ge) { u = sk_start(c, U, Ge); ue = sk_start(c + 1, U, Ge); }
-    else { u = 0; ue = 0; }
+  Part P;
+  long long w, we;
+  __device__ __forceinline__ SegIter(const Part& P_, int c) : P(P_) {
+    const int p = P.logical(c);
+    if (p >= 0) { w = P.start(p); we = P.start(p + 1); }
+    else { w = 0; we = 0; }
   }
   __device__ __forceinline__ bool next(int& tile, int& kb0, int& kb1) {
-    if (u >= ue) return false;
-    tile = (int)(u / KB);
-    kb0 = (int)(u - (long long)tile * KB);
-    const long long left = ue - u;
-    kb1 = (left < (long long)(KB - kb0)) ? kb0 + (int)left : KB;
-    u += kb1 - kb0;
+    if (w >= we) return false;
+    tile = (int)(w / P.SK);
+    const int j0 = (int)(w - (long long)tile * P.SK);
+    const long long left = we - w;
+    const int j1 = (left < (long long)(P.SK - j0)) ? j0 + (int)left : P.SK;
+    kb0 = P.kb_of(j0);
+    kb1 = P.kb_of(j1);
+    w += j1 - j0;
     return true;
   }
 };
@@ -168,11 +184,21 @@ __device__ __forceinline__ void tensormap_acquire(const CUtensorMap* tm) {
 __device__ __forceinline__ void trace_mark(const int* trace, int cta, int role, int op, int step) {
   if (trace && cta == 0) ((volatile int*)trace)[role] = (op << 8) | step;
 }
+// timeline slots per operator: 0 epilogue reaches the operator, 1 its attention done (O only), 2 first accumulator
+// ready, 3 epilogue leaves the operator, 4 activation flag seen, 5 activation loads issued, 6 first MMA issued,
+// 7 weight loads issued
+__device__ __forceinline__ void tl_mark(long long* tl, bool on, int op, int slot) {
+  if (tl && on) {
+    long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    ((volatile long long*)tl)[op * 8 + slot] = t;
+  }
+}
 
 template <int M_PAD, int D>
 struct MgSmem {
   static constexpr int X_BYTES = M_PAD * 128;
-  static constexpr int ATT_BYTES = attn_smem_bytes<D>() > M_PAD * 128 * 4 ? attn_smem_bytes<D>() : M_PAD * 128 * 4;
+  static constexpr int ATT_BYTES = attn_smem_bytes<D>() > M_PAD * 132 * 4 ? attn_smem_bytes<D>() : M_PAD * 132 * 4;   // also the epilogues' exchange buffer
   static constexpr int BAR_BYTES = 2048;
   static constexpr int NW_RAW = (MG_SMEM_LIMIT - 1024 - BAR_BYTES - ATT_BYTES - MG_NX * X_BYTES) / MG_W_BYTES;
   static constexpr int NW = NW_RAW > 12 ? 12 : NW_RAW;
@@ -183,9 +209,8 @@ struct MgSmem {
   static constexpr int TOTAL = BAR_OFF + BAR_BYTES + 1024;
 };
 
-struct OpGeom { int T, KB; };
-__device__ __forceinline__ OpGeom op_geom(const MgModel& M, int kind) {
-  OpGeom g;
+__device__ __forceinline__ Part op_part(const MgModel& M, int kind, int G) {
+  Part g;
   switch (kind) {
     case OP_QKV: g.T = M.tq_begin[3]; g.KB = M.KB_h; break;
     case OP_O: g.T = M.T_o; g.KB = M.KB_q; break;
@@ -193,6 +218,7 @@ __device__ __forceinline__ OpGeom op_geom(const MgModel& M, int kind) {
     case OP_D: g.T = M.T_o; g.KB = M.KB_i; break;
     default: g.T = M.T_l; g.KB = M.KB_h; break;
   }
+  g.SK = M.op_sk[kind]; g.Ge = M.op_ge[kind]; g.off = M.op_off[kind]; g.G = G;
   return g;
 }
 
@@ -217,11 +243,57 @@ __device__ __forceinline__ void group_signal(int* flag, int etid) {
 __device__ __forceinline__ void load_rstd(const float* ssq, int nt, float inv_h, float eps, float* s_rstd, int row0, int rows,
                                           int etid) {
   if (etid < rows) {
+    const float* p = ssq + (size_t)(row0 + etid) * nt;
     float s = 0.f;
-    for (int t = 0; t < nt; ++t) s += __ldcg(&ssq[(size_t)(row0 + etid) * nt + t]);
+    for (int t0 = 0; t0 < nt; t0 += 8) {         // eight independent loads in flight, summed in index order
+      float r[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) r[i] = (t0 + i < nt) ? __ldcg(p + t0 + i) : 0.f;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) s += r[i];
+    }
     s_rstd[etid] = rsqrtf(s * inv_h + eps);
   }
   epi_bar();
+}
+
+// Merge of the key chunks of one (row, head) by one warp: out = sum_c w_c O_c / sum_c w_c l_c, w_c = 2^(m_c - max m).
+// Lane j owns D / 32 consecutive output features; the chunk statistics are spread over the lanes.
+template <int D>
+__device__ __forceinline__ void attn_merge_warp(const float* att_o, const float2* att_ml, bf16* out, size_t slot0, int n_chunks,
+                                                int lane) {
+  constexpr int VPL = D / 32;
+  float mx = -INFINITY;
+  for (int c = lane; c < n_chunks; c += 32) mx = fmaxf(mx, __ldcg(&att_ml[slot0 + c]).x);
+  mx = warp_max(mx);
+  float den = 0.f, acc[VPL];
+#pragma unroll
+  for (int i = 0; i < VPL; ++i) acc[i] = 0.f;
+  for (int c0 = 0; c0 < n_chunks; c0 += 32) {
+    const int c = c0 + lane;
+    float w = 0.f;
+    if (c < n_chunks) {
+      const float2 ml = __ldcg(&att_ml[slot0 + c]);
+      if (ml.y != 0.f) { w = exp2f(ml.x - mx); den = fmaf(w, ml.y, den); }
+    }
+    const int cn = min(32, n_chunks - c0);
+#pragma unroll 4
+    for (int cc = 0; cc < cn; ++cc) {
+      const float wc = __shfl_sync(0xffffffffu, w, cc);
+      const float* src = att_o + (slot0 + c0 + cc) * D + lane * VPL;
+      if (VPL == 4) {
+        const float4 o = __ldcg(reinterpret_cast<const float4*>(src));
+        acc[0] = fmaf(wc, o.x, acc[0]); acc[1] = fmaf(wc, o.y, acc[1]); acc[2] = fmaf(wc, o.z, acc[2]); acc[VPL - 1] = fmaf(wc, o.w, acc[VPL - 1]);
+      } else {
+        const float2 o = __ldcg(reinterpret_cast<const float2*>(src));
+        acc[0] = fmaf(wc, o.x, acc[0]); acc[VPL - 1] = fmaf(wc, o.y, acc[VPL - 1]);
+      }
+    }
+  }
+  den = warp_sum(den);
+  const float inv = 1.f / den;
+#pragma unroll
+  for (int i = 0; i < VPL; ++i) out[lane * VPL + i] = __float2bfloat16_rn(acc[i] * inv);
 }
 
 template <int M_PAD, int D>
@@ -242,7 +314,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
   volatile int* s_flag = (volatile int*)(sm + S::BAR_OFF + MISC + 16);     // epilogue group broadcast word
   float* s_rstd = (float*)(sm + S::BAR_OFF + MISC + 32);                    // [64]
   float* s_red = s_rstd + 64;                                               // [4][M_PAD <= 64]
-  float* s_xch = (float*)(sm + S::ATT_OFF);                                 // [M_PAD][128] exchange (GEMM epilogues only)
+  float* s_xch = (float*)(sm + S::ATT_OFF);                                 // [M_PAD][<=132] exchange (GEMM epilogues only)
 
   // the run description in registers
   const MgModel* const Mp = Rp.M;
@@ -272,6 +344,8 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
   int* const sync = M.sync;
   const int* const status = M.status;
   const int* const trace = M.trace;
+  long long* const tl = M.tline;
+  const bool tl_on = (cta == M.trace_cta);
   const int n_layers = M.n_layers, layer_stride = M.layer_stride, T_o = M.T_o, T_g = M.T_g;
   const int mpi = M_PAD / 16 - 1;
 
@@ -285,7 +359,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
       OpIter ops(n_layers, r_lm_rows);
       while (ok && ops.next()) {
         const int kind = ops.kind, l = ops.l;
-        const OpGeom g = op_geom(M, kind);
+        const Part g = op_part(M, kind, G);
         const MgLayer* Ly = &M.layers[kind == OP_LM ? 0 : l];
         trace_mark(trace, cta, 0, l * 4 + kind, 1);
         switch (kind) {
@@ -295,7 +369,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
           case OP_D: tensormap_acquire(&Ly->tm_d); break;
           default: tensormap_acquire(&M.tm_lm); break;
         }
-        SegIter seg(g.T, g.KB, cta, G);
+        SegIter seg(g, cta);
         int tile, kb0, kb1;
         while (ok && seg.next(tile, kb0, kb1)) {
           const CUtensorMap* tm = &M.tm_lm;
@@ -328,6 +402,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
             if (++stage == NW) { stage = 0; phase ^= 1u; }
           }
         }
+        tl_mark(tl, tl_on, l * 4 + kind, 7);
       }
       if (!ok) {
         atomicCAS(M.status, 0, MG_ERR_WPROD);
@@ -352,7 +427,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
       OpIter ops(n_layers, r_lm_rows);
       while (ok && ops.next()) {
         const int kind = ops.kind, l = ops.l;
-        const OpGeom g = op_geom(M, kind);
+        const Part g = op_part(M, kind, G);
         const int* lc = sync + (size_t)(kind == OP_LM ? l - 1 : l) * layer_stride;
         const CUtensorMap* tm = &M.tm_xg[mpi];
         const int* flag = lc;
@@ -367,8 +442,9 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
         trace_mark(trace, cta, 1, l * 4 + kind, 1);
         if (!wait_count(flag, target, abort_flag, status)) { ok = false; break; }
         trace_mark(trace, cta, 1, l * 4 + kind, 2);
+        tl_mark(tl, tl_on, l * 4 + kind, 4);
         fence_proxy_async_all();   // rows written by other SMs' generic stores are read by the async proxy below
-        SegIter seg(g.T, g.KB, cta, G);
+        SegIter seg(g, cta);
         int tile, kb0, kb1;
         while (ok && seg.next(tile, kb0, kb1)) {
           for (int kb = kb0; kb < kb1; ++kb) {
@@ -381,6 +457,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
             if (++stage == MG_NX) { stage = 0; phase ^= 1u; }
           }
         }
+        tl_mark(tl, tl_on, l * 4 + kind, 5);
       }
       if (!ok) {
         atomicCAS(M.status, 0, MG_ERR_XPROD);
@@ -403,8 +480,8 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
       while (ok && ops.next()) {
         const int kind = ops.kind, l = ops.l;
         trace_mark(trace, cta, 2, l * 4 + kind, 1);
-        const OpGeom g = op_geom(M, kind);
-        SegIter seg(g.T, g.KB, cta, G);
+        const Part g = op_part(M, kind, G);
+        SegIter seg(g, cta);
         int tile, kb0, kb1;
         while (ok && seg.next(tile, kb0, kb1)) {
           const int acc = nseg & 1;
@@ -416,6 +493,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
           for (int kb = kb0; kb < kb1; ++kb) {
             if (!mbar_wait(w_full0 + 8u * ws, wph, abort_flag) || !mbar_wait(x_full0 + 8u * xs, xph, abort_flag)) { ok = false; break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            if (kb == kb0) tl_mark(tl, tl_on, l * 4 + kind, 6);
             const uint64_t adesc = umma_desc_sw128(base + S::W_OFF + ws * MG_W_BYTES);
             const uint64_t bdesc = umma_desc_sw128(base + S::X_OFF + xs * S::X_BYTES);
 #pragma unroll
@@ -443,12 +521,12 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
     OpIter ops(n_layers, r_lm_rows);
     while (ok && ops.next()) {
       const int kind = ops.kind, l = ops.l;
-      const OpGeom g = op_geom(M, kind);
+      const Part g = op_part(M, kind, G);
       int* lc = sync + (size_t)(kind == OP_LM ? l - 1 : l) * layer_stride;
       const MgLayer* Ly = &M.layers[kind == OP_LM ? 0 : l];
       const int m = (kind == OP_LM) ? r_lm_rows : r_m;
       const int xrow0 = (kind == OP_LM) ? r_m - r_lm_rows : 0;
-      if (etid == 0) trace_mark(trace, cta, 3, l * 4 + kind, 1);
+      if (etid == 0) { trace_mark(trace, cta, 3, l * 4 + kind, 1); tl_mark(tl, tl_on, l * 4 + kind, 0); }
 
       if (kind == OP_O) {
         // ---------------- attention of this layer: split-KV items, then the merge of the key chunks ----------------
@@ -464,43 +542,51 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
         group_signal(lc + C_ATT, etid);
         if (!group_wait(lc + C_ATT, G, etid, s_flag, abort_flag, status)) { ok = false; break; }
         if (etid == 0) trace_mark(trace, cta, 3, l * 4 + kind, 3);
-        for (int p = cta; p < r_m * hq; p += G) {
+        // one warp per (row, head): the CTA's four warps take consecutive pairs
+        for (int p = cta * 4 + (warp - 2); p < r_m * hq; p += G * 4) {
           const int i = p / hq, head = p % hq;
-          if (etid < D) {
-            const size_t slot0 = ((size_t)head * r_m + i) * r_n_chunks;
-            float mx = -INFINITY;
-            for (int c = 0; c < r_n_chunks; ++c) mx = fmaxf(mx, __ldcg(&M.att_ml[slot0 + c]).x);
-            float den = 0.f, acc = 0.f;
-            for (int c = 0; c < r_n_chunks; ++c) {
-              const float2 ml = __ldcg(&M.att_ml[slot0 + c]);
-              if (ml.y == 0.f) continue;
-              const float w = exp2f(ml.x - mx);
-              den = fmaf(w, ml.y, den);
-              acc = fmaf(w, __ldcg(&M.att_o[(slot0 + c) * D + etid]), acc);
-            }
-            M.ao[((size_t)i * hq + head) * D + etid] = __float2bfloat16_rn(acc / den);
-          }
+          attn_merge_warp<D>(M.att_o, M.att_ml, M.ao + ((size_t)i * hq + head) * D, ((size_t)head * r_m + i) * r_n_chunks, r_n_chunks, lane);
         }
         group_signal(lc + C_AO, etid);
-        if (etid == 0) trace_mark(trace, cta, 3, l * 4 + kind, 4);
+        if (etid == 0) { trace_mark(trace, cta, 3, l * 4 + kind, 4); tl_mark(tl, tl_on, l * 4 + kind, 1); }
       }
 
       // the folded RMSNorm factor of this operator's input rows (QKV, GU, LM) is loaded before the first epilogue
       bool have_rstd = false;
+      (void)have_rstd;
       const int* rstd_flag = (kind == OP_QKV) ? lc - layer_stride + C_HOUT : (kind == OP_GU ? lc + C_H2 : lc + C_HOUT);
       const int rstd_target = (kind == OP_QKV && l == 0) ? 0 : T_o;
       const bool wants_rstd = (kind == OP_QKV || kind == OP_GU || kind == OP_LM);
 
-      SegIter seg(g.T, g.KB, cta, G);
+      SegIter seg(g, cta);
       int tile, kb0, kb1;
+      const bool is_resid = (kind == OP_O || kind == OP_D);
+      if (seg.w < seg.we) {
+        // inputs of the epilogues that do not depend on this operator's own MMAs are fetched while those run
+        if (wants_rstd) {
+          if (!group_wait(rstd_flag, rstd_target, etid, s_flag, abort_flag, status)) { ok = false; break; }
+          load_rstd(M.ssq, nt, inv_h, eps, s_rstd, xrow0, m, etid);
+          have_rstd = true;
+        } else if (is_resid) {
+          // the residual rows this operator adds to: complete once the previous residual operator has finished
+          const int* hflag = (kind == OP_O) ? lc - layer_stride + C_HOUT : lc + C_H2;
+          if (!group_wait(hflag, (kind == OP_O && l == 0) ? 0 : T_o, etid, s_flag, abort_flag, status)) { ok = false; break; }
+        }
+      }
       while (ok && seg.next(tile, kb0, kb1)) {
         const int acc = nseg & 1;
         const uint32_t acc_phase = (uint32_t)(nseg >> 1) & 1u;
         ++nseg;
+        float hold[M_PAD];
+        if (is_resid) {
+          const int c = tile * TC_BM + et;
+#pragma unroll
+          for (int b = 0; b < M_PAD; ++b) hold[b] = (c < H && b < m) ? __ldcg(&M.h[(size_t)b * H + c]) : 0.f;
+        }
         if (etid == 0) *s_flag = mbar_wait(t_full0 + 8u * acc, acc_phase, abort_flag) ? 1 : 0;
         epi_bar();
         if (*s_flag == 0) { ok = false; break; }
-        if (etid == 0) trace_mark(trace, cta, 3, l * 4 + kind, 5);
+        if (etid == 0) { trace_mark(trace, cta, 3, l * 4 + kind, 5); tl_mark(tl, tl_on, l * 4 + kind, 2); }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         float v[M_PAD];
         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * M_PAD);
@@ -513,16 +599,15 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
 
         // ---- split tile: leave a partial; the last CTA to arrive sums all partials in CTA order ----
         if (!(kb0 == 0 && kb1 == g.KB)) {
-          const long long U = (long long)g.T * g.KB;
-          const int Ge = sk_grid(U, G);
-          const int first_tile = (int)(sk_start(cta, U, Ge) / g.KB);
+          const int me = g.logical(cta);
+          const int first_tile = (int)(g.start(me) / g.SK);
           float* mine = M.part + ((size_t)(cta * 2 + (tile == first_tile ? 0 : 1)) * 64) * 128;
 #pragma unroll
           for (int b = 0; b < M_PAD; ++b)
             if (b < m) mine[b * 128 + et] = v[b];
           __threadfence();
           epi_bar();
-          const int cf = sk_owner((long long)tile * g.KB, U, Ge), cl = sk_owner((long long)tile * g.KB + g.KB - 1, U, Ge);
+          const int cf = g.owner((long long)tile * g.SK), cl = g.owner((long long)tile * g.SK + g.SK - 1);
           int* tcnt = lc + (kind == OP_LM ? M.off_lm : (kind == OP_QKV ? (int)C_TILES : (kind == OP_O ? M.off_to : (kind == OP_GU ? M.off_tg : M.off_td)))) + tile;
           if (etid == 0) *s_flag = (atomicAdd(tcnt, 1) == cl - cf) ? 1 : 0;
           epi_bar();
@@ -532,19 +617,25 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
           __threadfence();
 #pragma unroll
           for (int b = 0; b < M_PAD; ++b) v[b] = 0.f;
-          for (int c2 = cf; c2 <= cl; ++c2) {
-            const int ft = (int)(sk_start(c2, U, Ge) / g.KB);
-            const float* src = M.part + ((size_t)(c2 * 2 + (tile == ft ? 0 : 1)) * 64) * 128;
+          constexpr int CU = (M_PAD <= 16) ? 4 : (M_PAD <= 32 ? 2 : 1);   // partials loaded together (register budget)
+          for (int c2 = cf; c2 <= cl; c2 += CU) {
+            float pv[CU][M_PAD];
 #pragma unroll
-            for (int b = 0; b < M_PAD; ++b)
-              if (b < m) v[b] += __ldcg(&src[b * 128 + et]);
+            for (int u2 = 0; u2 < CU; ++u2) {
+              const int c3 = (c2 + u2 <= cl) ? c2 + u2 : cl;
+              const int ft = (int)(g.start(c3) / g.SK);
+              const float* src = M.part + ((size_t)(g.phys(c3) * 2 + (tile == ft ? 0 : 1)) * 64) * 128;
+#pragma unroll
+              for (int b = 0; b < M_PAD; ++b) pv[u2][b] = (b < m) ? __ldcg(&src[b * 128 + et]) : 0.f;
+            }
+#pragma unroll
+            for (int u2 = 0; u2 < CU; ++u2) {
+              if (c2 + u2 <= cl) {                 // summed in CTA order
+#pragma unroll
+                for (int b = 0; b < M_PAD; ++b) v[b] += pv[u2][b];
+              }
+            }
           }
-        }
-
-        if (wants_rstd && !have_rstd) {
-          if (!group_wait(rstd_flag, rstd_target, etid, s_flag, abort_flag, status)) { ok = false; break; }
-          load_rstd(M.ssq, nt, inv_h, eps, s_rstd, xrow0, m, etid);
-          have_rstd = true;
         }
 
         // ---- operator epilogue on a complete tile: v[b] = sum_k w[row et of the tile][k] x[b][k] ----
@@ -593,19 +684,26 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
           const bool in_range = c < H;
           const float* gain = (kind == OP_O) ? Ly->g_mlp : (l + 1 < n_layers ? M.layers[l + 1].g_attn : M.g_final);
           const float gn = in_range ? gain[c] : 0.f;
+          // squares go through shared memory ([row][132]: 4 x 33 per row, conflict-free both ways) for the per-row sums
 #pragma unroll
           for (int b = 0; b < M_PAD; ++b) {
             if (b < m) {                                   // uniform across the group
-              float hv = 0.f;
+              const float hv = hold[b] + v[b];
               if (in_range) {
                 const size_t idx = (size_t)b * H + c;
-                hv = __ldcg(&M.h[idx]) + v[b];
                 M.h[idx] = hv;
                 M.xg[idx] = __float2bfloat16_rn(hv * gn);
               }
-              const float ss = warp_sum(hv * hv);
-              if (lane == 0) s_red[(warp - 2) * M_PAD + b] = ss;
+              s_xch[b * 132 + (warp - 2) * 33 + lane] = in_range ? hv * hv : 0.f;
             }
+          }
+          epi_bar();
+          for (int w4 = etid; w4 < m * 4; w4 += 128) {
+            const int b = w4 >> 2, part = w4 & 3;
+            float ss = 0.f;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) ss += s_xch[b * 132 + part * 33 + i];
+            s_red[part * M_PAD + b] = ss;
           }
           epi_bar();
           if (etid < m) M.ssq[(size_t)etid * nt + tile] = s_red[etid] + s_red[M_PAD + etid] + s_red[2 * M_PAD + etid] + s_red[3 * M_PAD + etid];
@@ -646,6 +744,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
           }
         }
       }
+      if (etid == 0) tl_mark(tl, tl_on, l * 4 + kind, 3);
     }
     if (!ok && etid == 0) atomicCAS(M.status, 0, MG_ERR_EPI);
   }
@@ -699,6 +798,8 @@ struct MegaCtx {
   float2* d_att_ml = nullptr;
   size_t sync_bytes = 0;
   int* h_trace = nullptr;   // host-mapped, only with FDVLM_MEGA_TRACE=1
+  long long* h_tline = nullptr;
+  int n_ops = 0;
   int grid = 0;
 };
 
@@ -751,6 +852,18 @@ void mega_destroy(fdvlm_t* h) {
     fprintf(stderr, "fdvlm persistent kernel trace (CTA 0; op<<8|step): wprod %x  xprod %x  mma %x  epi %x\n", c->h_trace[0],
             c->h_trace[1], c->h_trace[2], c->h_trace[3]);
     cudaFreeHost(c->h_trace);
+  }
+  if (c->h_tline) {
+    // per operator: microseconds since the first stamp of the last traced forward
+    long long t0 = 0;
+    for (int i = 0; i < c->n_ops * 8; ++i) if (c->h_tline[i] && (!t0 || c->h_tline[i] < t0)) t0 = c->h_tline[i];
+    fprintf(stderr, "op: epi_in att_done acc0 epi_out | x_flag x_issued | mma0 | w_issued   (us)\n");
+    for (int o = 0; o < c->n_ops; ++o) {
+      fprintf(stderr, "%3d:", o);
+      for (int k = 0; k < 8; ++k) fprintf(stderr, " %9.2f", c->h_tline[o * 8 + k] ? (c->h_tline[o * 8 + k] - t0) / 1000.0 : -1.0);
+      fprintf(stderr, "\n");
+    }
+    cudaFreeHost(c->h_tline);
   }
   void* bufs[] = {c->d_model, c->d_layers, c->d_sync, c->d_part, c->d_att_o, c->d_att_ml};
   for (void* p : bufs) if (p) cudaFree(p);
@@ -806,6 +919,22 @@ bool mega_create(fdvlm_t* h) {
   mm.tq_begin[3] = mm.tq_begin[2] + ceil_div(NKV, 128);
   mm.T_o = ceil_div(H, 128); mm.T_g = ceil_div(I, 64); mm.T_l = ceil_div(cf.vocab, 128);
   mm.KB_h = ceil_div(H, 64); mm.KB_q = ceil_div(NQ, 64); mm.KB_i = ceil_div(I, 64);
+  // work partition per operator kind: whole tiles for QKV / O / gate-up (direct epilogues), a small split for the
+  // down projection (few tiles, long K), stream-K for the LM head
+  {
+    const int G = c->grid;
+    const int T[5] = {mm.tq_begin[3], mm.T_o, mm.T_g, mm.T_o, mm.T_l};
+    const int KB[5] = {mm.KB_h, mm.KB_q, mm.KB_h, mm.KB_i, mm.KB_h};
+    for (int k = 0; k < 5; ++k) {
+      int sk = 1;
+      if (k == OP_D) { sk = (G / 2) / T[k]; if (sk > KB[k] / 8) sk = KB[k] / 8; if (sk < 1) sk = 1; }
+      if (k == OP_LM) sk = KB[k];
+      const long long W = (long long)T[k] * sk;
+      mm.op_sk[k] = sk;
+      mm.op_ge[k] = W < G ? (int)W : G;
+      mm.op_off[k] = (k == OP_O) ? 3 : (k == OP_D ? 5 : 0);
+    }
+  }
   mm.off_to = C_TILES + mm.tq_begin[3]; mm.off_tg = mm.off_to + mm.T_o; mm.off_td = mm.off_tg + mm.T_g;
   mm.layer_stride = ((mm.off_td + mm.T_o + 31) / 32) * 32;
   mm.off_lm = mm.layer_stride + 32;   // relative to the last layer's counters
@@ -814,8 +943,13 @@ bool mega_create(fdvlm_t* h) {
   // attention partials: worst case over the block sizes this handle may see
   size_t worst = 0;
   for (int n = 1; n <= R; ++n) {
+    // the chunk count of a shorter sequence can exceed that of max_seq (chunks are whole key tiles), so take its bound
     const MgAttPlan p = mg_att_plan(n, cf.max_seq, cf.n_q_heads, cf.n_kv_heads, c->grid);
-    const size_t slots = (size_t)cf.n_q_heads * n * p.n_chunks;
+    int bound = c->grid / (cf.n_kv_heads * p.groups);
+    const int tiles_max = ceil_div(cf.max_seq, AT_KEYS);
+    if (bound > tiles_max) bound = tiles_max;
+    if (bound < 1) bound = 1;
+    const size_t slots = (size_t)cf.n_q_heads * n * bound;
     if (slots > worst) worst = slots;
   }
   bool alloc_ok = cudaMalloc((void**)&c->d_model, sizeof(MgModel)) == cudaSuccess &&
@@ -829,7 +963,14 @@ bool mega_create(fdvlm_t* h) {
     memset(c->h_trace, 0, 64);
     void* dp = nullptr;
     if (cudaHostGetDevicePointer(&dp, c->h_trace, 0) == cudaSuccess) mm.trace = (int*)dp;
+    c->n_ops = cf.n_layers * 4 + 1;
+    if (cudaHostAlloc((void**)&c->h_tline, (size_t)c->n_ops * 64, cudaHostAllocMapped) == cudaSuccess) {
+      memset(c->h_tline, 0, (size_t)c->n_ops * 64);
+      if (cudaHostGetDevicePointer(&dp, c->h_tline, 0) == cudaSuccess) mm.tline = (long long*)dp;
+    }
   }
+  mm.trace_cta = -1;
+  if (mm.tline) { const char* tc = getenv("FDVLM_MEGA_TRACE_CTA"); mm.trace_cta = tc ? atoi(tc) : 0; }
   if (alloc_ok) {
     mm.layers = c->d_layers; mm.sync = c->d_sync; mm.part = c->d_part; mm.att_o = c->d_att_o; mm.att_ml = c->d_att_ml;
     alloc_ok = cudaMemcpy(c->d_layers, layers.data(), sizeof(MgLayer) * cf.n_layers, cudaMemcpyHostToDevice) == cudaSuccess &&
