@@ -39,7 +39,6 @@
 namespace fdk {
 
 constexpr int MG_THREADS = 224;
-constexpr int MG_NX = 4;                 // activation ring stages
 constexpr int MG_W_BYTES = 16384;        // one weight stage: 128 rows x 64 k bf16
 constexpr long long MG_TIMEOUT = 1ll << 29;  // clock cycles (~0.3 s) before a global wait gives up
 constexpr int MG_SMEM_LIMIT = 232448;    // 227 KB
@@ -57,9 +56,16 @@ struct alignas(128) MgLayer {
   bf16 *kc, *vc;                              // cache planes [Hkv][max_seq][d]
 };
 
+// Tensor maps live in global memory (they are too many for the parameter block) ...
 struct alignas(128) MgModel {
   CUtensorMap tm_lm;
   CUtensorMap tm_xg[4], tm_ao[4], tm_act[4];  // activation maps, box {64 k, 16 / 32 / 48 / 64 rows}
+};
+static_assert(sizeof(MgLayer) % 128 == 0 && sizeof(CUtensorMap) == 128, "tensor maps must stay 128-byte aligned");
+
+// ... everything else the kernel reads travels by value in the parameter block (constant bank): a field kept in
+// global memory would have to be re-read after every global store of an epilogue loop.
+struct MgConst {
   const MgLayer* layers;
   int n_layers, H, I, NQ, NKV, hq, hkv, d, vocab, mask_id, max_seq, nt;
   float eps, inv_h;
@@ -68,7 +74,7 @@ struct alignas(128) MgModel {
   bf16 *xg, *q, *ao, *act;
   float* ssq;          // [R][nt]
   const float2* cs;    // [R][d/2]
-  float* part;         // [grid * 2][64][128] stream-K partial slots
+  float* part;         // [grid * 2][64][128] split-K partial slots
   float* att_o;
   float2* att_ml;
   float* logits;
@@ -83,10 +89,10 @@ struct alignas(128) MgModel {
   int layer_stride, off_to, off_tg, off_td, off_lm;
   int op_sk[5], op_ge[5], op_off[5];   // per operator kind: K-splits per tile, participating CTAs, first CTA
 };
-static_assert(sizeof(MgLayer) % 128 == 0 && sizeof(CUtensorMap) == 128, "tensor maps must stay 128-byte aligned");
 
 struct MgRun {
   const MgModel* M;
+  MgConst c;
   int m, L, causal;
   int lm_rows;         // 0: no LM head; 1: last row only; m: every row
   int write_logits;
@@ -195,21 +201,29 @@ __device__ __forceinline__ void tl_mark(long long* tl, bool on, int op, int slot
   }
 }
 
+// Shared memory: [weight ring][region R][barriers].  Region R holds the attention tiles while the epilogue group
+// runs attention, and the activation ring plus the epilogues' exchange buffer while GEMMs run: the two never overlap
+// in time inside a CTA (attention starts only after every QKV tile of the grid is finished, and the next
+// activation load waits for the counter that every CTA bumps after its attention work).
 template <int M_PAD, int D>
 struct MgSmem {
   static constexpr int X_BYTES = M_PAD * 128;
-  static constexpr int ATT_BYTES = attn_smem_bytes<D>() > M_PAD * 132 * 4 ? attn_smem_bytes<D>() : M_PAD * 132 * 4;   // also the epilogues' exchange buffer
+  static constexpr int NX = M_PAD <= 32 ? 12 : (M_PAD <= 48 ? 8 : 5);       // activation ring stages
+  static constexpr int XCH_OFF = NX * X_BYTES;                               // exchange buffer inside region R
+  static constexpr int XCH_BYTES = ((M_PAD * 132 * 4 + 1023) / 1024) * 1024;
+  static constexpr int GEMM_BYTES = XCH_OFF + XCH_BYTES;
+  static constexpr int ATT_BYTES = attn_smem_bytes<D>() > GEMM_BYTES ? attn_smem_bytes<D>() : GEMM_BYTES;
   static constexpr int BAR_BYTES = 2048;
-  static constexpr int NW_RAW = (MG_SMEM_LIMIT - 1024 - BAR_BYTES - ATT_BYTES - MG_NX * X_BYTES) / MG_W_BYTES;
+  static constexpr int NW_RAW = (MG_SMEM_LIMIT - 1024 - BAR_BYTES - ATT_BYTES) / MG_W_BYTES;
   static constexpr int NW = NW_RAW > 12 ? 12 : NW_RAW;
   static constexpr int W_OFF = 0;
-  static constexpr int X_OFF = NW * MG_W_BYTES;
-  static constexpr int ATT_OFF = X_OFF + MG_NX * X_BYTES;
+  static constexpr int ATT_OFF = NW * MG_W_BYTES;
+  static constexpr int X_OFF = ATT_OFF;
   static constexpr int BAR_OFF = ATT_OFF + ATT_BYTES;
   static constexpr int TOTAL = BAR_OFF + BAR_BYTES + 1024;
 };
 
-__device__ __forceinline__ Part op_part(const MgModel& M, int kind, int G) {
+__device__ __forceinline__ Part op_part(const MgConst& M, int kind, int G) {
   Part g;
   switch (kind) {
     case OP_QKV: g.T = M.tq_begin[3]; g.KB = M.KB_h; break;
@@ -299,7 +313,7 @@ __device__ __forceinline__ void attn_merge_warp(const float* att_o, const float2
 template <int M_PAD, int D>
 __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun Rp) {
   using S = MgSmem<M_PAD, D>;
-  constexpr int NW = S::NW;
+  constexpr int NW = S::NW, MG_NX = S::NX;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -308,13 +322,13 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
   // barrier slots (8 bytes each)
   const uint32_t w_full0 = bar0, w_empty0 = bar0 + 8u * NW, x_full0 = bar0 + 8u * (2 * NW), x_empty0 = bar0 + 8u * (2 * NW + MG_NX);
   const uint32_t t_full0 = bar0 + 8u * (2 * NW + 2 * MG_NX), t_empty0 = t_full0 + 16u;
-  constexpr int MISC = 8 * (2 * 12 + 2 * MG_NX + 4);   // 288
+  constexpr int MISC = 8 * (2 * 12 + 2 * 12 + 4);   // past the largest barrier set
   volatile uint32_t* tmem_slot = (volatile uint32_t*)(sm + S::BAR_OFF + MISC);
   volatile int* abort_flag = (volatile int*)(sm + S::BAR_OFF + MISC + 8);
   volatile int* s_flag = (volatile int*)(sm + S::BAR_OFF + MISC + 16);     // epilogue group broadcast word
   float* s_rstd = (float*)(sm + S::BAR_OFF + MISC + 32);                    // [64]
   float* s_red = s_rstd + 64;                                               // [4][M_PAD <= 64]
-  float* s_xch = (float*)(sm + S::ATT_OFF);                                 // [M_PAD][<=132] exchange (GEMM epilogues only)
+  float* s_xch = (float*)(sm + S::ATT_OFF + S::XCH_OFF);                                 // [M_PAD][<=132] exchange (GEMM epilogues only)
 
   // the run description in registers
   const MgModel* const Mp = Rp.M;
@@ -341,12 +355,12 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
-  int* const sync = M.sync;
-  const int* const status = M.status;
-  const int* const trace = M.trace;
-  long long* const tl = M.tline;
-  const bool tl_on = (cta == M.trace_cta);
-  const int n_layers = M.n_layers, layer_stride = M.layer_stride, T_o = M.T_o, T_g = M.T_g;
+  int* const sync = Rp.c.sync;
+  const int* const status = Rp.c.status;
+  const int* const trace = Rp.c.trace;
+  long long* const tl = Rp.c.tline;
+  const bool tl_on = (cta == Rp.c.trace_cta);
+  const int n_layers = Rp.c.n_layers, layer_stride = Rp.c.layer_stride, T_o = Rp.c.T_o, T_g = Rp.c.T_g;
   const int mpi = M_PAD / 16 - 1;
 
   if (warp == 0) {
@@ -359,8 +373,8 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
       OpIter ops(n_layers, r_lm_rows);
       while (ok && ops.next()) {
         const int kind = ops.kind, l = ops.l;
-        const Part g = op_part(M, kind, G);
-        const MgLayer* Ly = &M.layers[kind == OP_LM ? 0 : l];
+        const Part g = op_part(Rp.c, kind, G);
+        const MgLayer* Ly = &Rp.c.layers[kind == OP_LM ? 0 : l];
         trace_mark(trace, cta, 0, l * 4 + kind, 1);
         switch (kind) {
           case OP_QKV: tensormap_acquire(&Ly->tm_q); tensormap_acquire(&Ly->tm_k); tensormap_acquire(&Ly->tm_v); break;
@@ -376,9 +390,9 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
           int r0 = tile * TC_BM;
           if (kind == OP_QKV) {
             int mi = 0;
-            while (mi < 2 && tile >= M.tq_begin[mi + 1]) ++mi;
+            while (mi < 2 && tile >= Rp.c.tq_begin[mi + 1]) ++mi;
             tm = mi == 0 ? &Ly->tm_q : (mi == 1 ? &Ly->tm_k : &Ly->tm_v);
-            r0 = (tile - M.tq_begin[mi]) * TC_BM;
+            r0 = (tile - Rp.c.tq_begin[mi]) * TC_BM;
           } else if (kind == OP_O) tm = &Ly->tm_o;
           else if (kind == OP_D) tm = &Ly->tm_d;
           for (int kb = kb0; kb < kb1; ++kb) {
@@ -405,7 +419,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
         tl_mark(tl, tl_on, l * 4 + kind, 7);
       }
       if (!ok) {
-        atomicCAS(M.status, 0, MG_ERR_WPROD);
+        atomicCAS(Rp.c.status, 0, MG_ERR_WPROD);
         for (int s = 0; s < NW; ++s) {
           if (!(armed & (1u << s))) continue;
           const uint32_t par = (armed_parity >> s) & 1u;
@@ -427,7 +441,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
       OpIter ops(n_layers, r_lm_rows);
       while (ok && ops.next()) {
         const int kind = ops.kind, l = ops.l;
-        const Part g = op_part(M, kind, G);
+        const Part g = op_part(Rp.c, kind, G);
         const int* lc = sync + (size_t)(kind == OP_LM ? l - 1 : l) * layer_stride;
         const CUtensorMap* tm = &M.tm_xg[mpi];
         const int* flag = lc;
@@ -460,7 +474,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
         tl_mark(tl, tl_on, l * 4 + kind, 5);
       }
       if (!ok) {
-        atomicCAS(M.status, 0, MG_ERR_XPROD);
+        atomicCAS(Rp.c.status, 0, MG_ERR_XPROD);
         for (int s = 0; s < MG_NX; ++s) {
           if (!(armed & (1u << s))) continue;
           const uint32_t par = (armed_parity >> s) & 1u;
@@ -480,7 +494,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
       while (ok && ops.next()) {
         const int kind = ops.kind, l = ops.l;
         trace_mark(trace, cta, 2, l * 4 + kind, 1);
-        const Part g = op_part(M, kind, G);
+        const Part g = op_part(Rp.c, kind, G);
         SegIter seg(g, cta);
         int tile, kb0, kb1;
         while (ok && seg.next(tile, kb0, kb1)) {
@@ -507,35 +521,43 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
           if (ok) umma_commit(t_full0 + 8u * acc);
         }
       }
-      if (!ok) atomicCAS(M.status, 0, MG_ERR_MMA);
+      if (!ok) atomicCAS(Rp.c.status, 0, MG_ERR_MMA);
     }
   } else {
     // ================================ epilogue group (warps 2..5, 128 threads) ================================
     const int q = warp & 3;                       // tensor-memory lane quarter this warp may read
     const int et = q * 32 + lane;                 // accumulator row held by this thread (0..127)
     const int etid = (warp - 2) * 32 + lane;      // index inside the group
-    const int nt = M.nt, hq = M.hq, hkv = M.hkv, max_seq = M.max_seq, H = M.H, I = M.I, vocab = M.vocab, mask_id = M.mask_id;
-    const float inv_h = M.inv_h, eps = M.eps;
+    const int nt = Rp.c.nt, hq = Rp.c.hq, hkv = Rp.c.hkv, max_seq = Rp.c.max_seq, H = Rp.c.H, I = Rp.c.I, vocab = Rp.c.vocab, mask_id = Rp.c.mask_id;
+    const float inv_h = Rp.c.inv_h, eps = Rp.c.eps;
     int nseg = 0;
     bool ok = true;
     OpIter ops(n_layers, r_lm_rows);
     while (ok && ops.next()) {
       const int kind = ops.kind, l = ops.l;
-      const Part g = op_part(M, kind, G);
+      const Part g = op_part(Rp.c, kind, G);
       int* lc = sync + (size_t)(kind == OP_LM ? l - 1 : l) * layer_stride;
-      const MgLayer* Ly = &M.layers[kind == OP_LM ? 0 : l];
+      const MgLayer* Ly = &Rp.c.layers[kind == OP_LM ? 0 : l];
+      // per-layer pointers of this operator, read once (the layer table is in global memory)
+      bf16* const kc = Ly->kc;
+      bf16* const vc = Ly->vc;
+      const float* const bq = (kind == OP_QKV) ? Ly->bq : nullptr;
+      const float* const bk = (kind == OP_QKV) ? Ly->bk : nullptr;
+      const float* const bv = (kind == OP_QKV) ? Ly->bv : nullptr;
+      const float* const res_gain = (kind == OP_O) ? Ly->g_mlp
+                                    : (kind == OP_D ? (l + 1 < n_layers ? Rp.c.layers[l + 1].g_attn : Rp.c.g_final) : nullptr);
       const int m = (kind == OP_LM) ? r_lm_rows : r_m;
       const int xrow0 = (kind == OP_LM) ? r_m - r_lm_rows : 0;
       if (etid == 0) { trace_mark(trace, cta, 3, l * 4 + kind, 1); tl_mark(tl, tl_on, l * 4 + kind, 0); }
 
       if (kind == OP_O) {
         // ---------------- attention of this layer: split-KV items, then the merge of the key chunks ----------------
-        if (!group_wait(lc + C_QKV, M.tq_begin[3], etid, s_flag, abort_flag, status)) { ok = false; break; }
+        if (!group_wait(lc + C_QKV, Rp.c.tq_begin[3], etid, s_flag, abort_flag, status)) { ok = false; break; }
         const int n_items = hkv * r_groups * r_n_chunks;
         for (int item = cta; item < n_items; item += G) {
           const int chunk = item % r_n_chunks, rest = item / r_n_chunks;
           const int grp = rest % r_groups, hk = rest / r_groups;
-          attn_item<D>(M.q, Ly->kc, Ly->vc, M.att_o, M.att_ml, r_m, r_L, max_seq, hq, hkv, r_qh, r_chunk_keys, r_n_chunks,
+          attn_item<D>(Rp.c.q, kc, vc, Rp.c.att_o, Rp.c.att_ml, r_m, r_L, max_seq, hq, hkv, r_qh, r_chunk_keys, r_n_chunks,
                        r_causal, chunk, grp, hk, base + S::ATT_OFF, etid);
         }
         if (etid == 0) trace_mark(trace, cta, 3, l * 4 + kind, 2);
@@ -545,7 +567,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
         // one warp per (row, head): the CTA's four warps take consecutive pairs
         for (int p = cta * 4 + (warp - 2); p < r_m * hq; p += G * 4) {
           const int i = p / hq, head = p % hq;
-          attn_merge_warp<D>(M.att_o, M.att_ml, M.ao + ((size_t)i * hq + head) * D, ((size_t)head * r_m + i) * r_n_chunks, r_n_chunks, lane);
+          attn_merge_warp<D>(Rp.c.att_o, Rp.c.att_ml, Rp.c.ao + ((size_t)i * hq + head) * D, ((size_t)head * r_m + i) * r_n_chunks, r_n_chunks, lane);
         }
         group_signal(lc + C_AO, etid);
         if (etid == 0) { trace_mark(trace, cta, 3, l * 4 + kind, 4); tl_mark(tl, tl_on, l * 4 + kind, 1); }
@@ -565,7 +587,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
         // inputs of the epilogues that do not depend on this operator's own MMAs are fetched while those run
         if (wants_rstd) {
           if (!group_wait(rstd_flag, rstd_target, etid, s_flag, abort_flag, status)) { ok = false; break; }
-          load_rstd(M.ssq, nt, inv_h, eps, s_rstd, xrow0, m, etid);
+          load_rstd(Rp.c.ssq, nt, inv_h, eps, s_rstd, xrow0, m, etid);
           have_rstd = true;
         } else if (is_resid) {
           // the residual rows this operator adds to: complete once the previous residual operator has finished
@@ -581,7 +603,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
         if (is_resid) {
           const int c = tile * TC_BM + et;
 #pragma unroll
-          for (int b = 0; b < M_PAD; ++b) hold[b] = (c < H && b < m) ? __ldcg(&M.h[(size_t)b * H + c]) : 0.f;
+          for (int b = 0; b < M_PAD; ++b) hold[b] = (c < H && b < m) ? __ldcg(&Rp.c.h[(size_t)b * H + c]) : 0.f;
         }
         if (etid == 0) *s_flag = mbar_wait(t_full0 + 8u * acc, acc_phase, abort_flag) ? 1 : 0;
         epi_bar();
@@ -601,14 +623,14 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
         if (!(kb0 == 0 && kb1 == g.KB)) {
           const int me = g.logical(cta);
           const int first_tile = (int)(g.start(me) / g.SK);
-          float* mine = M.part + ((size_t)(cta * 2 + (tile == first_tile ? 0 : 1)) * 64) * 128;
+          float* mine = Rp.c.part + ((size_t)(cta * 2 + (tile == first_tile ? 0 : 1)) * 64) * 128;
 #pragma unroll
           for (int b = 0; b < M_PAD; ++b)
             if (b < m) mine[b * 128 + et] = v[b];
           __threadfence();
           epi_bar();
           const int cf = g.owner((long long)tile * g.SK), cl = g.owner((long long)tile * g.SK + g.SK - 1);
-          int* tcnt = lc + (kind == OP_LM ? M.off_lm : (kind == OP_QKV ? (int)C_TILES : (kind == OP_O ? M.off_to : (kind == OP_GU ? M.off_tg : M.off_td)))) + tile;
+          int* tcnt = lc + (kind == OP_LM ? Rp.c.off_lm : (kind == OP_QKV ? (int)C_TILES : (kind == OP_O ? Rp.c.off_to : (kind == OP_GU ? Rp.c.off_tg : Rp.c.off_td)))) + tile;
           if (etid == 0) *s_flag = (atomicAdd(tcnt, 1) == cl - cf) ? 1 : 0;
           epi_bar();
           const bool last = *s_flag != 0;
@@ -624,7 +646,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
             for (int u2 = 0; u2 < CU; ++u2) {
               const int c3 = (c2 + u2 <= cl) ? c2 + u2 : cl;
               const int ft = (int)(g.start(c3) / g.SK);
-              const float* src = M.part + ((size_t)(g.phys(c3) * 2 + (tile == ft ? 0 : 1)) * 64) * 128;
+              const float* src = Rp.c.part + ((size_t)(g.phys(c3) * 2 + (tile == ft ? 0 : 1)) * 64) * 128;
 #pragma unroll
               for (int b = 0; b < M_PAD; ++b) pv[u2][b] = (b < m) ? __ldcg(&src[b * 128 + et]) : 0.f;
             }
@@ -641,11 +663,11 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
         // ---- operator epilogue on a complete tile: v[b] = sum_k w[row et of the tile][k] x[b][k] ----
         if (kind == OP_QKV) {
           int mi = 0;
-          while (mi < 2 && tile >= M.tq_begin[mi + 1]) ++mi;
-          const int n = (tile - M.tq_begin[mi]) * TC_BM + et;          // feature inside its matrix
-          const int n_out = (mi == 0) ? M.NQ : M.NKV;
+          while (mi < 2 && tile >= Rp.c.tq_begin[mi + 1]) ++mi;
+          const int n = (tile - Rp.c.tq_begin[mi]) * TC_BM + et;          // feature inside its matrix
+          const int n_out = (mi == 0) ? Rp.c.NQ : Rp.c.NKV;
           const bool in_range = n < n_out;
-          const float* bias = (mi == 0) ? Ly->bq : (mi == 1 ? Ly->bk : Ly->bv);
+          const float* bias = (mi == 0) ? bq : (mi == 1 ? bk : bv);
           const float bi = (in_range && bias) ? bias[n] : 0.f;
           const int head = n / D, j = n % D;
           constexpr int half = D / 2;
@@ -663,7 +685,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
             for (int b = 0; b < M_PAD; ++b) {
               if (b < m) {
                 const float other = s_xch[b * 128 + pt];
-                const float2 c = M.cs[b * half + jj];
+                const float2 c = Rp.c.cs[b * half + jj];
                 v[b] = lo ? v[b] * c.x - other * c.y : v[b] * c.x + other * c.y;
               }
             }
@@ -672,18 +694,18 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
           if (in_range) {
             bf16* dst;
             size_t stride;
-            if (mi == 0) { dst = M.q + (size_t)head * D + j; stride = (size_t)hq * D; }
-            else { dst = (mi == 1 ? Ly->kc : Ly->vc) + ((size_t)head * max_seq + r_L) * D + j; stride = D; }
+            if (mi == 0) { dst = Rp.c.q + (size_t)head * D + j; stride = (size_t)hq * D; }
+            else { dst = (mi == 1 ? kc : vc) + ((size_t)head * max_seq + r_L) * D + j; stride = D; }
 #pragma unroll
             for (int b = 0; b < M_PAD; ++b)
               if (b < m) dst[(size_t)b * stride] = __float2bfloat16_rn(v[b]);
           }
+          if (etid == 0) tl_mark(tl, tl_on, l * 4 + kind, 1);
           group_signal(lc + C_QKV, etid);
         } else if (kind == OP_O || kind == OP_D) {
           const int c = tile * TC_BM + et;
           const bool in_range = c < H;
-          const float* gain = (kind == OP_O) ? Ly->g_mlp : (l + 1 < n_layers ? M.layers[l + 1].g_attn : M.g_final);
-          const float gn = in_range ? gain[c] : 0.f;
+          const float gn = in_range ? res_gain[c] : 0.f;
           // squares go through shared memory ([row][132]: 4 x 33 per row, conflict-free both ways) for the per-row sums
 #pragma unroll
           for (int b = 0; b < M_PAD; ++b) {
@@ -691,8 +713,8 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
               const float hv = hold[b] + v[b];
               if (in_range) {
                 const size_t idx = (size_t)b * H + c;
-                M.h[idx] = hv;
-                M.xg[idx] = __float2bfloat16_rn(hv * gn);
+                Rp.c.h[idx] = hv;
+                Rp.c.xg[idx] = __float2bfloat16_rn(hv * gn);
               }
               s_xch[b * 132 + (warp - 2) * 33 + lane] = in_range ? hv * hv : 0.f;
             }
@@ -706,7 +728,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
             s_red[part * M_PAD + b] = ss;
           }
           epi_bar();
-          if (etid < m) M.ssq[(size_t)etid * nt + tile] = s_red[etid] + s_red[M_PAD + etid] + s_red[2 * M_PAD + etid] + s_red[3 * M_PAD + etid];
+          if (etid < m) Rp.c.ssq[(size_t)etid * nt + tile] = s_red[etid] + s_red[M_PAD + etid] + s_red[2 * M_PAD + etid] + s_red[3 * M_PAD + etid];
           group_signal(lc + (kind == OP_O ? C_H2 : C_HOUT), etid);
         } else if (kind == OP_GU) {
           const int col = tile * 64 + q * 16 + (lane & 15);
@@ -717,9 +739,10 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
             if (live && b < m) {
               const float rs = s_rstd[b];
               const float gt = v[b] * rs;
-              M.act[(size_t)b * I + col] = __float2bfloat16_rn(gt / (1.f + __expf(-gt)) * (other * rs));
+              Rp.c.act[(size_t)b * I + col] = __float2bfloat16_rn(gt / (1.f + __expf(-gt)) * (other * rs));
             }
           }
+          if (etid == 0) tl_mark(tl, tl_on, l * 4 + kind, 1);
           group_signal(lc + C_ACT, etid);
         } else {
           const int n = tile * TC_BM + et;                    // vocabulary id held by this thread
@@ -729,7 +752,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
           for (int b = 0; b < M_PAD; ++b) {
             if (b >= m) break;                                // uniform across the group
             const float lg = v[b] * s_rstd[b];
-            if (r_write_logits && in_range) M.logits[(size_t)b * vocab + n] = lg;
+            if (r_write_logits && in_range) Rp.c.logits[(size_t)b * vocab + n] = lg;
             float mx = counted ? lg : -INFINITY;
             int ix = counted ? n : 0x7fffffff;
 #pragma unroll
@@ -740,13 +763,13 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
             }
             float e = (counted && mx > -INFINITY) ? __expf(lg - mx) : 0.f;
             e = warp_sum(e);
-            if (lane == 0) M.stats[(size_t)(tile * 4 + q) * m + b] = make_float4(mx, e, __int_as_float(ix), 0.f);
+            if (lane == 0) Rp.c.stats[(size_t)(tile * 4 + q) * m + b] = make_float4(mx, e, __int_as_float(ix), 0.f);
           }
         }
       }
       if (etid == 0) tl_mark(tl, tl_on, l * 4 + kind, 3);
     }
-    if (!ok && etid == 0) atomicCAS(M.status, 0, MG_ERR_EPI);
+    if (!ok && etid == 0) atomicCAS(Rp.c.status, 0, MG_ERR_EPI);
   }
 
   // ---- teardown: every thread arrives here, whatever happened ----
@@ -797,6 +820,7 @@ struct MegaCtx {
   float* d_att_o = nullptr;
   float2* d_att_ml = nullptr;
   size_t sync_bytes = 0;
+  MgConst cst;              // by-value part of the kernel parameter
   int* h_trace = nullptr;   // host-mapped, only with FDVLM_MEGA_TRACE=1
   long long* h_tline = nullptr;
   int n_ops = 0;
@@ -888,7 +912,9 @@ bool mega_create(fdvlm_t* h) {
 
   MegaCtx* c = new MegaCtx;
   c->grid = sms;
-  MgModel mm;
+  MgModel mt;               // tensor maps (device copy)
+  memset(&mt, 0, sizeof(mt));
+  MgConst& mm = c->cst;
   memset(&mm, 0, sizeof(mm));
   std::vector<MgLayer> layers(cf.n_layers);
   bool ok = true;
@@ -904,10 +930,10 @@ bool mega_create(fdvlm_t* h) {
   }
   const void* table = cf.tie_embeddings ? h->w.embed : h->w.lm_head;
   const int R = cf.max_block;
-  ok = ok && mg_tmap(&mm.tm_lm, table, cf.vocab, H, 128);
+  ok = ok && mg_tmap(&mt.tm_lm, table, cf.vocab, H, 128);
   for (int i = 0; i < 4 && ok; ++i)
-    ok = mg_tmap(&mm.tm_xg[i], h->a, R, H, 16 * (i + 1)) && mg_tmap(&mm.tm_ao[i], h->ao, R, NQ, 16 * (i + 1)) &&
-         mg_tmap(&mm.tm_act[i], h->act, R, I, 16 * (i + 1));
+    ok = mg_tmap(&mt.tm_xg[i], h->a, R, H, 16 * (i + 1)) && mg_tmap(&mt.tm_ao[i], h->ao, R, NQ, 16 * (i + 1)) &&
+         mg_tmap(&mt.tm_act[i], h->act, R, I, 16 * (i + 1));
   if (!ok) { delete c; return false; }
 
   mm.n_layers = cf.n_layers; mm.H = H; mm.I = I; mm.NQ = NQ; mm.NKV = NKV; mm.hq = cf.n_q_heads; mm.hkv = cf.n_kv_heads;
@@ -974,7 +1000,7 @@ bool mega_create(fdvlm_t* h) {
   if (alloc_ok) {
     mm.layers = c->d_layers; mm.sync = c->d_sync; mm.part = c->d_part; mm.att_o = c->d_att_o; mm.att_ml = c->d_att_ml;
     alloc_ok = cudaMemcpy(c->d_layers, layers.data(), sizeof(MgLayer) * cf.n_layers, cudaMemcpyHostToDevice) == cudaSuccess &&
-               cudaMemcpy(c->d_model, &mm, sizeof(MgModel), cudaMemcpyHostToDevice) == cudaSuccess;
+               cudaMemcpy(c->d_model, &mt, sizeof(MgModel), cudaMemcpyHostToDevice) == cudaSuccess;
   }
   h->mega = c;
   if (!alloc_ok) {
@@ -993,7 +1019,7 @@ int mega_forward(fdvlm_t* h, int n, int mode, int logits_rows, int want_logits) 
   CU(h, cudaMemsetAsync(c->d_sync, 0, c->sync_bytes, h->st));
   const MgAttPlan p = mg_att_plan(n, h->cache_len + n, cf.n_q_heads, cf.n_kv_heads, c->grid);
   MgRun run;
-  run.M = c->d_model; run.m = n; run.L = h->cache_len; run.causal = (mode == MODE_CAUSAL);
+  run.M = c->d_model; run.c = c->cst; run.m = n; run.L = h->cache_len; run.causal = (mode == MODE_CAUSAL);
   run.lm_rows = (logits_rows == 0) ? 0 : (logits_rows == n ? n : 1);
   run.write_logits = (logits_rows == n) ? want_logits : 1;
   run.qh = p.qh; run.att_groups = p.groups; run.chunk_keys = p.chunk_keys; run.n_chunks = p.n_chunks;
