@@ -32,9 +32,8 @@ extern "C" const char* fdvlm_last_error(const fdvlm_t* h) { return h ? h->err : 
 extern "C" void fdvlm_destroy(fdvlm_t* h) {
   if (!h) return;
   mega_destroy(h);
-  void* bufs[] = {h->kv, h->h, h->a, h->ao, h->act, h->q, h->y, h->cs, h->ssq, h->stats, h->logits, h->conf, h->pred,
-                  h->unmask, h->blk_tokens, h->blk_masked, h->info, h->init_stage, h->ws};
-  for (void* p : bufs) if (p) cudaFree(p);
+  if (h->kv) cudaFree(h->kv);
+  if (h->slab) cudaFree(h->slab);
   for (cudaEvent_t ev : h->prof_ev) cudaEventDestroy(ev);
   if (h->info_host) cudaFreeHost(h->info_host);
   if (h->host_stage) cudaFreeHost(h->host_stage);
@@ -84,6 +83,8 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
   h->blk_masked = nullptr; h->info = nullptr; h->init_stage = nullptr; h->ws = nullptr; h->info_host = nullptr;
   h->host_stage = nullptr;
   h->mega = nullptr;
+  h->slab = nullptr;
+  h->mega_slab = nullptr;
   cudaGetDevice(&h->device);
 
   const int R = cfg->max_block, H = cfg->hidden, I = cfg->intermediate, d = cfg->head_dim;
@@ -101,35 +102,42 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
     for (size_t b : g3) if (b > ws) ws = b;
   }
   h->ws_bytes = ws;
+  // Every buffer but the KV cache is carved out of one slab, the small hot ones first: with gigabytes of weights
+  // streaming through the TLBs, each separately allocated buffer would cost its own page walk whenever it is touched.
   struct { void** p; size_t bytes; } allocs[] = {
-      {(void**)&h->kv, (size_t)cfg->n_layers * 2 * kv_plane(h)},
-      {(void**)&h->h, (size_t)R * H * 4},
-      {(void**)&h->a, (size_t)R * H * h->act_sz},
-      {(void**)&h->ao, (size_t)R * NQ * h->act_sz},
-      {(void**)&h->act, (size_t)R * I * h->act_sz},
-      {(void**)&h->q, (size_t)R * NQ * h->act_sz},
-      {(void**)&h->y, (size_t)R * (NQKV > 2 * I ? NQKV : 2 * I) * 4},
-      {(void**)&h->cs, (size_t)R * d * 4},
-      {(void**)&h->ssq, (size_t)R * h->nt * 4},
-      {(void**)&h->stats, (size_t)((cfg->vocab + 127) / 128) * 4 * R * 16},
-      {(void**)&h->logits, (size_t)R * cfg->vocab * 4},
+      {(void**)&h->info, 16},
       {(void**)&h->conf, (size_t)R * 4},
       {(void**)&h->pred, (size_t)R * 4},
       {(void**)&h->unmask, 64},
       {(void**)&h->blk_tokens, 64 * 4},
       {(void**)&h->blk_masked, 64},
-      {(void**)&h->info, 16},
       {(void**)&h->init_stage, 64 * 4},
+      {(void**)&h->ssq, (size_t)R * h->nt * 4},
+      {(void**)&h->cs, (size_t)R * d * 4},
+      {(void**)&h->mega_slab, mega_slab_bytes(h)},
+      {(void**)&h->h, (size_t)R * H * 4},
+      {(void**)&h->a, (size_t)R * H * h->act_sz},
+      {(void**)&h->ao, (size_t)R * NQ * h->act_sz},
+      {(void**)&h->q, (size_t)R * NQ * h->act_sz},
+      {(void**)&h->act, (size_t)R * I * h->act_sz},
+      {(void**)&h->stats, (size_t)((cfg->vocab + 127) / 128) * 4 * R * 16},
+      {(void**)&h->y, (size_t)R * (NQKV > 2 * I ? NQKV : 2 * I) * 4},
       {(void**)&h->ws, ws ? ws : 16},
+      {(void**)&h->logits, (size_t)R * cfg->vocab * 4},
   };
-  for (auto& a : allocs) {
-    e = cudaMalloc(a.p, a.bytes);
-    if (e != cudaSuccess) {
-      fail(nullptr, FDVLM_ERR_OOM, "cudaMalloc of %zu bytes failed: %s", a.bytes, cudaGetErrorString(e));
-      cudaGetLastError();
-      fdvlm_destroy(h);
-      return FDVLM_ERR_OOM;
-    }
+  size_t slab_bytes = 0;
+  for (auto& a : allocs) slab_bytes += (a.bytes + 255) / 256 * 256;
+  e = cudaMalloc((void**)&h->slab, slab_bytes);
+  if (e == cudaSuccess) e = cudaMalloc((void**)&h->kv, (size_t)cfg->n_layers * 2 * kv_plane(h));
+  if (e != cudaSuccess) {
+    fail(nullptr, FDVLM_ERR_OOM, "cudaMalloc of the work buffers (%zu bytes) or the KV cache failed: %s", slab_bytes, cudaGetErrorString(e));
+    cudaGetLastError();
+    fdvlm_destroy(h);
+    return FDVLM_ERR_OOM;
+  }
+  {
+    char* cur = h->slab;
+    for (auto& a : allocs) { *a.p = cur; cur += (a.bytes + 255) / 256 * 256; }
   }
   if (cudaMallocHost((void**)&h->info_host, 16) != cudaSuccess || cudaMallocHost((void**)&h->host_stage, 64 * 16) != cudaSuccess) {
     fail(nullptr, FDVLM_ERR_OOM, "pinned host allocation failed");

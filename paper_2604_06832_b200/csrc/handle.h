@@ -20,6 +20,8 @@ struct fdvlm {
   size_t act_sz;   // bytes per activation / KV element
   int use_tc;      // bf16 weights: tcgen05 + TMA GEMMs, tensor-core attention, folded norms
   void* mega;      // persistent forward kernel context (null: kernel-per-operator path)
+  char* slab;      // one allocation behind every device buffer below except the KV cache
+  char* mega_slab; // the persistent kernel's share of the slab (counters, tensor maps, partial sums)
   // device buffers (R = max_block rows)
   char* kv;        // [n_layers][2][Hkv][max_seq][d]
   float* h;        // [R, H] residual stream, fp32
@@ -108,6 +110,7 @@ size_t linear_workspace_bytes(int m, int n, int k, int dtype);
 size_t attention_workspace_bytes(int n, int hq, int hkv, int d);
 
 // mega.cu: the persistent whole-forward kernel of the bf16 path
+size_t mega_slab_bytes(const fdvlm_t* h);   // device bytes mega_create will carve out of h->mega_slab
 bool mega_create(fdvlm_t* h);
 void mega_destroy(fdvlm_t* h);
 int mega_forward(fdvlm_t* h, int n, int mode, int logits_rows, int want_logits);

@@ -10,6 +10,10 @@
 //            are complete, then streams the matching activation k-blocks by TMA into a small second ring.
 //   warp 1   MMA issuer: tcgen05.mma, weights = A operand (128 rows), block rows = N, fp32 accumulators in
 //            tensor memory (two buffers).
+//   warp 7   L2 prefetcher: while the latency-bound phases of a layer run (QKV, attention, O) HBM would idle, so
+//            this warp asks for the layer's down-projection and O weights, its K/V cache rows and, later, the next
+//            layer's QKV weights to be brought into L2 (each CTA a 1/grid share); one CTA then streams them at
+//            L2 latency instead of DRAM latency.
 //   warps 2-5 epilogue group: tcgen05.ld, split-K bookkeeping and the fused operator epilogues; the same four
 //            warps run the attention items and the split-KV merge between the QKV and O projections.
 //
@@ -38,7 +42,7 @@
 
 namespace fdk {
 
-constexpr int MG_THREADS = 224;
+constexpr int MG_THREADS = 256;
 constexpr int MG_W_BYTES = 16384;        // one weight stage: 128 rows x 64 k bf16
 constexpr long long MG_TIMEOUT = 1ll << 29;  // clock cycles (~0.3 s) before a global wait gives up
 constexpr int MG_SMEM_LIMIT = 232448;    // 227 KB
@@ -54,12 +58,12 @@ struct alignas(128) MgLayer {
   CUtensorMap tm_g, tm_u;                     // box {64 k, 16 rows}: gate / up rows interleaved per 16
   const float *bq, *bk, *bv, *g_attn, *g_mlp;
   bf16 *kc, *vc;                              // cache planes [Hkv][max_seq][d]
+  const bf16 *wq, *wk, *wv, *wo, *wd;         // raw weight pointers (L2 prefetch)
 };
 
 // Tensor maps live in global memory (they are too many for the parameter block) ...
 struct alignas(128) MgModel {
   CUtensorMap tm_lm;
-  CUtensorMap tm_xg[4], tm_ao[4], tm_act[4];  // activation maps, box {64 k, 16 / 32 / 48 / 64 rows}
 };
 static_assert(sizeof(MgLayer) % 128 == 0 && sizeof(CUtensorMap) == 128, "tensor maps must stay 128-byte aligned");
 
@@ -68,6 +72,7 @@ static_assert(sizeof(MgLayer) % 128 == 0 && sizeof(CUtensorMap) == 128, "tensor 
 struct MgConst {
   const MgLayer* layers;
   int n_layers, H, I, NQ, NKV, hq, hkv, d, vocab, mask_id, max_seq, nt;
+  int R;               // rows allocated in the activation buffers (max_block)
   float eps, inv_h;
   const float* g_final;
   float* h;            // [R][H] residual stream
@@ -82,7 +87,7 @@ struct MgConst {
   int* sync;
   int* status;
   int* trace;          // optional host-mapped words, one per role of CTA 0: (operator index << 8) | step last reached
-  long long* tline;    // optional host-mapped timeline of one traced CTA: [operator][8] globaltimer stamps
+  long long* tline;    // optional host-mapped timeline of one traced CTA: [operator][16] globaltimer stamps
   int trace_cta;
   int tq_begin[4];     // first tile of q, k, v; [3] = T_qkv
   int T_o, T_g, T_l, KB_h, KB_q, KB_i;
@@ -166,6 +171,11 @@ __device__ __forceinline__ int ld_relaxed(const int* p) {
   asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
+__device__ __forceinline__ int atom_add_acq_rel(int* p, int v) {
+  int old;
+  asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+  return old;
+}
 __device__ __forceinline__ void red_release_add(int* p, int v) {
   asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
@@ -175,6 +185,7 @@ __device__ __forceinline__ bool wait_count(const int* p, int target, volatile in
   if (ld_acquire(p) >= target) return true;
   const long long t0 = clock64();
   for (int it = 1;; ++it) {
+    __nanosleep(64);               // a polling thread must not starve the warps that share its scheduler
     if (ld_acquire(p) >= target) return true;
     if (*abort_flag) return false;
     if ((it & 127) == 0 && (ld_relaxed(status) != 0 || clock64() - t0 > MG_TIMEOUT)) { *abort_flag = 1; return false; }
@@ -187,6 +198,30 @@ __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.pr
 __device__ __forceinline__ void tensormap_acquire(const CUtensorMap* tm) {
   asm volatile("fence.proxy.tensormap::generic.acquire.sys [%0], 128;" ::"l"(tm) : "memory");
 }
+// Ask for [p, p + bytes) (16-byte granules) to be brought into L2; no data returns to the SM.
+__device__ __forceinline__ void l2_prefetch(const void* p, size_t bytes) {
+  const char* c = (const char*)p;
+  while (bytes > 0) {
+    const uint32_t n = bytes > 32768 ? 32768u : (uint32_t)bytes;
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(c), "r"(n) : "memory");
+    c += n;
+    bytes -= n;
+  }
+}
+// This CTA's share (by rows) of a row-major [rows][row_bytes] matrix.
+__device__ __forceinline__ void l2_prefetch_rows(const void* base, int rows, size_t row_bytes, int cta, int G) {
+  const int r0 = (int)(((long long)cta * rows) / G), r1 = (int)(((long long)(cta + 1) * rows) / G);
+  if (r1 > r0) l2_prefetch((const char*)base + (size_t)r0 * row_bytes, (size_t)(r1 - r0) * row_bytes);
+}
+// Best-effort wait of the prefetch warp until this CTA has seen operator `op` start; false ends the prefetching.
+__device__ __forceinline__ bool prefetch_wait(volatile int* cur_op, int op, volatile int* abort_flag) {
+  const long long t0 = clock64();
+  while (*cur_op < op + 1) {
+    if (*abort_flag || clock64() - t0 > TC_TIMEOUT) return false;
+    __nanosleep(200);
+  }
+  return true;
+}
 __device__ __forceinline__ void trace_mark(const int* trace, int cta, int role, int op, int step) {
   if (trace && cta == 0) ((volatile int*)trace)[role] = (op << 8) | step;
 }
@@ -197,7 +232,7 @@ __device__ __forceinline__ void tl_mark(long long* tl, bool on, int op, int slot
   if (tl && on) {
     long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    ((volatile long long*)tl)[op * 8 + slot] = t;
+    ((volatile long long*)tl)[op * 16 + slot] = t;
   }
 }
 
@@ -246,12 +281,15 @@ __device__ __forceinline__ bool group_wait(const int* flag, int target, int etid
   epi_bar();
   return r;
 }
-// release: every thread's stores, then one counter increment
+// release: every thread's stores are ordered before the barrier; one thread then fences (cumulative) and bumps the
+// counter.  Each thread orders its own generic stores ahead of later async-proxy (TMA) reads of the same rows.
 __device__ __forceinline__ void group_signal(int* flag, int etid) {
-  __threadfence();
   fence_proxy_async_all();
   epi_bar();
-  if (etid == 0) red_release_add(flag, 1);
+  if (etid == 0) {
+    __threadfence();
+    red_release_add(flag, 1);
+  }
 }
 // s_rstd[i] = rsqrt(mean(h[row0 + i]^2) + eps) from the per-tile sums of squares
 __device__ __forceinline__ void load_rstd(const float* ssq, int nt, float inv_h, float eps, float* s_rstd, int row0, int rows,
@@ -291,7 +329,7 @@ __device__ __forceinline__ void attn_merge_warp(const float* att_o, const float2
       if (ml.y != 0.f) { w = exp2f(ml.x - mx); den = fmaf(w, ml.y, den); }
     }
     const int cn = min(32, n_chunks - c0);
-#pragma unroll 4
+#pragma unroll 8
     for (int cc = 0; cc < cn; ++cc) {
       const float wc = __shfl_sync(0xffffffffu, w, cc);
       const float* src = att_o + (slot0 + c0 + cc) * D + lane * VPL;
@@ -326,6 +364,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
   volatile uint32_t* tmem_slot = (volatile uint32_t*)(sm + S::BAR_OFF + MISC);
   volatile int* abort_flag = (volatile int*)(sm + S::BAR_OFF + MISC + 8);
   volatile int* s_flag = (volatile int*)(sm + S::BAR_OFF + MISC + 16);     // epilogue group broadcast word
+  volatile int* s_cur_op = (volatile int*)(sm + S::BAR_OFF + MISC + 24);   // 1 + index of the operator whose inputs are ready
   float* s_rstd = (float*)(sm + S::BAR_OFF + MISC + 32);                    // [64]
   float* s_red = s_rstd + 64;                                               // [4][M_PAD <= 64]
   float* s_xch = (float*)(sm + S::ATT_OFF + S::XCH_OFF);                                 // [M_PAD][<=132] exchange (GEMM epilogues only)
@@ -337,13 +376,18 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
   const MgModel& M = *Mp;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cta = blockIdx.x, G = gridDim.x;
-  constexpr int TMEM_COLS = (2 * M_PAD <= 32) ? 32 : ((2 * M_PAD <= 64) ? 64 : 128);
+  // Two accumulator buffers of NACC accumulators each: the NACC K sub-steps of a k-block go to different accumulators,
+  // so consecutive MMAs do not wait for one another's accumulate (with N <= 64 an MMA is far shorter than its latency).
+  constexpr int NACC = TC_BK / 16;
+  constexpr int ACC_COLS = NACC * M_PAD;
+  constexpr int TMEM_COLS = (2 * ACC_COLS <= 128) ? 128 : ((2 * ACC_COLS <= 256) ? 256 : 512);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < NW; ++s) { mbar_init(w_full0 + 8u * s, 1); mbar_init(w_empty0 + 8u * s, 1); }
     for (int s = 0; s < MG_NX; ++s) { mbar_init(x_full0 + 8u * s, 1); mbar_init(x_empty0 + 8u * s, 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(t_full0 + 8u * a, 1); mbar_init(t_empty0 + 8u * a, 4); }
     *abort_flag = 0;
+    *s_cur_op = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -361,7 +405,6 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
   long long* const tl = Rp.c.tline;
   const bool tl_on = (cta == Rp.c.trace_cta);
   const int n_layers = Rp.c.n_layers, layer_stride = Rp.c.layer_stride, T_o = Rp.c.T_o, T_g = Rp.c.T_g;
-  const int mpi = M_PAD / 16 - 1;
 
   if (warp == 0) {
     // =========================================== weight producer ===========================================
@@ -430,56 +473,112 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
     }
   } else if (warp == 6) {
     // ========================================= activation producer =========================================
-    if (lane == 0) {
-      const uint64_t pol_x = policy_evict_last();
-      tensormap_acquire(&M.tm_xg[mpi]);
-      tensormap_acquire(&M.tm_ao[mpi]);
-      tensormap_acquire(&M.tm_act[mpi]);
-      int stage = 0;
-      uint32_t phase = 0, armed = 0, armed_parity = 0;
-      bool ok = true;
-      OpIter ops(n_layers, r_lm_rows);
-      while (ok && ops.next()) {
-        const int kind = ops.kind, l = ops.l;
-        const Part g = op_part(Rp.c, kind, G);
-        const int* lc = sync + (size_t)(kind == OP_LM ? l - 1 : l) * layer_stride;
-        const CUtensorMap* tm = &M.tm_xg[mpi];
-        const int* flag = lc;
-        int target = 0, row0 = 0;
-        switch (kind) {
-          case OP_QKV: if (l > 0) { flag = lc - layer_stride + C_HOUT; target = T_o; } break;
-          case OP_O: tm = &M.tm_ao[mpi]; flag = lc + C_AO; target = G; break;
-          case OP_GU: flag = lc + C_H2; target = T_o; break;
-          case OP_D: tm = &M.tm_act[mpi]; flag = lc + C_ACT; target = T_g; break;
-          default: flag = lc + C_HOUT; target = T_o; row0 = r_m - r_lm_rows; break;
-        }
+    // The whole warp copies the [M_PAD x 64] bf16 activation tile of each k-block from L2 with plain 16-byte loads
+    // and writes it in the 128-byte-swizzled layout the MMA expects.  (Bulk tensor copies of these small,
+    // latency-critical tiles would queue behind the weight stream in the SM's copy engine.)
+    bool ok = true;
+    int stage = 0;
+    uint32_t phase = 0;
+    constexpr int CPL = M_PAD * 8 / 32;        // 16-byte chunks per lane and tile
+    OpIter ops(n_layers, r_lm_rows);
+    while (ok && ops.next()) {
+      const int kind = ops.kind, l = ops.l;
+      const Part g = op_part(Rp.c, kind, G);
+      const int* lc = sync + (size_t)(kind == OP_LM ? l - 1 : l) * layer_stride;
+      const bf16* xb = Rp.c.xg;
+      int K = Rp.c.H;
+      const int* flag = lc;
+      int target = 0, row0 = 0;
+      switch (kind) {
+        case OP_QKV: if (l > 0) { flag = lc - layer_stride + C_HOUT; target = T_o; } break;
+        case OP_O: xb = Rp.c.ao; K = Rp.c.NQ; flag = lc + C_AO; target = G; break;
+        case OP_GU: flag = lc + C_H2; target = T_o; break;
+        case OP_D: xb = Rp.c.act; K = Rp.c.I; flag = lc + C_ACT; target = T_g; break;
+        default: flag = lc + C_HOUT; target = T_o; row0 = r_m - r_lm_rows; break;
+      }
+      if (lane == 0) {
         trace_mark(trace, cta, 1, l * 4 + kind, 1);
-        if (!wait_count(flag, target, abort_flag, status)) { ok = false; break; }
+        ok = wait_count(flag, target, abort_flag, status);
         trace_mark(trace, cta, 1, l * 4 + kind, 2);
         tl_mark(tl, tl_on, l * 4 + kind, 4);
-        fence_proxy_async_all();   // rows written by other SMs' generic stores are read by the async proxy below
-        SegIter seg(g, cta);
-        int tile, kb0, kb1;
-        while (ok && seg.next(tile, kb0, kb1)) {
-          for (int kb = kb0; kb < kb1; ++kb) {
-            if (!mbar_wait(x_empty0 + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
-            const uint32_t fb = x_full0 + 8u * stage;
-            mbar_expect_tx(fb, S::X_BYTES);
-            armed |= 1u << stage;
-            armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
-            tma_load_2d(base + S::X_OFF + stage * S::X_BYTES, tm, fb, kb * TC_BK, row0, pol_x);
-            if (++stage == MG_NX) { stage = 0; phase ^= 1u; }
+        *s_cur_op = l * 4 + kind + 1;
+      }
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      __syncwarp();                                        // lane 0's acquire orders the whole warp's loads below
+      if (!ok) break;
+      // k-blocks are handled NB at a time: all their loads are in flight together (one L2 round trip per group),
+      // and only the stores wait for free stages
+      constexpr int NB = (32 / CPL) < 2 ? 2 : (32 / CPL);
+      SegIter seg(g, cta);
+      int tile, kb0 = 0, kb1 = 0;
+      bool more = true;
+      int ngrp = 0;
+      if (lane == 0) tl_mark(tl, tl_on, l * 4 + kind, 12);
+      while (ok && more) {
+        int kbs[NB];
+        int n = 0;
+        while (n < NB) {
+          if (kb0 >= kb1 && !seg.next(tile, kb0, kb1)) { more = false; break; }
+          kbs[n++] = kb0++;
+        }
+        if (n == 0) break;
+        uint4 val[NB][CPL];
+#pragma unroll
+        for (int j = 0; j < NB; ++j) {
+#pragma unroll
+          for (int i = 0; i < CPL; ++i) {
+            const int ch = lane + 32 * i, r = ch >> 3, c = ch & 7;
+            const int col = kbs[j < n ? j : 0] * TC_BK + c * 8;
+            const bool valid = j < n && (row0 + r) < Rp.c.R && col < K;
+            val[j][i] = valid ? __ldcg(reinterpret_cast<const uint4*>(xb + (size_t)(row0 + r) * K + col)) : make_uint4(0u, 0u, 0u, 0u);
           }
         }
-        tl_mark(tl, tl_on, l * 4 + kind, 5);
+        if (lane == 0 && ngrp == 0) { tl_mark(tl, tl_on && (val[0][0].x != 0x12345u), l * 4 + kind, 13); }
+#pragma unroll
+        for (int j = 0; j < NB; ++j) {
+          if (j < n) {                                      // uniform across the warp
+            if (lane == 0) ok = mbar_wait(x_empty0 + 8u * stage, phase ^ 1u, abort_flag);
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (ok) {
+              const uint32_t dst = base + S::X_OFF + stage * S::X_BYTES;
+#pragma unroll
+              for (int i = 0; i < CPL; ++i) {
+                const int ch = lane + 32 * i, r = ch >> 3, c = ch & 7;
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + r * 128 + ((c ^ (r & 7)) << 4)), "r"(val[j][i].x),
+                             "r"(val[j][i].y), "r"(val[j][i].z), "r"(val[j][i].w) : "memory");
+              }
+              asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> the MMA's async-proxy reads
+              __syncwarp();
+              if (lane == 0) mbar_arrive(x_full0 + 8u * stage);
+              if (++stage == MG_NX) { stage = 0; phase ^= 1u; }
+            }
+          }
+        }
+        if (lane == 0 && ngrp == 0) tl_mark(tl, tl_on, l * 4 + kind, 14);
+        ++ngrp;
       }
-      if (!ok) {
-        atomicCAS(Rp.c.status, 0, MG_ERR_XPROD);
-        for (int s = 0; s < MG_NX; ++s) {
-          if (!(armed & (1u << s))) continue;
-          const uint32_t par = (armed_parity >> s) & 1u;
-          const long long t0 = clock64();
-          while (!mbar_try_wait(x_full0 + 8u * s, par) && clock64() - t0 < TC_TIMEOUT) {}
+      if (lane == 0) tl_mark(tl, tl_on, l * 4 + kind, 5);
+    }
+    if (!ok && lane == 0) atomicCAS(Rp.c.status, 0, MG_ERR_XPROD);
+  } else if (warp == 7) {
+    // ============================================== L2 prefetcher ============================================
+    if (lane == 0) {
+      const size_t rb_h = (size_t)Rp.c.H * 2, rb_q = (size_t)Rp.c.NQ * 2, rb_i = (size_t)Rp.c.I * 2;
+      for (int l = 0; l < n_layers; ++l) {
+        const MgLayer* Ly = &Rp.c.layers[l];
+        if (!prefetch_wait(s_cur_op, l * 4 + OP_QKV, abort_flag)) break;
+        l2_prefetch_rows(Ly->wo, Rp.c.H, rb_q, cta, G);
+        for (int hk = 0; hk < Rp.c.hkv; ++hk) {
+          l2_prefetch_rows(Ly->kc + (size_t)hk * Rp.c.max_seq * D, r_L, (size_t)D * 2, cta, G);
+          l2_prefetch_rows(Ly->vc + (size_t)hk * Rp.c.max_seq * D, r_L, (size_t)D * 2, cta, G);
+        }
+        l2_prefetch_rows(Ly->wd, Rp.c.H, rb_i, cta, G);
+        if (l + 1 < n_layers) {
+          if (!prefetch_wait(s_cur_op, l * 4 + OP_GU, abort_flag)) break;
+          const MgLayer* Ln = &Rp.c.layers[l + 1];
+          l2_prefetch_rows(Ln->wq, Rp.c.NQ, rb_h, cta, G);
+          l2_prefetch_rows(Ln->wk, Rp.c.NKV, rb_h, cta, G);
+          l2_prefetch_rows(Ln->wv, Rp.c.NKV, rb_h, cta, G);
         }
       }
     }
@@ -503,7 +602,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
           ++nseg;
           if (!mbar_wait(t_empty0 + 8u * acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint32_t d_tmem = tmem_base + (uint32_t)(acc * M_PAD);
+          const uint32_t d_tmem = tmem_base + (uint32_t)(acc * ACC_COLS);
           for (int kb = kb0; kb < kb1; ++kb) {
             if (!mbar_wait(w_full0 + 8u * ws, wph, abort_flag) || !mbar_wait(x_full0 + 8u * xs, xph, abort_flag)) { ok = false; break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -512,7 +611,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
             const uint64_t bdesc = umma_desc_sw128(base + S::X_OFF + xs * S::X_BYTES);
 #pragma unroll
             for (int kk = 0; kk < TC_BK / 16; ++kk)
-              umma_bf16(d_tmem, adesc + 2u * kk, bdesc + 2u * kk, idesc, (kb > kb0 || kk > 0) ? 1u : 0u);
+              umma_bf16(d_tmem + (uint32_t)(kk * M_PAD), adesc + 2u * kk, bdesc + 2u * kk, idesc, (kb > kb0) ? 1u : 0u);
             umma_commit(w_empty0 + 8u * ws);
             umma_commit(x_empty0 + 8u * xs);
             if (++ws == NW) { ws = 0; wph ^= 1u; }
@@ -599,11 +698,23 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
         const int acc = nseg & 1;
         const uint32_t acc_phase = (uint32_t)(nseg >> 1) & 1u;
         ++nseg;
-        float hold[M_PAD];
+        // epilogue inputs that do not depend on the MMAs: residual rows (O, D) or the rotary table entries (QKV)
+        constexpr bool PRE_CS = (M_PAD <= 32);
+        float pre[PRE_CS ? 2 * M_PAD : M_PAD];
+        float pre_gain = 0.f;
         if (is_resid) {
           const int c = tile * TC_BM + et;
+          pre_gain = (c < H) ? res_gain[c] : 0.f;
 #pragma unroll
-          for (int b = 0; b < M_PAD; ++b) hold[b] = (c < H && b < m) ? __ldcg(&Rp.c.h[(size_t)b * H + c]) : 0.f;
+          for (int b = 0; b < M_PAD; ++b) pre[b] = (c < H && b < m) ? __ldcg(&Rp.c.h[(size_t)b * H + c]) : 0.f;
+        } else if (PRE_CS && kind == OP_QKV) {
+          const int jq = et % (D / 2);
+#pragma unroll
+          for (int b = 0; b < M_PAD; ++b) {
+            const float2 c2 = Rp.c.cs[(b < m ? b : 0) * (D / 2) + jq];
+            pre[(2 * b) % (PRE_CS ? 2 * M_PAD : M_PAD)] = c2.x;
+            pre[(2 * b + 1) % (PRE_CS ? 2 * M_PAD : M_PAD)] = c2.y;
+          }
         }
         if (etid == 0) *s_flag = mbar_wait(t_full0 + 8u * acc, acc_phase, abort_flag) ? 1 : 0;
         epi_bar();
@@ -611,13 +722,23 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
         if (etid == 0) { trace_mark(trace, cta, 3, l * 4 + kind, 5); tl_mark(tl, tl_on, l * 4 + kind, 2); }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         float v[M_PAD];
-        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * M_PAD);
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * ACC_COLS);
 #pragma unroll
         for (int c = 0; c < M_PAD; c += 16) tmem_ld16(taddr + c, v + c);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+        for (int a = 1; a < NACC; ++a) {                 // sum of the K sub-step accumulators, fixed order
+          float t[M_PAD];
+#pragma unroll
+          for (int c = 0; c < M_PAD; c += 16) tmem_ld16(taddr + (uint32_t)(a * M_PAD + c), t + c);
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+          for (int i = 0; i < M_PAD; ++i) v[i] += t[i];
+        }
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncwarp();
         if (lane == 0) mbar_arrive(t_empty0 + 8u * acc);
+        if (etid == 0) tl_mark(tl, tl_on, l * 4 + kind, 8);
 
         // ---- split tile: leave a partial; the last CTA to arrive sums all partials in CTA order ----
         if (!(kb0 == 0 && kb1 == g.KB)) {
@@ -627,16 +748,16 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
 #pragma unroll
           for (int b = 0; b < M_PAD; ++b)
             if (b < m) mine[b * 128 + et] = v[b];
-          __threadfence();
           epi_bar();
           const int cf = g.owner((long long)tile * g.SK), cl = g.owner((long long)tile * g.SK + g.SK - 1);
           int* tcnt = lc + (kind == OP_LM ? Rp.c.off_lm : (kind == OP_QKV ? (int)C_TILES : (kind == OP_O ? Rp.c.off_to : (kind == OP_GU ? Rp.c.off_tg : Rp.c.off_td)))) + tile;
-          if (etid == 0) *s_flag = (atomicAdd(tcnt, 1) == cl - cf) ? 1 : 0;
+          // one acq_rel atomic after the barrier: releases every thread's partial stores (cumulative) and, for the
+          // last arriver, acquires the other CTAs' partials for the whole group (through the second barrier)
+          if (etid == 0) *s_flag = (atom_add_acq_rel(tcnt, 1) == cl - cf) ? 1 : 0;
           epi_bar();
           const bool last = *s_flag != 0;
-          epi_bar();
+          epi_bar();                               // s_flag may be rewritten from here on
           if (!last) continue;
-          __threadfence();
 #pragma unroll
           for (int b = 0; b < M_PAD; ++b) v[b] = 0.f;
           constexpr int CU = (M_PAD <= 16) ? 4 : (M_PAD <= 32 ? 2 : 1);   // partials loaded together (register budget)
@@ -660,6 +781,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
           }
         }
 
+        if (etid == 0) tl_mark(tl, tl_on, l * 4 + kind, 9);
         // ---- operator epilogue on a complete tile: v[b] = sum_k w[row et of the tile][k] x[b][k] ----
         if (kind == OP_QKV) {
           int mi = 0;
@@ -685,12 +807,15 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
             for (int b = 0; b < M_PAD; ++b) {
               if (b < m) {
                 const float other = s_xch[b * 128 + pt];
-                const float2 c = Rp.c.cs[b * half + jj];
+                float2 c;
+                if (PRE_CS) { c.x = pre[(2 * b) % (PRE_CS ? 2 * M_PAD : M_PAD)]; c.y = pre[(2 * b + 1) % (PRE_CS ? 2 * M_PAD : M_PAD)]; }
+                else c = Rp.c.cs[b * half + jj];
                 v[b] = lo ? v[b] * c.x - other * c.y : v[b] * c.x + other * c.y;
               }
             }
             epi_bar();
           }
+          if (etid == 0) tl_mark(tl, tl_on, l * 4 + kind, 10);
           if (in_range) {
             bf16* dst;
             size_t stride;
@@ -702,15 +827,16 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
           }
           if (etid == 0) tl_mark(tl, tl_on, l * 4 + kind, 1);
           group_signal(lc + C_QKV, etid);
+          if (etid == 0) tl_mark(tl, tl_on, l * 4 + kind, 11);
         } else if (kind == OP_O || kind == OP_D) {
           const int c = tile * TC_BM + et;
           const bool in_range = c < H;
-          const float gn = in_range ? res_gain[c] : 0.f;
+          const float gn = pre_gain;
           // squares go through shared memory ([row][132]: 4 x 33 per row, conflict-free both ways) for the per-row sums
 #pragma unroll
           for (int b = 0; b < M_PAD; ++b) {
             if (b < m) {                                   // uniform across the group
-              const float hv = hold[b] + v[b];
+              const float hv = pre[b] + v[b];
               if (in_range) {
                 const size_t idx = (size_t)b * H + c;
                 Rp.c.h[idx] = hv;
@@ -719,6 +845,7 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
               s_xch[b * 132 + (warp - 2) * 33 + lane] = in_range ? hv * hv : 0.f;
             }
           }
+          if (etid == 0) tl_mark(tl, tl_on, l * 4 + kind, 10);
           epi_bar();
           for (int w4 = etid; w4 < m * 4; w4 += 128) {
             const int b = w4 >> 2, part = w4 & 3;
@@ -729,7 +856,9 @@ __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun
           }
           epi_bar();
           if (etid < m) Rp.c.ssq[(size_t)etid * nt + tile] = s_red[etid] + s_red[M_PAD + etid] + s_red[2 * M_PAD + etid] + s_red[3 * M_PAD + etid];
+          if (etid == 0) tl_mark(tl, tl_on, l * 4 + kind, 1);
           group_signal(lc + (kind == OP_O ? C_H2 : C_HOUT), etid);
+          if (etid == 0) tl_mark(tl, tl_on, l * 4 + kind, 11);
         } else if (kind == OP_GU) {
           const int col = tile * 64 + q * 16 + (lane & 15);
           const bool live = lane < 16 && col < I;
@@ -880,19 +1009,57 @@ void mega_destroy(fdvlm_t* h) {
   if (c->h_tline) {
     // per operator: microseconds since the first stamp of the last traced forward
     long long t0 = 0;
-    for (int i = 0; i < c->n_ops * 8; ++i) if (c->h_tline[i] && (!t0 || c->h_tline[i] < t0)) t0 = c->h_tline[i];
-    fprintf(stderr, "op: epi_in att_done acc0 epi_out | x_flag x_issued | mma0 | w_issued   (us)\n");
+    for (int i = 0; i < c->n_ops * 16; ++i) if (c->h_tline[i] && (!t0 || c->h_tline[i] < t0)) t0 = c->h_tline[i];
+    fprintf(stderr, "op: epi_in att/pre_sig acc0 epi_out | x_flag x_issued | mma0 | w_issued | tmem_ld partial_done mid_epi after_signal  (us)\n");
     for (int o = 0; o < c->n_ops; ++o) {
       fprintf(stderr, "%3d:", o);
-      for (int k = 0; k < 8; ++k) fprintf(stderr, " %9.2f", c->h_tline[o * 8 + k] ? (c->h_tline[o * 8 + k] - t0) / 1000.0 : -1.0);
+      for (int k = 0; k < 16; ++k) fprintf(stderr, " %8.2f", c->h_tline[o * 16 + k] ? (c->h_tline[o * 16 + k] - t0) / 1000.0 : -1.0);
       fprintf(stderr, "\n");
     }
     cudaFreeHost(c->h_tline);
   }
-  void* bufs[] = {c->d_model, c->d_layers, c->d_sync, c->d_part, c->d_att_o, c->d_att_ml};
-  for (void* p : bufs) if (p) cudaFree(p);
-  delete c;
+  delete c;       // the device buffers belong to the handle's slab
   h->mega = nullptr;
+}
+
+// Sizes of the persistent kernel's device buffers, in carving order (hot and small first).
+struct MegaSizes { size_t sync, model, layers, att_ml, att_o, part, total; int grid; size_t att_slots; };
+static MegaSizes mega_sizes(const fdvlm_t* h) {
+  const fdvlm_config& cf = h->cfg;
+  MegaSizes z;
+  memset(&z, 0, sizeof(z));
+  int dev = 0, sms = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  z.grid = sms > 0 ? sms : 1;
+  const int d = cf.head_dim, H = cf.hidden, I = cf.intermediate, NQ = cf.n_q_heads * d, NKV = cf.n_kv_heads * d;
+  const int tq = ceil_div(NQ, 128) + 2 * ceil_div(NKV, 128), T_o = ceil_div(H, 128), T_g = ceil_div(I, 64), T_l = ceil_div(cf.vocab, 128);
+  const int stride = ((C_TILES + tq + T_o + T_g + T_o + 31) / 32) * 32;
+  z.sync = ((size_t)cf.n_layers * stride + 32 + T_l + 32) * sizeof(int);
+  z.model = sizeof(MgModel);
+  z.layers = sizeof(MgLayer) * cf.n_layers;
+  size_t worst = 0;
+  for (int n = 1; n <= cf.max_block; ++n) {
+    // the chunk count of a shorter sequence can exceed that of max_seq (chunks are whole key tiles), so take its bound
+    const MgAttPlan p = mg_att_plan(n, cf.max_seq, cf.n_q_heads, cf.n_kv_heads, z.grid);
+    int bound = z.grid / (cf.n_kv_heads * p.groups);
+    const int tiles_max = ceil_div(cf.max_seq, AT_KEYS);
+    if (bound > tiles_max) bound = tiles_max;
+    if (bound < 1) bound = 1;
+    const size_t slots = (size_t)cf.n_q_heads * n * bound;
+    if (slots > worst) worst = slots;
+  }
+  z.att_slots = worst;
+  z.att_ml = worst * sizeof(float2);
+  z.att_o = worst * d * sizeof(float);
+  z.part = (size_t)z.grid * 2 * 64 * 128 * sizeof(float);
+  auto up = [](size_t b) { return (b + 255) / 256 * 256; };
+  z.total = up(z.sync) + up(z.model) + up(z.layers) + up(z.att_ml) + up(z.att_o) + up(z.part);
+  return z;
+}
+size_t mega_slab_bytes(const fdvlm_t* h) {
+  if (h->dt != DT_BF16) return 16;
+  return mega_sizes(h).total;
 }
 
 // Builds the device-side model description.  Returns false (and leaves h->mega null) when the shape or the
@@ -927,17 +1094,15 @@ bool mega_create(fdvlm_t* h) {
          mg_tmap(&L.tm_u, lw.w_up, I, H, 16);
     L.bq = lw.bq; L.bk = lw.bk; L.bv = lw.bv; L.g_attn = lw.g_attn; L.g_mlp = lw.g_mlp;
     L.kc = (bf16*)kv_ptr(h, l, 0); L.vc = (bf16*)kv_ptr(h, l, 1);
+    L.wq = (const bf16*)lw.wq; L.wk = (const bf16*)lw.wk; L.wv = (const bf16*)lw.wv; L.wo = (const bf16*)lw.wo; L.wd = (const bf16*)lw.w_down;
   }
   const void* table = cf.tie_embeddings ? h->w.embed : h->w.lm_head;
   const int R = cf.max_block;
   ok = ok && mg_tmap(&mt.tm_lm, table, cf.vocab, H, 128);
-  for (int i = 0; i < 4 && ok; ++i)
-    ok = mg_tmap(&mt.tm_xg[i], h->a, R, H, 16 * (i + 1)) && mg_tmap(&mt.tm_ao[i], h->ao, R, NQ, 16 * (i + 1)) &&
-         mg_tmap(&mt.tm_act[i], h->act, R, I, 16 * (i + 1));
   if (!ok) { delete c; return false; }
 
   mm.n_layers = cf.n_layers; mm.H = H; mm.I = I; mm.NQ = NQ; mm.NKV = NKV; mm.hq = cf.n_q_heads; mm.hkv = cf.n_kv_heads;
-  mm.d = d; mm.vocab = cf.vocab; mm.mask_id = cf.mask_id; mm.max_seq = cf.max_seq; mm.nt = h->nt;
+  mm.R = R; mm.d = d; mm.vocab = cf.vocab; mm.mask_id = cf.mask_id; mm.max_seq = cf.max_seq; mm.nt = h->nt;
   mm.eps = cf.rms_eps; mm.inv_h = 1.f / (float)H; mm.g_final = h->w.g_final;
   mm.h = h->h; mm.xg = (bf16*)h->a; mm.q = (bf16*)h->q; mm.ao = (bf16*)h->ao; mm.act = (bf16*)h->act; mm.ssq = h->ssq;
   mm.cs = (const float2*)h->cs; mm.logits = h->logits; mm.stats = (float4*)h->stats; mm.status = h->info + 3;
@@ -945,16 +1110,20 @@ bool mega_create(fdvlm_t* h) {
   mm.tq_begin[3] = mm.tq_begin[2] + ceil_div(NKV, 128);
   mm.T_o = ceil_div(H, 128); mm.T_g = ceil_div(I, 64); mm.T_l = ceil_div(cf.vocab, 128);
   mm.KB_h = ceil_div(H, 64); mm.KB_q = ceil_div(NQ, 64); mm.KB_i = ceil_div(I, 64);
-  // work partition per operator kind: whole tiles for QKV / O / gate-up (direct epilogues), a small split for the
-  // down projection (few tiles, long K), stream-K for the LM head
+  // work partition per operator kind
   {
     const int G = c->grid;
     const int T[5] = {mm.tq_begin[3], mm.T_o, mm.T_g, mm.T_o, mm.T_l};
     const int KB[5] = {mm.KB_h, mm.KB_q, mm.KB_h, mm.KB_i, mm.KB_h};
     for (int k = 0; k < 5; ++k) {
-      int sk = 1;
-      if (k == OP_D) { sk = (G / 2) / T[k]; if (sk > KB[k] / 8) sk = KB[k] / 8; if (sk < 1) sk = 1; }
-      if (k == OP_LM) sk = KB[k];
+      // QKV / O: few tiles, short K -> a small split whose shares fit the run-ahead ring (the weights are already in
+      // shared memory when the activations arrive); D: few tiles, long K -> enough splits to occupy most SMs;
+      // gate/up and the LM head: stream-K, every SM streams the same number of bytes.
+      int sk = KB[k];
+      if (k == OP_QKV || k == OP_O) { sk = (G / 2 + T[k] - 1) / T[k]; if (sk > KB[k] / 4) sk = KB[k] / 4; }
+      if (k == OP_D) { sk = (G - G / 8) / T[k]; if (sk > KB[k] / 8) sk = KB[k] / 8; }
+      if (sk < 1) sk = 1;
+      if (sk > KB[k]) sk = KB[k];
       const long long W = (long long)T[k] * sk;
       mm.op_sk[k] = sk;
       mm.op_ge[k] = W < G ? (int)W : G;
@@ -966,32 +1135,26 @@ bool mega_create(fdvlm_t* h) {
   mm.off_lm = mm.layer_stride + 32;   // relative to the last layer's counters
   c->sync_bytes = ((size_t)cf.n_layers * mm.layer_stride + 32 + mm.T_l + 32) * sizeof(int);
 
-  // attention partials: worst case over the block sizes this handle may see
-  size_t worst = 0;
-  for (int n = 1; n <= R; ++n) {
-    // the chunk count of a shorter sequence can exceed that of max_seq (chunks are whole key tiles), so take its bound
-    const MgAttPlan p = mg_att_plan(n, cf.max_seq, cf.n_q_heads, cf.n_kv_heads, c->grid);
-    int bound = c->grid / (cf.n_kv_heads * p.groups);
-    const int tiles_max = ceil_div(cf.max_seq, AT_KEYS);
-    if (bound > tiles_max) bound = tiles_max;
-    if (bound < 1) bound = 1;
-    const size_t slots = (size_t)cf.n_q_heads * n * bound;
-    if (slots > worst) worst = slots;
+  const MegaSizes z = mega_sizes(h);
+  bool alloc_ok = h->mega_slab != nullptr && z.sync == c->sync_bytes;
+  if (alloc_ok) {
+    auto up = [](size_t b) { return (b + 255) / 256 * 256; };
+    char* cur = h->mega_slab;
+    c->d_sync = (int*)cur; cur += up(z.sync);
+    c->d_model = (MgModel*)cur; cur += up(z.model);
+    c->d_layers = (MgLayer*)cur; cur += up(z.layers);
+    c->d_att_ml = (float2*)cur; cur += up(z.att_ml);
+    c->d_att_o = (float*)cur; cur += up(z.att_o);
+    c->d_part = (float*)cur;
   }
-  bool alloc_ok = cudaMalloc((void**)&c->d_model, sizeof(MgModel)) == cudaSuccess &&
-                  cudaMalloc((void**)&c->d_layers, sizeof(MgLayer) * cf.n_layers) == cudaSuccess &&
-                  cudaMalloc((void**)&c->d_sync, c->sync_bytes) == cudaSuccess &&
-                  cudaMalloc((void**)&c->d_part, (size_t)c->grid * 2 * 64 * 128 * sizeof(float)) == cudaSuccess &&
-                  cudaMalloc((void**)&c->d_att_o, worst * d * sizeof(float)) == cudaSuccess &&
-                  cudaMalloc((void**)&c->d_att_ml, worst * sizeof(float2)) == cudaSuccess;
   const char* tr = getenv("FDVLM_MEGA_TRACE");
   if (alloc_ok && tr && tr[0] == '1' && cudaHostAlloc((void**)&c->h_trace, 64, cudaHostAllocMapped) == cudaSuccess) {
     memset(c->h_trace, 0, 64);
     void* dp = nullptr;
     if (cudaHostGetDevicePointer(&dp, c->h_trace, 0) == cudaSuccess) mm.trace = (int*)dp;
     c->n_ops = cf.n_layers * 4 + 1;
-    if (cudaHostAlloc((void**)&c->h_tline, (size_t)c->n_ops * 64, cudaHostAllocMapped) == cudaSuccess) {
-      memset(c->h_tline, 0, (size_t)c->n_ops * 64);
+    if (cudaHostAlloc((void**)&c->h_tline, (size_t)c->n_ops * 128, cudaHostAllocMapped) == cudaSuccess) {
+      memset(c->h_tline, 0, (size_t)c->n_ops * 128);
       if (cudaHostGetDevicePointer(&dp, c->h_tline, 0) == cudaSuccess) mm.tline = (long long*)dp;
     }
   }
