@@ -18,27 +18,22 @@ __global__ void __launch_bounds__(128) attn_mma_kernel(const bf16* __restrict__ 
                                                        float2* __restrict__ part_ml, int n, int L, int max_seq, int hq,
                                                        int hkv, int qh, int chunk_keys, int n_chunks, int causal) {
   extern __shared__ __align__(128) uint8_t smem[];
+  pdl_trigger();
+  pdl_wait();
   attn_item<D>(q, kc, vc, part_o, part_ml, n, L, max_seq, hq, hkv, qh, chunk_keys, n_chunks, causal, blockIdx.x, blockIdx.y,
                blockIdx.z, (uint32_t)__cvta_generic_to_shared(smem), threadIdx.x);
 }
 
-// out[i][head] = sum_c w_c O_c / sum_c w_c l_c, w_c = 2^(m_c - max_c m_c)
+// out[i][head] = sum_c w_c O_c / sum_c w_c l_c, w_c = 2^(m_c - max_c m_c): one warp per (row, head), four per CTA
 template <int D>
-__global__ void __launch_bounds__(D) attn_combine_kernel(const float* __restrict__ part_o, const float2* __restrict__ part_ml,
-                                                        bf16* __restrict__ out, int n, int hq, int n_chunks) {
-  const int i = blockIdx.x, head = blockIdx.y, dd = threadIdx.x;
-  const size_t slot0 = ((size_t)head * n + i) * n_chunks;
-  float mx = -INFINITY;
-  for (int c = 0; c < n_chunks; ++c) mx = fmaxf(mx, part_ml[slot0 + c].x);
-  float den = 0.f, acc = 0.f;
-  for (int c = 0; c < n_chunks; ++c) {
-    const float2 ml = part_ml[slot0 + c];
-    if (ml.y == 0.f) continue;
-    const float w = exp2f(ml.x - mx);
-    den = fmaf(w, ml.y, den);
-    acc = fmaf(w, part_o[(slot0 + c) * D + dd], acc);
-  }
-  out[((size_t)i * hq + head) * D + dd] = __float2bfloat16_rn(acc / den);
+__global__ void __launch_bounds__(128) attn_combine_kernel(const float* __restrict__ part_o, const float2* __restrict__ part_ml,
+                                                          bf16* __restrict__ out, int n, int hq, int n_chunks) {
+  pdl_trigger();
+  pdl_wait();
+  const int p = blockIdx.x * 4 + (threadIdx.x >> 5);
+  if (p >= n * hq) return;
+  const int i = p / hq, head = p % hq;
+  attn_merge_warp<D>(part_o, part_ml, out + ((size_t)i * hq + head) * D, ((size_t)head * n + i) * n_chunks, n_chunks, threadIdx.x & 31);
 }
 
 // ---- host side -------------------------------------------------------------------------------------
@@ -93,9 +88,12 @@ static cudaError_t attn_launch_t(const AttnArgs& a, const AttnPlan& p, cudaStrea
     attr_set = true;
   }
   dim3 grid(p.n_chunks, p.groups, a.hkv);
-  attn_mma_kernel<D><<<grid, 128, smem, st>>>((const bf16*)a.q, (const bf16*)a.kc, (const bf16*)a.vc, part_o, part_ml, a.n,
-                                               a.cache_len, a.max_seq, a.hq, a.hkv, p.qh, p.chunk_keys, p.n_chunks, a.causal);
-  attn_combine_kernel<D><<<dim3(a.n, a.hq), D, 0, st>>>(part_o, part_ml, (bf16*)a.out, a.n, a.hq, p.n_chunks);
+  cudaError_t e = launch_pdl(attn_mma_kernel<D>, grid, dim3(128), (size_t)smem, st, (const bf16*)a.q, (const bf16*)a.kc, (const bf16*)a.vc,
+                             part_o, part_ml, a.n, a.cache_len, a.max_seq, a.hq, a.hkv, p.qh, p.chunk_keys, p.n_chunks, a.causal);
+  if (e != cudaSuccess) return e;
+  e = launch_pdl(attn_combine_kernel<D>, dim3((a.n * a.hq + 3) / 4), dim3(128), 0, st, (const float*)part_o, (const float2*)part_ml,
+                 (bf16*)a.out, a.n, a.hq, p.n_chunks);
+  if (e != cudaSuccess) return e;
   return cudaGetLastError();
 }
 

@@ -4,6 +4,7 @@
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <string.h>
 
 namespace fdk {
 
@@ -55,6 +56,25 @@ __device__ __forceinline__ float block_max(float v, float* red) {
   float r = (lane < nw) ? red[lane] : -INFINITY;
   r = warp_max(r);
   return r;
+}
+
+// Programmatic dependent launch: a kernel launched with launch_pdl may start while its predecessor in the stream is
+// still running.  pdl_trigger lets the successor's CTAs be scheduled early; pdl_wait returns once the predecessor grid
+// has completed and its writes are visible -- every thread calls it before it reads the predecessor's results or
+// overwrites anything the predecessor may still read.  Launched the ordinary way both are no-ops.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
 }
 
 enum { MODE_BIDIR = 0, MODE_CAUSAL = 1 };

@@ -95,6 +95,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_con
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
+  pdl_trigger();
 
   const int total_tiles = p.tile_begin[p.n_mats];
   const int n_items = total_tiles * p.splits;
@@ -108,6 +109,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_con
       uint32_t armed = 0;           // bit s: full[s] armed and not yet known complete
       uint32_t armed_parity = 0;    // bit s: parity of that arming
       bool ok = true;
+      bool waited = false;
+      int n_pend = 0, pend_stage[TC_STAGES], pend_kb[TC_STAGES];
       for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
         const int tile = it % total_tiles, split = it / total_tiles;
         int mi = 0, r0 = 0;
@@ -135,9 +138,26 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_con
             tma_load_2d(a_dst, &p.tm_w[mi], full_bar(stage), kb * TC_BK, r0, pol_w);
             tma_load_2d(a_dst + TC_A_BYTES / 2, &p.tm_w[mi], full_bar(stage), kb * TC_BK, r0 + 64, pol_w);
           }
-          tma_load_2d(a_dst + TC_A_BYTES, &p.tm_x, full_bar(stage), kb * TC_BK, 0, pol_x);
+          // The weights do not depend on the predecessor kernel: the first ring of weight loads is issued before waiting
+          // for it; the activation tiles of those stages follow once it has completed.
+          if (waited) {
+            tma_load_2d(a_dst + TC_A_BYTES, &p.tm_x, full_bar(stage), kb * TC_BK, 0, pol_x);
+          } else {
+            pend_stage[n_pend] = stage; pend_kb[n_pend] = kb;
+            if (++n_pend == TC_STAGES) {
+              pdl_wait();
+              waited = true;
+              for (int j = 0; j < n_pend; ++j)
+                tma_load_2d(base + pend_stage[j] * L::STAGE_BYTES + TC_A_BYTES, &p.tm_x, full_bar(pend_stage[j]), pend_kb[j] * TC_BK, 0, pol_x);
+            }
+          }
           if (++stage == TC_STAGES) { stage = 0; phase ^= 1u; }
         }
+      }
+      if (!waited) {
+        pdl_wait();
+        for (int j = 0; j < n_pend; ++j)
+          tma_load_2d(base + pend_stage[j] * L::STAGE_BYTES + TC_A_BYTES, &p.tm_x, full_bar(pend_stage[j]), pend_kb[j] * TC_BK, 0, pol_x);
       }
       if (!ok) {
         atomicCAS(p.status, 0, TC_ERR_PRODUCER);
@@ -188,6 +208,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_con
     const int q = warp & 3;  // TMEM lane quarter this warp may read
     int local = 0;
     bool ok = true;
+    pdl_wait();   // the epilogue reads the predecessor's row statistics and overwrites buffers it may still be reading
     // folded RMSNorm: lane l keeps the factor of rows l and l + 32; broadcast by shuffle where needed
     float rs0 = 1.f, rs1 = 1.f;
     if (p.ssq_in) {
@@ -383,8 +404,7 @@ static cudaError_t tc_launch_t(const TcParams& p, int grid, cudaStream_t st) {
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  gemm_tc_kernel<M_PAD><<<grid, TC_THREADS, TcSmem<M_PAD>::TOTAL, st>>>(p);
-  return cudaGetLastError();
+  return launch_pdl(gemm_tc_kernel<M_PAD>, dim3(grid), dim3(TC_THREADS), (size_t)TcSmem<M_PAD>::TOTAL, st, p);
 }
 
 static cudaError_t tc_launch(const TcParams& p, cudaStream_t st) {

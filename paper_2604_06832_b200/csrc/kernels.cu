@@ -117,6 +117,8 @@ linear_simt_kernel(const XT* __restrict__ x, const WT* __restrict__ w, float* __
 __global__ void splitk_epilogue_kernel(const float* __restrict__ part, int S, int m, int N,
                                        const float* __restrict__ scale, const float* __restrict__ bias,
                                        float* __restrict__ y, int ldy, int accumulate) {
+  pdl_trigger();
+  pdl_wait();
   size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   size_t total = (size_t)m * N;
   if (idx >= total) return;
@@ -223,6 +225,8 @@ void launch_rmsnorm(const float* h, const float* g, void* out, int n, int hidden
 // rotary table: cs[r][j] = (cos, sin)(pos * theta^(-2j/d)), angles formed in fp64
 // ================================================================================================
 __global__ void rope_table_kernel(float2* __restrict__ cs, int n, int pos0, int half, double theta) {
+  pdl_trigger();
+  pdl_wait();
   int idx = blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= n * half) return;
   int r = idx / half, j = idx % half;
@@ -233,7 +237,7 @@ __global__ void rope_table_kernel(float2* __restrict__ cs, int n, int pos0, int 
 }
 void launch_rope_table(float* cs, int n, int pos0, int head_dim, float theta, cudaStream_t st) {
   int half = head_dim / 2, total = n * half;
-  rope_table_kernel<<<(total + 127) / 128, 128, 0, st>>>((float2*)cs, n, pos0, half, (double)theta);
+  launch_pdl(rope_table_kernel, dim3((total + 127) / 128), dim3(128), 0, st, (float2*)cs, n, pos0, half, (double)theta);
 }
 
 // rotate-half pairing (j, j + d/2); q -> q buffer, k -> cache K plane, v -> cache V plane
@@ -279,6 +283,8 @@ void launch_qkv_post(const float* qkv, const float* cs, void* q, void* kc, void*
 __global__ void embed_prep_kernel(const bf16* __restrict__ table, const int32_t* __restrict__ tokens,
                                   const bf16* __restrict__ rows, float* __restrict__ h, bf16* __restrict__ xg,
                                   const float* __restrict__ g, float* __restrict__ ssq, int nt, int hidden) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float red[32];
   const int r = blockIdx.x;
   const bf16* src = tokens ? table + (size_t)tokens[r] * hidden : rows + (size_t)r * hidden;
@@ -297,6 +303,19 @@ void launch_embed_prep(const void* table, const int32_t* tokens, const void* row
   embed_prep_kernel<<<n, 256, 0, st>>>((const bf16*)table, tokens, (const bf16*)rows, h, (bf16*)xg, g, ssq, nt, hidden);
 }
 
+// Sum of S split-K partials p[i * stride], eight loads in flight at a time, added in index order (deterministic).
+__device__ __forceinline__ float sum_partials(const float* __restrict__ p, size_t stride, int S) {
+  float s = 0.f;
+  for (int i0 = 0; i0 < S; i0 += 8) {
+    float r[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) r[j] = (i0 + j < S) ? __ldcg(p + (size_t)(i0 + j) * stride) : 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) s += r[j];
+  }
+  return s;
+}
+
 // QKV finalisation: sum the split-K partials, apply the folded norm factor and the bias, rotate q and k
 // (rotate-half pairs j, j + d/2), write q to its buffer and k, v into the layer's cache planes.
 // grid (hq + 2 hkv heads, m rows), d/2 threads: thread j owns the pair (j, j + d/2) of one head.
@@ -305,6 +324,8 @@ __global__ void fin_qkv_kernel(const float* __restrict__ part, int S, int m, con
                                const float* __restrict__ bq, const float* __restrict__ bk, const float* __restrict__ bv,
                                bf16* __restrict__ q, bf16* __restrict__ kc, bf16* __restrict__ vc, int pos0, int hq, int hkv,
                                int d, int max_seq) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float s_rstd;
   const int head = blockIdx.x, r = blockIdx.y, j = threadIdx.x, half = d >> 1;
   if (threadIdx.x < 32) {
@@ -319,8 +340,7 @@ __global__ void fin_qkv_kernel(const float* __restrict__ part, int S, int m, con
   const int width = (hq + 2 * hkv) * d;
   const size_t sstride = (size_t)m * width;
   const float* pa = part + (size_t)r * width + head * d + j;
-  float a = 0.f, b = 0.f;
-  for (int i = 0; i < S; ++i) { a += pa[i * sstride]; b += pa[i * sstride + half]; }
+  float a = sum_partials(pa, sstride, S), b = sum_partials(pa + half, sstride, S);
   a *= rstd; b *= rstd;
   if (head < hq) {
     if (bq) { a += bq[head * d + j]; b += bq[head * d + j + half]; }
@@ -346,7 +366,7 @@ __global__ void fin_qkv_kernel(const float* __restrict__ part, int S, int m, con
 void launch_fin_qkv(const float* part, int S, int m, const float* cs, const float* ssq, int nt, int hidden, float eps,
                     const float* bq, const float* bk, const float* bv, void* q, void* kc, void* vc, int pos0, int hq,
                     int hkv, int d, int max_seq, cudaStream_t st) {
-  fin_qkv_kernel<<<dim3(hq + 2 * hkv, m), d / 2, 0, st>>>(part, S, m, (const float2*)cs, ssq, nt, 1.f / (float)hidden, eps, bq, bk,
+  launch_pdl(fin_qkv_kernel, dim3(hq + 2 * hkv, m), dim3(d / 2), 0, st, part, S, m, (const float2*)cs, ssq, nt, 1.f / (float)hidden, eps, bq, bk,
                                                           bv, (bf16*)q, (bf16*)kc, (bf16*)vc, pos0, hq, hkv, d, max_seq);
 }
 
@@ -355,14 +375,15 @@ void launch_fin_qkv(const float* part, int S, int m, const float* cs, const floa
 __global__ void __launch_bounds__(128) fin_resid_kernel(const float* __restrict__ part, int S, int m, int hidden,
                                                         float* __restrict__ h, const float* __restrict__ g,
                                                         bf16* __restrict__ xg, float* __restrict__ ssq, int nt) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float red[32];
   const int t = blockIdx.x, r = blockIdx.y, c = t * 128 + threadIdx.x;
   float v = 0.f;
   if (c < hidden) {
     const size_t idx = (size_t)r * hidden + c, sstride = (size_t)m * hidden;
-    float s = 0.f;
-    for (int i = 0; i < S; ++i) s += part[i * sstride + idx];
-    v = h[idx] + s;
+    const float hv = h[idx];
+    v = hv + sum_partials(part + idx, sstride, S);
     h[idx] = v;
     xg[idx] = __float2bfloat16_rn(v * g[c]);
   }
@@ -371,13 +392,15 @@ __global__ void __launch_bounds__(128) fin_resid_kernel(const float* __restrict_
 }
 void launch_fin_resid(const float* part, int S, int m, int hidden, float* h, const float* g, void* xg, float* ssq, int nt,
                       cudaStream_t st) {
-  fin_resid_kernel<<<dim3(nt, m), 128, 0, st>>>(part, S, m, hidden, h, g, (bf16*)xg, ssq, nt);
+  launch_pdl(fin_resid_kernel, dim3(nt, m), dim3(128), 0, st, part, S, m, hidden, h, g, (bf16*)xg, ssq, nt);
 }
 
 // Merge the per-warp softmax statistics of the LM-head epilogue into confidence and prediction per row.
 // stats[e * m + row] = (max, sum exp(l - max), argmax id) for e in [0, n_part).  grid m rows, 256 threads.
 __global__ void __launch_bounds__(256) stats_merge_kernel(const float4* __restrict__ stats, int n_part, int m,
                                                           float* __restrict__ conf, int32_t* __restrict__ pred) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float sm_m[8], sm_s[8];
   __shared__ int sm_i[8];
   const int r = blockIdx.x;
@@ -412,7 +435,7 @@ __global__ void __launch_bounds__(256) stats_merge_kernel(const float4* __restri
   }
 }
 void launch_stats_merge(const void* stats, int n_part, int m, float* conf, int32_t* pred, cudaStream_t st) {
-  stats_merge_kernel<<<m, 256, 0, st>>>((const float4*)stats, n_part, m, conf, pred);
+  launch_pdl(stats_merge_kernel, dim3(m), dim3(256), 0, st, (const float4*)stats, n_part, m, conf, pred);
 }
 
 // ================================================================================================
@@ -489,6 +512,8 @@ __global__ void select_kernel(const float* __restrict__ conf, const int32_t* __r
                               int32_t* __restrict__ tokens, uint8_t* __restrict__ masked,
                               uint8_t* __restrict__ unmask, int32_t* __restrict__ info, int n, int rule,
                               float threshold, int k) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float c[64];
   __shared__ int mk[64];
   int i = threadIdx.x;

@@ -309,45 +309,6 @@ __device__ __forceinline__ void load_rstd(const float* ssq, int nt, float inv_h,
   epi_bar();
 }
 
-// Merge of the key chunks of one (row, head) by one warp: out = sum_c w_c O_c / sum_c w_c l_c, w_c = 2^(m_c - max m).
-// Lane j owns D / 32 consecutive output features; the chunk statistics are spread over the lanes.
-template <int D>
-__device__ __forceinline__ void attn_merge_warp(const float* att_o, const float2* att_ml, bf16* out, size_t slot0, int n_chunks,
-                                                int lane) {
-  constexpr int VPL = D / 32;
-  float mx = -INFINITY;
-  for (int c = lane; c < n_chunks; c += 32) mx = fmaxf(mx, __ldcg(&att_ml[slot0 + c]).x);
-  mx = warp_max(mx);
-  float den = 0.f, acc[VPL];
-#pragma unroll
-  for (int i = 0; i < VPL; ++i) acc[i] = 0.f;
-  for (int c0 = 0; c0 < n_chunks; c0 += 32) {
-    const int c = c0 + lane;
-    float w = 0.f;
-    if (c < n_chunks) {
-      const float2 ml = __ldcg(&att_ml[slot0 + c]);
-      if (ml.y != 0.f) { w = exp2f(ml.x - mx); den = fmaf(w, ml.y, den); }
-    }
-    const int cn = min(32, n_chunks - c0);
-#pragma unroll 8
-    for (int cc = 0; cc < cn; ++cc) {
-      const float wc = __shfl_sync(0xffffffffu, w, cc);
-      const float* src = att_o + (slot0 + c0 + cc) * D + lane * VPL;
-      if (VPL == 4) {
-        const float4 o = __ldcg(reinterpret_cast<const float4*>(src));
-        acc[0] = fmaf(wc, o.x, acc[0]); acc[1] = fmaf(wc, o.y, acc[1]); acc[2] = fmaf(wc, o.z, acc[2]); acc[VPL - 1] = fmaf(wc, o.w, acc[VPL - 1]);
-      } else {
-        const float2 o = __ldcg(reinterpret_cast<const float2*>(src));
-        acc[0] = fmaf(wc, o.x, acc[0]); acc[VPL - 1] = fmaf(wc, o.y, acc[VPL - 1]);
-      }
-    }
-  }
-  den = warp_sum(den);
-  const float inv = 1.f / den;
-#pragma unroll
-  for (int i = 0; i < VPL; ++i) out[lane * VPL + i] = __float2bfloat16_rn(acc[i] * inv);
-}
-
 template <int M_PAD, int D>
 __global__ void __launch_bounds__(MG_THREADS, 1) forward_mega_kernel(const MgRun Rp) {
   using S = MgSmem<M_PAD, D>;
