@@ -95,7 +95,7 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
   for (auto& s : shapes) { size_t b = linear_workspace_bytes(R, s[0], s[1], h->dt); if (b > ws) ws = b; }
   size_t wa = attention_workspace_bytes(R, cfg->n_q_heads, cfg->n_kv_heads, d);
   if (wa > ws) ws = wa;
-  h->use_tc = (h->dt == DT_BF16) && tc_linear_supported(R, NQ, H, DT_BF16);
+  h->use_tc = (h->dt == DT_BF16 || h->dt == DT_FP8) && tc_linear_supported(R, NQ, H, h->dt) && tc_linear_supported(R, H, I, h->dt);
   if (h->use_tc) {
     const size_t g3[] = {tc_workspace_bytes(R, NQKV, (NQ + 127) / 128 + 2 * ((NKV + 127) / 128), H),
                          tc_workspace_bytes(R, H, (H + 127) / 128, NQ), tc_workspace_bytes(R, H, (H + 127) / 128, I)};

@@ -38,6 +38,7 @@ int launch_linear(const LinearArgs& a, cudaStream_t st, cudaError_t* err) {
   TcGroup g;
   memset(&g, 0, sizeof(g));
   g.x = a.x; g.m = a.m; g.k = a.k; g.w[0] = a.w; g.n[0] = a.n; g.n_mats = 1;
+  g.fp8 = (a.dtype == DT_FP8);
   int splits = 0;
   TcOut o;
   memset(&o, 0, sizeof(o));
@@ -158,6 +159,7 @@ static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int wan
     memset(&g, 0, sizeof(g));
     g.x = x; g.m = m; g.k = k; g.n_mats = nm;
     g.w[0] = w0; g.n[0] = n0; g.w[1] = w1; g.n[1] = n1; g.w[2] = w2; g.n[2] = n2;
+    g.fp8 = (h->dt == DT_FP8);
     return g;
   };
   auto out = [&](int tc_mode) {
@@ -182,7 +184,7 @@ static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int wan
     o.ld = NQKV; o.splits_out = &S;
     if (!gemm(group(h->a, n, H, 3, lw.wq, NQ, lw.wk, NKV, lw.wv, NKV), o))
       return fail(h, FDVLM_ERR_CUDA, "qkv projection launch: %s", cudaGetErrorString(e));
-    launch_fin_qkv(part, S, n, h->cs, h->ssq, nt, H, c.rms_eps, lw.bq, lw.bk, lw.bv, h->q, kv_ptr(h, l, 0), kv_ptr(h, l, 1),
+    launch_fin_qkv(part, S, n, h->cs, h->ssq, nt, H, c.rms_eps, lw.bq, lw.bk, lw.bv, lw.s_q, lw.s_k, lw.s_v, h->q, kv_ptr(h, l, 0), kv_ptr(h, l, 1),
                    h->cache_len, c.n_q_heads, c.n_kv_heads, d, c.max_seq, h->st);
     AttnArgs at;
     at.q = h->q; at.kc = kv_ptr(h, l, 0); at.vc = kv_ptr(h, l, 1); at.out = h->ao; at.n = n; at.cache_len = h->cache_len;
@@ -197,17 +199,19 @@ static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int wan
     o.ld = H; o.splits_out = &S;
     if (!gemm(group(h->ao, n, NQ, 1, lw.wo, H, nullptr, 0, nullptr, 0), o))
       return fail(h, FDVLM_ERR_CUDA, "o projection launch: %s", cudaGetErrorString(e));
-    launch_fin_resid(part, S, n, H, h->h, lw.g_mlp, h->a, h->ssq, nt, h->st);
+    launch_fin_resid(part, S, n, H, h->h, lw.g_mlp, h->a, h->ssq, nt, lw.s_o, h->st);
     o = out(TC_MODE_SWIGLU);
     o.act = h->act; o.ssq_in = h->ssq; o.nt_in = nt; o.hidden = H; o.eps = c.rms_eps;
-    if (!gemm(group(h->a, n, H, 2, lw.w_gate, I, lw.w_up, I, nullptr, 0), o))
+    TcGroup gu = group(h->a, n, H, 2, lw.w_gate, I, lw.w_up, I, nullptr, 0);
+    gu.scale[0] = lw.s_gate; gu.scale[1] = lw.s_up;
+    if (!gemm(gu, o))
       return fail(h, FDVLM_ERR_CUDA, "gate/up projection launch: %s", cudaGetErrorString(e));
     o = out(TC_MODE_PARTIAL);
     o.ld = H; o.splits_out = &S;
     if (!gemm(group(h->act, n, I, 1, lw.w_down, H, nullptr, 0, nullptr, 0), o))
       return fail(h, FDVLM_ERR_CUDA, "down projection launch: %s", cudaGetErrorString(e));
     const float* g_next = (l + 1 < c.n_layers) ? h->layers[l + 1].g_attn : h->w.g_final;
-    launch_fin_resid(part, S, n, H, h->h, g_next, h->a, h->ssq, nt, h->st);
+    launch_fin_resid(part, S, n, H, h->h, g_next, h->a, h->ssq, nt, lw.s_down, h->st);
     h->launches += 2;
   }
   if (logits_rows > 0) {
@@ -218,7 +222,10 @@ static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int wan
     o.y = h->logits; o.ld = c.vocab; o.write_logits = (logits_rows == n) ? want_logits : 1;
     o.ssq_in = h->ssq + (size_t)first * nt; o.nt_in = nt; o.hidden = H; o.eps = c.rms_eps;
     o.stats = h->stats; o.mask_id = c.mask_id;
-    if (!gemm(group((const char*)h->a + (size_t)first * H * 2, m, H, 1, table, c.vocab, nullptr, 0, nullptr, 0), o))
+    TcGroup lm = group((const char*)h->a + (size_t)first * H * 2, m, H, 1, table, c.vocab, nullptr, 0, nullptr, 0);
+    if (c.tie_embeddings) lm.fp8 = 0;                 // a tied table is the bf16 embedding
+    else lm.scale[0] = h->w.s_lm_head;
+    if (!gemm(lm, o))
       return fail(h, FDVLM_ERR_CUDA, "lm head launch: %s", cudaGetErrorString(e));
     if (logits_rows == n) {
       launch_stats_merge(h->stats, ceil_div(c.vocab, 128) * 4, n, h->conf, h->pred, h->st);

@@ -7,7 +7,10 @@
 // one elected thread issues tcgen05.mma with fp32 accumulators in tensor memory (two accumulator
 // buffers, so the epilogue of one work item overlaps the mainloop of the next); four epilogue warps
 // read the accumulators with tcgen05.ld.  CTAs are persistent over a static round-robin list of
-// work items (tile, K-split).  Every mbarrier wait is bounded: on a timeout the CTA records an
+// work items (tile, K-split).  FP8-E4M3 weights take the same road with half the bytes: the byte tile lands in
+// the stage, four converter warps widen it exactly to bf16 (e4m3 -> f16 -> f32 -> bf16, all exact) into a
+// swizzled buffer of its own, and the MMA reads that buffer; the per-channel scales are applied by the epilogues.
+// Every mbarrier wait is bounded: on a timeout the CTA records an
 // error code in a status word, drains its own bulk copies, frees its tensor memory and returns.
 #include <cuda.h>
 
@@ -20,9 +23,10 @@
 
 namespace fdk {
 
-constexpr int TC_STAGES = 4;
-constexpr int TC_THREADS = 192;  // warp 0 TMA producer, warp 1 MMA issuer, warps 2..5 epilogue
-constexpr int TC_A_BYTES = TC_BM * TC_BK * 2;
+constexpr int TC_THREADS = 192;       // warp 0 TMA producer, warp 1 MMA issuer, warps 2..5 epilogue
+constexpr int TC_THREADS_FP8 = 320;   // + warps 6..9: e4m3 -> bf16 converters
+constexpr int TC_A_BYTES = TC_BM * TC_BK * 2;   // a bf16 weight tile
+constexpr int TC_NCONV = 2;           // converted-tile buffers (fp8 only)
 
 enum { TC_ERR_PRODUCER = 1, TC_ERR_MMA = 2, TC_ERR_EPILOGUE = 3 };
 
@@ -53,29 +57,57 @@ struct TcParams {
   int* status;          // device word, set non-zero when a wait timed out
 };
 
-template <int M_PAD>
+template <int M_PAD, bool FP8>
 struct TcSmem {
+  static constexpr int STAGES = FP8 ? 6 : 4;
+  static constexpr int W_BYTES = FP8 ? TC_BM * TC_BK : TC_A_BYTES;     // weight tile as it is streamed
+  static constexpr int W_ROW = FP8 ? TC_BK : TC_BK * 2;                // bytes per weight row in the stage
   static constexpr int B_BYTES = M_PAD * TC_BK * 2;
-  static constexpr int STAGE_BYTES = TC_A_BYTES + B_BYTES;
-  static constexpr int BAR_OFF = TC_STAGES * STAGE_BYTES;
+  static constexpr int STAGE_BYTES = W_BYTES + B_BYTES;
+  static constexpr int CONV_OFF = STAGES * STAGE_BYTES;                // bf16 tiles made by the converters
+  static constexpr int BAR_OFF = CONV_OFF + (FP8 ? TC_NCONV * TC_A_BYTES : 0);
   static constexpr int TOTAL = BAR_OFF + 256 + 1024;  // barriers + alignment slack
 };
 
-template <int M_PAD>
-__global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_constant__ TcParams p) {
+// sixteen e4m3 bytes -> sixteen bf16 (exact: every e4m3 value is a bf16 value)
+__device__ __forceinline__ void e4m3x16_to_bf16(const uint4& in, uint4& lo, uint4& hi) {
+  const uint32_t w[4] = {in.x, in.y, in.z, in.w};
+  uint32_t o[8];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+#pragma unroll
+    for (int hsel = 0; hsel < 2; ++hsel) {
+      const unsigned short two = (unsigned short)(hsel ? (w[i] >> 16) : (w[i] & 0xffffu));
+      uint32_t h2;
+      asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(two));
+      const float f0 = __half2float(__ushort_as_half((unsigned short)(h2 & 0xffffu)));
+      const float f1 = __half2float(__ushort_as_half((unsigned short)(h2 >> 16)));
+      __nv_bfloat162 b2 = __floats2bfloat162_rn(f0, f1);
+      o[2 * i + hsel] = *reinterpret_cast<uint32_t*>(&b2);
+    }
+  }
+  lo = make_uint4(o[0], o[1], o[2], o[3]);
+  hi = make_uint4(o[4], o[5], o[6], o[7]);
+}
+
+template <int M_PAD, bool FP8>
+__global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_kernel(const __grid_constant__ TcParams p) {
   extern __shared__ uint8_t smem_raw[];
-  using L = TcSmem<M_PAD>;
+  using L = TcSmem<M_PAD, FP8>;
+  constexpr int TC_STAGES = L::STAGES;
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* sm = smem_raw + (base - raw);
   const uint32_t bar0 = base + L::BAR_OFF;
-  // barrier slots (8 bytes each): full[S], empty[S], tmem_full[2], tmem_empty[2]
+  // barrier slots (8 bytes each): full[S], empty[S], tmem_full[2], tmem_empty[2], conv_full[2], conv_empty[2]
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (TC_STAGES + s); };
   auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * TC_STAGES + a); };
   auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * TC_STAGES + 2 + a); };
-  volatile uint32_t* tmem_slot = (volatile uint32_t*)(sm + L::BAR_OFF + 8 * (2 * TC_STAGES + 4));
-  volatile int* abort_flag = (volatile int*)(sm + L::BAR_OFF + 8 * (2 * TC_STAGES + 4) + 8);
+  auto cfull_bar = [&](int c) { return bar0 + 8u * (2 * TC_STAGES + 4 + c); };
+  auto cempty_bar = [&](int c) { return bar0 + 8u * (2 * TC_STAGES + 6 + c); };
+  volatile uint32_t* tmem_slot = (volatile uint32_t*)(sm + L::BAR_OFF + 8 * (2 * TC_STAGES + 8));
+  volatile int* abort_flag = (volatile int*)(sm + L::BAR_OFF + 8 * (2 * TC_STAGES + 8) + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   constexpr int TMEM_COLS = (2 * M_PAD <= 32) ? 32 : ((2 * M_PAD <= 64) ? 64 : 128);
@@ -83,6 +115,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_con
   if (threadIdx.x == 0) {
     for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    for (int c = 0; c < TC_NCONV; ++c) { mbar_init(cfull_bar(c), 4); mbar_init(cempty_bar(c), 1); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -131,24 +164,24 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_con
             // 0..15 and the matching up rows in lanes 16..31, so the epilogue pairs them with one shuffle
 #pragma unroll
             for (int qq = 0; qq < 4; ++qq) {
-              tma_load_2d(a_dst + (32 * qq) * 128, &p.tm_w[0], full_bar(stage), kb * TC_BK, tile * 64 + 16 * qq, pol_w);
-              tma_load_2d(a_dst + (32 * qq + 16) * 128, &p.tm_w[1], full_bar(stage), kb * TC_BK, tile * 64 + 16 * qq, pol_w);
+              tma_load_2d(a_dst + (32 * qq) * L::W_ROW, &p.tm_w[0], full_bar(stage), kb * TC_BK, tile * 64 + 16 * qq, pol_w);
+              tma_load_2d(a_dst + (32 * qq + 16) * L::W_ROW, &p.tm_w[1], full_bar(stage), kb * TC_BK, tile * 64 + 16 * qq, pol_w);
             }
           } else {
             tma_load_2d(a_dst, &p.tm_w[mi], full_bar(stage), kb * TC_BK, r0, pol_w);
-            tma_load_2d(a_dst + TC_A_BYTES / 2, &p.tm_w[mi], full_bar(stage), kb * TC_BK, r0 + 64, pol_w);
+            tma_load_2d(a_dst + L::W_BYTES / 2, &p.tm_w[mi], full_bar(stage), kb * TC_BK, r0 + 64, pol_w);
           }
           // The weights do not depend on the predecessor kernel: the first ring of weight loads is issued before waiting
           // for it; the activation tiles of those stages follow once it has completed.
           if (waited) {
-            tma_load_2d(a_dst + TC_A_BYTES, &p.tm_x, full_bar(stage), kb * TC_BK, 0, pol_x);
+            tma_load_2d(a_dst + L::W_BYTES, &p.tm_x, full_bar(stage), kb * TC_BK, 0, pol_x);
           } else {
             pend_stage[n_pend] = stage; pend_kb[n_pend] = kb;
             if (++n_pend == TC_STAGES) {
               pdl_wait();
               waited = true;
               for (int j = 0; j < n_pend; ++j)
-                tma_load_2d(base + pend_stage[j] * L::STAGE_BYTES + TC_A_BYTES, &p.tm_x, full_bar(pend_stage[j]), pend_kb[j] * TC_BK, 0, pol_x);
+                tma_load_2d(base + pend_stage[j] * L::STAGE_BYTES + L::W_BYTES, &p.tm_x, full_bar(pend_stage[j]), pend_kb[j] * TC_BK, 0, pol_x);
             }
           }
           if (++stage == TC_STAGES) { stage = 0; phase ^= 1u; }
@@ -157,7 +190,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_con
       if (!waited) {
         pdl_wait();
         for (int j = 0; j < n_pend; ++j)
-          tma_load_2d(base + pend_stage[j] * L::STAGE_BYTES + TC_A_BYTES, &p.tm_x, full_bar(pend_stage[j]), pend_kb[j] * TC_BK, 0, pol_x);
+          tma_load_2d(base + pend_stage[j] * L::STAGE_BYTES + L::W_BYTES, &p.tm_x, full_bar(pend_stage[j]), pend_kb[j] * TC_BK, 0, pol_x);
       }
       if (!ok) {
         atomicCAS(p.status, 0, TC_ERR_PRODUCER);
@@ -174,8 +207,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_con
     // ------------------------------------------------ MMA issuer --------------------------------------------------
     if (lane == 0) {
       const uint32_t idesc = umma_idesc_bf16(M_PAD);
-      int stage = 0;
-      uint32_t phase = 0;
+      int stage = 0, cbuf = 0;
+      uint32_t phase = 0, cphase = 0;
       int local = 0;
       bool ok = true;
       for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++local) {
@@ -188,21 +221,60 @@ __global__ void __launch_bounds__(TC_THREADS, 1) gemm_tc_kernel(const __grid_con
         const int kb0 = split * p.kb_per_split;
         const int kb1 = min(p.kblocks, kb0 + p.kb_per_split);
         for (int kb = kb0; kb < kb1; ++kb) {
-          if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+          // fp8: the converters have waited for the stage and left the widened tile in buffer cbuf
+          if (!mbar_wait(FP8 ? cfull_bar(cbuf) : full_bar(stage), FP8 ? cphase : phase, abort_flag)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t a_addr = base + stage * L::STAGE_BYTES;
-          const uint64_t adesc = umma_desc_sw128(a_addr);
-          const uint64_t bdesc = umma_desc_sw128(a_addr + TC_A_BYTES);
+          const uint64_t adesc = umma_desc_sw128(FP8 ? base + L::CONV_OFF + cbuf * TC_A_BYTES : a_addr);
+          const uint64_t bdesc = umma_desc_sw128(a_addr + L::W_BYTES);
 #pragma unroll
           for (int kk = 0; kk < TC_BK / 16; ++kk)
             umma_bf16(d_tmem, adesc + 2u * kk, bdesc + 2u * kk, idesc, (kb > kb0 || kk > 0) ? 1u : 0u);
           umma_commit(empty_bar(stage));
+          if (FP8) {
+            umma_commit(cempty_bar(cbuf));
+            if (++cbuf == TC_NCONV) { cbuf = 0; cphase ^= 1u; }
+          }
           if (++stage == TC_STAGES) { stage = 0; phase ^= 1u; }
         }
         if (ok) umma_commit(tfull_bar(acc));
       }
       if (!ok) atomicCAS(p.status, 0, TC_ERR_MMA);
     }
+  } else if (FP8 && warp >= 6) {
+    // ------------------------------------------------ e4m3 -> bf16 converters ---------------------------------------
+    // 128 threads; thread t widens the 16-byte pieces t, t + 128, t + 256, t + 384 of the 8 KB byte tile (rows of 64
+    // bytes) into the 128-byte-swizzled bf16 tile the MMA descriptor expects.
+    const int ct = threadIdx.x - 192;
+    int stage = 0, cbuf = 0;
+    uint32_t phase = 0, cphase = 0;
+    bool ok = true;
+    for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+      const int split = it / total_tiles;
+      const int kb0 = split * p.kb_per_split;
+      const int kb1 = min(p.kblocks, kb0 + p.kb_per_split);
+      for (int kb = kb0; kb < kb1; ++kb) {
+        if (!mbar_wait(full_bar(stage), phase, abort_flag) || !mbar_wait(cempty_bar(cbuf), cphase ^ 1u, abort_flag)) { ok = false; break; }
+        const uint8_t* src = sm + stage * L::STAGE_BYTES;
+        const uint32_t dst = base + L::CONV_OFF + cbuf * TC_A_BYTES;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int piece = ct + 128 * i, r = piece >> 2, c = piece & 3;     // row, 16-byte piece of the row
+          const uint4 in = *reinterpret_cast<const uint4*>(src + piece * 16);
+          uint4 lo, hi;
+          e4m3x16_to_bf16(in, lo, hi);
+          const uint32_t row = dst + r * 128;
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + (((2 * c) ^ (r & 7)) << 4)), "r"(lo.x), "r"(lo.y), "r"(lo.z), "r"(lo.w) : "memory");
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + (((2 * c + 1) ^ (r & 7)) << 4)), "r"(hi.x), "r"(hi.y), "r"(hi.z), "r"(hi.w) : "memory");
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> the MMA's async-proxy reads
+        __syncwarp();
+        if (lane == 0) mbar_arrive(cfull_bar(cbuf));
+        if (++cbuf == TC_NCONV) { cbuf = 0; cphase ^= 1u; }
+        if (++stage == TC_STAGES) { stage = 0; phase ^= 1u; }
+      }
+    }
+    if (!ok && ct == 0) atomicCAS(p.status, 0, TC_ERR_MMA);
   } else {
     // ------------------------------------------------ epilogue warps ----------------------------------------------
     const int q = warp & 3;  // TMEM lane quarter this warp may read
@@ -336,24 +408,25 @@ static EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// 2-D bf16 row-major [rows, cols] tensor, box {64 columns, box_rows}, 128-byte swizzle, zero OOB fill.
-static bool make_tmap(CUtensorMap* tm, const void* ptr, int rows, int cols, int box_rows) {
-  typedef std::tuple<const void*, int, int, int> Key;
+// 2-D row-major [rows, cols] tensor, box {64 columns, box_rows}, zero OOB fill.  bf16: 128-byte swizzle (rows of the
+// box are 128 bytes); e4m3 bytes: no swizzle (rows of 64 bytes, widened by the converter warps).
+static bool make_tmap(CUtensorMap* tm, const void* ptr, int rows, int cols, int box_rows, bool fp8 = false) {
+  typedef std::tuple<const void*, int, int, int, bool> Key;
   static std::map<Key, CUtensorMap> cache;
   static std::mutex mu;
   std::lock_guard<std::mutex> lock(mu);
-  Key key(ptr, rows, cols, box_rows);
+  Key key(ptr, rows, cols, box_rows, fp8);
   auto it = cache.find(key);
   if (it != cache.end()) { *tm = it->second; return true; }
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * (fp8 ? 1 : 2)};
   cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  CUresult r = fn(tm, fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides,
+                  box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, fp8 ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return false;
   if (cache.size() > 4096) cache.clear();
   cache[key] = *tm;
@@ -387,7 +460,10 @@ static void tc_plan(int tiles, int kblocks, int* splits, int* kbps) {
 }
 
 bool tc_linear_supported(int m, int n, int k, int dtype) {
-  return dtype == DT_BF16 && m >= 1 && m <= 64 && n >= 1 && k >= 8 && (k % 8) == 0 && encode_fn() != nullptr;
+  if (m < 1 || m > 64 || n < 1 || encode_fn() == nullptr) return false;
+  if (dtype == DT_BF16) return k >= 8 && (k % 8) == 0;
+  if (dtype == DT_FP8) return k >= 16 && (k % 16) == 0;     // byte rows must be 16-byte multiples for TMA
+  return false;
 }
 
 size_t tc_workspace_bytes(int m, int ld, int tiles, int k) {
@@ -396,25 +472,26 @@ size_t tc_workspace_bytes(int m, int ld, int tiles, int k) {
   return (size_t)s * m * ld * sizeof(float);
 }
 
-template <int M_PAD>
+template <int M_PAD, bool FP8>
 static cudaError_t tc_launch_t(const TcParams& p, int grid, cudaStream_t st) {
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<M_PAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<M_PAD>::TOTAL);
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<M_PAD, FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<M_PAD, FP8>::TOTAL);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  return launch_pdl(gemm_tc_kernel<M_PAD>, dim3(grid), dim3(TC_THREADS), (size_t)TcSmem<M_PAD>::TOTAL, st, p);
+  return launch_pdl(gemm_tc_kernel<M_PAD, FP8>, dim3(grid), dim3(FP8 ? TC_THREADS_FP8 : TC_THREADS), (size_t)TcSmem<M_PAD, FP8>::TOTAL, st, p);
 }
 
-static cudaError_t tc_launch(const TcParams& p, cudaStream_t st) {
+template <bool FP8>
+static cudaError_t tc_launch_f(const TcParams& p, cudaStream_t st) {
   const int items = p.tile_begin[p.n_mats] * p.splits;
   const int grid = items < 2 * sm_count() ? items : 2 * sm_count();
   switch (pad_m(p.m)) {
-    case 16: return tc_launch_t<16>(p, grid, st);
-    case 32: return tc_launch_t<32>(p, grid, st);
-    case 48: return tc_launch_t<48>(p, grid, st);
-    default: return tc_launch_t<64>(p, grid, st);
+    case 16: return tc_launch_t<16, FP8>(p, grid, st);
+    case 32: return tc_launch_t<32, FP8>(p, grid, st);
+    case 48: return tc_launch_t<48, FP8>(p, grid, st);
+    default: return tc_launch_t<64, FP8>(p, grid, st);
   }
 }
 
@@ -431,7 +508,7 @@ cudaError_t tc_group_launch(const TcGroup& g, const TcOut& o, cudaStream_t st) {
   if (!make_tmap(&p.tm_x, g.x, g.m, g.k, mp)) return cudaErrorInvalidValue;
   int tiles = 0, col = 0;
   for (int i = 0; i < g.n_mats; ++i) {
-    if (!make_tmap(&p.tm_w[i], g.w[i], g.n[i], g.k, mode == TC_MODE_SWIGLU ? 16 : 64)) return cudaErrorInvalidValue;
+    if (!make_tmap(&p.tm_w[i], g.w[i], g.n[i], g.k, mode == TC_MODE_SWIGLU ? 16 : 64, g.fp8 != 0)) return cudaErrorInvalidValue;
     p.n_out[i] = g.n[i];
     p.tile_begin[i] = tiles;
     p.out_col[i] = col;
@@ -462,7 +539,7 @@ cudaError_t tc_group_launch(const TcGroup& g, const TcOut& o, cudaStream_t st) {
     if (mode == TC_MODE_LOGITS && (g.n_mats != 1 || !o.stats)) return cudaErrorInvalidValue;
   }
   if (o.splits_out) *o.splits_out = p.splits;
-  return tc_launch(p, st);
+  return g.fp8 ? tc_launch_f<true>(p, st) : tc_launch_f<false>(p, st);
 }
 
 }  // namespace fdk

@@ -322,6 +322,7 @@ __device__ __forceinline__ float sum_partials(const float* __restrict__ p, size_
 __global__ void fin_qkv_kernel(const float* __restrict__ part, int S, int m, const float2* __restrict__ cs,
                                const float* __restrict__ ssq, int nt, float inv_h, float eps,
                                const float* __restrict__ bq, const float* __restrict__ bk, const float* __restrict__ bv,
+                               const float* __restrict__ sq, const float* __restrict__ sk, const float* __restrict__ sv,
                                bf16* __restrict__ q, bf16* __restrict__ kc, bf16* __restrict__ vc, int pos0, int hq, int hkv,
                                int d, int max_seq) {
   pdl_trigger();
@@ -342,6 +343,10 @@ __global__ void fin_qkv_kernel(const float* __restrict__ part, int S, int m, con
   const float* pa = part + (size_t)r * width + head * d + j;
   float a = sum_partials(pa, sstride, S), b = sum_partials(pa + half, sstride, S);
   a *= rstd; b *= rstd;
+  if (sq) {   // fp8 weights: per-output-channel factors
+    const float* sc = head < hq ? sq + head * d : (head < hq + hkv ? sk + (head - hq) * d : sv + (head - hq - hkv) * d);
+    a *= sc[j]; b *= sc[j + half];
+  }
   if (head < hq) {
     if (bq) { a += bq[head * d + j]; b += bq[head * d + j + half]; }
     const float2 c = cs[r * half + j];
@@ -364,17 +369,18 @@ __global__ void fin_qkv_kernel(const float* __restrict__ part, int S, int m, con
   }
 }
 void launch_fin_qkv(const float* part, int S, int m, const float* cs, const float* ssq, int nt, int hidden, float eps,
-                    const float* bq, const float* bk, const float* bv, void* q, void* kc, void* vc, int pos0, int hq,
+                    const float* bq, const float* bk, const float* bv, const float* sq, const float* sk, const float* sv, void* q, void* kc, void* vc, int pos0, int hq,
                     int hkv, int d, int max_seq, cudaStream_t st) {
   launch_pdl(fin_qkv_kernel, dim3(hq + 2 * hkv, m), dim3(d / 2), 0, st, part, S, m, (const float2*)cs, ssq, nt, 1.f / (float)hidden, eps, bq, bk,
-                                                          bv, (bf16*)q, (bf16*)kc, (bf16*)vc, pos0, hq, hkv, d, max_seq);
+                                                          bv, sq, sk, sv, (bf16*)q, (bf16*)kc, (bf16*)vc, pos0, hq, hkv, d, max_seq);
 }
 
 // Residual finalisation: h += sum of split-K partials; xg = bf16(h * gain of the next norm); ssq[row][tile] =
 // sum of h^2 over the tile's 128 columns.  grid (nt tiles, m rows), 128 threads.
 __global__ void __launch_bounds__(128) fin_resid_kernel(const float* __restrict__ part, int S, int m, int hidden,
                                                         float* __restrict__ h, const float* __restrict__ g,
-                                                        bf16* __restrict__ xg, float* __restrict__ ssq, int nt) {
+                                                        bf16* __restrict__ xg, float* __restrict__ ssq, int nt,
+                                                        const float* __restrict__ scale) {
   pdl_trigger();
   pdl_wait();
   __shared__ float red[32];
@@ -383,7 +389,7 @@ __global__ void __launch_bounds__(128) fin_resid_kernel(const float* __restrict_
   if (c < hidden) {
     const size_t idx = (size_t)r * hidden + c, sstride = (size_t)m * hidden;
     const float hv = h[idx];
-    v = hv + sum_partials(part + idx, sstride, S);
+    v = hv + sum_partials(part + idx, sstride, S) * (scale ? scale[c] : 1.f);
     h[idx] = v;
     xg[idx] = __float2bfloat16_rn(v * g[c]);
   }
@@ -391,8 +397,8 @@ __global__ void __launch_bounds__(128) fin_resid_kernel(const float* __restrict_
   if (threadIdx.x == 0) ssq[(size_t)r * nt + t] = ss;
 }
 void launch_fin_resid(const float* part, int S, int m, int hidden, float* h, const float* g, void* xg, float* ssq, int nt,
-                      cudaStream_t st) {
-  launch_pdl(fin_resid_kernel, dim3(nt, m), dim3(128), 0, st, part, S, m, hidden, h, g, (bf16*)xg, ssq, nt);
+                      const float* scale, cudaStream_t st) {
+  launch_pdl(fin_resid_kernel, dim3(nt, m), dim3(128), 0, st, part, S, m, hidden, h, g, (bf16*)xg, ssq, nt, scale);
 }
 
 // Merge the per-warp softmax statistics of the LM-head epilogue into confidence and prediction per row.

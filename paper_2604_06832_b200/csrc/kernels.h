@@ -47,6 +47,7 @@ struct TcGroup {
   const void* x; int m, k;
   const void* w[3]; int n[3]; int n_mats;
   const float* scale[3]; const float* bias[3];
+  int fp8;   // weights are e4m3 bytes (scale[] holds the per-output-channel factors)
 };
 // What the GEMM leaves behind.
 //   PARTIAL: part[split][m][ld] = split-K partial sums (*splits_out of them) for the caller's reduce kernel
@@ -73,10 +74,11 @@ cudaError_t tc_group_launch(const TcGroup& g, const TcOut& o, cudaStream_t st);
 void launch_embed_prep(const void* table, const int32_t* tokens, const void* rows, float* h, void* xg, const float* g,
                        float* ssq, int nt, int n, int hidden, cudaStream_t st);
 void launch_fin_qkv(const float* part, int S, int m, const float* cs, const float* ssq, int nt, int hidden, float eps,
-                    const float* bq, const float* bk, const float* bv, void* q, void* kc, void* vc, int pos0, int hq,
+                    const float* bq, const float* bk, const float* bv, const float* sq, const float* sk, const float* sv, void* q,
+                    void* kc, void* vc, int pos0, int hq,
                     int hkv, int d, int max_seq, cudaStream_t st);
 void launch_fin_resid(const float* part, int S, int m, int hidden, float* h, const float* g, void* xg, float* ssq, int nt,
-                      cudaStream_t st);
+                      const float* scale, cudaStream_t st);
 void launch_stats_merge(const void* stats, int n_part, int m, float* conf, int32_t* pred, cudaStream_t st);
 
 // ---- attention -----------------------------------------------------------------------------------

@@ -72,6 +72,7 @@ extern "C" int fdvlm_op_linear_static(const void* x, const void* w, const float*
   TcGroup g;
   memset(&g, 0, sizeof(g));
   g.x = x; g.m = m; g.k = k; g.w[0] = w; g.n[0] = n; g.n_mats = 1;
+  g.fp8 = (dtype == FDVLM_W_FP8E4M3);
   int splits = 0;
   TcOut o;
   memset(&o, 0, sizeof(o));
