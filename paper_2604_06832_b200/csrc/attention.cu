@@ -12,14 +12,22 @@
 
 namespace fdk {
 
+// len_ptr (nullable): the cache length is read from device memory instead of L, and the chunking is derived from
+// it and `bound` (= gridDim.x) on the device -- lets one captured launch serve every cache length.
 template <int D>
 __global__ void __launch_bounds__(128) attn_mma_kernel(const bf16* __restrict__ q, const bf16* __restrict__ kc,
                                                        const bf16* __restrict__ vc, float* __restrict__ part_o,
                                                        float2* __restrict__ part_ml, int n, int L, int max_seq, int hq,
-                                                       int hkv, int qh, int chunk_keys, int n_chunks, int causal) {
+                                                       int hkv, int qh, int chunk_keys, int n_chunks, int causal,
+                                                       const int* __restrict__ len_ptr) {
   extern __shared__ __align__(128) uint8_t smem[];
   pdl_trigger();
   pdl_wait();
+  if (len_ptr) {
+    L = *len_ptr;
+    attn_chunking(L + n, (int)gridDim.x, &chunk_keys, &n_chunks);
+    if ((int)blockIdx.x >= n_chunks) return;
+  }
   attn_item<D>(q, kc, vc, part_o, part_ml, n, L, max_seq, hq, hkv, qh, chunk_keys, n_chunks, causal, blockIdx.x, blockIdx.y,
                blockIdx.z, (uint32_t)__cvta_generic_to_shared(smem), threadIdx.x);
 }
@@ -27,9 +35,14 @@ __global__ void __launch_bounds__(128) attn_mma_kernel(const bf16* __restrict__ 
 // out[i][head] = sum_c w_c O_c / sum_c w_c l_c, w_c = 2^(m_c - max_c m_c): one warp per (row, head), four per CTA
 template <int D>
 __global__ void __launch_bounds__(128) attn_combine_kernel(const float* __restrict__ part_o, const float2* __restrict__ part_ml,
-                                                          bf16* __restrict__ out, int n, int hq, int n_chunks) {
+                                                          bf16* __restrict__ out, int n, int hq, int n_chunks,
+                                                          const int* __restrict__ len_ptr, int bound) {
   pdl_trigger();
   pdl_wait();
+  if (len_ptr) {
+    int ck;
+    attn_chunking(*len_ptr + n, bound, &ck, &n_chunks);
+  }
   const int p = blockIdx.x * 4 + (threadIdx.x >> 5);
   if (p >= n * hq) return;
   const int i = p / hq, head = p % hq;
@@ -37,7 +50,15 @@ __global__ void __launch_bounds__(128) attn_combine_kernel(const float* __restri
 }
 
 // ---- host side -------------------------------------------------------------------------------------
-struct AttnPlan { int qh, groups, chunk_keys, n_chunks; };
+struct AttnPlan { int qh, groups, chunk_keys, n_chunks, bound; };
+
+static int attn_max_chunks(int n, int hq, int hkv) {
+  const int G = hq / hkv;
+  int qh = 1;
+  for (int c = G; c >= 1; --c)
+    if (c * n <= AT_ROWS) { qh = c; break; }
+  return ceil_div(2 * 148, hkv * ceil_div(G, qh));
+}
 
 static AttnPlan attn_plan(int n, int T, int hq, int hkv) {
   const int G = hq / hkv;
@@ -46,22 +67,9 @@ static AttnPlan attn_plan(int n, int T, int hq, int hkv) {
   for (int c = G; c >= 1; --c)                 // most heads per CTA that still fit 64 rows
     if (c * n <= AT_ROWS) { p.qh = c; break; }
   p.groups = ceil_div(G, p.qh);
-  const int ctas_per_chunk = hkv * p.groups;
-  const int tiles = ceil_div(T, AT_KEYS);
-  int want = ceil_div(2 * 148, ctas_per_chunk);
-  if (want > tiles) want = tiles;
-  if (want < 1) want = 1;
-  p.chunk_keys = ceil_div(tiles, want) * AT_KEYS;
-  p.n_chunks = ceil_div(T, p.chunk_keys);
+  p.bound = attn_max_chunks(n, hq, hkv);
+  attn_chunking(T, p.bound, &p.chunk_keys, &p.n_chunks);
   return p;
-}
-
-static int attn_max_chunks(int n, int hq, int hkv) {
-  const int G = hq / hkv;
-  int qh = 1;
-  for (int c = G; c >= 1; --c)
-    if (c * n <= AT_ROWS) { qh = c; break; }
-  return ceil_div(2 * 148, hkv * ceil_div(G, qh));
 }
 
 size_t attention_mma_workspace_bytes(int n, int hq, int hkv, int d) {
@@ -75,9 +83,10 @@ size_t attention_mma_workspace_bytes(int n, int hq, int hkv, int d) {
 
 template <int D>
 static cudaError_t attn_launch_t(const AttnArgs& a, const AttnPlan& p, cudaStream_t st) {
-  const int T = a.cache_len + a.n;
-  (void)T;
-  const size_t slots = (size_t)a.hq * a.n * p.n_chunks;
+  // with the length on the device the grid is sized for the most chunks any length can give
+  int grid_x = p.n_chunks;
+  if (a.len_ptr) { grid_x = p.bound; const int tmax = ceil_div(a.max_seq, AT_KEYS); if (grid_x > tmax) grid_x = tmax; }
+  const size_t slots = (size_t)a.hq * a.n * grid_x;
   float* part_o = (float*)a.workspace;
   float2* part_ml = (float2*)((char*)a.workspace + ((slots * D * 4 + 255) / 256) * 256);
   const int smem = AT_ROWS * D * 2 + 4 * AT_KEYS * D * 2;
@@ -87,12 +96,12 @@ static cudaError_t attn_launch_t(const AttnArgs& a, const AttnPlan& p, cudaStrea
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  dim3 grid(p.n_chunks, p.groups, a.hkv);
+  dim3 grid(grid_x, p.groups, a.hkv);
   cudaError_t e = launch_pdl(attn_mma_kernel<D>, grid, dim3(128), (size_t)smem, st, (const bf16*)a.q, (const bf16*)a.kc, (const bf16*)a.vc,
-                             part_o, part_ml, a.n, a.cache_len, a.max_seq, a.hq, a.hkv, p.qh, p.chunk_keys, p.n_chunks, a.causal);
+                             part_o, part_ml, a.n, a.cache_len, a.max_seq, a.hq, a.hkv, p.qh, p.chunk_keys, p.n_chunks, a.causal, a.len_ptr);
   if (e != cudaSuccess) return e;
   e = launch_pdl(attn_combine_kernel<D>, dim3((a.n * a.hq + 3) / 4), dim3(128), 0, st, (const float*)part_o, (const float2*)part_ml,
-                 (bf16*)a.out, a.n, a.hq, p.n_chunks);
+                 (bf16*)a.out, a.n, a.hq, p.n_chunks, a.len_ptr, grid_x);
   if (e != cudaSuccess) return e;
   return cudaGetLastError();
 }

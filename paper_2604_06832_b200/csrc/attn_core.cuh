@@ -37,6 +37,16 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) {
   return (uint32_t)(row * (D * 2) + ((chunk ^ (row & 7)) << 4));
 }
 
+// Split of T keys into chunks of whole 64-key tiles, at most `bound` chunks (the same on host and device, so a launch
+// whose grid was sized for `bound` can take the sequence length from device memory).
+__host__ __device__ inline void attn_chunking(int T, int bound, int* chunk_keys, int* n_chunks) {
+  const int tiles = (T + AT_KEYS - 1) / AT_KEYS;
+  int want = bound < tiles ? bound : tiles;
+  if (want < 1) want = 1;
+  *chunk_keys = ((tiles + want - 1) / want) * AT_KEYS;
+  *n_chunks = (T + *chunk_keys - 1) / *chunk_keys;
+}
+
 // Barrier of the 128 threads that work on one attention item (named barrier 1, so the threads may be a
 // subset of a larger CTA).
 __device__ __forceinline__ void attn_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }

@@ -32,6 +32,8 @@ extern "C" const char* fdvlm_last_error(const fdvlm_t* h) { return h ? h->err : 
 extern "C" void fdvlm_destroy(fdvlm_t* h) {
   if (!h) return;
   mega_destroy(h);
+  for (auto& g : h->graphs) if (g.exec) cudaGraphExecDestroy(g.exec);
+  h->graphs.clear();
   if (h->kv) cudaFree(h->kv);
   if (h->slab) cudaFree(h->slab);
   for (cudaEvent_t ev : h->prof_ev) cudaEventDestroy(ev);
@@ -84,6 +86,8 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
   h->host_stage = nullptr;
   h->mega = nullptr;
   h->slab = nullptr;
+  h->dev_len = nullptr;
+  h->use_graphs = 0;
   h->mega_slab = nullptr;
   cudaGetDevice(&h->device);
 
@@ -106,6 +110,7 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
   // streaming through the TLBs, each separately allocated buffer would cost its own page walk whenever it is touched.
   struct { void** p; size_t bytes; } allocs[] = {
       {(void**)&h->info, 16},
+      {(void**)&h->dev_len, 16},
       {(void**)&h->conf, (size_t)R * 4},
       {(void**)&h->pred, (size_t)R * 4},
       {(void**)&h->unmask, 64},
@@ -152,6 +157,10 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
     return FDVLM_ERR_CUDA;
   }
   // bf16 weights: the persistent forward kernel, for now only on request (FDVLM_MEGA=1)
+  // the tensor-core forward is replayed from captured CUDA graphs (FDVLM_NO_GRAPH=1: launch kernel by kernel)
+  const char* no_graph = getenv("FDVLM_NO_GRAPH");
+  // (the legacy default stream cannot be captured: a handle created on it launches kernel by kernel)
+  h->use_graphs = h->use_tc && h->st != nullptr && !(no_graph && no_graph[0] == '1');
   const char* want_mega = getenv("FDVLM_MEGA");
   if (h->use_tc && want_mega && want_mega[0] == '1') mega_create(h);
   *out = h;
@@ -414,6 +423,7 @@ extern "C" int fdvlm_op_attention(const void* q, const void* k_cache, const void
     return FDVLM_ERR_INVALID_ARG;
   if (dtype != FDVLM_F32 && dtype != FDVLM_BF16 && dtype != FDVLM_W_FP8E4M3) return FDVLM_ERR_INVALID_ARG;
   AttnArgs a;
+  a.len_ptr = nullptr;
   a.q = q; a.kc = k_cache; a.vc = v_cache; a.out = out; a.n = n_rows; a.cache_len = cache_len; a.max_seq = max_seq;
   a.hq = n_q_heads; a.hkv = n_kv_heads; a.d = head_dim; a.causal = causal ? 1 : 0; a.dtype = (int)dtype; a.workspace = workspace;
   cudaError_t e;

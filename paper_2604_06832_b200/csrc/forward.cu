@@ -104,6 +104,7 @@ static int forward_rows_simt(fdvlm_t* h, int n, int mode, int logits_rows) {
     launch_qkv_post(h->y, h->cs, h->q, kv_ptr(h, l, 0), kv_ptr(h, l, 1), n, h->cache_len, c.n_q_heads, c.n_kv_heads, d,
                     c.max_seq, dt, h->st);
     AttnArgs at;
+    at.len_ptr = nullptr;
     at.q = h->q; at.kc = kv_ptr(h, l, 0); at.vc = kv_ptr(h, l, 1); at.out = h->ao; at.n = n; at.cache_len = h->cache_len;
     at.max_seq = c.max_seq; at.hq = c.n_q_heads; at.hkv = c.n_kv_heads; at.d = d; at.causal = (mode == MODE_CAUSAL);
     at.dtype = dt; at.workspace = h->ws;
@@ -148,7 +149,7 @@ static int forward_rows_simt(fdvlm_t* h, int n, int mode, int logits_rows) {
 //            [O GEMM -> partials] [sum + residual + gain + ssq] [gate/up GEMM, folded norm + SwiGLU epilogue]
 //            [down GEMM -> partials] [sum + residual + gain + ssq]
 // head:      [LM-head GEMM, folded final norm, logits + softmax statistics epilogue] [statistics merge]
-static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int want_logits) {
+static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int want_logits, const int* len_ptr) {
   const fdvlm_config& c = h->cfg;
   const int H = c.hidden, I = c.intermediate, d = c.head_dim, nt = h->nt;
   const int NQ = c.n_q_heads * d, NKV = c.n_kv_heads * d, NQKV = NQ + 2 * NKV;
@@ -175,7 +176,7 @@ static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int wan
     h->launches++;
     return e == cudaSuccess;
   };
-  launch_rope_table(h->cs, n, h->cache_len, d, c.rope_theta, h->st);
+  launch_rope_table(h->cs, n, h->cache_len, d, c.rope_theta, h->st, len_ptr);
   h->launches++;
   for (int l = 0; l < c.n_layers; ++l) {
     const fdvlm_layer_weights& lw = h->layers[l];
@@ -185,8 +186,9 @@ static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int wan
     if (!gemm(group(h->a, n, H, 3, lw.wq, NQ, lw.wk, NKV, lw.wv, NKV), o))
       return fail(h, FDVLM_ERR_CUDA, "qkv projection launch: %s", cudaGetErrorString(e));
     launch_fin_qkv(part, S, n, h->cs, h->ssq, nt, H, c.rms_eps, lw.bq, lw.bk, lw.bv, lw.s_q, lw.s_k, lw.s_v, h->q, kv_ptr(h, l, 0), kv_ptr(h, l, 1),
-                   h->cache_len, c.n_q_heads, c.n_kv_heads, d, c.max_seq, h->st);
+                   h->cache_len, c.n_q_heads, c.n_kv_heads, d, c.max_seq, h->st, len_ptr);
     AttnArgs at;
+    at.len_ptr = len_ptr;
     at.q = h->q; at.kc = kv_ptr(h, l, 0); at.vc = kv_ptr(h, l, 1); at.out = h->ao; at.n = n; at.cache_len = h->cache_len;
     at.max_seq = c.max_seq; at.hq = c.n_q_heads; at.hkv = c.n_kv_heads; at.d = d; at.causal = (mode == MODE_CAUSAL);
     at.dtype = h->dt; at.workspace = h->ws;
@@ -237,9 +239,41 @@ static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int wan
   return FDVLM_OK;
 }
 
+// The tensor-core forward as a replayed CUDA graph: every kernel takes the cache length from a device word, so one
+// capture per (rows, mode, logits mode) serves every later call; the programmatic-dependent-launch edges are kept.
+static int forward_rows_graph(fdvlm_t* h, int n, int mode, int logits_rows, int want_logits) {
+  launch_set_len(h->dev_len, h->cache_len, h->st);
+  h->launches++;
+  for (auto& g : h->graphs) {
+    if (g.n == n && g.mode == mode && g.logits_rows == logits_rows && g.want_logits == want_logits) {
+      CU(h, cudaGraphLaunch(g.exec, h->st));
+      h->launches += g.launches;
+      return FDVLM_OK;
+    }
+  }
+  const int before = h->launches;
+  CU(h, cudaStreamBeginCapture(h->st, cudaStreamCaptureModeThreadLocal));
+  const int rc = forward_rows_tc(h, n, mode, logits_rows, want_logits, h->dev_len);
+  cudaGraph_t graph = nullptr;
+  cudaError_t e = cudaStreamEndCapture(h->st, &graph);
+  if (rc != FDVLM_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
+  if (e != cudaSuccess) return fail(h, FDVLM_ERR_CUDA, "graph capture: %s", cudaGetErrorString(e));
+  fdvlm::FwdGraph g;
+  g.n = n; g.mode = mode; g.logits_rows = logits_rows; g.want_logits = want_logits; g.launches = h->launches - before; g.exec = nullptr;
+  e = cudaGraphInstantiate(&g.exec, graph, 0);
+  cudaGraphDestroy(graph);
+  if (e != cudaSuccess) return fail(h, FDVLM_ERR_CUDA, "graph instantiate: %s", cudaGetErrorString(e));
+  h->graphs.push_back(g);
+  CU(h, cudaGraphLaunch(g.exec, h->st));
+  return FDVLM_OK;
+}
+
 int forward_rows(fdvlm_t* h, int n, int mode, int logits_rows, int want_logits) {
   if (h->mega) return mega_forward(h, n, mode, logits_rows, want_logits);
-  return h->use_tc ? forward_rows_tc(h, n, mode, logits_rows, want_logits) : forward_rows_simt(h, n, mode, logits_rows);
+  if (!h->use_tc) return forward_rows_simt(h, n, mode, logits_rows);
+  // per-kernel timing needs the kernels launched one by one
+  if (h->use_graphs && !h->prof_on) return forward_rows_graph(h, n, mode, logits_rows, want_logits);
+  return forward_rows_tc(h, n, mode, logits_rows, want_logits, nullptr);
 }
 
 }  // namespace fdk

@@ -21,6 +21,10 @@ struct fdvlm {
   int use_tc;      // bf16 weights: tcgen05 + TMA GEMMs, tensor-core attention, folded norms
   void* mega;      // persistent forward kernel context (null: kernel-per-operator path)
   char* slab;      // one allocation behind every device buffer below except the KV cache
+  int32_t* dev_len;   // device copy of cache_len, read by the captured forward graphs
+  int use_graphs;     // tensor-core path: replay one captured CUDA graph per (rows, mode, logits mode)
+  struct FwdGraph { int n, mode, logits_rows, want_logits, launches; cudaGraphExec_t exec; };
+  std::vector<FwdGraph> graphs;
   char* mega_slab; // the persistent kernel's share of the slab (counters, tensor maps, partial sums)
   // device buffers (R = max_block rows)
   char* kv;        // [n_layers][2][Hkv][max_seq][d]

@@ -224,9 +224,17 @@ void launch_rmsnorm(const float* h, const float* g, void* out, int n, int hidden
 // ================================================================================================
 // rotary table: cs[r][j] = (cos, sin)(pos * theta^(-2j/d)), angles formed in fp64
 // ================================================================================================
-__global__ void rope_table_kernel(float2* __restrict__ cs, int n, int pos0, int half, double theta) {
+__global__ void set_len_kernel(int* len_ptr, int value) {
   pdl_trigger();
   pdl_wait();
+  *len_ptr = value;
+}
+void launch_set_len(int* len_ptr, int value, cudaStream_t st) { set_len_kernel<<<1, 1, 0, st>>>(len_ptr, value); }
+
+__global__ void rope_table_kernel(float2* __restrict__ cs, int n, int pos0, int half, double theta, const int* __restrict__ len_ptr) {
+  pdl_trigger();
+  pdl_wait();
+  if (len_ptr) pos0 = *len_ptr;
   int idx = blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= n * half) return;
   int r = idx / half, j = idx % half;
@@ -235,9 +243,9 @@ __global__ void rope_table_kernel(float2* __restrict__ cs, int n, int pos0, int 
   sincos(ang, &s, &c);
   cs[idx] = make_float2((float)c, (float)s);
 }
-void launch_rope_table(float* cs, int n, int pos0, int head_dim, float theta, cudaStream_t st) {
+void launch_rope_table(float* cs, int n, int pos0, int head_dim, float theta, cudaStream_t st, const int* len_ptr) {
   int half = head_dim / 2, total = n * half;
-  launch_pdl(rope_table_kernel, dim3((total + 127) / 128), dim3(128), 0, st, (float2*)cs, n, pos0, half, (double)theta);
+  launch_pdl(rope_table_kernel, dim3((total + 127) / 128), dim3(128), 0, st, (float2*)cs, n, pos0, half, (double)theta, len_ptr);
 }
 
 // rotate-half pairing (j, j + d/2); q -> q buffer, k -> cache K plane, v -> cache V plane
@@ -324,9 +332,10 @@ __global__ void fin_qkv_kernel(const float* __restrict__ part, int S, int m, con
                                const float* __restrict__ bq, const float* __restrict__ bk, const float* __restrict__ bv,
                                const float* __restrict__ sq, const float* __restrict__ sk, const float* __restrict__ sv,
                                bf16* __restrict__ q, bf16* __restrict__ kc, bf16* __restrict__ vc, int pos0, int hq, int hkv,
-                               int d, int max_seq) {
+                               int d, int max_seq, const int* __restrict__ len_ptr) {
   pdl_trigger();
   pdl_wait();
+  if (len_ptr) pos0 = *len_ptr;
   __shared__ float s_rstd;
   const int head = blockIdx.x, r = blockIdx.y, j = threadIdx.x, half = d >> 1;
   if (threadIdx.x < 32) {
@@ -370,9 +379,9 @@ __global__ void fin_qkv_kernel(const float* __restrict__ part, int S, int m, con
 }
 void launch_fin_qkv(const float* part, int S, int m, const float* cs, const float* ssq, int nt, int hidden, float eps,
                     const float* bq, const float* bk, const float* bv, const float* sq, const float* sk, const float* sv, void* q, void* kc, void* vc, int pos0, int hq,
-                    int hkv, int d, int max_seq, cudaStream_t st) {
+                    int hkv, int d, int max_seq, cudaStream_t st, const int* len_ptr) {
   launch_pdl(fin_qkv_kernel, dim3(hq + 2 * hkv, m), dim3(d / 2), 0, st, part, S, m, (const float2*)cs, ssq, nt, 1.f / (float)hidden, eps, bq, bk,
-                                                          bv, sq, sk, sv, (bf16*)q, (bf16*)kc, (bf16*)vc, pos0, hq, hkv, d, max_seq);
+                                                          bv, sq, sk, sv, (bf16*)q, (bf16*)kc, (bf16*)vc, pos0, hq, hkv, d, max_seq, len_ptr);
 }
 
 // Residual finalisation: h += sum of split-K partials; xg = bf16(h * gain of the next norm); ssq[row][tile] =

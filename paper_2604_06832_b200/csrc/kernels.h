@@ -27,7 +27,8 @@ int launch_linear(const LinearArgs& a, cudaStream_t st, cudaError_t* err);
 void launch_embed(const void* table, const int32_t* tokens, float* h, int n, int hidden, int dtype, cudaStream_t st);
 void launch_rows_to_f32(const void* rows, float* h, int n, int hidden, int dtype, cudaStream_t st);
 void launch_rmsnorm(const float* h, const float* g, void* out, int n, int hidden, float eps, int dtype, cudaStream_t st);
-void launch_rope_table(float* cs, int n, int pos0, int head_dim, float theta, cudaStream_t st);
+void launch_rope_table(float* cs, int n, int pos0, int head_dim, float theta, cudaStream_t st, const int* len_ptr = nullptr);
+void launch_set_len(int* len_ptr, int value, cudaStream_t st);
 // qkv fp32 [n, (Hq + 2 Hkv) d] -> q (act type) [n, Hq, d] rotated; K (rotated) and V written into the
 // layer's cache planes [Hkv, max_seq, d] at positions pos0 .. pos0 + n - 1.
 void launch_qkv_post(const float* qkv, const float* cs, void* q, void* kc, void* vc, int n, int pos0,
@@ -76,7 +77,7 @@ void launch_embed_prep(const void* table, const int32_t* tokens, const void* row
 void launch_fin_qkv(const float* part, int S, int m, const float* cs, const float* ssq, int nt, int hidden, float eps,
                     const float* bq, const float* bk, const float* bv, const float* sq, const float* sk, const float* sv, void* q,
                     void* kc, void* vc, int pos0, int hq,
-                    int hkv, int d, int max_seq, cudaStream_t st);
+                    int hkv, int d, int max_seq, cudaStream_t st, const int* len_ptr = nullptr);
 void launch_fin_resid(const float* part, int S, int m, int hidden, float* h, const float* g, void* xg, float* ssq, int nt,
                       const float* scale, cudaStream_t st);
 void launch_stats_merge(const void* stats, int n_part, int m, float* conf, int32_t* pred, cudaStream_t st);
@@ -89,6 +90,7 @@ struct AttnArgs {
   void* out;       // [n, Hq*d]
   int n, cache_len, max_seq, hq, hkv, d, causal, dtype;
   void* workspace;
+  const int* len_ptr;   // nullable: device word holding the cache length (overrides cache_len; bf16 kernel only)
 };
 size_t attention_workspace_bytes(int n, int hq, int hkv, int d);
 int launch_attention(const AttnArgs& a, cudaStream_t st, cudaError_t* err);

@@ -11,11 +11,13 @@ TOL = {I.F32: dict(logits=1e-4, conf=1e-4), I.BF16: dict(logits=3e-2, conf=5e-3)
 MARGIN = 1e-3
 
 
-def make_pair(shape, seed, max_seq, max_block=64, **wkw):
+def make_pair(shape, seed, max_seq, max_block=64, stream=None, **wkw):
+    """`stream`: a torch.cuda.Stream for the handle (the library then replays captured CUDA graphs; on the default
+    stream it launches kernel by kernel)."""
     from paper_2604_06832_b200 import binding as B
     w = I.make_weights(shape, seed, **wkw)
     oracle = orc.Oracle(shape, I.weights_to_numpy(w))
-    handle = B.Handle(shape, B.weights_to_device(w), max_seq=max_seq, max_block=max_block)
+    handle = B.Handle(shape, B.weights_to_device(w), max_seq=max_seq, max_block=max_block, stream=stream)
     return oracle, handle, w
 
 

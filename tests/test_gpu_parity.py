@@ -161,6 +161,24 @@ def test_small_bf16_fp8_parity(shape, B_, L_e, L_t, rule, k):
     handle.close()
 
 
+@pytest.mark.parametrize("shape,B_", [(SMALL_BF16, 32), (SMALL_BF16, 5), (SMALL_FP8, 16)])
+def test_parity_through_captured_graphs_on_a_user_stream(shape, B_):
+    """On a caller-given stream the forward is replayed from CUDA graphs captured once per (rows, mode): several blocks
+    at growing cache lengths must keep matching the oracle (the cache length travels through device memory)."""
+    stream = torch.cuda.Stream()
+    oracle, handle, _ = make_pair(shape, 21, max_seq=400, stream=stream, qkv_bias=True)
+    emb, toks = I.make_prefix(shape, 37, 30, 6)
+    ref_last = oracle.prefill(I.as_numpy_storage(emb), toks.numpy())
+    last = torch.empty(shape.vocab, dtype=torch.float32, device="cuda")
+    with torch.cuda.stream(stream):
+        handle.prefill(*upload_prefix(emb, toks), last)
+        stream.synchronize()
+        assert np.abs(last.double().cpu().numpy() - ref_last).max() <= TOL[shape.dtype]["logits"]
+        stats = replay_decode(oracle, handle, shape, B_, orc.TOPK, 0.9, 4, n_blocks=3)
+    assert stats["steps"] >= 3 and handle.cache_len() == 67 + 3 * B_
+    handle.close()
+
+
 def test_small_bf16_peaked_discrete_parity():
     oracle, handle, _ = make_pair(SMALL_BF16, 9, max_seq=256, final_gain=16.0)
     emb, toks = I.make_prefix(SMALL_BF16, 20, 20, 4)
