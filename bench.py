@@ -281,6 +281,13 @@ def run_ours(args, wl, block):
     wbytes = shape.weight_bytes()
     gemm_ms_per_fwd = prof["ms_linear"] / n_steps
     gemm_gbs = wbytes / (gemm_ms_per_fwd / 1000.0) / 1e9
+    # DRAM bytes of the same launches, from the ncu captures summarised under profiles/ (dram read + write over
+    # algorithmic bytes of the four layer projections, measured on the 4-layer cut of the shape and scaled by the
+    # weight bytes: traffic grows in proportion).  None for shapes without a capture.
+    ratio = {"cfg2_3b_bf16_p1024_b32_top8": 158.55 / 154.15, "cfg3_3b_bf16_p2048_sweep": 158.55 / 154.15,
+             "cfg4_3b_bf16_p8192_b32_top8": 158.55 / 154.15, "cfg5_7b_fp8_p1024_b32": 240.71 / 233.06}.get(wl.name)
+    traffic = None if ratio is None or block != 32 else wbytes * ratio
+    traffic_note = None if traffic is None else "scaled from the 4-layer ncu capture of the same layer shapes (profiles/)"
     step_bytes = wbytes + shape.kv_bytes_per_token() * L_step
     step_med = statistics.median(lat)
     line = {
@@ -295,7 +302,9 @@ def run_ours(args, wl, block):
         "gpu_launches": n_launch,
         "clocks": clocks,
         "roofline": {"bound": "hbm", "achieved": gemm_gbs, "peak": peak, "unit": "GB/s", "frac": gemm_gbs / peak,
-                     "traffic": None, "peak_kind": peak_kind, "kernel": "projection GEMMs (all linear weights of one forward)",
+                     "traffic": traffic, "traffic_note": traffic_note, "peak_kind": peak_kind,
+                     "kernel": "gemm_tc_kernel: all projection launches of one forward (timed one by one with CUDA events, "
+                               "i.e. without the overlap of the live chain)",
                      "algorithmic_bytes_per_forward": wbytes, "ms_per_forward": gemm_ms_per_fwd},
         "step": {"latency_ms_median": step_med, "latency_ms_all": lat, "cache_len": L_step, "bytes": step_bytes,
                  "gbs": step_bytes / (step_med / 1000.0) / 1e9, "frac_of_peak": step_bytes / (step_med / 1000.0) / 1e9 / peak,
