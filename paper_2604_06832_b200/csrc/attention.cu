@@ -22,12 +22,12 @@ __global__ void __launch_bounds__(128) attn_mma_kernel(const bf16* __restrict__ 
                                                        const int* __restrict__ len_ptr) {
   extern __shared__ __align__(128) uint8_t smem[];
   pdl_trigger();
-  pdl_wait();
-  if (len_ptr) {
+  if (len_ptr) {   // the length word is written before the forward starts, not by a predecessor kernel
     L = *len_ptr;
     attn_chunking(L + n, (int)gridDim.x, &chunk_keys, &n_chunks);
-    if ((int)blockIdx.x >= n_chunks) return;
   }
+  pdl_wait();
+  if ((int)blockIdx.x >= n_chunks) return;
   attn_item<D>(q, kc, vc, part_o, part_ml, n, L, max_seq, hq, hkv, qh, chunk_keys, n_chunks, causal, blockIdx.x, blockIdx.y,
                blockIdx.z, (uint32_t)__cvta_generic_to_shared(smem), threadIdx.x);
 }
@@ -38,11 +38,11 @@ __global__ void __launch_bounds__(128) attn_combine_kernel(const float* __restri
                                                           bf16* __restrict__ out, int n, int hq, int n_chunks,
                                                           const int* __restrict__ len_ptr, int bound) {
   pdl_trigger();
-  pdl_wait();
   if (len_ptr) {
     int ck;
     attn_chunking(*len_ptr + n, bound, &ck, &n_chunks);
   }
+  pdl_wait();
   const int p = blockIdx.x * 4 + (threadIdx.x >> 5);
   if (p >= n * hq) return;
   const int i = p / hq, head = p % hq;

@@ -222,8 +222,32 @@ template <int D>
 __device__ __forceinline__ void attn_merge_warp(const float* att_o, const float2* att_ml, bf16* out, size_t slot0, int n_chunks,
                                                 int lane) {
   constexpr int VPL = D / 32;
-  float mx = -INFINITY;
-  for (int c = lane; c < n_chunks; c += 32) mx = fmaxf(mx, __ldcg(&att_ml[slot0 + c]).x);
+  constexpr int CB = 16;     // chunks whose partial outputs are in flight together
+  // The statistics and the first CB partial outputs are requested together: one L2 round trip for up to 16 chunks.
+  float2 ml0 = make_float2(-INFINITY, 0.f);
+  if (lane < n_chunks) ml0 = __ldcg(&att_ml[slot0 + lane]);
+  float ov[CB][VPL];
+  auto issue = [&](int c0) {
+#pragma unroll
+    for (int cc = 0; cc < CB; ++cc) {
+      const float* src = att_o + (slot0 + c0 + cc) * D + lane * VPL;
+      if (c0 + cc < n_chunks) {
+        if (VPL == 4) {
+          const float4 o = __ldcg(reinterpret_cast<const float4*>(src));
+          ov[cc][0] = o.x; ov[cc][1] = o.y; ov[cc][2] = o.z; ov[cc][VPL - 1] = o.w;
+        } else {
+          const float2 o = __ldcg(reinterpret_cast<const float2*>(src));
+          ov[cc][0] = o.x; ov[cc][VPL - 1] = o.y;
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < VPL; ++i) ov[cc][i] = 0.f;
+      }
+    }
+  };
+  issue(0);
+  float mx = ml0.x;
+  for (int c = lane + 32; c < n_chunks; c += 32) mx = fmaxf(mx, __ldcg(&att_ml[slot0 + c]).x);
   mx = warp_max(mx);
   float den = 0.f, acc[VPL];
 #pragma unroll
@@ -232,20 +256,16 @@ __device__ __forceinline__ void attn_merge_warp(const float* att_o, const float2
     const int c = c0 + lane;
     float w = 0.f;
     if (c < n_chunks) {
-      const float2 ml = __ldcg(&att_ml[slot0 + c]);
+      const float2 ml = (c0 == 0) ? ml0 : __ldcg(&att_ml[slot0 + c]);
       if (ml.y != 0.f) { w = exp2f(ml.x - mx); den = fmaf(w, ml.y, den); }
     }
-    const int cn = min(32, n_chunks - c0);
-#pragma unroll 8
-    for (int cc = 0; cc < cn; ++cc) {
-      const float wc = __shfl_sync(0xffffffffu, w, cc);
-      const float* src = att_o + (slot0 + c0 + cc) * D + lane * VPL;
-      if (VPL == 4) {
-        const float4 o = __ldcg(reinterpret_cast<const float4*>(src));
-        acc[0] = fmaf(wc, o.x, acc[0]); acc[1] = fmaf(wc, o.y, acc[1]); acc[2] = fmaf(wc, o.z, acc[2]); acc[VPL - 1] = fmaf(wc, o.w, acc[VPL - 1]);
-      } else {
-        const float2 o = __ldcg(reinterpret_cast<const float2*>(src));
-        acc[0] = fmaf(wc, o.x, acc[0]); acc[VPL - 1] = fmaf(wc, o.y, acc[VPL - 1]);
+    for (int h0 = 0; h0 < 32 && c0 + h0 < n_chunks; h0 += CB) {
+      if (c0 + h0 > 0) issue(c0 + h0);
+#pragma unroll
+      for (int cc = 0; cc < CB; ++cc) {
+        const float wc = __shfl_sync(0xffffffffu, w, h0 + cc);     // zero for chunks past the end
+#pragma unroll
+        for (int i = 0; i < VPL; ++i) acc[i] = fmaf(wc, ov[cc][i], acc[i]);
       }
     }
   }

@@ -311,15 +311,26 @@ void launch_embed_prep(const void* table, const int32_t* tokens, const void* row
   embed_prep_kernel<<<n, 256, 0, st>>>((const bf16*)table, tokens, (const bf16*)rows, h, (bf16*)xg, g, ssq, nt, hidden);
 }
 
-// Sum of S split-K partials p[i * stride], eight loads in flight at a time, added in index order (deterministic).
-__device__ __forceinline__ float sum_partials(const float* __restrict__ p, size_t stride, int S) {
-  float s = 0.f;
-  for (int i0 = 0; i0 < S; i0 += 8) {
-    float r[8];
+// Sum of S split-K partials p[i * stride].  These kernels are a handful of dependent L2 round trips long, so every
+// load that can be issued at once is: N loads in flight per call, added in index order (deterministic).
+template <int N> struct Partials { float r[N]; };
+template <int N>
+__device__ __forceinline__ void issue_partials(Partials<N>& v, const float* __restrict__ p, size_t stride, int i0, int S) {
 #pragma unroll
-    for (int j = 0; j < 8; ++j) r[j] = (i0 + j < S) ? __ldcg(p + (size_t)(i0 + j) * stride) : 0.f;
+  for (int j = 0; j < N; ++j) v.r[j] = (i0 + j < S) ? __ldcg(p + (size_t)(i0 + j) * stride) : 0.f;
+}
+template <int N>
+__device__ __forceinline__ float add_partials(const Partials<N>& v, float s) {
 #pragma unroll
-    for (int j = 0; j < 8; ++j) s += r[j];
+  for (int j = 0; j < N; ++j) s += v.r[j];
+  return s;
+}
+// the partials from index i0 on, added to s
+__device__ __forceinline__ float sum_partials_from(const float* __restrict__ p, size_t stride, int i0, int S, float s) {
+  for (; i0 < S; i0 += 16) {
+    Partials<16> v;
+    issue_partials(v, p, stride, i0, S);
+    s = add_partials(v, s);
   }
   return s;
 }
@@ -334,44 +345,53 @@ __global__ void fin_qkv_kernel(const float* __restrict__ part, int S, int m, con
                                bf16* __restrict__ q, bf16* __restrict__ kc, bf16* __restrict__ vc, int pos0, int hq, int hkv,
                                int d, int max_seq, const int* __restrict__ len_ptr) {
   pdl_trigger();
-  pdl_wait();
-  if (len_ptr) pos0 = *len_ptr;
-  __shared__ float s_rstd;
   const int head = blockIdx.x, r = blockIdx.y, j = threadIdx.x, half = d >> 1;
-  if (threadIdx.x < 32) {
-    float s = 0.f;
-    for (int t = threadIdx.x; t < nt; t += 32) s += ssq[(size_t)r * nt + t];
-    // fixed order: lanes hold disjoint strided subsets, combined by the butterfly below
-    s = warp_sum(s);
-    if (threadIdx.x == 0) s_rstd = rsqrtf(s * inv_h + eps);
+  // not written by any kernel of this forward: the cache length word, the scales and the biases
+  if (len_ptr) pos0 = *len_ptr;
+  float sc_a = 1.f, sc_b = 1.f, bi_a = 0.f, bi_b = 0.f;
+  {
+    const int hl = head < hq ? head : (head < hq + hkv ? head - hq : head - hq - hkv);
+    const float* sc = head < hq ? sq : (head < hq + hkv ? sk : sv);
+    const float* bi = head < hq ? bq : (head < hq + hkv ? bk : bv);
+    if (sc) { sc_a = sc[hl * d + j]; sc_b = sc[hl * d + j + half]; }   // fp8 weights: per-output-channel factors
+    if (bi) { bi_a = bi[hl * d + j]; bi_b = bi[hl * d + j + half]; }
   }
-  __syncthreads();
-  const float rstd = s_rstd;
+  pdl_wait();
+  __shared__ float s_rstd;
+  // every load of this kernel is issued before the first result is needed
   const int width = (hq + 2 * hkv) * d;
   const size_t sstride = (size_t)m * width;
   const float* pa = part + (size_t)r * width + head * d + j;
-  float a = sum_partials(pa, sstride, S), b = sum_partials(pa + half, sstride, S);
-  a *= rstd; b *= rstd;
-  if (sq) {   // fp8 weights: per-output-channel factors
-    const float* sc = head < hq ? sq + head * d : (head < hq + hkv ? sk + (head - hq) * d : sv + (head - hq - hkv) * d);
-    a *= sc[j]; b *= sc[j + half];
+  float ssq_v = 0.f;
+  if (threadIdx.x < 32)
+    for (int t = threadIdx.x; t < nt; t += 32) ssq_v += __ldcg(ssq + (size_t)r * nt + t);
+  const float2 c = (head < hq + hkv) ? __ldcg(&cs[r * half + j]) : make_float2(1.f, 0.f);
+  Partials<16> va, vb;
+  issue_partials(va, pa, sstride, 0, S);
+  issue_partials(vb, pa + half, sstride, 0, S);
+  if (threadIdx.x < 32) {
+    // fixed order: lanes hold disjoint strided subsets, combined by the butterfly below
+    const float t = warp_sum(ssq_v);
+    if (threadIdx.x == 0) s_rstd = rsqrtf(t * inv_h + eps);
   }
+  float a = add_partials(va, 0.f), b = add_partials(vb, 0.f);
+  a = sum_partials_from(pa, sstride, 16, S, a);
+  b = sum_partials_from(pa + half, sstride, 16, S, b);
+  __syncthreads();
+  const float rstd = s_rstd;
+  a = a * rstd * sc_a + bi_a;
+  b = b * rstd * sc_b + bi_b;
   if (head < hq) {
-    if (bq) { a += bq[head * d + j]; b += bq[head * d + j + half]; }
-    const float2 c = cs[r * half + j];
     bf16* o = q + ((size_t)r * hq + head) * d;
     o[j] = __float2bfloat16_rn(a * c.x - b * c.y);
     o[j + half] = __float2bfloat16_rn(b * c.x + a * c.y);
   } else if (head < hq + hkv) {
     const int hk = head - hq;
-    if (bk) { a += bk[hk * d + j]; b += bk[hk * d + j + half]; }
-    const float2 c = cs[r * half + j];
     bf16* o = kc + ((size_t)hk * max_seq + pos0 + r) * d;
     o[j] = __float2bfloat16_rn(a * c.x - b * c.y);
     o[j + half] = __float2bfloat16_rn(b * c.x + a * c.y);
   } else {
     const int hk = head - hq - hkv;
-    if (bv) { a += bv[hk * d + j]; b += bv[hk * d + j + half]; }
     bf16* o = vc + ((size_t)hk * max_seq + pos0 + r) * d;
     o[j] = __float2bfloat16_rn(a);
     o[j + half] = __float2bfloat16_rn(b);
@@ -391,16 +411,21 @@ __global__ void __launch_bounds__(128) fin_resid_kernel(const float* __restrict_
                                                         bf16* __restrict__ xg, float* __restrict__ ssq, int nt,
                                                         const float* __restrict__ scale) {
   pdl_trigger();
-  pdl_wait();
   __shared__ float red[32];
   const int t = blockIdx.x, r = blockIdx.y, c = t * 128 + threadIdx.x;
+  // weights (gain, scale) do not depend on the predecessor
+  const float gc = (c < hidden) ? g[c] : 0.f;
+  const float sc = (c < hidden && scale) ? scale[c] : 1.f;
+  pdl_wait();
   float v = 0.f;
   if (c < hidden) {
     const size_t idx = (size_t)r * hidden + c, sstride = (size_t)m * hidden;
-    const float hv = h[idx];
-    v = hv + sum_partials(part + idx, sstride, S) * (scale ? scale[c] : 1.f);
+    Partials<32> pv;
+    issue_partials(pv, part + idx, sstride, 0, S);
+    const float hv = __ldcg(h + idx);
+    v = hv + sum_partials_from(part + idx, sstride, 32, S, add_partials(pv, 0.f)) * sc;
     h[idx] = v;
-    xg[idx] = __float2bfloat16_rn(v * g[c]);
+    xg[idx] = __float2bfloat16_rn(v * gc);
   }
   const float ss = block_sum(v * v, red);
   if (threadIdx.x == 0) ssq[(size_t)r * nt + t] = ss;
