@@ -65,7 +65,11 @@ struct TcSmem {
   static constexpr int B_BYTES = M_PAD * TC_BK * 2;
   static constexpr int STAGE_BYTES = W_BYTES + B_BYTES;
   static constexpr int CONV_OFF = STAGES * STAGE_BYTES;                // bf16 tiles made by the converters
-  static constexpr int BAR_OFF = CONV_OFF + (FP8 ? TC_NCONV * TC_A_BYTES : 0);
+  static constexpr int EX_OFF = CONV_OFF + (FP8 ? TC_NCONV * TC_A_BYTES : 0);   // SwiGLU epilogue: gate/up exchange
+  static constexpr int EX_ROWS = FP8 ? 16 : 32;                         // rows that pass through it per round
+  static constexpr int EX_ROUNDS = (M_PAD + EX_ROWS - 1) / EX_ROWS;
+  static constexpr int EX_BYTES = (M_PAD / EX_ROUNDS) * 256;
+  static constexpr int BAR_OFF = EX_OFF + EX_BYTES;
   static constexpr int TOTAL = BAR_OFF + 256 + 1024;  // barriers + alignment slack
 };
 
@@ -106,6 +110,9 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
   auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * TC_STAGES + 2 + a); };
   auto cfull_bar = [&](int c) { return bar0 + 8u * (2 * TC_STAGES + 4 + c); };
   auto cempty_bar = [&](int c) { return bar0 + 8u * (2 * TC_STAGES + 6 + c); };
+  // SwiGLU epilogue, per warp pair pr: exchange buffer written (exw) / read (exr), two arrivals each
+  auto exw_bar = [&](int pr) { return bar0 + 8u * (2 * TC_STAGES + 10 + pr); };
+  auto exr_bar = [&](int pr) { return bar0 + 8u * (2 * TC_STAGES + 12 + pr); };
   volatile uint32_t* tmem_slot = (volatile uint32_t*)(sm + L::BAR_OFF + 8 * (2 * TC_STAGES + 8));
   volatile int* abort_flag = (volatile int*)(sm + L::BAR_OFF + 8 * (2 * TC_STAGES + 8) + 8);
 
@@ -116,6 +123,7 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
     for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
     for (int c = 0; c < TC_NCONV; ++c) { mbar_init(cfull_bar(c), 4); mbar_init(cempty_bar(c), 1); }
+    for (int pr = 0; pr < 2; ++pr) { mbar_init(exw_bar(pr), 2); mbar_init(exr_bar(pr), 2); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -160,13 +168,9 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
           armed |= 1u << stage;
           armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
           if (p.mode == TC_MODE_SWIGLU) {
-            // 64 features per tile; TMEM lane quarter qq holds gate rows of features 16qq..16qq+15 in its lanes
-            // 0..15 and the matching up rows in lanes 16..31, so the epilogue pairs them with one shuffle
-#pragma unroll
-            for (int qq = 0; qq < 4; ++qq) {
-              tma_load_2d(a_dst + (32 * qq) * L::W_ROW, &p.tm_w[0], full_bar(stage), kb * TC_BK, tile * 64 + 16 * qq, pol_w);
-              tma_load_2d(a_dst + (32 * qq + 16) * L::W_ROW, &p.tm_w[1], full_bar(stage), kb * TC_BK, tile * 64 + 16 * qq, pol_w);
-            }
+            // 64 features per tile: their gate rows fill TMEM lanes 0..63, their up rows lanes 64..127
+            tma_load_2d(a_dst, &p.tm_w[0], full_bar(stage), kb * TC_BK, tile * 64, pol_w);
+            tma_load_2d(a_dst + L::W_BYTES / 2, &p.tm_w[1], full_bar(stage), kb * TC_BK, tile * 64, pol_w);
           } else {
             tma_load_2d(a_dst, &p.tm_w[mi], full_bar(stage), kb * TC_BK, r0, pol_w);
             tma_load_2d(a_dst + L::W_BYTES / 2, &p.tm_w[mi], full_bar(stage), kb * TC_BK, r0 + 64, pol_w);
@@ -311,19 +315,49 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
       if (lane == 0) mbar_arrive(tempty_bar(acc));
 
       if (p.mode == TC_MODE_SWIGLU) {
-        const int col = tile * 64 + q * 16 + (lane & 15);
-        const bool live = lane < 16 && col < p.inter;
-        const float sg = (live && p.scale[0]) ? p.scale[0][col] : 1.f;
-        const float su = (live && p.scale[1]) ? p.scale[1][col] : 1.f;
+        // Warps 0, 1 of the epilogue hold the gate values of features 32 pr + lane, warps 2, 3 the up values of the
+        // same features.  Each warp of a pair finishes half of the rows: it hands the other half of its values
+        // (scaled) to its partner through shared memory and takes the partner's values for its own rows.
+        constexpr int HALF = M_PAD / 2;
+        constexpr int ROUNDS = L::EX_ROUNDS;
+        static_assert(HALF % ROUNDS == 0, "rows per round");
+        constexpr int HR = HALF / ROUNDS;
+        const int side = q >> 1, pr = q & 1;
+        const int col = tile * 64 + pr * 32 + lane;
+        const bool live = col < p.inter;
+        const float sc = (live && p.scale[side]) ? p.scale[side][col] : 1.f;
+        float* ex = reinterpret_cast<float*>(sm + L::EX_OFF) + pr * (2 * HR * 32);   // [side][HR rows][32 lanes]
 #pragma unroll
-        for (int b = 0; b < M_PAD; ++b) {
-          const float other = __shfl_xor_sync(0xffffffffu, v[b], 16);   // lanes 0..15: the matching "up" value
-          const float rs = __shfl_sync(0xffffffffu, (b < 32) ? rs0 : rs1, b & 31);
-          if (live && b < p.m) {
-            const float g = v[b] * sg * rs;
-            p.act[(size_t)b * p.inter + col] = __float2bfloat16_rn(g / (1.f + __expf(-g)) * (other * su * rs));
+        for (int r = 0; r < ROUNDS; ++r) {
+          const uint32_t par = (uint32_t)(local * ROUNDS + r) & 1u;
+#pragma unroll
+          for (int b = 0; b < HR; ++b) {
+            // the gate side finishes rows 0 .. HALF-1 and sends its values of rows HALF ..; the up side the reverse
+            const int lo = r * HR + b, hi = HALF + r * HR + b;
+            const float rs_lo = __shfl_sync(0xffffffffu, (lo < 32) ? rs0 : rs1, lo & 31);
+            const float rs_hi = __shfl_sync(0xffffffffu, (hi < 32) ? rs0 : rs1, hi & 31);
+            ex[(side * HR + b) * 32 + lane] = side ? v[lo] * sc * rs_lo : v[hi] * sc * rs_hi;
           }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(exw_bar(pr));
+          if (!mbar_wait(exw_bar(pr), par, abort_flag)) { ok = false; break; }
+#pragma unroll
+          for (int b = 0; b < HR; ++b) {
+            const int lo = r * HR + b, hi = HALF + r * HR + b;
+            const float rs_lo = __shfl_sync(0xffffffffu, (lo < 32) ? rs0 : rs1, lo & 31);
+            const float rs_hi = __shfl_sync(0xffffffffu, (hi < 32) ? rs0 : rs1, hi & 31);
+            const float other = ex[((1 - side) * HR + b) * 32 + lane];
+            const float mine = side ? v[hi] * sc * rs_hi : v[lo] * sc * rs_lo;
+            const float g = side ? other : mine, u = side ? mine : other;
+            const int row = side ? hi : lo;
+            if (live && row < p.m) p.act[(size_t)row * p.inter + col] = __float2bfloat16_rn(g / (1.f + __expf(-g)) * u);
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(exr_bar(pr));
+          // the buffer may be rewritten once the partner has read it too
+          if (!mbar_wait(exr_bar(pr), par, abort_flag)) { ok = false; break; }
         }
+        if (!ok) break;
       } else if (p.mode == TC_MODE_LOGITS) {
         const int n = tile * TC_BM + q * 32 + lane;          // vocabulary id held by this lane
         const bool in_range = n < p.n_out[0];
@@ -508,7 +542,7 @@ cudaError_t tc_group_launch(const TcGroup& g, const TcOut& o, cudaStream_t st) {
   if (!make_tmap(&p.tm_x, g.x, g.m, g.k, mp)) return cudaErrorInvalidValue;
   int tiles = 0, col = 0;
   for (int i = 0; i < g.n_mats; ++i) {
-    if (!make_tmap(&p.tm_w[i], g.w[i], g.n[i], g.k, mode == TC_MODE_SWIGLU ? 16 : 64, g.fp8 != 0)) return cudaErrorInvalidValue;
+    if (!make_tmap(&p.tm_w[i], g.w[i], g.n[i], g.k, 64, g.fp8 != 0)) return cudaErrorInvalidValue;
     p.n_out[i] = g.n[i];
     p.tile_begin[i] = tiles;
     p.out_col[i] = col;
