@@ -26,9 +26,8 @@ __global__ void __launch_bounds__(128) attn_mma_kernel(const bf16* __restrict__ 
     L = *len_ptr;
     attn_chunking(L + n, (int)gridDim.x, &chunk_keys, &n_chunks);
   }
-  pdl_wait();
-  if ((int)blockIdx.x >= n_chunks) return;
-  attn_item<D>(q, kc, vc, part_o, part_ml, n, L, max_seq, hq, hkv, qh, chunk_keys, n_chunks, causal, blockIdx.x, blockIdx.y,
+  if ((int)blockIdx.x >= n_chunks) { pdl_wait(); return; }
+  attn_item<D, true>(q, kc, vc, part_o, part_ml, n, L, max_seq, hq, hkv, qh, chunk_keys, n_chunks, causal, blockIdx.x, blockIdx.y,
                blockIdx.z, (uint32_t)__cvta_generic_to_shared(smem), threadIdx.x);
 }
 

@@ -54,7 +54,10 @@ __device__ __forceinline__ void attn_bar() { asm volatile("bar.sync 1, 128;" :::
 // One attention work item: the query heads [hk * G + grp * qh, +qh) of KV head hk against the keys of `chunk`.
 // Called by 128 threads (tid 0..127) that own attn_smem_bytes<D>() bytes of shared memory at address sQ (128-byte
 // aligned).  Leaves the unnormalised partial (O, running max, running sum) of every row in part_o / part_ml.
-template <int D>
+// PDL: the caller is a kernel launched with programmatic dependent launch that has not yet waited for its predecessor
+// (which writes q and the K/V rows of positions >= L); a first key tile that lies wholly in the committed cache is
+// then requested before that wait.
+template <int D, bool PDL = false>
 __device__ __forceinline__ void attn_item(const bf16* q, const bf16* kc, const bf16* vc, float* part_o, float2* part_ml,
                                           int n, int L, int max_seq, int hq, int hkv, int qh, int chunk_keys, int n_chunks,
                                           int causal, int chunk, int grp, int hk, uint32_t sQ, int tid) {
@@ -74,14 +77,6 @@ __device__ __forceinline__ void attn_item(const bf16* q, const bf16* kc, const b
   const bf16* kbase = kc + (size_t)hk * max_seq * D;
   const bf16* vbase = vc + (size_t)hk * max_seq * D;
 
-  // ---- stage Q (rows = heads_here x n; row r -> head r / n, token r % n) ----
-  for (int v = tid; v < AT_ROWS * CH; v += 128) {
-    const int r = v / CH, c = v % CH;
-    const bool ok = r < m_valid;
-    const int hl = ok ? r / n : 0, i = ok ? r % n : 0;
-    const bf16* src = q + ((size_t)i * hq + head0 + hl) * D + c * 8;
-    cp_async16(sQ + swz<D>(r, c), src, ok ? 16 : 0);
-  }
   auto load_tile = [&](int t, int buf) {
     const int j0 = key_begin + t * AT_KEYS;
     for (int v = tid; v < AT_KEYS * CH; v += 128) {
@@ -93,7 +88,25 @@ __device__ __forceinline__ void attn_item(const bf16* q, const bf16* kc, const b
       cp_async16(sV + buf * TILE_BYTES + swz<D>(r, c), vbase + off, ok ? 16 : 0);
     }
   };
-  if (n_tiles > 0) load_tile(0, 0);
+  const bool early = PDL && n_tiles > 0 && key_begin + AT_KEYS <= L;
+  if (early) load_tile(0, 0);
+  // ---- stage Q (rows = heads_here x n; row r -> head r / n, token r % n); addresses worked out before the wait ----
+  constexpr int QV = AT_ROWS * CH / 128;
+  const bf16* q_src[QV];
+  uint32_t q_dst[QV];
+#pragma unroll
+  for (int u = 0; u < QV; ++u) {
+    const int v = tid + u * 128;
+    const int r = v / CH, c = v % CH;
+    const bool ok = r < m_valid;
+    const int hl = ok ? r / n : 0, i = ok ? r % n : 0;
+    q_src[u] = ok ? q + ((size_t)i * hq + head0 + hl) * D + c * 8 : nullptr;
+    q_dst[u] = sQ + swz<D>(r, c);
+  }
+  if (PDL) pdl_wait();
+#pragma unroll
+  for (int u = 0; u < QV; ++u) cp_async16(q_dst[u], q_src[u] ? q_src[u] : q, q_src[u] ? 16 : 0);
+  if (n_tiles > 0 && !early) load_tile(0, 0);
   cp_async_commit();
 
   const int row0 = warp * 16;                       // this warp's rows of the CTA tile
