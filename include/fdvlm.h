@@ -93,7 +93,10 @@ typedef struct {
  *  TOPK:      reveal the min(k, #masked) masked positions of highest confidence.
  *  Ties go to the lowest position index; the vocabulary argmax takes the lowest token id. */
 typedef enum { FDVLM_RULE_THRESHOLD = 0, FDVLM_RULE_TOPK = 1 } fdvlm_rule;
-typedef struct { fdvlm_rule rule; float threshold; int k; } fdvlm_step_params;
+/* pred_shift = 0: row i of the forward predicts position i (a block of B masks).  pred_shift = 1: the paper's
+ * convention (Appendix B, Alg. 1 "shift-by-one"): row i-1 predicts position i, so position 0 can never be predicted
+ * and must be a given token -- the AR seed of Sec. 3.4 "causal context decoding" (pass it through init_tokens). */
+typedef struct { fdvlm_rule rule; float threshold; int k; int pred_shift; } fdvlm_step_params;
 typedef struct { int n_unmasked, n_remaining, step_index; } fdvlm_step_info;
 
 /* Create a handle on the current CUDA device.  `cuda_stream` is a cudaStream_t (NULL = default
@@ -145,6 +148,31 @@ int fdvlm_block_set_tokens(fdvlm_t *h, const int32_t *tokens);
  * next_logits (device fp32 [vocab], nullable) = logits of the block's last row.
  * Errors: STATE if no block is open or masked positions remain. */
 int fdvlm_commit_block(fdvlm_t *h, float *next_logits);
+
+/* Commit as above and also return, for every row i of the block, the argmax token (mask_id excluded) and its
+ * confidence under the causal pass: row_pred[i] is the autoregressive prediction for the position after block row i
+ * (Appendix B, Alg. 1 "verify step": a_i = argmax h^v_i).  row_pred device int32 [B], row_conf device fp32 [B],
+ * next_logits device fp32 [vocab]; all nullable. */
+int fdvlm_commit_block_verify(fdvlm_t *h, int32_t *row_pred, float *row_conf, float *next_logits);
+
+/* Drop committed positions from the end of the cache: cache_len = new_len (Alg. 1 "Crop").  The dropped K/V rows
+ * are simply overwritten by later commits.  Errors: STATE inside an open block; INVALID_ARG unless
+ * 0 <= new_len <= cache_len. */
+int fdvlm_truncate(fdvlm_t *h, int new_len);
+
+/* One iteration of linear self-speculative decoding (Sec. 3.4 "self-speculative block decoding"; Appendix B,
+ * Alg. 1) with block size B: the block [seed, MASK x (B-1)] is drafted in one denoise pass (shift-by-one, every
+ * masked position filled), verified by one causal pass with cache update, and the longest prefix on which the
+ * causal predictions agree with the draft is accepted: k = 1 + (first j in [0, B-2] with a_j != d_{j+1}; B-1 if
+ * none).  The cache keeps block rows 0 .. k-1 (cache_len += k) and a_{k-1} is the next iteration's seed.
+ *   seed_token     the block's first token (from fdvlm_prefill's last_logits, or the previous call's next_token)
+ *   draft_tokens   device int32 [B], nullable: the block after the draft pass
+ *   verify_pred    device int32 [B], nullable: a_0 .. a_{B-1}
+ *   info           HOST, required: accepted k, next_token = a_{k-1}, cache_len after the call
+ * Always synchronous (the accepted length decides the cache length).  Errors as block_begin / block_step. */
+typedef struct { int accepted; int32_t next_token; int cache_len; } fdvlm_spec_info;
+int fdvlm_spec_block(fdvlm_t *h, int block_size, int32_t seed_token, int32_t *draft_tokens,
+                     int32_t *verify_pred, fdvlm_spec_info *info);
 
 /* Committed positions, or a negative status for a NULL handle. */
 int fdvlm_cache_len(const fdvlm_t *h);

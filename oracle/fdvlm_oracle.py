@@ -297,40 +297,103 @@ class Oracle:
         h = self.forward_rows(self.embed_tokens(self.block_tokens), BIDIR, update_cache=False)
         return self.logits_of(h)
 
-    def block_step(self, rule: str = THRESHOLD, threshold: float = 0.9, k: int = 8):
+    def block_step(self, rule: str = THRESHOLD, threshold: float = 0.9, k: int = 8, pred_shift: int = 0):
         """One denoise step (Sec. 3.4): forward, confidence, selection, reveal.
 
-        Returns dict(logits, conf, pred, margin, unmask, block_tokens, n_unmasked, n_remaining,
+        pred_shift = 0: row i predicts position i.  pred_shift = 1 (Appendix B, Alg. 1 "shift-by-one"): row i-1
+        predicts position i; position 0 has no predictor, it must already hold a given token (the AR seed of Sec. 3.4
+        "causal context decoding").  `conf` / `pred` in the record are per ROW; `pos_conf` / `pos_pred` are what
+        the selection used per POSITION.
+
+        Returns dict(logits, conf, pred, margin, pos_conf, pos_pred, unmask, block_tokens, n_unmasked, n_remaining,
         masked_before)."""
+        assert pred_shift in (0, 1)
         logits = self.block_forward()
         pred, conf, margin = confidence(logits, self.s.mask_id)
+        if pred_shift:
+            assert not self.masked[0], "with shift-by-one the first position of the block must be given"
+            pos_pred = np.concatenate([[-1], pred[:-1]])
+            pos_conf = np.concatenate([[NEG_INF], conf[:-1]])
+        else:
+            pos_pred, pos_conf = pred, conf
         before = self.masked.copy()
-        sel = select_unmask(conf, self.masked, rule, threshold, k)
-        self.block_tokens[sel] = pred[sel]
+        sel = select_unmask(pos_conf, self.masked, rule, threshold, k)
+        self.block_tokens[sel] = pos_pred[sel]
         self.masked = self.masked & ~sel
         self.step_index += 1
-        return dict(logits=logits, conf=conf, pred=pred, margin=margin, unmask=sel,
+        return dict(logits=logits, conf=conf, pred=pred, margin=margin, pos_conf=pos_conf, pos_pred=pos_pred, unmask=sel,
                     block_tokens=self.block_tokens.copy(), n_unmasked=int(sel.sum()),
                     n_remaining=int(self.masked.sum()), masked_before=before)
 
-    def commit_block(self, want_logits: bool = True):
+    def commit_block(self, want_logits: bool = True, all_rows: bool = False):
         """Causal pass over the finished block with cache update (Alg. 1 verify pass; clean context
         is token-causal, Sec. 3.3 M_C2C).  K/V computed during denoise passes are never stored.
-        Returns the last row's logits."""
+        Returns the last row's logits, or with all_rows the logits of every block row [B, vocab]
+        (row i = the autoregressive distribution of the token after block position i)."""
         assert self.block_tokens is not None and not self.masked.any()
         h = self.forward_rows(self.embed_tokens(self.block_tokens), CAUSAL, update_cache=True)
         self.block_tokens, self.masked = None, None
+        if all_rows:
+            return self.logits_of(h)
         return self.logits_of(h[-1:])[0] if want_logits else None
 
-    def decode_block(self, block_size: int, rule: str, threshold: float = 0.9, k: int = 8, init_tokens=None):
+    def truncate(self, new_len: int):
+        """Drop the cache entries of positions >= new_len (Alg. 1 "Crop")."""
+        assert self.block_tokens is None and 0 <= new_len <= self.cache_len
+        for l in range(self.s.n_layers):
+            self.K[l] = self.K[l][:new_len]
+            self.V[l] = self.V[l][:new_len]
+        self.cache_len = new_len
+
+    def decode_block(self, block_size: int, rule: str, threshold: float = 0.9, k: int = 8, init_tokens=None,
+                     pred_shift: int = 0):
         """Denoise one block to completion and commit it; returns the list of step records."""
         self.block_begin(block_size, init_tokens)
         steps = []
         while self.masked.any():
-            steps.append(self.block_step(rule, threshold, k))
+            steps.append(self.block_step(rule, threshold, k, pred_shift))
             assert steps[-1]["n_unmasked"] >= 1 and len(steps) <= block_size
         next_logits = self.commit_block()
         return steps, next_logits
+
+    def decode_block_seeded(self, block_size: int, seed_token: int, rule: str, threshold: float = 0.9, k: int = 8):
+        """A block decoded the paper's way (Sec. 3.4 "causal context decoding"; Alg. 1's block layout): the first
+        position holds the AR seed, the other B-1 are masks filled under shift-by-one; then the causal commit, whose
+        last row's argmax (mask token excluded) is the next block's seed.  Returns (block tokens, steps, next seed)."""
+        init = np.full(block_size, self.s.mask_id, dtype=np.int64)
+        init[0] = seed_token
+        self.block_begin(block_size, init)
+        steps = []
+        while self.masked.any():
+            steps.append(self.block_step(rule, threshold, k, pred_shift=1))
+            assert steps[-1]["n_unmasked"] >= 1 and len(steps) <= block_size - 1
+        tokens = self.block_tokens.copy()
+        next_logits = self.commit_block()
+        return tokens, steps, int(confidence(next_logits[None, :], self.s.mask_id)[0][0])
+
+    def spec_block(self, block_size: int, seed_token: int):
+        """One iteration of linear self-speculative decoding (Sec. 3.4; Appendix B, Alg. 1), in its notation:
+
+        d = [x_n, M, ..., M]; draft pass (denoise attention, no cache update): d_i <- argmax of row i-1 for the mask
+        positions i; verify pass (causal, cache updated with all B rows): a_i = argmax of row i; accept
+        k = 1 + min{ j in [0, B-2] : a_j != d_{j+1} } (no mismatch: k = B, the reading taken where Alg. 1 leaves the
+        minimum of an empty set undefined); the sequence gains a_0 .. a_{k-1}; the cache is cropped to the entries of
+        d_0 .. d_{k-1}.  a_{k-1} is the next iteration's x_n.  Argmax excludes the mask token.
+        Returns dict(draft, a, accepted, new_tokens, next_token)."""
+        B = block_size
+        L0 = self.cache_len
+        init = np.full(B, self.s.mask_id, dtype=np.int64)
+        init[0] = seed_token
+        self.block_begin(B, init)
+        if B > 1:
+            rec = self.block_step(THRESHOLD, NEG_INF, 0, pred_shift=1)      # every mask position filled in one pass
+            assert rec["n_remaining"] == 0
+        d = self.block_tokens.copy()
+        a = confidence(self.commit_block(all_rows=True), self.s.mask_id)[0]
+        mism = [j for j in range(0, B - 1) if a[j] != d[j + 1]]
+        k = (mism[0] if mism else B - 1) + 1
+        self.truncate(L0 + k)
+        return dict(draft=d, a=a, accepted=k, new_tokens=a[:k].copy(), next_token=int(a[k - 1]))
 
     # -- brute force: no cache, explicit [T, T] mask ----------------------------------------------
     def forward_dense(self, x: np.ndarray, allowed: np.ndarray, positions=None) -> np.ndarray:

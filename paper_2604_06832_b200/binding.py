@@ -46,11 +46,15 @@ class Weights(C.Structure):
 
 
 class StepParams(C.Structure):
-    _fields_ = [("rule", C.c_int), ("threshold", C.c_float), ("k", C.c_int)]
+    _fields_ = [("rule", C.c_int), ("threshold", C.c_float), ("k", C.c_int), ("pred_shift", C.c_int)]
 
 
 class StepInfo(C.Structure):
     _fields_ = [("n_unmasked", C.c_int), ("n_remaining", C.c_int), ("step_index", C.c_int)]
+
+
+class SpecInfo(C.Structure):
+    _fields_ = [("accepted", C.c_int), ("next_token", C.c_int32), ("cache_len", C.c_int)]
 
 
 EXPORTS = {
@@ -66,6 +70,9 @@ EXPORTS = {
                                         C.c_void_p, C.POINTER(StepInfo)]),
     "fdvlm_block_set_tokens": (C.c_int, [C.c_void_p, C.c_void_p]),
     "fdvlm_commit_block": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "fdvlm_commit_block_verify": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "fdvlm_truncate": (C.c_int, [C.c_void_p, C.c_int]),
+    "fdvlm_spec_block": (C.c_int, [C.c_void_p, C.c_int, C.c_int32, C.c_void_p, C.c_void_p, C.POINTER(SpecInfo)]),
     "fdvlm_cache_len": (C.c_int, [C.c_void_p]),
     "fdvlm_cache_read": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p]),
     "fdvlm_last_launch_count": (C.c_int, [C.c_void_p]),
@@ -177,15 +184,15 @@ class Handle:
         self._check(lib().fdvlm_block_begin_host(self._h, block_size, _ptr(init_tokens_host)))
 
     def block_step(self, rule: int, threshold: float = 0.9, k: int = 8, logits=None, conf=None, pred=None,
-                   unmask=None, block_tokens=None) -> StepInfo:
-        p, info = StepParams(rule, threshold, k), StepInfo()
+                   unmask=None, block_tokens=None, pred_shift: int = 0) -> StepInfo:
+        p, info = StepParams(rule, threshold, k, pred_shift), StepInfo()
         self._check(lib().fdvlm_block_step(self._h, C.byref(p), _ptr(logits), _ptr(conf), _ptr(pred), _ptr(unmask),
                                            _ptr(block_tokens), C.byref(info)))
         return info
 
     def block_step_host(self, rule: int, threshold: float = 0.9, k: int = 8, conf=None, pred=None, unmask=None,
-                        block_tokens=None) -> StepInfo:
-        p, info = StepParams(rule, threshold, k), StepInfo()
+                        block_tokens=None, pred_shift: int = 0) -> StepInfo:
+        p, info = StepParams(rule, threshold, k, pred_shift), StepInfo()
         self._check(lib().fdvlm_block_step_host(self._h, C.byref(p), _ptr(conf), _ptr(pred), _ptr(unmask),
                                                 _ptr(block_tokens), C.byref(info)))
         return info
@@ -195,6 +202,20 @@ class Handle:
 
     def commit_block(self, next_logits: Optional[torch.Tensor] = None):
         self._check(lib().fdvlm_commit_block(self._h, _ptr(next_logits)))
+
+    def commit_block_verify(self, row_pred: Optional[torch.Tensor] = None, row_conf: Optional[torch.Tensor] = None,
+                            next_logits: Optional[torch.Tensor] = None):
+        self._check(lib().fdvlm_commit_block_verify(self._h, _ptr(row_pred), _ptr(row_conf), _ptr(next_logits)))
+
+    def truncate(self, new_len: int):
+        self._check(lib().fdvlm_truncate(self._h, new_len))
+
+    def spec_block(self, block_size: int, seed_token: int, draft_tokens: Optional[torch.Tensor] = None,
+                   verify_pred: Optional[torch.Tensor] = None) -> SpecInfo:
+        info = SpecInfo()
+        self._check(lib().fdvlm_spec_block(self._h, block_size, seed_token, _ptr(draft_tokens), _ptr(verify_pred),
+                                           C.byref(info)))
+        return info
 
     def cache_len(self) -> int:
         return lib().fdvlm_cache_len(self._h)

@@ -273,6 +273,7 @@ static int step_core(fdvlm_t* h, const fdvlm_step_params* p, int want_logits) {
   if (p->rule != FDVLM_RULE_THRESHOLD && p->rule != FDVLM_RULE_TOPK) return fail(h, FDVLM_ERR_INVALID_ARG, "unknown rule");
   if (p->rule == FDVLM_RULE_TOPK && p->k < 1) return fail(h, FDVLM_ERR_INVALID_ARG, "top-k needs k >= 1");
   if (p->rule == FDVLM_RULE_THRESHOLD && !(p->threshold == p->threshold)) return fail(h, FDVLM_ERR_INVALID_ARG, "threshold is NaN");
+  if (p->pred_shift != 0 && p->pred_shift != 1) return fail(h, FDVLM_ERR_INVALID_ARG, "pred_shift is 0 or 1");
   if (!h->block_open) return fail(h, FDVLM_ERR_STATE, "block_step without an open block");
   if (h->n_remaining == 0) return fail(h, FDVLM_ERR_STATE, "block_step with no masked position left");
   const int B = h->block_size;
@@ -281,7 +282,8 @@ static int step_core(fdvlm_t* h, const fdvlm_step_params* p, int want_logits) {
   if (rc) return rc;
   rc = forward_rows(h, B, MODE_BIDIR, B, want_logits);
   if (rc) return rc;
-  launch_select(h->conf, h->pred, h->blk_tokens, h->blk_masked, h->unmask, h->info, B, (int)p->rule, p->threshold, p->k, h->st);
+  launch_select(h->conf, h->pred, h->blk_tokens, h->blk_masked, h->unmask, h->info, B, (int)p->rule, p->threshold, p->k, h->st,
+                p->pred_shift);
   h->launches++;
   CU(h, cudaGetLastError());
   h->step_index++;
@@ -292,6 +294,8 @@ static int finish_info(fdvlm_t* h, fdvlm_step_info* info) {
   int rc = sync_info(h);
   if (rc) return rc;
   if (info) { info->n_unmasked = h->info_host[0]; info->n_remaining = h->info_host[1]; info->step_index = h->info_host[2]; }
+  if (h->info_host[0] == 0 && h->info_host[1] > 0)
+    return fail(h, FDVLM_ERR_STATE, "no position could be revealed: with pred_shift = 1 position 0 of the block must be a given token");
   return FDVLM_OK;
 }
 
@@ -330,7 +334,9 @@ extern "C" int fdvlm_block_step_host(fdvlm_t* h, const fdvlm_step_params* p, flo
   return FDVLM_OK;
 }
 
-extern "C" int fdvlm_commit_block(fdvlm_t* h, float* next_logits) {
+// Causal pass over the finished block with cache update.  all_rows: confidence / prediction of every row are left in
+// h->conf / h->pred (and, with want_logits, all rows' logits in h->logits); else only the last row's logits.
+static int commit_core(fdvlm_t* h, int all_rows, int want_logits) {
   if (!h) return FDVLM_ERR_INVALID_ARG;
   if (!h->block_open) return fail(h, FDVLM_ERR_STATE, "commit without an open block");
   if (h->n_remaining != 0) return fail(h, FDVLM_ERR_STATE, "commit with %d masked positions left", h->n_remaining);
@@ -338,12 +344,84 @@ extern "C" int fdvlm_commit_block(fdvlm_t* h, float* next_logits) {
   h->launches = 0;
   int rc = stage_rows(h, 0, B, h->blk_tokens, nullptr);
   if (rc) return rc;
-  rc = forward_rows(h, B, MODE_CAUSAL, next_logits ? 1 : 0, 1);
+  rc = forward_rows(h, B, MODE_CAUSAL, all_rows ? B : (want_logits ? 1 : 0), all_rows ? want_logits : 1);
   if (rc) return rc;
-  if (next_logits) CU(h, cudaMemcpyAsync(next_logits, h->logits, (size_t)h->cfg.vocab * 4, cudaMemcpyDeviceToDevice, h->st));
   h->cache_len += B;
   h->block_open = 0;
   h->block_size = 0;
+  return FDVLM_OK;
+}
+
+extern "C" int fdvlm_commit_block(fdvlm_t* h, float* next_logits) {
+  int rc = commit_core(h, 0, next_logits != nullptr);
+  if (rc) return rc;
+  if (next_logits) CU(h, cudaMemcpyAsync(next_logits, h->logits, (size_t)h->cfg.vocab * 4, cudaMemcpyDeviceToDevice, h->st));
+  return FDVLM_OK;
+}
+
+extern "C" int fdvlm_commit_block_verify(fdvlm_t* h, int32_t* row_pred, float* row_conf, float* next_logits) {
+  if (!h) return FDVLM_ERR_INVALID_ARG;
+  const int B = h->block_size;
+  int rc = commit_core(h, 1, next_logits != nullptr);
+  if (rc) return rc;
+  const cudaMemcpyKind DD = cudaMemcpyDeviceToDevice;
+  if (row_pred) CU(h, cudaMemcpyAsync(row_pred, h->pred, (size_t)B * 4, DD, h->st));
+  if (row_conf) CU(h, cudaMemcpyAsync(row_conf, h->conf, (size_t)B * 4, DD, h->st));
+  if (next_logits) CU(h, cudaMemcpyAsync(next_logits, h->logits + (size_t)(B - 1) * h->cfg.vocab, (size_t)h->cfg.vocab * 4, DD, h->st));
+  return FDVLM_OK;
+}
+
+extern "C" int fdvlm_truncate(fdvlm_t* h, int new_len) {
+  if (!h) return FDVLM_ERR_INVALID_ARG;
+  if (h->block_open) return fail(h, FDVLM_ERR_STATE, "truncate inside an open block");
+  if (new_len < 0 || new_len > h->cache_len) return fail(h, FDVLM_ERR_INVALID_ARG, "truncate to %d of %d committed positions", new_len, h->cache_len);
+  h->cache_len = new_len;
+  return FDVLM_OK;
+}
+
+extern "C" int fdvlm_spec_block(fdvlm_t* h, int block_size, int32_t seed_token, int32_t* draft_tokens, int32_t* verify_pred,
+                                fdvlm_spec_info* info) {
+  if (!h) return FDVLM_ERR_INVALID_ARG;
+  if (!info) return fail(h, FDVLM_ERR_INVALID_ARG, "spec_block needs the host info struct");
+  if (seed_token < 0 || seed_token >= h->cfg.vocab || seed_token == h->cfg.mask_id)
+    return fail(h, FDVLM_ERR_INVALID_ARG, "seed token %d is not a vocabulary token", (int)seed_token);
+  int rc = block_begin_common(h, block_size);
+  if (rc) return rc;
+  const int B = block_size, L0 = h->cache_len;
+  int32_t init[64];
+  init[0] = seed_token;
+  for (int i = 1; i < B; ++i) init[i] = h->cfg.mask_id;
+  rc = fdvlm_block_begin_host(h, B, init);
+  if (rc) return rc;
+  if (B > 1) {
+    // draft: one denoise pass, shift-by-one, every masked position filled (threshold below any confidence)
+    fdvlm_step_params p;
+    p.rule = FDVLM_RULE_THRESHOLD; p.threshold = -1.f; p.k = 0; p.pred_shift = 1;
+    rc = step_core(h, &p, 0);
+    if (rc) return rc;
+    rc = sync_info(h);
+    if (rc) return rc;
+    if (h->n_remaining != 0) return fail(h, FDVLM_ERR_STATE, "draft pass left %d masked positions", h->n_remaining);
+  }
+  const cudaMemcpyKind DD = cudaMemcpyDeviceToDevice;
+  if (draft_tokens) CU(h, cudaMemcpyAsync(draft_tokens, h->blk_tokens, (size_t)B * 4, DD, h->st));
+  // verify: causal pass with cache update, predictions of every row
+  const int draft_launches = h->launches;
+  rc = commit_core(h, 1, 0);
+  if (rc) return rc;
+  if (verify_pred) CU(h, cudaMemcpyAsync(verify_pred, h->pred, (size_t)B * 4, DD, h->st));
+  launch_accept(h->pred, h->blk_tokens, B, h->init_stage, h->st);
+  h->launches += draft_launches + 1;
+  CU(h, cudaGetLastError());
+  CU(h, cudaMemcpyAsync(h->host_stage, h->init_stage, 8, cudaMemcpyDeviceToHost, h->st));
+  rc = sync_info(h);              // synchronises, and reports a timed-out device wait of either pass
+  if (rc) return rc;
+  const int k = ((const int32_t*)h->host_stage)[0];
+  if (k < 1 || k > B) return fail(h, FDVLM_ERR_CUDA, "accept kernel returned %d", k);
+  h->cache_len = L0 + k;          // crop: the rows after the accepted prefix are dropped
+  info->accepted = k;
+  info->next_token = ((const int32_t*)h->host_stage)[1];
+  info->cache_len = h->cache_len;
   return FDVLM_OK;
 }
 

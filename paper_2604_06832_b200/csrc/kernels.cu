@@ -551,14 +551,17 @@ void launch_row_stats(const float* logits, int n, int vocab, int mask_id, float*
 __global__ void select_kernel(const float* __restrict__ conf, const int32_t* __restrict__ pred,
                               int32_t* __restrict__ tokens, uint8_t* __restrict__ masked,
                               uint8_t* __restrict__ unmask, int32_t* __restrict__ info, int n, int rule,
-                              float threshold, int k) {
+                              float threshold, int k, int shift) {
   pdl_trigger();
   pdl_wait();
   __shared__ float c[64];
   __shared__ int mk[64];
   int i = threadIdx.x;
-  c[i] = i < n ? conf[i] : -1.f;
-  mk[i] = i < n ? (int)masked[i] : 0;
+  // shift = 1: position i is predicted by row i - 1; position 0 has no predictor and is never selected
+  c[i] = (i < n && i >= shift) ? conf[i - shift] : -1.f;
+  mk[i] = (i < n && i >= shift) ? (int)masked[i] : 0;
+  // a masked position 0 under shift = 1 has no predictor: nothing is revealed and it is reported as remaining
+  const int stuck = (shift && n > 0 && masked[0]) ? 1 : 0;
   __syncthreads();
   int is_m = mk[i];
   int rank = 0, n_masked = 0;
@@ -575,16 +578,32 @@ __global__ void select_kernel(const float* __restrict__ conf, const int32_t* __r
   } else {
     sel = is_m && rank < k;
   }
+  if (stuck) sel = 0;
   int n_sel = __syncthreads_count(sel);
   if (i < n) {
     unmask[i] = (uint8_t)sel;
-    if (sel) { tokens[i] = pred[i]; masked[i] = 0; }
+    if (sel) { tokens[i] = pred[i - shift]; masked[i] = 0; }
   }
-  if (i == 0) { info[0] = n_sel; info[1] = n_masked - n_sel; info[2] = info[2] + 1; }
+  if (i == 0) { info[0] = n_sel; info[1] = n_masked - n_sel + stuck; info[2] = info[2] + 1; }
 }
 void launch_select(const float* conf, const int32_t* pred, int32_t* tokens, uint8_t* masked, uint8_t* unmask,
-                   int32_t* info, int n, int rule, float threshold, int k, cudaStream_t st) {
-  select_kernel<<<1, 64, 0, st>>>(conf, pred, tokens, masked, unmask, info, n, rule, threshold, k);
+                   int32_t* info, int n, int rule, float threshold, int k, cudaStream_t st, int shift) {
+  select_kernel<<<1, 64, 0, st>>>(conf, pred, tokens, masked, unmask, info, n, rule, threshold, k, shift);
+}
+
+// Longest accepted prefix of a drafted block d against the causal predictions a (a[j] predicts the token after d[j]):
+// k = 1 + (first j in [0, n-2] with a[j] != d[j+1]; n-1 if none).  out = {k, a[k-1]}.
+__global__ void accept_kernel(const int32_t* __restrict__ a, const int32_t* __restrict__ d, int n, int32_t* __restrict__ out) {
+  __shared__ int first;
+  if (threadIdx.x == 0) first = n - 1;
+  __syncthreads();
+  const int j = threadIdx.x;
+  if (j < n - 1 && a[j] != d[j + 1]) atomicMin(&first, j);
+  __syncthreads();
+  if (threadIdx.x == 0) { out[0] = first + 1; out[1] = a[first]; }
+}
+void launch_accept(const int32_t* a, const int32_t* d, int n, int32_t* out, cudaStream_t st) {
+  accept_kernel<<<1, 64, 0, st>>>(a, d, n, out);
 }
 
 __global__ void init_block_kernel(int32_t* tokens, uint8_t* masked, int32_t* info, const int32_t* init, int n, int mask_id,

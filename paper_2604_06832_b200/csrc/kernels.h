@@ -37,7 +37,9 @@ void launch_swiglu(const float* gu, void* act, int n, int inter, int dtype, cuda
 void launch_row_stats(const float* logits, int n, int vocab, int mask_id, float* conf, int32_t* pred, cudaStream_t st);
 // Unmask selection + block-state update.  info = {n_unmasked, n_remaining, step_index}.
 void launch_select(const float* conf, const int32_t* pred, int32_t* tokens, uint8_t* masked, uint8_t* unmask,
-                   int32_t* info, int n, int rule, float threshold, int k, cudaStream_t st);
+                   int32_t* info, int n, int rule, float threshold, int k, cudaStream_t st, int shift = 0);
+// out[0] = accepted length k, out[1] = a[k - 1] (Alg. 1 "Accept: left-to-right comparison")
+void launch_accept(const int32_t* a, const int32_t* d, int n, int32_t* out, cudaStream_t st);
 void launch_init_block(int32_t* tokens, uint8_t* masked, int32_t* info, const int32_t* init, int n, int mask_id,
                        int step, cudaStream_t st);
 
