@@ -94,6 +94,22 @@ __device__ __forceinline__ void e4m3x16_to_bf16(const uint4& in, uint4& lo, uint
   hi = make_uint4(o[4], o[5], o[6], o[7]);
 }
 
+// Widen NP 16-byte pieces (tid, tid + stride, ...) of an 8 KB e4m3 tile (rows of 64 bytes) into the 128-byte-swizzled
+// bf16 tile the MMA descriptor expects.
+template <int NP>
+__device__ __forceinline__ void convert_pieces(const uint8_t* src, uint32_t dst, int tid, int stride) {
+#pragma unroll
+  for (int i = 0; i < NP; ++i) {
+    const int piece = tid + stride * i, r = piece >> 2, c = piece & 3;     // row, 16-byte piece of the row
+    const uint4 in = *reinterpret_cast<const uint4*>(src + piece * 16);
+    uint4 lo, hi;
+    e4m3x16_to_bf16(in, lo, hi);
+    const uint32_t row = dst + r * 128;
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + (((2 * c) ^ (r & 7)) << 4)), "r"(lo.x), "r"(lo.y), "r"(lo.z), "r"(lo.w) : "memory");
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + (((2 * c + 1) ^ (r & 7)) << 4)), "r"(hi.x), "r"(hi.y), "r"(hi.z), "r"(hi.w) : "memory");
+  }
+}
+
 template <int M_PAD, bool FP8>
 __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_kernel(const __grid_constant__ TcParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -119,10 +135,13 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   constexpr int TMEM_COLS = (2 * M_PAD <= 32) ? 32 : ((2 * M_PAD <= 64) ? 64 : 128);
 
+  // fp8 launches in which no CTA has a second work item: the epilogue warps, idle until the accumulator is complete,
+  // widen half of every weight tile beside the four converter warps
+  const bool helpers = FP8 && p.tile_begin[p.n_mats] * p.splits <= (int)gridDim.x;
   if (threadIdx.x == 0) {
     for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
-    for (int c = 0; c < TC_NCONV; ++c) { mbar_init(cfull_bar(c), 4); mbar_init(cempty_bar(c), 1); }
+    for (int c = 0; c < TC_NCONV; ++c) { mbar_init(cfull_bar(c), helpers ? 8 : 4); mbar_init(cempty_bar(c), 1); }
     for (int pr = 0; pr < 2; ++pr) { mbar_init(exw_bar(pr), 2); mbar_init(exr_bar(pr), 2); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -140,6 +159,30 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
 
   const int total_tiles = p.tile_begin[p.n_mats];
   const int n_items = total_tiles * p.splits;
+
+  const int kbps = p.kb_per_split, kblocks = p.kblocks;
+  auto convert_all = [&](int cvt_tid) -> bool {
+    int stage = 0, cbuf = 0;
+    uint32_t phase = 0, cphase = 0;
+    for (int it = blockIdx.x; it < n_items; it += gridDim.x) {
+      const int split = it / total_tiles;
+      const int kb0 = split * kbps;
+      const int kb1 = min(kblocks, kb0 + kbps);
+      for (int kb = kb0; kb < kb1; ++kb) {
+        if (!mbar_wait(full_bar(stage), phase, abort_flag) || !mbar_wait(cempty_bar(cbuf), cphase ^ 1u, abort_flag)) return false;
+        const uint8_t* src = sm + stage * L::STAGE_BYTES;
+        const uint32_t dst = base + L::CONV_OFF + cbuf * TC_A_BYTES;
+        if (helpers) convert_pieces<2>(src, dst, cvt_tid, 256);
+        else convert_pieces<4>(src, dst, cvt_tid, 128);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> the MMA's async-proxy reads
+        __syncwarp();
+        if (lane == 0) mbar_arrive(cfull_bar(cbuf));
+        if (++cbuf == TC_NCONV) { cbuf = 0; cphase ^= 1u; }
+        if (++stage == TC_STAGES) { stage = 0; phase ^= 1u; }
+      }
+    }
+    return true;
+  };
 
   if (warp == 0) {
     // ------------------------------------------------ TMA producer ------------------------------------------------
@@ -247,43 +290,15 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
     }
   } else if (FP8 && warp >= 6) {
     // ------------------------------------------------ e4m3 -> bf16 converters ---------------------------------------
-    // 128 threads; thread t widens the 16-byte pieces t, t + 128, t + 256, t + 384 of the 8 KB byte tile (rows of 64
-    // bytes) into the 128-byte-swizzled bf16 tile the MMA descriptor expects.
-    const int ct = threadIdx.x - 192;
-    int stage = 0, cbuf = 0;
-    uint32_t phase = 0, cphase = 0;
-    bool ok = true;
-    for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
-      const int split = it / total_tiles;
-      const int kb0 = split * p.kb_per_split;
-      const int kb1 = min(p.kblocks, kb0 + p.kb_per_split);
-      for (int kb = kb0; kb < kb1; ++kb) {
-        if (!mbar_wait(full_bar(stage), phase, abort_flag) || !mbar_wait(cempty_bar(cbuf), cphase ^ 1u, abort_flag)) { ok = false; break; }
-        const uint8_t* src = sm + stage * L::STAGE_BYTES;
-        const uint32_t dst = base + L::CONV_OFF + cbuf * TC_A_BYTES;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int piece = ct + 128 * i, r = piece >> 2, c = piece & 3;     // row, 16-byte piece of the row
-          const uint4 in = *reinterpret_cast<const uint4*>(src + piece * 16);
-          uint4 lo, hi;
-          e4m3x16_to_bf16(in, lo, hi);
-          const uint32_t row = dst + r * 128;
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + (((2 * c) ^ (r & 7)) << 4)), "r"(lo.x), "r"(lo.y), "r"(lo.z), "r"(lo.w) : "memory");
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + (((2 * c + 1) ^ (r & 7)) << 4)), "r"(hi.x), "r"(hi.y), "r"(hi.z), "r"(hi.w) : "memory");
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> the MMA's async-proxy reads
-        __syncwarp();
-        if (lane == 0) mbar_arrive(cfull_bar(cbuf));
-        if (++cbuf == TC_NCONV) { cbuf = 0; cphase ^= 1u; }
-        if (++stage == TC_STAGES) { stage = 0; phase ^= 1u; }
-      }
-    }
-    if (!ok && ct == 0) atomicCAS(p.status, 0, TC_ERR_MMA);
+    // 128 threads (256 with the epilogue warps helping): thread t widens the 16-byte pieces t, t + 128 (256), ... of
+    // each 8 KB byte tile
+    if (!convert_all(threadIdx.x - 192) && threadIdx.x == 192) atomicCAS(p.status, 0, TC_ERR_MMA);
   } else {
     // ------------------------------------------------ epilogue warps ----------------------------------------------
     const int q = warp & 3;  // TMEM lane quarter this warp may read
     int local = 0;
     bool ok = true;
+    if (helpers) ok = convert_all(128 + (int)threadIdx.x - 64);
     pdl_wait();   // the epilogue reads the predecessor's row statistics and overwrites buffers it may still be reading
     // folded RMSNorm: lane l keeps the factor of rows l and l + 32; broadcast by shuffle where needed
     float rs0 = 1.f, rs1 = 1.f;

@@ -267,3 +267,23 @@ def test_host_buffer_variants_match_device_variants():
     assert torch.equal(conf_d.cpu(), conf_h) and torch.equal(pred_d.cpu(), pred_h)
     assert tok_h[0] == 17 and um_h[0] == 0 and um_h.sum() == 3
     handle.close()
+
+
+def test_fp8_weight_codes_are_widened_exactly():
+    # one-hot activation rows pick single weights: the output must be the decoded e4m3 value times the row scale,
+    # bit for bit, for every finite code (normals, subnormals, both zeros)
+    b = B()
+    codes = np.array([c for c in range(256) if c not in (0x7F, 0xFF)], dtype=np.uint8)
+    n, k, m = 128, 256, 32
+    rng = np.random.default_rng(0)
+    w = rng.choice(codes, size=(n, k)).astype(np.uint8)
+    w[:, :254] = codes[None, :]                      # every code in every row
+    cols = rng.choice(k, size=m, replace=False)
+    cols[:8] = [0, 1, 7, 8, 0x78, 0x80 - 1, 200, 253]
+    x = np.zeros((m, k), dtype=np.float32)
+    x[np.arange(m), cols] = 1.0
+    scale = (2.0 ** rng.integers(-3, 3, size=n)).astype(np.float32)      # powers of two keep the product exact
+    y = b.op_linear(torch.from_numpy(x).to(torch.bfloat16).cuda(), torch.from_numpy(w).cuda(), torch.from_numpy(scale).cuda(),
+                    None, dtype=b.DT_FP8).cpu().numpy()
+    want = (orc.decode_e4m3(w)[:, cols] * scale[:, None].astype(np.float64)).T
+    assert np.array_equal(y.astype(np.float64), want)
