@@ -326,7 +326,7 @@ def run_ours(args, wl, block):
     # algorithmic bytes of the four layer projections, measured on the 4-layer cut of the shape and scaled by the
     # weight bytes: traffic grows in proportion).  None for shapes without a capture.
     ratio = {"cfg2_3b_bf16_p1024_b32_top8": 158.91 / 154.15, "cfg3_3b_bf16_p2048_sweep": 158.91 / 154.15,
-             "cfg4_3b_bf16_p8192_b32_top8": 158.91 / 154.15, "cfg5_7b_fp8_p1024_b32": 240.61 / 233.06}.get(wl.name)
+             "cfg4_3b_bf16_p8192_b32_top8": 158.91 / 154.15, "cfg5_7b_fp8_p1024_b32": 240.66 / 233.06}.get(wl.name)
     traffic = None if ratio is None or block != 32 else wbytes * ratio
     traffic_note = None if traffic is None else "scaled from the 4-layer ncu capture of the same layer shapes (profiles/)"
     step_bytes = wbytes + shape.kv_bytes_per_token() * L_step
