@@ -118,8 +118,8 @@ def oracle_sample(wl: I.Workload, block: int, weights_cpu: dict, reps: int = 1):
 
 
 def run_reference(args, wl, block):
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    from paper_2604_06832_b200 import replicas as R
+    if not R.prints_result(int(os.environ.get("RANK", "0"))):
         return
     shape = wl.shape
     weights = I.make_weights(shape, wl.weight_seed)
@@ -153,6 +153,7 @@ def run_reference(args, wl, block):
 def run_ours(args, wl, block):
     from paper_2604_06832_b200 import binding as B
     from paper_2604_06832_b200 import build as build_mod
+    from paper_2604_06832_b200 import replicas as R
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -227,12 +228,7 @@ def run_ours(args, wl, block):
                 fn()
             b.record(stream)
             torch.cuda.synchronize()
-            ms = a.elapsed_time(b)
-            if dist is not None:
-                t = torch.tensor([ms], device="cuda")
-                dist.all_reduce(t, op=dist.ReduceOp.MAX)
-                ms = float(t.item())
-            return ms
+            return R.max_over_ranks_ms(a.elapsed_time(b), dist, torch.device("cuda", local))
 
         for _ in range(W):
             steps_seen = one_block_device()
@@ -315,9 +311,8 @@ def run_ours(args, wl, block):
                      "self_speculative_linear": {"tok_s": state["accepted"] * world / (ms_spec / 1000.0), "ms_per_iteration": ms_spec / K,
                                                  "accepted_per_iteration": state["accepted"] / K}}
 
-    tokens = K * block * world
-    value = tokens / (ms_dev / 1000.0)
-    e2e_value = tokens / (ms_e2e / 1000.0)
+    value = R.whole_job_rate(K * block, world, ms_dev)
+    e2e_value = R.whole_job_rate(K * block, world, ms_e2e)
     peak, peak_kind = measured_peaks()
     wbytes = shape.weight_bytes()
     gemm_ms_per_fwd = prof["ms_linear"] / n_steps
@@ -361,7 +356,7 @@ def run_ours(args, wl, block):
                                 "sample": f"one denoise forward ({ts:.1f} s) + one commit forward ({tc:.1f} s) of a {block}-token block "
                                           f"at cache length 32, extrapolated over {n_steps} denoise steps + 1 commit per block"}
     handle.close()
-    if rank == 0:
+    if R.prints_result(rank):
         print(json.dumps(line), flush=True)
     if dist is not None:
         dist.barrier()
