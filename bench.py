@@ -192,6 +192,12 @@ def run_ours(args, wl, block):
         launches = [0]
 
         def one_block_device():
+            if wl.rule == "topk":      # fixed schedule: every step enqueued without a host round trip in between
+                info = handle.decode_block_topk(block, wl.k)
+                launches[0] += handle.last_launch_count()
+                handle.commit_block()
+                launches[0] += handle.last_launch_count()
+                return info.step_index
             handle.block_begin(block)
             n = 0
             while True:

@@ -140,6 +140,17 @@ int fdvlm_block_step_host(fdvlm_t *h, const fdvlm_step_params *p, float *conf_ho
                           int32_t *pred_host, uint8_t *unmask_host, int32_t *block_tokens_host,
                           fdvlm_step_info *info);
 
+/* Open a block and run the whole top-k schedule on it without a host round trip between the steps: with k positions
+ * revealed per step the number of denoise steps is known in advance (ceil(masked / k)), so all of them are enqueued
+ * back to back and the host reads the block state once at the end.  init_tokens as in fdvlm_block_begin (device,
+ * nullable); pred_shift as in fdvlm_step_params (with 1, position 0 must be given).  block_tokens (device int32 [B],
+ * nullable) receives the finished block; info (HOST, required) the counts after the last step and the number of steps
+ * in step_index.  The block is left open and fully revealed: commit it with fdvlm_commit_block(_verify).
+ * Errors as fdvlm_block_begin / fdvlm_block_step; STATE if masked positions remain (a masked position 0 under
+ * pred_shift = 1). */
+int fdvlm_decode_block_topk(fdvlm_t *h, int block_size, const int32_t *init_tokens, int k, int pred_shift,
+                            int32_t *block_tokens, fdvlm_step_info *info);
+
 /* Replace the open block's tokens / masked flags (device int32 [B]; mask_id = masked) without
  * touching the step counter: lets a test replay another implementation's block state. */
 int fdvlm_block_set_tokens(fdvlm_t *h, const int32_t *tokens);

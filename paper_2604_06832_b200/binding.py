@@ -69,6 +69,7 @@ EXPORTS = {
     "fdvlm_block_step_host": (C.c_int, [C.c_void_p, C.POINTER(StepParams), C.c_void_p, C.c_void_p, C.c_void_p,
                                         C.c_void_p, C.POINTER(StepInfo)]),
     "fdvlm_block_set_tokens": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "fdvlm_decode_block_topk": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.POINTER(StepInfo)]),
     "fdvlm_commit_block": (C.c_int, [C.c_void_p, C.c_void_p]),
     "fdvlm_commit_block_verify": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "fdvlm_truncate": (C.c_int, [C.c_void_p, C.c_int]),
@@ -195,6 +196,13 @@ class Handle:
         p, info = StepParams(rule, threshold, k, pred_shift), StepInfo()
         self._check(lib().fdvlm_block_step_host(self._h, C.byref(p), _ptr(conf), _ptr(pred), _ptr(unmask),
                                                 _ptr(block_tokens), C.byref(info)))
+        return info
+
+    def decode_block_topk(self, block_size: int, k: int, init_tokens: Optional[torch.Tensor] = None, pred_shift: int = 0,
+                          block_tokens: Optional[torch.Tensor] = None) -> StepInfo:
+        info = StepInfo()
+        self._check(lib().fdvlm_decode_block_topk(self._h, block_size, _ptr(init_tokens), k, pred_shift, _ptr(block_tokens),
+                                                  C.byref(info)))
         return info
 
     def block_set_tokens(self, tokens: torch.Tensor):

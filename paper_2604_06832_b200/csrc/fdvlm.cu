@@ -314,6 +314,32 @@ extern "C" int fdvlm_block_step(fdvlm_t* h, const fdvlm_step_params* p, float* l
   return finish_info(h, info);
 }
 
+extern "C" int fdvlm_decode_block_topk(fdvlm_t* h, int block_size, const int32_t* init_tokens, int k, int pred_shift,
+                                       int32_t* block_tokens, fdvlm_step_info* info) {
+  if (!h) return FDVLM_ERR_INVALID_ARG;
+  if (!info) return fail(h, FDVLM_ERR_INVALID_ARG, "decode_block_topk needs the host info struct");
+  if (k < 1) return fail(h, FDVLM_ERR_INVALID_ARG, "top-k needs k >= 1");
+  int rc = fdvlm_block_begin(h, block_size, init_tokens);      // (reads the masked count back when tokens are given)
+  if (rc) return rc;
+  fdvlm_step_params p;
+  p.rule = FDVLM_RULE_TOPK; p.threshold = 0.f; p.k = k; p.pred_shift = pred_shift;
+  const int steps = (h->n_remaining + k - 1) / k;
+  int launches = 0;
+  for (int s = 0; s < steps; ++s) {
+    h->n_remaining = 1;            // the device keeps the true count; the host checks it once, below
+    rc = step_core(h, &p, 0);
+    if (rc) return rc;
+    launches += h->launches;
+  }
+  h->launches = launches;
+  if (block_tokens) CU(h, cudaMemcpyAsync(block_tokens, h->blk_tokens, (size_t)block_size * 4, cudaMemcpyDeviceToDevice, h->st));
+  rc = sync_info(h);
+  if (rc) return rc;
+  info->n_unmasked = h->info_host[0]; info->n_remaining = h->info_host[1]; info->step_index = h->info_host[2];
+  if (h->n_remaining != 0) return fail(h, FDVLM_ERR_STATE, "%d masked positions left after %d top-%d steps", h->n_remaining, steps, k);
+  return FDVLM_OK;
+}
+
 extern "C" int fdvlm_block_step_host(fdvlm_t* h, const fdvlm_step_params* p, float* conf_host, int32_t* pred_host,
                                      uint8_t* unmask_host, int32_t* block_tokens_host, fdvlm_step_info* info) {
   int rc = step_core(h, p, 0);

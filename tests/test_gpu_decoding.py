@@ -194,6 +194,46 @@ def test_speculative_decoding_on_the_gpu_is_lossless():
     assert outs[0] == outs[1]
 
 
+@pytest.mark.parametrize("shift", [0, 1])
+def test_topk_block_decode_without_host_round_trips_equals_stepwise(shift):
+    b = B()
+    shape, Bsz, k = I.TINY, 8, 3
+    _, handle, _ = make_pair(shape, 4, max_seq=128, final_gain=16.0)
+    toks = I.random_tokens(shape, 30, 2).cuda()
+    init = torch.full((Bsz,), shape.mask_id, dtype=torch.int32, device="cuda")
+    if shift:
+        init[0] = 77
+    out = []
+    for mode in ("stepwise", "fused"):
+        handle.reset()
+        handle.prefill(None, toks)
+        got = torch.empty(Bsz, dtype=torch.int32, device="cuda")
+        if mode == "stepwise":
+            handle.block_begin(Bsz, init)
+            n = 0
+            while True:
+                info = handle.block_step(b.RULE_TOPK, 0.0, k, block_tokens=got, pred_shift=shift)
+                n += 1
+                if info.n_remaining == 0:
+                    break
+        else:
+            info = handle.decode_block_topk(Bsz, k, init, shift, got)
+            n = info.step_index
+        assert info.n_remaining == 0 and n == -(-(Bsz - shift) // k)
+        nxt = torch.empty(shape.vocab, dtype=torch.float32, device="cuda")
+        handle.commit_block(nxt)
+        out.append((got.cpu().numpy().copy(), nxt.cpu().numpy().copy(), n))
+    assert np.array_equal(out[0][0], out[1][0]) and np.array_equal(out[0][1], out[1][1]) and out[0][2] == out[1][2]
+    assert (out[1][0] != shape.mask_id).all()
+    # shift-by-one needs a given first position
+    handle.reset()
+    handle.prefill(None, toks)
+    with pytest.raises(b.FdvlmError) as e:
+        handle.decode_block_topk(Bsz, k, None, 1)
+    assert e.value.code == b.ERR_STATE
+    handle.close()
+
+
 def test_decoding_entry_point_errors():
     b = B()
     _, handle, _ = make_pair(I.TINY, 0, max_seq=64, max_block=8)
