@@ -287,3 +287,22 @@ def test_fp8_weight_codes_are_widened_exactly():
                     None, dtype=b.DT_FP8).cpu().numpy()
     want = (orc.decode_e4m3(w)[:, cols] * scale[:, None].astype(np.float64)).T
     assert np.array_equal(y.astype(np.float64), want)
+
+
+# ---- edge sizes: single-row and maximum blocks (every activation-tile width of the GEMM: 16, 32, 48, 64 rows), an
+# ---- empty cache, and a decode that ends exactly at max_seq ------------------------------------------------------
+@pytest.mark.parametrize("shape,B_,L_t", [(SMALL_BF16, 1, 9), (SMALL_BF16, 40, 17), (SMALL_BF16, 64, 30), (SMALL_FP8, 64, 12),
+                                          (SMALL_FP8, 48, 5), (SMALL_BF16, 16, 0), (SMALL_FP8, 3, 0)])
+def test_edge_block_sizes_and_empty_cache(shape, B_, L_t):
+    n_blocks = 2
+    oracle, handle, _ = make_pair(shape, 13, max_seq=L_t + n_blocks * B_, max_block=B_)      # the last commit fills the cache
+    if L_t:
+        toks = I.random_tokens(shape, L_t, 6)
+        oracle.prefill(None, toks.numpy(), want_logits=False)
+        handle.prefill(None, toks.cuda())
+    stats = replay_decode(oracle, handle, shape, B_, orc.TOPK, 0.9, 7, n_blocks=n_blocks)
+    assert stats["steps"] == n_blocks * -(-B_ // 7) and handle.cache_len() == L_t + n_blocks * B_
+    with pytest.raises(B().FdvlmError) as e:
+        handle.block_begin(1)                            # the cache is full
+    assert e.value.code == B().ERR_CAPACITY
+    handle.close()
