@@ -297,11 +297,36 @@ __global__ void embed_prep_kernel(const bf16* __restrict__ table, const int32_t*
   const int r = blockIdx.x;
   const bf16* src = tokens ? table + (size_t)tokens[r] * hidden : rows + (size_t)r * hidden;
   float ss = 0.f;
-  for (int c = threadIdx.x; c < hidden; c += blockDim.x) {
-    const float v = __bfloat162float(src[c]);
-    h[(size_t)r * hidden + c] = v;
-    xg[(size_t)r * hidden + c] = __float2bfloat16_rn(v * g[c]);
-    ss = fmaf(v, v, ss);
+  if ((hidden & 7) == 0) {
+    // eight values per thread and pass: one 16-byte load of the row and two of the gain, all issued before use
+    for (int c8 = threadIdx.x; c8 < hidden / 8; c8 += blockDim.x) {
+      const uint4 raw = *reinterpret_cast<const uint4*>(src + 8 * c8);
+      const float4 g0 = *reinterpret_cast<const float4*>(g + 8 * c8), g1 = *reinterpret_cast<const float4*>(g + 8 * c8 + 4);
+      const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+      const float gg[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+      float v[8];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { v[2 * i] = __uint_as_float(w[i] << 16); v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u); }
+      float* hd = h + (size_t)r * hidden + 8 * c8;
+      *reinterpret_cast<float4*>(hd) = make_float4(v[0], v[1], v[2], v[3]);
+      *reinterpret_cast<float4*>(hd + 4) = make_float4(v[4], v[5], v[6], v[7]);
+      uint32_t o[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        __nv_bfloat162 b2 = __floats2bfloat162_rn(v[2 * i] * gg[2 * i], v[2 * i + 1] * gg[2 * i + 1]);
+        o[i] = *reinterpret_cast<uint32_t*>(&b2);
+        ss = fmaf(v[2 * i], v[2 * i], ss);
+        ss = fmaf(v[2 * i + 1], v[2 * i + 1], ss);
+      }
+      *reinterpret_cast<uint4*>(xg + (size_t)r * hidden + 8 * c8) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+  } else {
+    for (int c = threadIdx.x; c < hidden; c += blockDim.x) {
+      const float v = __bfloat162float(src[c]);
+      h[(size_t)r * hidden + c] = v;
+      xg[(size_t)r * hidden + c] = __float2bfloat16_rn(v * g[c]);
+      ss = fmaf(v, v, ss);
+    }
   }
   ss = block_sum(ss, red);
   for (int t = threadIdx.x; t < nt; t += blockDim.x) ssq[(size_t)r * nt + t] = (t == 0) ? ss : 0.f;
@@ -437,12 +462,12 @@ void launch_fin_resid(const float* part, int S, int m, int hidden, float* h, con
 
 // Merge the per-warp softmax statistics of the LM-head epilogue into confidence and prediction per row.
 // stats[e * m + row] = (max, sum exp(l - max), argmax id) for e in [0, n_part).  grid m rows, 256 threads.
-__global__ void __launch_bounds__(256) stats_merge_kernel(const float4* __restrict__ stats, int n_part, int m,
+__global__ void __launch_bounds__(512) stats_merge_kernel(const float4* __restrict__ stats, int n_part, int m,
                                                           float* __restrict__ conf, int32_t* __restrict__ pred) {
   pdl_trigger();
   pdl_wait();
-  __shared__ float sm_m[8], sm_s[8];
-  __shared__ int sm_i[8];
+  __shared__ float sm_m[16], sm_s[16];
+  __shared__ int sm_i[16];
   const int r = blockIdx.x;
   float mx = -INFINITY, s = 0.f;
   int ix = 0x7fffffff;
@@ -454,9 +479,16 @@ __global__ void __launch_bounds__(256) stats_merge_kernel(const float4* __restri
     if (m2 > mx || (m2 == mx && i2 < ix)) ix = i2;
     mx = mn;
   };
-  for (int e = threadIdx.x; e < n_part; e += blockDim.x) {
-    const float4 v = stats[(size_t)e * m + r];
-    merge(v.x, v.y, __float_as_int(v.z));
+  // ten loads in flight per thread: at the 3B / 7B vocabularies (4.7k partials per row) one L2 round trip in all
+  for (int e0 = threadIdx.x; e0 < n_part; e0 += 10 * blockDim.x) {
+    float4 v[10];
+#pragma unroll
+    for (int j = 0; j < 10; ++j) {
+      const int e = e0 + j * blockDim.x;
+      v[j] = e < n_part ? __ldcg(&stats[(size_t)e * m + r]) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int j = 0; j < 10; ++j) merge(v[j].x, v[j].y, __float_as_int(v[j].z));
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
@@ -469,13 +501,13 @@ __global__ void __launch_bounds__(256) stats_merge_kernel(const float4* __restri
   __syncthreads();
   if (threadIdx.x == 0) {
     mx = sm_m[0]; s = sm_s[0]; ix = sm_i[0];
-    for (int k = 1; k < 8; ++k) merge(sm_m[k], sm_s[k], sm_i[k]);
+    for (int k = 1; k < (int)(blockDim.x >> 5); ++k) merge(sm_m[k], sm_s[k], sm_i[k]);
     conf[r] = 1.f / s;
     pred[r] = ix;
   }
 }
 void launch_stats_merge(const void* stats, int n_part, int m, float* conf, int32_t* pred, cudaStream_t st) {
-  launch_pdl(stats_merge_kernel, dim3(m), dim3(256), 0, st, (const float4*)stats, n_part, m, conf, pred);
+  launch_pdl(stats_merge_kernel, dim3(m), dim3(512), 0, st, (const float4*)stats, n_part, m, conf, pred);
 }
 
 // ================================================================================================
