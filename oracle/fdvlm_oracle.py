@@ -390,8 +390,7 @@ class Oracle:
             assert rec["n_remaining"] == 0
         d = self.block_tokens.copy()
         a = confidence(self.commit_block(all_rows=True), self.s.mask_id)[0]
-        mism = [j for j in range(0, B - 1) if a[j] != d[j + 1]]
-        k = (mism[0] if mism else B - 1) + 1
+        k = accept_length(a, d)
         self.truncate(L0 + k)
         return dict(draft=d, a=a, accepted=k, new_tokens=a[:k].copy(), next_token=int(a[k - 1]))
 
@@ -432,6 +431,21 @@ class Oracle:
             act = silu(m @ self._lin(l, "w_gate").T.astype(np.float64)) * (m @ self._lin(l, "w_up").T.astype(np.float64))
             h = h + act @ self._lin(l, "w_down").T.astype(np.float64)
         return np.asarray(self.logits_of(h.astype(self.ft)), dtype=np.float64)
+
+
+def accept_length(a, d) -> int:
+    """Alg. 1 "Accept: left-to-right comparison": k = min{ j in [0, B-2] : a_j != d_{j+1} }, then k + 1; with no
+    mismatch the minimum is taken as B-1 (all B accepted)."""
+    B = len(d)
+    mism = [j for j in range(0, B - 1) if a[j] != d[j + 1]]
+    return (mism[0] if mism else B - 1) + 1
+
+
+def verify_mask(L: int, B: int) -> np.ndarray:
+    """Boolean [B, L+B] mask of Alg. 1's verify step: the whole cache, and block keys j <= i (A_ij = 1[i >= j])."""
+    m = np.ones((B, L + B), dtype=bool)
+    m[:, L:] = np.tril(np.ones((B, B), dtype=bool))
+    return m
 
 
 def draft_mask(L: int, B: int) -> np.ndarray:

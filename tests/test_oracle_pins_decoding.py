@@ -144,3 +144,25 @@ def test_planted_off_by_one_in_crop_is_caught(monkeypatch):
         partial = partial or rec["accepted"] < 4
         got.extend(int(t) for t in rec["new_tokens"])
     assert partial and got[:12] != want
+
+
+def test_golden_masks_and_accept_rule_of_algorithm_1():
+    import os
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "alg1_masks_and_accept.txt")
+    lines = [l.strip() for l in open(path) if l.strip() and not l.startswith("#")]
+    i = n_accept = 0
+    while i < len(lines):
+        parts = lines[i].split()
+        if parts[0] in ("draft_mask", "verify_mask"):
+            L, B_ = int(parts[1]), int(parts[2])
+            want = np.array([[int(x) for x in lines[i + 1 + r].split()] for r in range(B_)], dtype=bool)
+            got = orc.draft_mask(L, B_)[L:] if parts[0] == "draft_mask" else orc.verify_mask(L, B_)
+            assert got.shape == want.shape and np.array_equal(got, want)
+            i += 1 + B_
+        else:
+            assert parts[0] == "accept"
+            d, a, k, new = [[int(x) for x in f.split()] for f in lines[i][len("accept"):].split("|")]
+            assert orc.accept_length(np.array(a), np.array(d)) == k[0] and a[:k[0]] == new
+            n_accept += 1
+            i += 1
+    assert n_accept == 5
