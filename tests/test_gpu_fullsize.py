@@ -2,8 +2,8 @@
 stream, i.e. graph replay + programmatic dependent launch, real tile counts and the full 151936-row LM head).
 
 The oracle needs ~13 s per forward of the 3B shape, so the 3B case keeps the prefix short (one 32-row prefill chunk)
-and checks one denoise step and the commit; the FP8 case uses the 4-layer cut of the 7B shape (same per-layer
-matrices).  Confidence keeps the stated tolerance; the logit tolerance is the stated one or, for the 36-layer shape,
+and checks one denoise step and the commit; the FP8 cases are the 4-layer cut of the 7B shape (same per-layer
+matrices, two blocks) and the full 28-layer 7B shape (one block).  Confidence keeps the stated tolerance; the logit tolerance is the stated one or, for the 36-layer shape,
 the bound `helpers.depth_tolerance` derives from the arithmetic (accumulated bf16 rounding grows with sqrt(layers):
 measured 0.026 / 0.045 / 0.081 / 0.119 max-abs at 1 / 4 / 18 / 36 layers of the 3B width)."""
 import numpy as np
@@ -18,7 +18,8 @@ from helpers import depth_tolerance, make_pair, replay_decode, upload_prefix
 pytestmark = [pytest.mark.gpu, pytest.mark.slow]
 
 
-@pytest.mark.parametrize("wl_name,n_blocks", [("cfg2_3b_bf16_p1024_b32_top8", 1), ("prof_7b_fp8_4layers", 2)])
+@pytest.mark.parametrize("wl_name,n_blocks", [("cfg2_3b_bf16_p1024_b32_top8", 1), ("prof_7b_fp8_4layers", 2),
+                                              ("cfg5_7b_fp8_p1024_b32", 1)])
 def test_full_layer_shapes_block32_on_stream(wl_name, n_blocks):
     wl = I.WORKLOADS[wl_name]
     shape = wl.shape
