@@ -175,7 +175,9 @@ def run_ours(args, wl, block):
     max_seq = L0 + (2 * (K + W) + 2) * block + (2 * K + 4) * block + 64
     weights = I.make_weights(shape, wl.weight_seed, device="cuda")
     stream = torch.cuda.Stream()
-    handle = B.Handle(shape, weights, max_seq=max_seq, max_block=max(block, 32), stream=stream)
+    # the 7B configuration prescribes a bf16 KV cache; the others leave the cache's element type open
+    kv_dtype = B.KV_BF16 if shape.dtype == I.FP8 else B.KV_F16
+    handle = B.Handle(shape, weights, max_seq=max_seq, max_block=max(block, 32), stream=stream, kv_dtype=kv_dtype)
     emb, toks = I.make_prefix(shape, wl.n_embeds, wl.n_tokens, wl.prefix_seed)
     emb_d, toks_d = emb.cuda(), toks.cuda()
     rule = B.RULE_TOPK if wl.rule == "topk" else B.RULE_THRESHOLD

@@ -51,13 +51,21 @@ typedef enum {
   FDVLM_ERR_OOM = -7          /* device allocation failed in fdvlm_create                          */
 } fdvlm_status;
 
-/* Storage type of the linear weights.  Activations, KV cache and the embedding table are fp32 for
- * FDVLM_F32 and bf16 otherwise; accumulation, residual stream, norms and softmax are always fp32. */
+/* Storage type of the linear weights.  For FDVLM_F32 everything is fp32.  Otherwise the embedding table and the
+ * embedding rows given to fdvlm_prefill are bf16, and the accumulation, residual stream, norms and softmax are
+ * fp32; the 16-bit tensors between the operators are internal: GEMM inputs are pairs of bf16 (value = hi + lo, ~16
+ * significant bits) for bf16 weights and f16 for fp8 weights (e4m3 widens exactly to f16), q and the KV cache are
+ * of fdvlm_kv_dtype. */
 typedef enum {
   FDVLM_F32 = 0,
   FDVLM_BF16 = 1,
   FDVLM_W_FP8E4M3 = 2 /* OCP e4m3fn bytes + fp32 per-output-channel scale: w = e4m3(byte) * scale[out] */
 } fdvlm_dtype;
+
+/* Element type of the KV cache (and of q, and of the attention probabilities in the P.V product) for the bf16 /
+ * fp8 weight types; same bytes either way.  F16 keeps 11 significant bits instead of 8 -- what the stated logit
+ * tolerances need at 28-36 layers -- and saturates at +-65504.  Ignored for FDVLM_F32 (fp32 cache). */
+typedef enum { FDVLM_KV_BF16 = 0, FDVLM_KV_F16 = 1 } fdvlm_kv_dtype;
 
 typedef struct {
   int n_layers, hidden, n_q_heads, n_kv_heads, head_dim, intermediate, vocab;
@@ -69,6 +77,7 @@ typedef struct {
   fdvlm_dtype dtype;
   int max_seq;        /* KV-cache capacity in positions; every call needs cache_len + rows <= max_seq */
   int max_block;      /* largest block size (1..64) */
+  fdvlm_kv_dtype kv_dtype;
 } fdvlm_config;
 
 typedef struct {
@@ -108,6 +117,13 @@ void fdvlm_destroy(fdvlm_t *h);
 
 /* Forget the cache and any open block (cache_len = 0). */
 int fdvlm_reset(fdvlm_t *h);
+
+/* Wait for everything issued on the handle's stream and report what the device left in its status word since the
+ * last report: FDVLM_ERR_TIMEOUT if a bounded device-side wait gave up, FDVLM_ERR_INVALID_ARG if a token id outside
+ * [0, vocab) was met (the embedding of token 0 was used in its place; nothing out of bounds was read), else FDVLM_OK.
+ * The asynchronous calls (fdvlm_prefill, fdvlm_commit_block, fdvlm_block_step without `info`) cannot report these
+ * themselves; every synchronous call does, and so does this one. */
+int fdvlm_synchronize(fdvlm_t *h);
 
 /* Append `n_embeds` embedding rows (device, [n_embeds, hidden], fp32 for F32 else bf16; may be NULL
  * when n_embeds = 0) and then `n_tokens` token ids (device int32; may be NULL when 0) to the cache
@@ -151,6 +167,15 @@ int fdvlm_block_step_host(fdvlm_t *h, const fdvlm_step_params *p, float *conf_ho
 int fdvlm_decode_block_topk(fdvlm_t *h, int block_size, const int32_t *init_tokens, int k, int pred_shift,
                             int32_t *block_tokens, fdvlm_step_info *info);
 
+/* Open a block and denoise it to the end under either rule without a host round trip between the steps (Sec. 3.4
+ * "confidence-aware parallel decoding": the number of steps of the threshold rule depends on the confidences, so
+ * the loop itself runs on the device and stops as soon as no masked position is left).  Arguments as
+ * fdvlm_decode_block_topk with the rule in `p`; info (HOST, required) receives the counts after the last step and
+ * the number of steps taken in step_index.  Needs a handle created on a non-default stream (the loop is a CUDA graph
+ * with a conditional node); UNSUPPORTED otherwise. */
+int fdvlm_decode_block(fdvlm_t *h, int block_size, const int32_t *init_tokens, const fdvlm_step_params *p,
+                       int32_t *block_tokens, fdvlm_step_info *info);
+
 /* Replace the open block's tokens / masked flags (device int32 [B]; mask_id = masked) without
  * touching the step counter: lets a test replay another implementation's block state. */
 int fdvlm_block_set_tokens(fdvlm_t *h, const int32_t *tokens);
@@ -189,18 +214,37 @@ int fdvlm_spec_block(fdvlm_t *h, int block_size, int32_t seed_token, int32_t *dr
 int fdvlm_cache_len(const fdvlm_t *h);
 
 /* Copy cached K (which = 0, post-rotary) or V (which = 1) of `layer`, positions [pos0, pos0 + n), to
- * dst (device, [n, n_kv_heads, head_dim], fp32 for F32 else bf16).  For tests and checkpointing. */
+ * dst (device, [n, n_kv_heads, head_dim], fp32 for F32 else the handle's kv_dtype).  For tests and checkpointing. */
 int fdvlm_cache_read(const fdvlm_t *h, int layer, int which, int pos0, int n, void *dst);
 
 /* Number of kernel launches issued by the last prefill / step / commit call of this handle. */
 int fdvlm_last_launch_count(const fdvlm_t *h);
 
-/* Instrumentation: while enabled, every projection (GEMM) launch group and every attention launch of
- * this handle is bracketed by CUDA events on the handle's stream.  fdvlm_profile_read synchronises
- * the stream, returns the summed device time (milliseconds) and the number of bracketed groups per
- * family since the last enable / read, and clears the counters.  Any output pointer may be NULL. */
-int fdvlm_profile_enable(fdvlm_t *h, int on);
+/* Instrumentation.  mode 0: off.  mode 1: every projection (GEMM) launch group and every attention launch of this
+ * handle is bracketed by CUDA events on the handle's stream and the kernels are launched one by one (so without the
+ * overlap of the production chain); fdvlm_profile_read synchronises the stream, returns the summed device time
+ * (milliseconds) and the number of bracketed groups per family since the last enable / read, and clears the
+ * counters.  mode 2 (in-chain timing): the forward runs exactly as in production (graph replay, dependent launches),
+ * and every kernel records, from the GPU's global nanosecond timer, the earliest start of any of its CTAs, the
+ * earliest return of a CTA from its wait for the predecessor kernel, and the latest end of any CTA;
+ * fdvlm_profile_read_chain synchronises and returns the records of the LAST forward in launch order (at most `cap`;
+ * *n = how many there were).  Any output pointer may be NULL. */
+typedef enum {
+  FDVLM_K_ROPE_TABLE = 0, FDVLM_K_GEMM_QKV = 1, FDVLM_K_FIN_QKV = 2, FDVLM_K_ATTENTION = 3, FDVLM_K_ATTN_MERGE = 4,
+  FDVLM_K_GEMM_O = 5, FDVLM_K_FIN_RESID = 6, FDVLM_K_GEMM_GATE_UP = 7, FDVLM_K_GEMM_DOWN = 8, FDVLM_K_GEMM_LM_HEAD = 9,
+  FDVLM_K_STATS_MERGE = 10
+} fdvlm_kernel_kind;
+typedef struct { int kind; /* fdvlm_kernel_kind */ double start_us, released_us, end_us; /* relative to the first start */ } fdvlm_kernel_record;
+int fdvlm_profile_enable(fdvlm_t *h, int mode);
 int fdvlm_profile_read(fdvlm_t *h, double *ms_linear, int *n_linear, double *ms_attention, int *n_attention);
+int fdvlm_profile_read_chain(fdvlm_t *h, fdvlm_kernel_record *records, int cap, int *n);
+
+/* Test hook for the give-up path of the kernels' bounded waits.  While `on` is non-zero, every tensor-core GEMM of
+ * this handle reads the flag when it starts and each of its roles (TMA producer, MMA issuer, converters, epilogue)
+ * leaves at once by the path a timed-out wait takes -- nothing issued, nothing in flight, tensor memory freed -- and
+ * records its role in the status word, so the next synchronous call returns FDVLM_ERR_TIMEOUT.  Outputs of such
+ * calls are undefined; committed cache positions are not written.  Takes effect in stream order. */
+int fdvlm_debug_poison(fdvlm_t *h, int on);
 
 /* Message of the last error on this handle ("" if none); valid until the next call on it.
  * With h = NULL returns the message of the last failed fdvlm_create on this thread. */
@@ -212,11 +256,16 @@ const char *fdvlm_last_error(const fdvlm_t *h);
  * every projection of the decoder is (QKV, O, gate/up, down, LM head; M = block size <= 64).
  * x: device [m, k], fp32 for F32 else bf16; w: device [n, k] in `dtype` storage; scale: device fp32
  * [n] (fp8) or NULL; bias: device fp32 [n] or NULL; y: device fp32 [m, n].
- * workspace: device scratch of at least fdvlm_op_linear_workspace_bytes(m, n, k, dtype) bytes (used
- * for split-K partial sums; may be NULL when that size is 0). */
+ * workspace: device scratch of at least fdvlm_op_linear_workspace_bytes(m, n, k, dtype) bytes (never 0): the
+ * kernels' status words, split-K partial sums and, for fp8 weights, the f16 copy of x that GEMM multiplies by.
+ * The call is asynchronous; fdvlm_op_linear_status(workspace, stream) waits for the stream and returns
+ * FDVLM_ERR_TIMEOUT if a bounded wait inside the kernels of the LAST call on that workspace gave up (y is then
+ * undefined), else FDVLM_OK.  workspace = NULL asks about the built-in scratch of fdvlm_op_linear_static on the
+ * current device. */
 int fdvlm_op_linear(const void *x, const void *w, const float *scale, const float *bias, float *y,
                     int m, int n, int k, fdvlm_dtype dtype, void *workspace, void *cuda_stream);
 size_t fdvlm_op_linear_workspace_bytes(int m, int n, int k, fdvlm_dtype dtype);
+int fdvlm_op_linear_status(const void *workspace, void *cuda_stream);
 
 /* (No counterpart in the paper: an integration convenience of this library.)
  * The same projection as fdvlm_op_linear for callers that cannot allocate device memory -- code running
@@ -225,8 +274,8 @@ size_t fdvlm_op_linear_workspace_bytes(int m, int n, int k, fdvlm_dtype dtype);
  * fdvlm_op_linear takes as `workspace` is instead a fixed array of FDVLM_STATIC_SCRATCH_BYTES bytes
  * built into the library's device image; every GPU that loads the library holds it until the process
  * exits.  The call allocates nothing (no cudaMalloc / cudaFree, no allocating library routine).
- *   - Shapes whose scratch need (see fdvlm_op_linear_workspace_bytes) exceeds the array less its first
- *     256 bytes are refused with FDVLM_ERR_CAPACITY; the message (fdvlm_last_error(NULL)) names both sizes.
+ *   - Shapes whose scratch need (see fdvlm_op_linear_workspace_bytes) exceeds the array are refused with
+ *     FDVLM_ERR_CAPACITY; the message (fdvlm_last_error(NULL)) names both sizes.
  *   - The first call on each device looks up the array's device address (with that device current);
  *     make that first call before any stream capture.
  *   - All calls on one device share the array: two calls whose kernels may overlap on the GPU (different
@@ -242,11 +291,12 @@ int fdvlm_op_linear_static(const void *x, const void *w, const float *scale, con
  * k_cache / v_cache: device [n_kv_heads, max_seq, head_dim] holding cache_len committed positions
  * followed by the n_rows new positions; causal = 0: every row reads all cache_len + n_rows keys,
  * causal = 1: row i reads keys 0 .. cache_len + i.  out: device [n_rows, n_q_heads * head_dim].
- * Element type fp32 for F32, bf16 otherwise.  workspace: device scratch of at least
- * fdvlm_op_attention_workspace_bytes(...) bytes for the split-KV partial results. */
+ * Element type of q, the caches and out: fp32 for F32, otherwise bf16 or f16 as kv_dtype says.  workspace: device
+ * scratch of at least fdvlm_op_attention_workspace_bytes(...) bytes for the split-KV partial results. */
 int fdvlm_op_attention(const void *q, const void *k_cache, const void *v_cache, void *out,
                        int n_rows, int cache_len, int max_seq, int n_q_heads, int n_kv_heads,
-                       int head_dim, int causal, fdvlm_dtype dtype, void *workspace, void *cuda_stream);
+                       int head_dim, int causal, fdvlm_dtype dtype, fdvlm_kv_dtype kv_dtype, void *workspace,
+                       void *cuda_stream);
 size_t fdvlm_op_attention_workspace_bytes(int n_rows, int n_q_heads, int n_kv_heads, int head_dim);
 
 /* Version string of the library. */

@@ -21,7 +21,10 @@ LIB_PATH = os.path.join(_HERE, "libfdvlm.so")
 FDVLM_OK = 0
 ERR_INVALID_ARG, ERR_STATE, ERR_CAPACITY, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_OOM = -1, -2, -3, -4, -5, -6, -7
 DT_F32, DT_BF16, DT_FP8 = 0, 1, 2
+KV_BF16, KV_F16 = 0, 1
 RULE_THRESHOLD, RULE_TOPK = 0, 1
+KERNEL_KINDS = ("rope_table", "gemm_qkv", "fin_qkv", "attention", "attn_merge", "gemm_o", "fin_resid", "gemm_gate_up",
+                "gemm_down", "gemm_lm_head", "stats_merge")
 _DTYPE_CODE = {_in.F32: DT_F32, _in.BF16: DT_BF16, _in.FP8: DT_FP8}
 
 
@@ -29,7 +32,7 @@ class Config(C.Structure):
     _fields_ = [(n, C.c_int) for n in ("n_layers", "hidden", "n_q_heads", "n_kv_heads", "head_dim", "intermediate",
                                        "vocab", "mask_id")] + \
                [("rms_eps", C.c_float), ("rope_theta", C.c_float), ("tie_embeddings", C.c_int), ("dtype", C.c_int),
-                ("max_seq", C.c_int), ("max_block", C.c_int)]
+                ("max_seq", C.c_int), ("max_block", C.c_int), ("kv_dtype", C.c_int)]
 
 
 _LW_FIELDS = ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down", "bq", "bk", "bv",
@@ -53,6 +56,10 @@ class StepInfo(C.Structure):
     _fields_ = [("n_unmasked", C.c_int), ("n_remaining", C.c_int), ("step_index", C.c_int)]
 
 
+class KernelRecord(C.Structure):
+    _fields_ = [("kind", C.c_int), ("start_us", C.c_double), ("released_us", C.c_double), ("end_us", C.c_double)]
+
+
 class SpecInfo(C.Structure):
     _fields_ = [("accepted", C.c_int), ("next_token", C.c_int32), ("cache_len", C.c_int)]
 
@@ -61,6 +68,11 @@ EXPORTS = {
     "fdvlm_create": (C.c_int, [C.POINTER(Config), C.POINTER(Weights), C.c_void_p, C.POINTER(C.c_void_p)]),
     "fdvlm_destroy": (None, [C.c_void_p]),
     "fdvlm_reset": (C.c_int, [C.c_void_p]),
+    "fdvlm_synchronize": (C.c_int, [C.c_void_p]),
+    "fdvlm_debug_poison": (C.c_int, [C.c_void_p, C.c_int]),
+    "fdvlm_decode_block": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.POINTER(StepParams), C.c_void_p, C.POINTER(StepInfo)]),
+    "fdvlm_profile_read_chain": (C.c_int, [C.c_void_p, C.POINTER(KernelRecord), C.c_int, C.POINTER(C.c_int)]),
+    "fdvlm_op_linear_status": (C.c_int, [C.c_void_p, C.c_void_p]),
     "fdvlm_prefill": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_void_p]),
     "fdvlm_block_begin": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p]),
     "fdvlm_block_begin_host": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p]),
@@ -87,7 +99,7 @@ EXPORTS = {
                                          C.c_int, C.c_void_p]),
     "fdvlm_op_linear_workspace_bytes": (C.c_size_t, [C.c_int, C.c_int, C.c_int, C.c_int]),
     "fdvlm_op_attention": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int,
-                                     C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p]),
+                                     C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p]),
     "fdvlm_op_attention_workspace_bytes": (C.c_size_t, [C.c_int, C.c_int, C.c_int, C.c_int]),
     "fdvlm_version": (C.c_char_p, []),
 }
@@ -136,12 +148,13 @@ class Handle:
     `inputs.make_weights`; it is kept alive by this object because the library borrows the pointers."""
 
     def __init__(self, shape: _in.ModelShape, weights: dict, max_seq: int, max_block: int = 64,
-                 stream: Optional[torch.cuda.Stream] = None):
+                 stream: Optional[torch.cuda.Stream] = None, kv_dtype: int = KV_F16):
         self.shape, self.weights, self.stream = shape, weights, stream
         self.max_seq, self.max_block = max_seq, max_block
+        self.kv_dtype = kv_dtype
         cfg = Config(shape.n_layers, shape.hidden, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
                      shape.intermediate, shape.vocab, shape.mask_id, shape.rms_eps, shape.rope_theta,
-                     int(shape.tie_embeddings), _DTYPE_CODE[shape.dtype], max_seq, max_block)
+                     int(shape.tie_embeddings), _DTYPE_CODE[shape.dtype], max_seq, max_block, kv_dtype)
         self._layers = (LayerWeights * shape.n_layers)()
         for i, lw in enumerate(weights["layers"]):
             for name in _LW_FIELDS:
@@ -153,6 +166,7 @@ class Handle:
         if rc != FDVLM_OK:
             raise FdvlmError(rc, lib().fdvlm_last_error(None).decode())
         self.act_dtype = torch.float32 if shape.dtype == _in.F32 else torch.bfloat16
+        self.kv_torch_dtype = torch.float32 if shape.dtype == _in.F32 else (torch.float16 if kv_dtype == KV_F16 else torch.bfloat16)
 
     def _check(self, rc: int):
         if rc != FDVLM_OK:
@@ -171,6 +185,19 @@ class Handle:
 
     def reset(self):
         self._check(lib().fdvlm_reset(self._h))
+
+    def synchronize(self):
+        self._check(lib().fdvlm_synchronize(self._h))
+
+    def debug_poison(self, on: bool):
+        self._check(lib().fdvlm_debug_poison(self._h, int(on)))
+
+    def decode_block(self, block_size: int, rule: int, threshold: float = 0.9, k: int = 8,
+                     init_tokens: Optional[torch.Tensor] = None, pred_shift: int = 0,
+                     block_tokens: Optional[torch.Tensor] = None) -> StepInfo:
+        p, info = StepParams(rule, threshold, k, pred_shift), StepInfo()
+        self._check(lib().fdvlm_decode_block(self._h, block_size, _ptr(init_tokens), C.byref(p), _ptr(block_tokens), C.byref(info)))
+        return info
 
     def prefill(self, embeds: Optional[torch.Tensor], tokens: Optional[torch.Tensor],
                 last_logits: Optional[torch.Tensor] = None):
@@ -229,15 +256,22 @@ class Handle:
         return lib().fdvlm_cache_len(self._h)
 
     def cache_read(self, layer: int, which: int, pos0: int, n: int) -> torch.Tensor:
-        dst = torch.empty(n, self.shape.n_kv_heads, self.shape.head_dim, dtype=self.act_dtype, device="cuda")
+        dst = torch.empty(n, self.shape.n_kv_heads, self.shape.head_dim, dtype=self.kv_torch_dtype, device="cuda")
         self._check(lib().fdvlm_cache_read(self._h, layer, which, pos0, n, _ptr(dst)))
         return dst
 
     def last_launch_count(self) -> int:
         return lib().fdvlm_last_launch_count(self._h)
 
-    def profile_enable(self, on: bool):
-        self._check(lib().fdvlm_profile_enable(self._h, int(on)))
+    def profile_enable(self, mode):
+        self._check(lib().fdvlm_profile_enable(self._h, int(mode)))
+
+    def profile_read_chain(self, cap: int = 1024) -> list:
+        """Records of the last forward under profile mode 2: dicts(kind, start_us, released_us, end_us) in launch order."""
+        recs, n = (KernelRecord * cap)(), C.c_int()
+        self._check(lib().fdvlm_profile_read_chain(self._h, recs, cap, C.byref(n)))
+        return [dict(kind=KERNEL_KINDS[r.kind], start_us=r.start_us, released_us=r.released_us, end_us=r.end_us)
+                for r in recs[:min(n.value, cap)]]
 
     def profile_read(self) -> dict:
         ml, ma, nl, na = C.c_double(), C.c_double(), C.c_int(), C.c_int()
@@ -254,6 +288,8 @@ def op_linear(x: torch.Tensor, w: torch.Tensor, scale=None, bias=None, dtype: in
     ws = torch.empty(max(nbytes, 16), dtype=torch.uint8, device=x.device)
     rc = lib().fdvlm_op_linear(_ptr(x), _ptr(w), _ptr(scale), _ptr(bias), _ptr(y), m, n, k, dtype, _ptr(ws),
                                _stream_ptr(stream))
+    if rc == FDVLM_OK:
+        rc = lib().fdvlm_op_linear_status(_ptr(ws), _stream_ptr(stream))
     if rc != FDVLM_OK:
         raise FdvlmError(rc, "fdvlm_op_linear")
     return y
@@ -268,6 +304,8 @@ def op_linear_static(x: torch.Tensor, w: torch.Tensor, scale=None, bias=None, dt
     if y is None:
         y = torch.empty(m, n, dtype=torch.float32, device=x.device)
     rc = lib().fdvlm_op_linear_static(_ptr(x), _ptr(w), _ptr(scale), _ptr(bias), _ptr(y), m, n, k, dtype, _stream_ptr(stream))
+    if rc == FDVLM_OK:
+        rc = lib().fdvlm_op_linear_status(None, _stream_ptr(stream))
     if rc != FDVLM_OK:
         raise FdvlmError(rc, lib().fdvlm_last_error(None).decode())
     return y
@@ -275,13 +313,15 @@ def op_linear_static(x: torch.Tensor, w: torch.Tensor, scale=None, bias=None, dt
 
 def op_attention(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, cache_len: int, causal: bool,
                  dtype: int = DT_BF16, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """Element type of q / caches / result: fp32 with DT_F32, else the tensors' own 16-bit type (bf16 or f16)."""
+    kv = KV_F16 if q.dtype == torch.float16 else KV_BF16
     n, hq, d = q.shape
     hkv, max_seq, _ = k_cache.shape
     out = torch.empty(n, hq * d, dtype=q.dtype, device=q.device)
     nbytes = lib().fdvlm_op_attention_workspace_bytes(n, hq, hkv, d)
     ws = torch.empty(max(nbytes, 16), dtype=torch.uint8, device=q.device)
     rc = lib().fdvlm_op_attention(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(out), n, cache_len, max_seq, hq, hkv, d,
-                                  int(causal), dtype, _ptr(ws), _stream_ptr(stream))
+                                  int(causal), dtype, kv, _ptr(ws), _stream_ptr(stream))
     if rc != FDVLM_OK:
         raise FdvlmError(rc, "fdvlm_op_attention")
     return out

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfdvlm.so")
-SOURCES = ["fdvlm.cu", "forward.cu", "kernels.cu", "gemm_tc.cu", "attention.cu", "op_static.cu", "mega.cu"]
+SOURCES = ["fdvlm.cu", "forward.cu", "kernels.cu", "gemm_tc.cu", "attention.cu", "op_static.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-cudart", "static", "--expt-relaxed-constexpr"]
 
@@ -32,16 +32,19 @@ def build(force: bool = False, verbose: bool = False) -> str:
     """Compile every .cu of the library and link the shared object; returns its path."""
     if not force and not _stale():
         return LIB
-    objs = []
+    objs, procs = [], []
     os.makedirs(os.path.join(HERE, "_build"), exist_ok=True)
-    for src in SOURCES:
+    for src in SOURCES:       # one nvcc per translation unit, side by side
         obj = os.path.join(HERE, "_build", src.replace(".cu", ".o"))
         cmd = [_nvcc(), *NVCC_FLAGS, "-c", os.path.join(CSRC, src), "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas")
             cmd.insert(2, "-v")
-        subprocess.run(cmd, check=True)
+        procs.append((cmd, subprocess.Popen(cmd)))
         objs.append(obj)
+    for cmd, proc in procs:
+        if proc.wait() != 0:
+            raise subprocess.CalledProcessError(proc.returncode, cmd)
     subprocess.run([_nvcc(), *NVCC_FLAGS, "-shared", *objs, "-o", LIB], check=True)
     return LIB
 

@@ -1,5 +1,5 @@
-// Core of the split-KV, block-masked GQA attention (bf16, mma.sync m16n8k16, online softmax in fp32),
-// as a device function that both the stand-alone kernel and the persistent forward kernel call.
+// Core of the split-KV, block-masked GQA attention (bf16 or f16 operands, mma.sync m16n8k16, online softmax in
+// fp32).  T is the element type of q and of the KV cache; the probabilities are rounded to T for the P.V product.
 #pragma once
 #include "common.cuh"
 
@@ -21,13 +21,24 @@ __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r
 __device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
 }
-__device__ __forceinline__ void mma_bf16(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+template <typename T> __device__ __forceinline__ void mma_16816(float* c, const uint32_t* a, uint32_t b0, uint32_t b1);
+template <> __device__ __forceinline__ void mma_16816<bf16>(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
   asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+template <> __device__ __forceinline__ void mma_16816<__half>(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+template <typename T> __device__ __forceinline__ uint32_t pack2(float lo, float hi);
+template <> __device__ __forceinline__ uint32_t pack2<bf16>(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+template <> __device__ __forceinline__ uint32_t pack2<__half>(float lo, float hi) {
+  __half2 v = __floats2half2_rn(lo, hi);       // probabilities lie in [0, 1]: no range concern
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
@@ -57,8 +68,8 @@ __device__ __forceinline__ void attn_bar() { asm volatile("bar.sync 1, 128;" :::
 // PDL: the caller is a kernel launched with programmatic dependent launch that has not yet waited for its predecessor
 // (which writes q and the K/V rows of positions >= L); a first key tile that lies wholly in the committed cache is
 // then requested before that wait.
-template <int D, bool PDL = false>
-__device__ __forceinline__ void attn_item(const bf16* q, const bf16* kc, const bf16* vc, float* part_o, float2* part_ml,
+template <int D, typename E, bool PDL = false>
+__device__ __forceinline__ void attn_item(const E* q, const E* kc, const E* vc, float* part_o, float2* part_ml,
                                           int n, int L, int max_seq, int hq, int hkv, int qh, int chunk_keys, int n_chunks,
                                           int causal, int chunk, int grp, int hk, uint32_t sQ, int tid) {
   constexpr int CH = D / 8;                 // 16-byte chunks per row
@@ -74,8 +85,8 @@ __device__ __forceinline__ void attn_item(const bf16* q, const bf16* kc, const b
   const int key_end = min(T, key_begin + chunk_keys);
   const int n_tiles = (key_end - key_begin + AT_KEYS - 1) / AT_KEYS;
   const int warp = tid >> 5, lane = tid & 31;
-  const bf16* kbase = kc + (size_t)hk * max_seq * D;
-  const bf16* vbase = vc + (size_t)hk * max_seq * D;
+  const E* kbase = kc + (size_t)hk * max_seq * D;
+  const E* vbase = vc + (size_t)hk * max_seq * D;
 
   auto load_tile = [&](int t, int buf) {
     const int j0 = key_begin + t * AT_KEYS;
@@ -92,7 +103,7 @@ __device__ __forceinline__ void attn_item(const bf16* q, const bf16* kc, const b
   if (early) load_tile(0, 0);
   // ---- stage Q (rows = heads_here x n; row r -> head r / n, token r % n); addresses worked out before the wait ----
   constexpr int QV = AT_ROWS * CH / 128;
-  const bf16* q_src[QV];
+  const E* q_src[QV];
   uint32_t q_dst[QV];
 #pragma unroll
   for (int u = 0; u < QV; ++u) {
@@ -146,8 +157,8 @@ __device__ __forceinline__ void attn_item(const bf16* q, const bf16* kc, const b
         for (int np = 0; np < AT_KEYS / 16; ++np) {
           uint32_t b0, b1, b2, b3;
           ldsm_x4(kt + swz<D>(np * 16 + (lane & 7) + ((lane >> 4) << 3), kk * 2 + ((lane >> 3) & 1)), b0, b1, b2, b3);
-          mma_bf16(s[2 * np], qf[kk], b0, b1);
-          mma_bf16(s[2 * np + 1], qf[kk], b2, b3);
+          mma_16816<E>(s[2 * np], qf[kk], b0, b1);
+          mma_16816<E>(s[2 * np + 1], qf[kk], b2, b3);
         }
       }
       // mask + running max
@@ -187,16 +198,16 @@ __device__ __forceinline__ void attn_item(const bf16* q, const bf16* kc, const b
 #pragma unroll
       for (int kk = 0; kk < AT_KEYS / 16; ++kk) {
         uint32_t pa[4];
-        pa[0] = pack_bf16(s[2 * kk][0], s[2 * kk][1]);
-        pa[1] = pack_bf16(s[2 * kk][2], s[2 * kk][3]);
-        pa[2] = pack_bf16(s[2 * kk + 1][0], s[2 * kk + 1][1]);
-        pa[3] = pack_bf16(s[2 * kk + 1][2], s[2 * kk + 1][3]);
+        pa[0] = pack2<E>(s[2 * kk][0], s[2 * kk][1]);
+        pa[1] = pack2<E>(s[2 * kk][2], s[2 * kk][3]);
+        pa[2] = pack2<E>(s[2 * kk + 1][0], s[2 * kk + 1][1]);
+        pa[3] = pack2<E>(s[2 * kk + 1][2], s[2 * kk + 1][3]);
 #pragma unroll
         for (int dp = 0; dp < D / 16; ++dp) {
           uint32_t b0, b1, b2, b3;
           ldsm_x4_t(vt + swz<D>(kk * 16 + (lane & 7) + (((lane >> 3) & 1) << 3), dp * 2 + (lane >> 4)), b0, b1, b2, b3);
-          mma_bf16(o[2 * dp], pa, b0, b1);
-          mma_bf16(o[2 * dp + 1], pa, b2, b3);
+          mma_16816<E>(o[2 * dp], pa, b0, b1);
+          mma_16816<E>(o[2 * dp + 1], pa, b2, b3);
         }
       }
     }
@@ -231,9 +242,10 @@ template <int D> constexpr int attn_smem_bytes() { return AT_ROWS * D * 2 + 4 * 
 
 // Merge of the key chunks of one (row, head) by one warp: out = sum_c w_c O_c / sum_c w_c l_c, w_c = 2^(m_c - max m).
 // Lane j owns D / 32 consecutive output features; the chunk statistics are spread over the lanes.
+// The result is stored as `fmt` (XF_*) at element offset out_idx of `out`.
 template <int D>
-__device__ __forceinline__ void attn_merge_warp(const float* att_o, const float2* att_ml, bf16* out, size_t slot0, int n_chunks,
-                                                int lane) {
+__device__ __forceinline__ void attn_merge_warp(const float* att_o, const float2* att_ml, void* out, size_t out_idx, size_t lo_off,
+                                                int fmt, size_t slot0, int n_chunks, int lane) {
   constexpr int VPL = D / 32;
   constexpr int CB = 16;     // chunks whose partial outputs are in flight together
   // The statistics and the first CB partial outputs are requested together: one L2 round trip for up to 16 chunks.
@@ -285,7 +297,7 @@ __device__ __forceinline__ void attn_merge_warp(const float* att_o, const float2
   den = warp_sum(den);
   const float inv = 1.f / den;
 #pragma unroll
-  for (int i = 0; i < VPL; ++i) out[lane * VPL + i] = __float2bfloat16_rn(acc[i] * inv);
+  for (int i = 0; i < VPL; ++i) store_act(out, lo_off, out_idx + lane * VPL + i, acc[i] * inv, fmt);
 }
 
 }  // namespace fdk

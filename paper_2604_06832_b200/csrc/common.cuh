@@ -14,6 +14,7 @@ struct fp8e4m3 { uint8_t b; };  // OCP e4m3fn storage byte
 // ---- exact widening of storage types to fp32 -------------------------------------------------
 __device__ __forceinline__ float to_f32(float v) { return v; }
 __device__ __forceinline__ float to_f32(bf16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ float to_f32(__half v) { return __half2float(v); }
 // e4m3 (1-4-3, bias 7) placed in a half (1-5-10, bias 15): same sign, exponent field and top
 // mantissa bits; the bias difference is a factor 2^8.  Exact for normals and subnormals alike.
 __device__ __forceinline__ float to_f32(fp8e4m3 v) {
@@ -24,6 +25,11 @@ __device__ __forceinline__ float to_f32(fp8e4m3 v) {
 template <typename T> __device__ __forceinline__ T from_f32(float v);
 template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
 template <> __device__ __forceinline__ bf16 from_f32<bf16>(float v) { return __float2bfloat16_rn(v); }
+template <> __device__ __forceinline__ __half from_f32<__half>(float v) {
+  unsigned short r;
+  asm("cvt.rn.satfinite.f16.f32 %0, %1;" : "=h"(r) : "f"(v));
+  return __ushort_as_half(r);
+}
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
@@ -65,6 +71,12 @@ __device__ __forceinline__ float block_max(float v, float* red) {
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+// Set while a launch sequence is captured for a place that takes no programmatic edges: the kernels are then launched
+// the ordinary way (pdl_trigger / pdl_wait are no-ops).
+inline bool& pdl_disabled() {
+  static thread_local bool off = false;
+  return off;
+}
 template <typename... KArgs, typename... Args>
 static inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
   cudaLaunchConfig_t cfg;
@@ -73,12 +85,68 @@ static inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 blo
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr; cfg.numAttrs = 1;
+  cfg.attrs = attr; cfg.numAttrs = pdl_disabled() ? 0 : 1;
   return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
 }
 
+// In-chain timing of one kernel launch (only when profiling is on; a null pointer otherwise): the earliest start of
+// any of its CTAs, the earliest return of any CTA from its wait for the predecessor grid, the latest end of any CTA,
+// all in nanoseconds of the GPU's global timer.  Every field is kept as a minimum (the end as the minimum of the
+// complemented time), so the host presets the whole record to all-ones bytes.
+struct KStamp { unsigned long long start, released, end_inv, pad; };
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// each called by ONE thread of a CTA
+__device__ __forceinline__ void stamp_start(KStamp* s) { if (s) atomicMin(&s->start, global_ns()); }
+__device__ __forceinline__ void stamp_released(KStamp* s) { if (s) atomicMin(&s->released, global_ns()); }
+__device__ __forceinline__ void stamp_end(KStamp* s) { if (s) atomicMin(&s->end_inv, ~global_ns()); }
+
 enum { MODE_BIDIR = 0, MODE_CAUSAL = 1 };
 enum { DT_F32 = 0, DT_BF16 = 1, DT_FP8 = 2 };
+// Element type of q and the KV cache on the tensor-core path.
+enum { KV_BF16 = 0, KV_F16 = 1 };
+// How a 16-bit activation tensor that feeds a tensor-core GEMM is stored.
+//   XF_BF16X2: two bf16 planes, hi = bf16(v) and lo = bf16(v - hi), `lo_off` elements apart: the GEMM multiplies
+//              the streamed weight tile by both, so the activation carries ~16 significant bits (bf16 weights).
+//   XF_F16   : one f16 plane (fp8 weights widen exactly to f16, so that GEMM runs in f16: 11 significant bits).
+//   XF_BF16  : one bf16 plane (operator-level entry points that take caller-given bf16 rows).
+enum { XF_BF16X2 = 0, XF_F16 = 1, XF_BF16 = 2 };
+// Device status word: 0 = fine; 1..15 = a bounded wait gave up (the role that gave up); 16 = a token id outside
+// [0, vocab) was met (row 0 of the table was read instead).
+enum { ST_PRODUCER = 1, ST_MMA = 2, ST_EPILOGUE = 3, ST_ATTENTION = 4, ST_BAD_TOKEN = 16 };
+
+__device__ __forceinline__ unsigned short f16_bits_sat(float v) {
+  unsigned short r;
+  asm("cvt.rn.satfinite.f16.f32 %0, %1;" : "=h"(r) : "f"(v));
+  return r;
+}
+// one activation value into a tensor stored as `fmt` (see above); p points at the hi / only plane
+__device__ __forceinline__ void store_act(void* p, size_t lo_off, size_t idx, float v, int fmt) {
+  if (fmt == XF_F16) {
+    reinterpret_cast<unsigned short*>(p)[idx] = f16_bits_sat(v);
+  } else {
+    const bf16 hi = __float2bfloat16_rn(v);
+    reinterpret_cast<bf16*>(p)[idx] = hi;
+    if (fmt == XF_BF16X2) reinterpret_cast<bf16*>(p)[lo_off + idx] = __float2bfloat16_rn(v - __bfloat162float(hi));
+  }
+}
+
+constexpr int MAX_DEVICES = 64;
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) is a per-device setting: `done` is one flag per device.
+template <typename K>
+static inline cudaError_t ensure_dynamic_smem(K kern, int bytes, bool* done) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
+  if (done[dev]) return cudaSuccess;
+  e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) done[dev] = true;
+  return e;
+}
 
 static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 

@@ -22,18 +22,19 @@ static int check_config(const fdvlm_config* c) {
   if (c->max_block < 1 || c->max_block > 64) return fail(nullptr, FDVLM_ERR_INVALID_ARG, "max_block must be in 1..64");
   if (c->max_seq < c->max_block) return fail(nullptr, FDVLM_ERR_INVALID_ARG, "max_seq smaller than max_block");
   if (!(c->rms_eps > 0.f) || !(c->rope_theta > 0.f)) return fail(nullptr, FDVLM_ERR_INVALID_ARG, "rms_eps / rope_theta must be positive");
+  if (c->kv_dtype != FDVLM_KV_BF16 && c->kv_dtype != FDVLM_KV_F16) return fail(nullptr, FDVLM_ERR_INVALID_ARG, "unknown kv_dtype %d", (int)c->kv_dtype);
   return FDVLM_OK;
 }
 
-extern "C" const char* fdvlm_version(void) { return "fdvlm 0.2 (sm_100a)"; }
+extern "C" const char* fdvlm_version(void) { return "fdvlm 0.3 (sm_100a)"; }
 
 extern "C" const char* fdvlm_last_error(const fdvlm_t* h) { return h ? h->err : g_create_error; }
 
 extern "C" void fdvlm_destroy(fdvlm_t* h) {
   if (!h) return;
-  mega_destroy(h);
   for (auto& g : h->graphs) if (g.exec) cudaGraphExecDestroy(g.exec);
   h->graphs.clear();
+  if (h->loop_exec) cudaGraphExecDestroy(h->loop_exec);
   if (h->kv) cudaFree(h->kv);
   if (h->slab) cudaFree(h->slab);
   for (cudaEvent_t ev : h->prof_ev) cudaEventDestroy(ev);
@@ -84,11 +85,12 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
   h->stats = nullptr; h->logits = nullptr; h->conf = nullptr; h->pred = nullptr; h->unmask = nullptr; h->blk_tokens = nullptr;
   h->blk_masked = nullptr; h->info = nullptr; h->init_stage = nullptr; h->ws = nullptr; h->info_host = nullptr;
   h->host_stage = nullptr;
-  h->mega = nullptr;
   h->slab = nullptr;
   h->dev_len = nullptr;
   h->use_graphs = 0;
-  h->mega_slab = nullptr;
+  h->stamps = nullptr;
+  h->stamp_used = 0;
+  h->loop_exec = nullptr;
   cudaGetDevice(&h->device);
 
   const int R = cfg->max_block, H = cfg->hidden, I = cfg->intermediate, d = cfg->head_dim;
@@ -100,6 +102,17 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
   size_t wa = attention_workspace_bytes(R, cfg->n_q_heads, cfg->n_kv_heads, d);
   if (wa > ws) ws = wa;
   h->use_tc = (h->dt == DT_BF16 || h->dt == DT_FP8) && tc_linear_supported(R, NQ, H, h->dt) && tc_linear_supported(R, H, I, h->dt);
+  h->kv_type = (int)cfg->kv_dtype;
+  if (!h->use_tc && h->dt != DT_F32 && h->kv_type != KV_BF16) {
+    delete h;
+    return fail(nullptr, FDVLM_ERR_UNSUPPORTED, "an f16 KV cache needs shapes the tensor-core kernels take");
+  }
+  // GEMM inputs: bf16 hi + lo planes for bf16 weights, one f16 plane for fp8 weights (CUDA-core path: one plane)
+  h->xfmt = !h->use_tc ? XF_BF16 : (h->dt == DT_FP8 ? XF_F16 : XF_BF16X2);
+  h->head_fmt = (h->xfmt == XF_F16 && cfg->tie_embeddings) ? XF_BF16X2 : h->xfmt;
+  const int planes = h->xfmt == XF_BF16X2 ? 2 : 1;
+  const int a_planes = (h->xfmt == XF_BF16X2 || h->head_fmt == XF_BF16X2) ? 2 : 1;
+  h->a_lo = (size_t)R * H; h->ao_lo = (size_t)R * NQ; h->act_lo = (size_t)R * I;
   if (h->use_tc) {
     const size_t g3[] = {tc_workspace_bytes(R, NQKV, (NQ + 127) / 128 + 2 * ((NKV + 127) / 128), H),
                          tc_workspace_bytes(R, H, (H + 127) / 128, NQ), tc_workspace_bytes(R, H, (H + 127) / 128, I)};
@@ -109,7 +122,7 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
   // Every buffer but the KV cache is carved out of one slab, the small hot ones first: with gigabytes of weights
   // streaming through the TLBs, each separately allocated buffer would cost its own page walk whenever it is touched.
   struct { void** p; size_t bytes; } allocs[] = {
-      {(void**)&h->info, 16},
+      {(void**)&h->info, 32},
       {(void**)&h->dev_len, 16},
       {(void**)&h->conf, (size_t)R * 4},
       {(void**)&h->pred, (size_t)R * 4},
@@ -119,12 +132,12 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
       {(void**)&h->init_stage, 64 * 4},
       {(void**)&h->ssq, (size_t)R * h->nt * 4},
       {(void**)&h->cs, (size_t)R * d * 4},
-      {(void**)&h->mega_slab, mega_slab_bytes(h)},
+      {(void**)&h->stamps, h->use_tc ? sizeof(KStamp) * FDVLM_MAX_STAMPS : 16},
       {(void**)&h->h, (size_t)R * H * 4},
-      {(void**)&h->a, (size_t)R * H * h->act_sz},
-      {(void**)&h->ao, (size_t)R * NQ * h->act_sz},
+      {(void**)&h->a, (size_t)R * H * h->act_sz * a_planes},
+      {(void**)&h->ao, (size_t)R * NQ * h->act_sz * planes},
       {(void**)&h->q, (size_t)R * NQ * h->act_sz},
-      {(void**)&h->act, (size_t)R * I * h->act_sz},
+      {(void**)&h->act, (size_t)R * I * h->act_sz * planes},
       {(void**)&h->stats, (size_t)((cfg->vocab + 127) / 128) * 4 * R * 16},
       {(void**)&h->y, (size_t)R * (NQKV > 2 * I ? NQKV : 2 * I) * 4},
       {(void**)&h->ws, ws ? ws : 16},
@@ -144,25 +157,22 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
     char* cur = h->slab;
     for (auto& a : allocs) { *a.p = cur; cur += (a.bytes + 255) / 256 * 256; }
   }
-  if (cudaMallocHost((void**)&h->info_host, 16) != cudaSuccess || cudaMallocHost((void**)&h->host_stage, 64 * 16) != cudaSuccess) {
+  if (cudaMallocHost((void**)&h->info_host, 32) != cudaSuccess || cudaMallocHost((void**)&h->host_stage, 64 * 16) != cudaSuccess) {
     fail(nullptr, FDVLM_ERR_OOM, "pinned host allocation failed");
     fdvlm_destroy(h);
     return FDVLM_ERR_OOM;
   }
   e = cudaMemsetAsync(h->kv, 0, (size_t)cfg->n_layers * 2 * kv_plane(h), h->st);
-  if (e == cudaSuccess) e = cudaMemsetAsync(h->info, 0, 16, h->st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(h->info, 0, 32, h->st);
   if (e != cudaSuccess) {
     fail(nullptr, FDVLM_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
     fdvlm_destroy(h);
     return FDVLM_ERR_CUDA;
   }
-  // bf16 weights: the persistent forward kernel, for now only on request (FDVLM_MEGA=1)
   // the tensor-core forward is replayed from captured CUDA graphs (FDVLM_NO_GRAPH=1: launch kernel by kernel)
   const char* no_graph = getenv("FDVLM_NO_GRAPH");
   // (the legacy default stream cannot be captured: a handle created on it launches kernel by kernel)
   h->use_graphs = h->use_tc && h->st != nullptr && !(no_graph && no_graph[0] == '1');
-  const char* want_mega = getenv("FDVLM_MEGA");
-  if (h->use_tc && want_mega && want_mega[0] == '1') mega_create(h);
   *out = h;
   return FDVLM_OK;
 }
@@ -226,14 +236,33 @@ static int block_begin_common(fdvlm_t* h, int block_size) {
 
 // Read the 16-byte device record back: counts for the state machine, and the kernels' timeout word.
 static int sync_info(fdvlm_t* h) {
-  CU(h, cudaMemcpyAsync(h->info_host, h->info, 16, cudaMemcpyDeviceToHost, h->st));
+  CU(h, cudaMemcpyAsync(h->info_host, h->info, 32, cudaMemcpyDeviceToHost, h->st));
   CU(h, cudaStreamSynchronize(h->st));
   h->n_remaining = h->info_host[1];
   if (h->info_host[3] != 0) {
     const int code = h->info_host[3];
     cudaMemsetAsync(h->info + 3, 0, 4, h->st);
+    if (code == ST_BAD_TOKEN)
+      return fail(h, FDVLM_ERR_INVALID_ARG, "a token id outside [0, %d) was given; token 0 was embedded in its place", h->cfg.vocab);
     return fail(h, FDVLM_ERR_TIMEOUT, "a bounded device-side wait gave up (kernel role %d); results of this call are invalid", code);
   }
+  return FDVLM_OK;
+}
+
+extern "C" int fdvlm_synchronize(fdvlm_t* h) {
+  if (!h) return FDVLM_ERR_INVALID_ARG;
+  const int keep = h->n_remaining;        // the block state the host tracks is not this call's business
+  const int rc = sync_info(h);
+  h->n_remaining = keep;
+  return rc;
+}
+
+extern "C" int fdvlm_debug_poison(fdvlm_t* h, int on) {
+  if (!h) return FDVLM_ERR_INVALID_ARG;
+  int32_t* stage = (int32_t*)(h->host_stage + 960);      // pinned, beyond what the *_host variants use
+  CU(h, cudaStreamSynchronize(h->st));                   // an earlier value may still be in flight from the same slot
+  *stage = on ? 1 : 0;
+  CU(h, cudaMemcpyAsync(h->info + 4, stage, 4, cudaMemcpyHostToDevice, h->st));
   return FDVLM_OK;
 }
 
@@ -267,13 +296,19 @@ extern "C" int fdvlm_block_set_tokens(fdvlm_t* h, const int32_t* tokens) {
   return sync_info(h);
 }
 
-static int step_core(fdvlm_t* h, const fdvlm_step_params* p, int want_logits) {
-  if (!h) return FDVLM_ERR_INVALID_ARG;
+static int check_step_params(fdvlm_t* h, const fdvlm_step_params* p) {
   if (!p) return fail(h, FDVLM_ERR_INVALID_ARG, "NULL step params");
   if (p->rule != FDVLM_RULE_THRESHOLD && p->rule != FDVLM_RULE_TOPK) return fail(h, FDVLM_ERR_INVALID_ARG, "unknown rule");
   if (p->rule == FDVLM_RULE_TOPK && p->k < 1) return fail(h, FDVLM_ERR_INVALID_ARG, "top-k needs k >= 1");
   if (p->rule == FDVLM_RULE_THRESHOLD && !(p->threshold == p->threshold)) return fail(h, FDVLM_ERR_INVALID_ARG, "threshold is NaN");
   if (p->pred_shift != 0 && p->pred_shift != 1) return fail(h, FDVLM_ERR_INVALID_ARG, "pred_shift is 0 or 1");
+  return FDVLM_OK;
+}
+
+static int step_core(fdvlm_t* h, const fdvlm_step_params* p, int want_logits) {
+  if (!h) return FDVLM_ERR_INVALID_ARG;
+  int prc = check_step_params(h, p);
+  if (prc) return prc;
   if (!h->block_open) return fail(h, FDVLM_ERR_STATE, "block_step without an open block");
   if (h->n_remaining == 0) return fail(h, FDVLM_ERR_STATE, "block_step with no masked position left");
   const int B = h->block_size;
@@ -337,6 +372,92 @@ extern "C" int fdvlm_decode_block_topk(fdvlm_t* h, int block_size, const int32_t
   if (rc) return rc;
   info->n_unmasked = h->info_host[0]; info->n_remaining = h->info_host[1]; info->step_index = h->info_host[2];
   if (h->n_remaining != 0) return fail(h, FDVLM_ERR_STATE, "%d masked positions left after %d top-%d steps", h->n_remaining, steps, k);
+  return FDVLM_OK;
+}
+
+// The decode loop of one block as a CUDA graph: a conditional WHILE node whose body is one denoise step (embedding
+// of the block's tokens, the forward, the selection); the selection kernel sets the loop condition on the device.
+// Built once per (block size, step parameters) and kept.  Dependent-launch edges are tried first; if the runtime
+// refuses them inside a conditional body the kernels are recorded with ordinary edges.
+static int build_loop_graph(fdvlm_t* h, int B, const fdvlm_step_params* p, bool with_pdl) {
+  cudaGraph_t g = nullptr;
+  CU(h, cudaGraphCreate(&g, 0));
+  int rc = FDVLM_OK;
+  cudaGraphExec_t exec = nullptr;
+  int body_launches = 0;
+  do {
+    cudaGraphConditionalHandle cond;
+    cudaError_t e = cudaGraphConditionalHandleCreate(&cond, g, 1, cudaGraphCondAssignDefault);
+    if (e != cudaSuccess) { rc = fail(h, FDVLM_ERR_CUDA, "conditional handle: %s", cudaGetErrorString(e)); break; }
+    cudaGraphNodeParams np = {cudaGraphNodeTypeConditional};
+    np.type = cudaGraphNodeTypeConditional;
+    np.conditional.handle = cond;
+    np.conditional.type = cudaGraphCondTypeWhile;
+    np.conditional.size = 1;
+    cudaGraphNode_t node;
+    e = cudaGraphAddNode(&node, g, nullptr, 0, &np);
+    if (e != cudaSuccess) { rc = fail(h, FDVLM_ERR_CUDA, "conditional node: %s", cudaGetErrorString(e)); break; }
+    cudaGraph_t body = np.conditional.phGraph_out[0];
+    e = cudaStreamBeginCaptureToGraph(h->st, body, nullptr, nullptr, 0, cudaStreamCaptureModeThreadLocal);
+    if (e != cudaSuccess) { rc = fail(h, FDVLM_ERR_CUDA, "capture of the loop body: %s", cudaGetErrorString(e)); break; }
+    pdl_disabled() = !with_pdl;
+    const int before = h->launches;
+    rc = stage_rows(h, 0, B, h->blk_tokens, nullptr);
+    if (rc == FDVLM_OK) rc = forward_rows_enqueue(h, B, MODE_BIDIR, B, 0);
+    if (rc == FDVLM_OK) {
+      launch_select(h->conf, h->pred, h->blk_tokens, h->blk_masked, h->unmask, h->info, B, (int)p->rule, p->threshold, p->k, h->st,
+                    p->pred_shift, cond, 1);
+      h->launches++;
+    }
+    pdl_disabled() = false;
+    body_launches = h->launches - before;
+    cudaGraph_t captured = nullptr;
+    e = cudaStreamEndCapture(h->st, &captured);
+    if (rc != FDVLM_OK) break;
+    if (e != cudaSuccess) { rc = fail(h, FDVLM_ERR_CUDA, "capture of the loop body: %s", cudaGetErrorString(e)); break; }
+    e = cudaGraphInstantiate(&exec, g, 0);
+    if (e != cudaSuccess) { rc = fail(h, FDVLM_ERR_CUDA, "instantiate of the loop graph: %s", cudaGetErrorString(e)); break; }
+  } while (0);
+  cudaGraphDestroy(g);
+  if (rc != FDVLM_OK) { cudaGetLastError(); return rc; }
+  if (h->loop_exec) cudaGraphExecDestroy(h->loop_exec);
+  h->loop_exec = exec;
+  h->loop_n = B; h->loop_rule = (int)p->rule; h->loop_k = p->k; h->loop_shift = p->pred_shift; h->loop_threshold = p->threshold;
+  h->loop_body_launches = body_launches;
+  return FDVLM_OK;
+}
+
+extern "C" int fdvlm_decode_block(fdvlm_t* h, int block_size, const int32_t* init_tokens, const fdvlm_step_params* p,
+                                  int32_t* block_tokens, fdvlm_step_info* info) {
+  if (!h) return FDVLM_ERR_INVALID_ARG;
+  if (!info) return fail(h, FDVLM_ERR_INVALID_ARG, "decode_block needs the host info struct");
+  int rc = check_step_params(h, p);
+  if (rc) return rc;
+  if (!h->use_graphs) return fail(h, FDVLM_ERR_UNSUPPORTED, "decode_block needs the tensor-core path on a non-default stream");
+  rc = fdvlm_block_begin(h, block_size, init_tokens);      // (reads the masked count back when tokens are given)
+  if (rc) return rc;
+  h->launches = 0;
+  if (h->n_remaining > 0) {
+    const bool have = h->loop_exec && h->loop_n == block_size && h->loop_rule == (int)p->rule && h->loop_k == p->k &&
+                      h->loop_shift == p->pred_shift && h->loop_threshold == p->threshold;
+    if (!have) {
+      rc = build_loop_graph(h, block_size, p, true);
+      if (rc) rc = build_loop_graph(h, block_size, p, false);
+      if (rc) return rc;
+    }
+    launch_set_len(h->dev_len, h->cache_len, h->st);
+    CU(h, cudaMemsetAsync(h->info + 5, 0, 4, h->st));
+    CU(h, cudaGraphLaunch(h->loop_exec, h->st));
+  }
+  if (block_tokens) CU(h, cudaMemcpyAsync(block_tokens, h->blk_tokens, (size_t)block_size * 4, cudaMemcpyDeviceToDevice, h->st));
+  rc = sync_info(h);
+  if (rc) return rc;
+  info->n_unmasked = h->info_host[0]; info->n_remaining = h->info_host[1]; info->step_index = h->info_host[2];
+  h->step_index = h->info_host[2];
+  h->launches = 1 + h->info_host[5] * h->loop_body_launches;
+  if (h->n_remaining != 0)
+    return fail(h, FDVLM_ERR_STATE, "%d masked positions left after %d steps (a masked position 0 under pred_shift = 1 cannot be revealed)",
+                h->n_remaining, h->info_host[5]);
   return FDVLM_OK;
 }
 
@@ -468,10 +589,33 @@ extern "C" int fdvlm_cache_read(const fdvlm_t* hc, int layer, int which, int pos
 }
 
 // ---- instrumentation --------------------------------------------------------------------------------
-extern "C" int fdvlm_profile_enable(fdvlm_t* h, int on) {
+extern "C" int fdvlm_profile_enable(fdvlm_t* h, int mode) {
   if (!h) return FDVLM_ERR_INVALID_ARG;
-  h->prof_on = on ? 1 : 0;
+  if (mode < 0 || mode > 2) return fail(h, FDVLM_ERR_INVALID_ARG, "profile mode is 0, 1 or 2");
+  if (mode == 2 && !h->use_tc) return fail(h, FDVLM_ERR_UNSUPPORTED, "in-chain timing covers the tensor-core path only");
+  h->prof_on = mode;
   h->prof_used = 0;
+  h->stamp_used = 0;
+  return FDVLM_OK;
+}
+
+extern "C" int fdvlm_profile_read_chain(fdvlm_t* h, fdvlm_kernel_record* records, int cap, int* n) {
+  if (!h) return FDVLM_ERR_INVALID_ARG;
+  CU(h, cudaStreamSynchronize(h->st));
+  const int used = h->stamp_used;
+  if (n) *n = used;
+  if (!records || cap <= 0 || used == 0) return FDVLM_OK;
+  std::vector<KStamp> host((size_t)used);
+  CU(h, cudaMemcpy(host.data(), h->stamps, sizeof(KStamp) * used, cudaMemcpyDeviceToHost));
+  unsigned long long t0 = ~0ull;
+  for (const KStamp& k : host) if (k.start < t0) t0 = k.start;
+  for (int i = 0; i < used && i < cap; ++i) {
+    const KStamp& k = host[i];
+    records[i].kind = h->stamp_kind[i];
+    records[i].start_us = (k.start == ~0ull) ? -1.0 : (double)(k.start - t0) * 1e-3;
+    records[i].released_us = (k.released == ~0ull) ? -1.0 : (double)(k.released - t0) * 1e-3;
+    records[i].end_us = (k.end_inv == ~0ull) ? -1.0 : (double)(~k.end_inv - t0) * 1e-3;
+  }
   return FDVLM_OK;
 }
 
@@ -508,7 +652,7 @@ extern "C" int fdvlm_op_linear(const void* x, const void* w, const float* scale,
   LinearArgs a;
   a.x = x; a.w = w; a.scale = scale; a.bias = bias; a.y = y; a.m = m; a.n = n; a.k = k; a.ldy = n; a.accumulate = 0;
   a.dtype = (int)dtype; a.workspace = workspace; a.workspace_bytes = linear_workspace_bytes(m, n, k, (int)dtype);
-  if (a.workspace_bytes && !workspace) return FDVLM_ERR_INVALID_ARG;
+  if (!workspace) return FDVLM_ERR_INVALID_ARG;
   cudaError_t e;
   int r = launch_linear(a, (cudaStream_t)cuda_stream, &e);
   return r < 0 ? FDVLM_ERR_CUDA : FDVLM_OK;
@@ -521,13 +665,15 @@ extern "C" size_t fdvlm_op_attention_workspace_bytes(int n_rows, int n_q_heads, 
 
 extern "C" int fdvlm_op_attention(const void* q, const void* k_cache, const void* v_cache, void* out, int n_rows,
                                   int cache_len, int max_seq, int n_q_heads, int n_kv_heads, int head_dim, int causal,
-                                  fdvlm_dtype dtype, void* workspace, void* cuda_stream) {
+                                  fdvlm_dtype dtype, fdvlm_kv_dtype kv_dtype, void* workspace, void* cuda_stream) {
   if (!q || !k_cache || !v_cache || !out || n_rows < 1 || n_rows > 64 || cache_len < 0 || cache_len + n_rows > max_seq ||
       n_q_heads < 1 || n_kv_heads < 1 || (n_q_heads % n_kv_heads) || (head_dim != 64 && head_dim != 128))
     return FDVLM_ERR_INVALID_ARG;
   if (dtype != FDVLM_F32 && dtype != FDVLM_BF16 && dtype != FDVLM_W_FP8E4M3) return FDVLM_ERR_INVALID_ARG;
+  if (kv_dtype != FDVLM_KV_BF16 && kv_dtype != FDVLM_KV_F16) return FDVLM_ERR_INVALID_ARG;
   AttnArgs a;
-  a.len_ptr = nullptr;
+  memset(&a, 0, sizeof(a));
+  a.kv_type = (int)kv_dtype; a.out_fmt = kv_dtype == FDVLM_KV_F16 ? XF_F16 : XF_BF16;
   a.q = q; a.kc = k_cache; a.vc = v_cache; a.out = out; a.n = n_rows; a.cache_len = cache_len; a.max_seq = max_seq;
   a.hq = n_q_heads; a.hkv = n_kv_heads; a.d = head_dim; a.causal = causal ? 1 : 0; a.dtype = (int)dtype; a.workspace = workspace;
   cudaError_t e;

@@ -7,9 +7,12 @@
 // one elected thread issues tcgen05.mma with fp32 accumulators in tensor memory (two accumulator
 // buffers, so the epilogue of one work item overlaps the mainloop of the next); four epilogue warps
 // read the accumulators with tcgen05.ld.  CTAs are persistent over a static round-robin list of
-// work items (tile, K-split).  FP8-E4M3 weights take the same road with half the bytes: the byte tile lands in
-// the stage, four converter warps widen it exactly to bf16 (e4m3 -> f16 -> f32 -> bf16, all exact) into a
-// swizzled buffer of its own, and the MMA reads that buffer; the per-channel scales are applied by the epilogues.
+// work items (tile, K-split).  bf16 weights: the activations arrive as two bf16 planes, hi = bf16(v) and
+// lo = bf16(v - hi); every streamed weight tile is multiplied by both (two MMAs into the same accumulator), so the
+// activation side of the product carries ~16 significant bits at no extra HBM traffic.  FP8-E4M3 weights take the
+// same road with half the bytes: the byte tile lands in the stage, four converter warps widen it exactly to f16
+// (one cvt per pair) into a swizzled buffer of its own, and the MMA (f16 x f16, activations stored as f16) reads
+// that buffer; the per-channel scales are applied by the epilogues.
 // Every mbarrier wait is bounded: on a timeout the CTA records an
 // error code in a status word, drains its own bulk copies, frees its tensor memory and returns.
 #include <cuda.h>
@@ -28,11 +31,13 @@ constexpr int TC_THREADS_FP8 = 320;   // + warps 6..9: e4m3 -> bf16 converters
 constexpr int TC_A_BYTES = TC_BM * TC_BK * 2;   // a bf16 weight tile
 constexpr int TC_NCONV = 2;           // converted-tile buffers (fp8 only)
 
-enum { TC_ERR_PRODUCER = 1, TC_ERR_MMA = 2, TC_ERR_EPILOGUE = 3 };
+enum { TC_ERR_PRODUCER = ST_PRODUCER, TC_ERR_MMA = ST_MMA, TC_ERR_EPILOGUE = ST_EPILOGUE };
 
 struct TcParams {
   CUtensorMap tm_w[3];  // weight matrices, box {64 k, 64 rows}
-  CUtensorMap tm_x;     // activations, box {64 k, m_pad rows}
+  CUtensorMap tm_x;     // activations (hi plane, or the only one), box {64 k, m_pad rows}
+  CUtensorMap tm_xl;    // lo plane of the activations (has_lo)
+  int has_lo;
   int n_out[3];         // rows (output features) of each matrix
   int tile_begin[4];    // first tile of each matrix; [n_mats] = total tiles
   int out_col[3];       // column of each matrix's first feature in the output row
@@ -43,8 +48,9 @@ struct TcParams {
   int ldp;
   float* y;             // [m][ldy]             (DIRECT)
   int ldy, accumulate;
-  bf16* act;            // [m][inter]           (SWIGLU)
-  int inter;
+  void* act;            // [m][inter]           (SWIGLU), stored as act_fmt (XF_*), lo plane act_lo_off elements on
+  size_t act_lo_off;
+  int act_fmt, inter;
   // RMSNorm folded into the consumer: x holds bf16(h * gain); the per-row factor rsqrt(mean(h^2) + eps)
   // is applied to the accumulators.  ssq_in[row][nt_in] holds partial sums of h^2 (null: factor 1).
   const float* ssq_in;
@@ -54,16 +60,19 @@ struct TcParams {
   // mask token's column excluded: (max, sum exp(l - max), argmax column)
   float4* stats;        // [tiles * 4][m]
   int mask_id, write_logits;
-  int* status;          // device word, set non-zero when a wait timed out
+  int* status;          // device words: [0] set non-zero when a wait timed out; [1] read at start: non-zero makes
+                        // every role take its give-up path at once (a host-set test hook for that path)
+  KStamp* stamp;        // in-chain timing of this launch (null: off)
 };
 
 template <int M_PAD, bool FP8>
 struct TcSmem {
-  static constexpr int STAGES = FP8 ? 6 : 4;
+  static constexpr int STAGES = FP8 ? 6 : (M_PAD <= 32 ? 4 : 3);       // two CTAs per SM must fit
   static constexpr int W_BYTES = FP8 ? TC_BM * TC_BK : TC_A_BYTES;     // weight tile as it is streamed
   static constexpr int W_ROW = FP8 ? TC_BK : TC_BK * 2;                // bytes per weight row in the stage
-  static constexpr int B_BYTES = M_PAD * TC_BK * 2;
-  static constexpr int STAGE_BYTES = W_BYTES + B_BYTES;
+  static constexpr int B_BYTES = M_PAD * TC_BK * 2;                    // one activation plane
+  static constexpr int X_PLANES = FP8 ? 1 : 2;                         // f16, or bf16 hi + lo
+  static constexpr int STAGE_BYTES = W_BYTES + X_PLANES * B_BYTES;
   static constexpr int CONV_OFF = STAGES * STAGE_BYTES;                // bf16 tiles made by the converters
   static constexpr int EX_OFF = CONV_OFF + (FP8 ? TC_NCONV * TC_A_BYTES : 0);   // SwiGLU epilogue: gate/up exchange
   static constexpr int EX_ROWS = FP8 ? 16 : 32;                         // rows that pass through it per round
@@ -73,8 +82,8 @@ struct TcSmem {
   static constexpr int TOTAL = BAR_OFF + 256 + 1024;  // barriers + alignment slack
 };
 
-// sixteen e4m3 bytes -> sixteen bf16 (exact: every e4m3 value is a bf16 value)
-__device__ __forceinline__ void e4m3x16_to_bf16(const uint4& in, uint4& lo, uint4& hi) {
+// sixteen e4m3 bytes -> sixteen f16 (exact: every e4m3 value, subnormals included, is an f16 value)
+__device__ __forceinline__ void e4m3x16_to_f16(const uint4& in, uint4& lo, uint4& hi) {
   const uint32_t w[4] = {in.x, in.y, in.z, in.w};
   uint32_t o[8];
 #pragma unroll
@@ -82,12 +91,7 @@ __device__ __forceinline__ void e4m3x16_to_bf16(const uint4& in, uint4& lo, uint
 #pragma unroll
     for (int hsel = 0; hsel < 2; ++hsel) {
       const unsigned short two = (unsigned short)(hsel ? (w[i] >> 16) : (w[i] & 0xffffu));
-      uint32_t h2;
-      asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"(two));
-      const float f0 = __half2float(__ushort_as_half((unsigned short)(h2 & 0xffffu)));
-      const float f1 = __half2float(__ushort_as_half((unsigned short)(h2 >> 16)));
-      __nv_bfloat162 b2 = __floats2bfloat162_rn(f0, f1);
-      o[2 * i + hsel] = *reinterpret_cast<uint32_t*>(&b2);
+      asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(o[2 * i + hsel]) : "h"(two));
     }
   }
   lo = make_uint4(o[0], o[1], o[2], o[3]);
@@ -95,7 +99,7 @@ __device__ __forceinline__ void e4m3x16_to_bf16(const uint4& in, uint4& lo, uint
 }
 
 // Widen NP 16-byte pieces (tid, tid + stride, ...) of an 8 KB e4m3 tile (rows of 64 bytes) into the 128-byte-swizzled
-// bf16 tile the MMA descriptor expects.
+// f16 tile the MMA descriptor expects.
 template <int NP>
 __device__ __forceinline__ void convert_pieces(const uint8_t* src, uint32_t dst, int tid, int stride) {
 #pragma unroll
@@ -103,7 +107,7 @@ __device__ __forceinline__ void convert_pieces(const uint8_t* src, uint32_t dst,
     const int piece = tid + stride * i, r = piece >> 2, c = piece & 3;     // row, 16-byte piece of the row
     const uint4 in = *reinterpret_cast<const uint4*>(src + piece * 16);
     uint4 lo, hi;
-    e4m3x16_to_bf16(in, lo, hi);
+    e4m3x16_to_f16(in, lo, hi);
     const uint32_t row = dst + r * 128;
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + (((2 * c) ^ (r & 7)) << 4)), "r"(lo.x), "r"(lo.y), "r"(lo.z), "r"(lo.w) : "memory");
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + (((2 * c + 1) ^ (r & 7)) << 4)), "r"(hi.x), "r"(hi.y), "r"(hi.z), "r"(hi.w) : "memory");
@@ -143,7 +147,9 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
     for (int c = 0; c < TC_NCONV; ++c) { mbar_init(cfull_bar(c), helpers ? 8 : 4); mbar_init(cempty_bar(c), 1); }
     for (int pr = 0; pr < 2; ++pr) { mbar_init(exw_bar(pr), 2); mbar_init(exr_bar(pr), 2); }
-    *abort_flag = 0;
+    stamp_start(p.stamp);
+    // status[1] is written by the host only (never by a kernel of the chain), so it may be read before the wait
+    *abort_flag = (p.status && *reinterpret_cast<const volatile int*>(p.status + 1) != 0) ? 1 : 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -155,6 +161,7 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
+  const bool poisoned = *abort_flag != 0;   // every role then leaves by its give-up path without issuing anything
   pdl_trigger();
 
   const int total_tiles = p.tile_begin[p.n_mats];
@@ -164,6 +171,7 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
   auto convert_all = [&](int cvt_tid) -> bool {
     int stage = 0, cbuf = 0;
     uint32_t phase = 0, cphase = 0;
+    if (poisoned) return false;
     for (int it = blockIdx.x; it < n_items; it += gridDim.x) {
       const int split = it / total_tiles;
       const int kb0 = split * kbps;
@@ -192,9 +200,15 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
       uint32_t phase = 0;
       uint32_t armed = 0;           // bit s: full[s] armed and not yet known complete
       uint32_t armed_parity = 0;    // bit s: parity of that arming
-      bool ok = true;
+      bool ok = !poisoned;
       bool waited = false;
       int n_pend = 0, pend_stage[TC_STAGES], pend_kb[TC_STAGES];
+      const uint32_t stage_tx = L::W_BYTES + (p.has_lo ? 2 : 1) * L::B_BYTES;
+      auto load_x = [&](int st_, int kb_) {
+        const uint32_t dst = base + st_ * L::STAGE_BYTES + L::W_BYTES;
+        tma_load_2d(dst, &p.tm_x, full_bar(st_), kb_ * TC_BK, 0, pol_x);
+        if (!FP8 && p.has_lo) tma_load_2d(dst + L::B_BYTES, &p.tm_xl, full_bar(st_), kb_ * TC_BK, 0, pol_x);
+      };
       for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
         const int tile = it % total_tiles, split = it / total_tiles;
         int mi = 0, r0 = 0;
@@ -207,7 +221,7 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t a_dst = base + stage * L::STAGE_BYTES;
-          mbar_expect_tx(full_bar(stage), L::STAGE_BYTES);
+          mbar_expect_tx(full_bar(stage), stage_tx);
           armed |= 1u << stage;
           armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
           if (p.mode == TC_MODE_SWIGLU) {
@@ -221,14 +235,14 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
           // The weights do not depend on the predecessor kernel: the first ring of weight loads is issued before waiting
           // for it; the activation tiles of those stages follow once it has completed.
           if (waited) {
-            tma_load_2d(a_dst + L::W_BYTES, &p.tm_x, full_bar(stage), kb * TC_BK, 0, pol_x);
+            load_x(stage, kb);
           } else {
             pend_stage[n_pend] = stage; pend_kb[n_pend] = kb;
             if (++n_pend == TC_STAGES) {
               pdl_wait();
+              stamp_released(p.stamp);
               waited = true;
-              for (int j = 0; j < n_pend; ++j)
-                tma_load_2d(base + pend_stage[j] * L::STAGE_BYTES + L::W_BYTES, &p.tm_x, full_bar(pend_stage[j]), pend_kb[j] * TC_BK, 0, pol_x);
+              for (int j = 0; j < n_pend; ++j) load_x(pend_stage[j], pend_kb[j]);
             }
           }
           if (++stage == TC_STAGES) { stage = 0; phase ^= 1u; }
@@ -236,8 +250,8 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
       }
       if (!waited) {
         pdl_wait();
-        for (int j = 0; j < n_pend; ++j)
-          tma_load_2d(base + pend_stage[j] * L::STAGE_BYTES + L::W_BYTES, &p.tm_x, full_bar(pend_stage[j]), pend_kb[j] * TC_BK, 0, pol_x);
+        stamp_released(p.stamp);
+        for (int j = 0; j < n_pend; ++j) load_x(pend_stage[j], pend_kb[j]);
       }
       if (!ok) {
         atomicCAS(p.status, 0, TC_ERR_PRODUCER);
@@ -253,11 +267,12 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
   } else if (warp == 1) {
     // ------------------------------------------------ MMA issuer --------------------------------------------------
     if (lane == 0) {
-      const uint32_t idesc = umma_idesc_bf16(M_PAD);
+      const uint32_t idesc = FP8 ? umma_idesc_f16(M_PAD) : umma_idesc_bf16(M_PAD);
+      const bool two_planes = !FP8 && p.has_lo;
       int stage = 0, cbuf = 0;
       uint32_t phase = 0, cphase = 0;
       int local = 0;
-      bool ok = true;
+      bool ok = !poisoned;
       for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++local) {
         const int split = it / total_tiles;
         const int acc = local & 1;
@@ -277,6 +292,11 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
 #pragma unroll
           for (int kk = 0; kk < TC_BK / 16; ++kk)
             umma_bf16(d_tmem, adesc + 2u * kk, bdesc + 2u * kk, idesc, (kb > kb0 || kk > 0) ? 1u : 0u);
+          if (two_planes) {     // the same weight tile against the activations' low-order plane
+            const uint64_t ldesc = umma_desc_sw128(a_addr + L::W_BYTES + L::B_BYTES);
+#pragma unroll
+            for (int kk = 0; kk < TC_BK / 16; ++kk) umma_bf16(d_tmem, adesc + 2u * kk, ldesc + 2u * kk, idesc, 1u);
+          }
           umma_commit(empty_bar(stage));
           if (FP8) {
             umma_commit(cempty_bar(cbuf));
@@ -297,7 +317,7 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
     // ------------------------------------------------ epilogue warps ----------------------------------------------
     const int q = warp & 3;  // TMEM lane quarter this warp may read
     int local = 0;
-    bool ok = true;
+    bool ok = !poisoned;
     if (helpers) ok = convert_all(128 + (int)threadIdx.x - 64);
     pdl_wait();   // the epilogue reads the predecessor's row statistics and overwrites buffers it may still be reading
     // folded RMSNorm: lane l keeps the factor of rows l and l + 32; broadcast by shuffle where needed
@@ -365,7 +385,7 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
             const float mine = side ? v[hi] * sc * rs_hi : v[lo] * sc * rs_lo;
             const float g = side ? other : mine, u = side ? mine : other;
             const int row = side ? hi : lo;
-            if (live && row < p.m) p.act[(size_t)row * p.inter + col] = __float2bfloat16_rn(g / (1.f + __expf(-g)) * u);
+            if (live && row < p.m) store_act(p.act, p.act_lo_off, (size_t)row * p.inter + col, g / (1.f + __expf(-g)) * u, p.act_fmt);
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(exr_bar(pr));
@@ -435,6 +455,7 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
+  if (threadIdx.x == 0) stamp_end(p.stamp);
 }
 
 // ================================================================================================
@@ -457,14 +478,17 @@ static EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// 2-D row-major [rows, cols] tensor, box {64 columns, box_rows}, zero OOB fill.  bf16: 128-byte swizzle (rows of the
-// box are 128 bytes); e4m3 bytes: no swizzle (rows of 64 bytes, widened by the converter warps).
-static bool make_tmap(CUtensorMap* tm, const void* ptr, int rows, int cols, int box_rows, bool fp8 = false) {
-  typedef std::tuple<const void*, int, int, int, bool> Key;
+// 2-D row-major [rows, cols] tensor, box {64 columns, box_rows}, zero OOB fill.  16-bit elements (kind 0 = bf16,
+// 2 = f16): 128-byte swizzle (rows of the box are 128 bytes); e4m3 bytes (kind 1): no swizzle (rows of 64 bytes,
+// widened by the converter warps).
+enum { TM_BF16 = 0, TM_E4M3 = 1, TM_F16 = 2 };
+static bool make_tmap(CUtensorMap* tm, const void* ptr, int rows, int cols, int box_rows, int kind = TM_BF16) {
+  typedef std::tuple<const void*, int, int, int, int> Key;
   static std::map<Key, CUtensorMap> cache;
   static std::mutex mu;
   std::lock_guard<std::mutex> lock(mu);
-  Key key(ptr, rows, cols, box_rows, fp8);
+  const bool fp8 = kind == TM_E4M3;
+  Key key(ptr, rows, cols, box_rows, kind);
   auto it = cache.find(key);
   if (it != cache.end()) { *tm = it->second; return true; }
   EncodeTiledFn fn = encode_fn();
@@ -473,7 +497,8 @@ static bool make_tmap(CUtensorMap* tm, const void* ptr, int rows, int cols, int 
   cuuint64_t strides[1] = {(cuuint64_t)cols * (fp8 ? 1 : 2)};
   cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(tm, fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides,
+  const CUtensorMapDataType dt = fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : (kind == TM_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
+  CUresult r = fn(tm, dt, 2, const_cast<void*>(ptr), dims, strides,
                   box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, fp8 ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return false;
@@ -482,15 +507,17 @@ static bool make_tmap(CUtensorMap* tm, const void* ptr, int rows, int cols, int 
   return true;
 }
 
+// SM count of the current device (cached per device: one process may drive several GPUs)
 static int sm_count() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    if (n <= 0) n = 148;
+  static int n[MAX_DEVICES] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return 148;
+  if (!n[dev]) {
+    int v = 0;
+    cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
+    n[dev] = v > 0 ? v : 148;
   }
-  return n;
+  return n[dev];
 }
 
 static int pad_m(int m) { return m <= 16 ? 16 : (m <= 32 ? 32 : (m <= 48 ? 48 : 64)); }
@@ -523,12 +550,9 @@ size_t tc_workspace_bytes(int m, int ld, int tiles, int k) {
 
 template <int M_PAD, bool FP8>
 static cudaError_t tc_launch_t(const TcParams& p, int grid, cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<M_PAD, FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcSmem<M_PAD, FP8>::TOTAL);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static bool attr_set[MAX_DEVICES] = {};
+  cudaError_t e = ensure_dynamic_smem(gemm_tc_kernel<M_PAD, FP8>, TcSmem<M_PAD, FP8>::TOTAL, attr_set);
+  if (e != cudaSuccess) return e;
   return launch_pdl(gemm_tc_kernel<M_PAD, FP8>, dim3(grid), dim3(FP8 ? TC_THREADS_FP8 : TC_THREADS), (size_t)TcSmem<M_PAD, FP8>::TOTAL, st, p);
 }
 
@@ -554,10 +578,13 @@ cudaError_t tc_group_launch(const TcGroup& g, const TcOut& o, cudaStream_t st) {
   memset(&p, 0, sizeof(p));
   const int mode = o.mode;
   const int mp = pad_m(g.m);
-  if (!make_tmap(&p.tm_x, g.x, g.m, g.k, mp)) return cudaErrorInvalidValue;
+  const int xkind = g.fp8 ? TM_F16 : TM_BF16;     // fp8 weights are widened to f16 and meet f16 activations
+  if (!make_tmap(&p.tm_x, g.x, g.m, g.k, mp, xkind)) return cudaErrorInvalidValue;
+  p.has_lo = (!g.fp8 && g.x_lo) ? 1 : 0;
+  if (p.has_lo && !make_tmap(&p.tm_xl, g.x_lo, g.m, g.k, mp, xkind)) return cudaErrorInvalidValue;
   int tiles = 0, col = 0;
   for (int i = 0; i < g.n_mats; ++i) {
-    if (!make_tmap(&p.tm_w[i], g.w[i], g.n[i], g.k, 64, g.fp8 != 0)) return cudaErrorInvalidValue;
+    if (!make_tmap(&p.tm_w[i], g.w[i], g.n[i], g.k, 64, g.fp8 ? TM_E4M3 : TM_BF16)) return cudaErrorInvalidValue;
     p.n_out[i] = g.n[i];
     p.tile_begin[i] = tiles;
     p.out_col[i] = col;
@@ -571,13 +598,14 @@ cudaError_t tc_group_launch(const TcGroup& g, const TcOut& o, cudaStream_t st) {
   p.m = g.m;
   p.mode = mode;
   p.status = o.status;
+  p.stamp = o.stamp;
   p.ssq_in = o.ssq_in; p.nt_in = o.nt_in; p.inv_h = o.hidden > 0 ? 1.f / (float)o.hidden : 0.f; p.eps = o.eps;
   if (mode == TC_MODE_SWIGLU) {
     tiles = ceil_div(g.n[0], 64);      // one combined list of 64-feature tiles (gate + up rows interleaved)
     p.n_mats = 1;
     p.tile_begin[0] = 0; p.tile_begin[1] = tiles;
     p.splits = 1; p.kb_per_split = p.kblocks;
-    p.act = (bf16*)o.act; p.inter = g.n[0];
+    p.act = o.act; p.act_lo_off = o.act_lo_off; p.act_fmt = o.act_fmt; p.inter = g.n[0];
   } else {
     p.tile_begin[g.n_mats] = tiles;
     if (mode == TC_MODE_PARTIAL) tc_plan(tiles, p.kblocks, &p.splits, &p.kb_per_split);

@@ -18,14 +18,20 @@ struct fdvlm {
   int device;
   int dt;          // DT_*
   size_t act_sz;   // bytes per activation / KV element
-  int use_tc;      // bf16 weights: tcgen05 + TMA GEMMs, tensor-core attention, folded norms
-  void* mega;      // persistent forward kernel context (null: kernel-per-operator path)
+  int use_tc;      // bf16 / fp8 weights: tcgen05 + TMA GEMMs, tensor-core attention, folded norms
+  int kv_type;     // tensor-core path: element type of q and the KV cache (KV_BF16 / KV_F16)
+  int xfmt;        // tensor-core path: storage of the GEMM inputs a / ao / act (XF_BF16X2 for bf16 weights, XF_F16 for fp8)
+  int head_fmt;    // storage of the LM head's input (as xfmt, but bf16 planes when the head is a tied bf16 table)
+  size_t a_lo, ao_lo, act_lo;   // XF_BF16X2: element offset of each buffer's low-order plane
   char* slab;      // one allocation behind every device buffer below except the KV cache
   int32_t* dev_len;   // device copy of cache_len, read by the captured forward graphs
   int use_graphs;     // tensor-core path: replay one captured CUDA graph per (rows, mode, logits mode)
-  struct FwdGraph { int n, mode, logits_rows, want_logits, launches; cudaGraphExec_t exec; };
+  struct FwdGraph { int n, mode, logits_rows, want_logits, stamped, launches; cudaGraphExec_t exec; std::vector<int> kinds; };
   std::vector<FwdGraph> graphs;
-  char* mega_slab; // the persistent kernel's share of the slab (counters, tensor maps, partial sums)
+  // on-device decode loop (fdvlm_decode_block): a graph whose conditional WHILE node repeats the denoise step
+  cudaGraphExec_t loop_exec;
+  int loop_n, loop_rule, loop_k, loop_shift, loop_body_launches;
+  float loop_threshold;
   // device buffers (R = max_block rows)
   char* kv;        // [n_layers][2][Hkv][max_seq][d]
   float* h;        // [R, H] residual stream, fp32
@@ -43,7 +49,8 @@ struct fdvlm {
   uint8_t* unmask; // [R]
   int32_t* blk_tokens;
   uint8_t* blk_masked;
-  int32_t* info;   // {n_unmasked, n_remaining, step_index, device status}
+  int32_t* info;   // {n_unmasked, n_remaining, step_index, device status, poison (host-set test hook),
+                   //  iterations of the on-device decode loop, 2 spare}
   int32_t* init_stage;  // [64] device staging of host-given block tokens
   void* ws;        // GEMM split-K / attention split-KV workspace
   size_t ws_bytes;
@@ -53,8 +60,12 @@ struct fdvlm {
   // state
   int cache_len, block_size, n_remaining, step_index, block_open;
   int launches;
-  // optional per-kernel-family timing (events around each launch group), see fdvlm_profile_*
+  // optional timing, see fdvlm_profile_*: prof_on = 1: events around each launch group (kernels launched one by one);
+  // prof_on = 2: every kernel of the replayed forward stamps the GPU's global timer into `stamps` (in-chain timing)
   int prof_on;
+  fdk::KStamp* stamps;                     // device, FDVLM_MAX_STAMPS records
+  std::vector<int> stamp_kind;        // kind of each record used by the last stamped forward (fdvlm_kernel_kind)
+  int stamp_used;
   std::vector<cudaEvent_t> prof_ev;   // pairs (start, stop)
   std::vector<int> prof_kind;         // per pair: 0 = projection GEMM, 1 = attention
   size_t prof_used;
@@ -109,14 +120,16 @@ int stage_rows(fdvlm_t* h, int row0, int n, const int32_t* tokens, const void* e
 // logits_rows: 0 none; n = all rows (logits into h->logits when want_logits, and conf / pred always);
 // 1 = last row only, raw logits into h->logits[0 .. V).
 int forward_rows(fdvlm_t* h, int n, int mode, int logits_rows, int want_logits);
+int forward_rows_enqueue(fdvlm_t* h, int n, int mode, int logits_rows, int want_logits);
 
 size_t linear_workspace_bytes(int m, int n, int k, int dtype);
 size_t attention_workspace_bytes(int n, int hq, int hkv, int d);
 
-// mega.cu: the persistent whole-forward kernel of the bf16 path
-size_t mega_slab_bytes(const fdvlm_t* h);   // device bytes mega_create will carve out of h->mega_slab
-bool mega_create(fdvlm_t* h);
-void mega_destroy(fdvlm_t* h);
-int mega_forward(fdvlm_t* h, int n, int mode, int logits_rows, int want_logits);
+constexpr int FDVLM_MAX_STAMPS = 1024;
+// Bytes at the start of an operator-level workspace that hold the kernels' two status words.
+constexpr size_t OP_HEAD = 256;
+// Stand-alone projection on `st` (workspace laid out as fdvlm_op_linear documents).  Returns launches or -1.
+int launch_linear(const LinearArgs& a, cudaStream_t st, cudaError_t* err);
+int launch_attention(const AttnArgs& a, cudaStream_t st, cudaError_t* err);
 
 }  // namespace fdk

@@ -186,19 +186,27 @@ int launch_linear_simt(const LinearArgs& a, cudaStream_t st, cudaError_t* err) {
 // ================================================================================================
 // embedding gather / row conversion
 // ================================================================================================
+// A token id outside [0, vocab) is not dereferenced: row 0 is read instead and ST_BAD_TOKEN is left in the status word.
+__device__ __forceinline__ int checked_token(const int32_t* tokens, int r, int vocab, int* status) {
+  const int t = tokens[r];
+  if (t >= 0 && t < vocab) return t;
+  if (threadIdx.x == 0 && status) atomicCAS(status, 0, ST_BAD_TOKEN);
+  return 0;
+}
 template <typename ET>
 __global__ void embed_kernel(const ET* __restrict__ table, const int32_t* __restrict__ tokens,
-                             float* __restrict__ h, int hidden) {
+                             float* __restrict__ h, int hidden, int vocab, int* status) {
   int r = blockIdx.x;
-  const ET* src = table + (size_t)(tokens ? tokens[r] : r) * hidden;
+  const ET* src = table + (size_t)(tokens ? checked_token(tokens, r, vocab, status) : r) * hidden;
   for (int c = threadIdx.x; c < hidden; c += blockDim.x) h[(size_t)r * hidden + c] = to_f32(src[c]);
 }
-void launch_embed(const void* table, const int32_t* tokens, float* h, int n, int hidden, int dtype, cudaStream_t st) {
-  if (dtype == DT_F32) embed_kernel<float><<<n, 256, 0, st>>>((const float*)table, tokens, h, hidden);
-  else embed_kernel<bf16><<<n, 256, 0, st>>>((const bf16*)table, tokens, h, hidden);
+void launch_embed(const void* table, const int32_t* tokens, float* h, int n, int hidden, int dtype, int vocab, int* status,
+                  cudaStream_t st) {
+  if (dtype == DT_F32) embed_kernel<float><<<n, 256, 0, st>>>((const float*)table, tokens, h, hidden, vocab, status);
+  else embed_kernel<bf16><<<n, 256, 0, st>>>((const bf16*)table, tokens, h, hidden, vocab, status);
 }
 void launch_rows_to_f32(const void* rows, float* h, int n, int hidden, int dtype, cudaStream_t st) {
-  launch_embed(rows, nullptr, h, n, hidden, dtype, st);
+  launch_embed(rows, nullptr, h, n, hidden, dtype, 0, nullptr, st);
 }
 
 // ================================================================================================
@@ -231,9 +239,12 @@ __global__ void set_len_kernel(int* len_ptr, int value) {
 }
 void launch_set_len(int* len_ptr, int value, cudaStream_t st) { set_len_kernel<<<1, 1, 0, st>>>(len_ptr, value); }
 
-__global__ void rope_table_kernel(float2* __restrict__ cs, int n, int pos0, int half, double theta, const int* __restrict__ len_ptr) {
+__global__ void rope_table_kernel(float2* __restrict__ cs, int n, int pos0, int half, double theta, const int* __restrict__ len_ptr,
+                                  KStamp* stamp) {
+  if (threadIdx.x == 0) stamp_start(stamp);
   pdl_trigger();
   pdl_wait();
+  if (threadIdx.x == 0) { stamp_released(stamp); stamp_end(stamp); }
   if (len_ptr) pos0 = *len_ptr;
   int idx = blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= n * half) return;
@@ -243,9 +254,9 @@ __global__ void rope_table_kernel(float2* __restrict__ cs, int n, int pos0, int 
   sincos(ang, &s, &c);
   cs[idx] = make_float2((float)c, (float)s);
 }
-void launch_rope_table(float* cs, int n, int pos0, int head_dim, float theta, cudaStream_t st, const int* len_ptr) {
+void launch_rope_table(float* cs, int n, int pos0, int head_dim, float theta, cudaStream_t st, const int* len_ptr, KStamp* stamp) {
   int half = head_dim / 2, total = n * half;
-  launch_pdl(rope_table_kernel, dim3((total + 127) / 128), dim3(128), 0, st, (float2*)cs, n, pos0, half, (double)theta, len_ptr);
+  launch_pdl(rope_table_kernel, dim3((total + 127) / 128), dim3(128), 0, st, (float2*)cs, n, pos0, half, (double)theta, len_ptr, stamp);
 }
 
 // rotate-half pairing (j, j + d/2); q -> q buffer, k -> cache K plane, v -> cache V plane
@@ -284,56 +295,46 @@ void launch_qkv_post(const float* qkv, const float* cs, void* q, void* kc, void*
 }
 
 // ================================================================================================
-// Glue of the tensor-core path (bf16).  RMSNorm is folded into its consumer GEMM: producers leave
-// xg = bf16(h * gain) and per-128-column partial sums of h^2 (ssq[row][nt]); the consumer's epilogue
-// multiplies by rsqrt(sum(ssq) / hidden + eps).  All sums run in a fixed order => deterministic.
+// Glue of the tensor-core path.  RMSNorm is folded into its consumer GEMM: producers leave xg = h * gain as a GEMM
+// input (XF_* storage: bf16 hi + lo planes, or f16) and per-128-column partial sums of h^2 (ssq[row][nt]); the
+// consumer's epilogue multiplies by rsqrt(sum(ssq) / hidden + eps).  All sums run in a fixed order => deterministic.
 // ================================================================================================
 __global__ void embed_prep_kernel(const bf16* __restrict__ table, const int32_t* __restrict__ tokens,
-                                  const bf16* __restrict__ rows, float* __restrict__ h, bf16* __restrict__ xg,
-                                  const float* __restrict__ g, float* __restrict__ ssq, int nt, int hidden) {
+                                  const bf16* __restrict__ rows, float* __restrict__ h, void* __restrict__ xg,
+                                  size_t lo_off, int fmt, const float* __restrict__ g, float* __restrict__ ssq, int nt,
+                                  int hidden, int vocab, int* status, KStamp* stamp) {
+  if (threadIdx.x == 0) stamp_start(stamp);
   pdl_trigger();
   pdl_wait();
+  if (threadIdx.x == 0) stamp_released(stamp);
   __shared__ float red[32];
   const int r = blockIdx.x;
-  const bf16* src = tokens ? table + (size_t)tokens[r] * hidden : rows + (size_t)r * hidden;
+  const bf16* src = tokens ? table + (size_t)checked_token(tokens, r, vocab, status) * hidden : rows + (size_t)r * hidden;
   float ss = 0.f;
-  if ((hidden & 7) == 0) {
-    // eight values per thread and pass: one 16-byte load of the row and two of the gain, all issued before use
-    for (int c8 = threadIdx.x; c8 < hidden / 8; c8 += blockDim.x) {
-      const uint4 raw = *reinterpret_cast<const uint4*>(src + 8 * c8);
-      const float4 g0 = *reinterpret_cast<const float4*>(g + 8 * c8), g1 = *reinterpret_cast<const float4*>(g + 8 * c8 + 4);
-      const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-      const float gg[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
-      float v[8];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) { v[2 * i] = __uint_as_float(w[i] << 16); v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u); }
-      float* hd = h + (size_t)r * hidden + 8 * c8;
-      *reinterpret_cast<float4*>(hd) = make_float4(v[0], v[1], v[2], v[3]);
-      *reinterpret_cast<float4*>(hd + 4) = make_float4(v[4], v[5], v[6], v[7]);
-      uint32_t o[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        __nv_bfloat162 b2 = __floats2bfloat162_rn(v[2 * i] * gg[2 * i], v[2 * i + 1] * gg[2 * i + 1]);
-        o[i] = *reinterpret_cast<uint32_t*>(&b2);
-        ss = fmaf(v[2 * i], v[2 * i], ss);
-        ss = fmaf(v[2 * i + 1], v[2 * i + 1], ss);
-      }
-      *reinterpret_cast<uint4*>(xg + (size_t)r * hidden + 8 * c8) = make_uint4(o[0], o[1], o[2], o[3]);
-    }
-  } else {
-    for (int c = threadIdx.x; c < hidden; c += blockDim.x) {
-      const float v = __bfloat162float(src[c]);
-      h[(size_t)r * hidden + c] = v;
-      xg[(size_t)r * hidden + c] = __float2bfloat16_rn(v * g[c]);
-      ss = fmaf(v, v, ss);
-    }
+  for (int c = threadIdx.x; c < hidden; c += blockDim.x) {
+    const float v = __bfloat162float(src[c]);
+    h[(size_t)r * hidden + c] = v;
+    store_act(xg, lo_off, (size_t)r * hidden + c, v * g[c], fmt);
+    ss = fmaf(v, v, ss);
   }
   ss = block_sum(ss, red);
   for (int t = threadIdx.x; t < nt; t += blockDim.x) ssq[(size_t)r * nt + t] = (t == 0) ? ss : 0.f;
+  if (threadIdx.x == 0) stamp_end(stamp);
 }
-void launch_embed_prep(const void* table, const int32_t* tokens, const void* rows, float* h, void* xg, const float* g,
-                       float* ssq, int nt, int n, int hidden, cudaStream_t st) {
-  embed_prep_kernel<<<n, 256, 0, st>>>((const bf16*)table, tokens, (const bf16*)rows, h, (bf16*)xg, g, ssq, nt, hidden);
+void launch_embed_prep(const void* table, const int32_t* tokens, const void* rows, float* h, void* xg, size_t lo_off, int fmt,
+                       const float* g, float* ssq, int nt, int n, int hidden, int vocab, int* status, cudaStream_t st, KStamp* stamp) {
+  embed_prep_kernel<<<n, 256, 0, st>>>((const bf16*)table, tokens, (const bf16*)rows, h, xg, lo_off, fmt, g, ssq, nt, hidden, vocab,
+                                       status, stamp);
+}
+
+// bf16 rows -> f16 rows (saturating), for the operator-level entry points whose callers hand bf16 activations to an
+// fp8-weight projection
+__global__ void bf16_to_f16_kernel(const bf16* __restrict__ in, unsigned short* __restrict__ out, size_t n) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) out[i] = f16_bits_sat(__bfloat162float(in[i]));
+}
+void launch_bf16_to_f16(const void* in, void* out, size_t n, cudaStream_t st) {
+  bf16_to_f16_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>((const bf16*)in, (unsigned short*)out, n);
 }
 
 // Sum of S split-K partials p[i * stride].  These kernels are a handful of dependent L2 round trips long, so every
@@ -363,12 +364,14 @@ __device__ __forceinline__ float sum_partials_from(const float* __restrict__ p, 
 // QKV finalisation: sum the split-K partials, apply the folded norm factor and the bias, rotate q and k
 // (rotate-half pairs j, j + d/2), write q to its buffer and k, v into the layer's cache planes.
 // grid (hq + 2 hkv heads, m rows), d/2 threads: thread j owns the pair (j, j + d/2) of one head.
+template <typename T>
 __global__ void fin_qkv_kernel(const float* __restrict__ part, int S, int m, const float2* __restrict__ cs,
                                const float* __restrict__ ssq, int nt, float inv_h, float eps,
                                const float* __restrict__ bq, const float* __restrict__ bk, const float* __restrict__ bv,
                                const float* __restrict__ sq, const float* __restrict__ sk, const float* __restrict__ sv,
-                               bf16* __restrict__ q, bf16* __restrict__ kc, bf16* __restrict__ vc, int pos0, int hq, int hkv,
-                               int d, int max_seq, const int* __restrict__ len_ptr) {
+                               T* __restrict__ q, T* __restrict__ kc, T* __restrict__ vc, int pos0, int hq, int hkv,
+                               int d, int max_seq, const int* __restrict__ len_ptr, KStamp* stamp) {
+  if (threadIdx.x == 0) stamp_start(stamp);
   pdl_trigger();
   const int head = blockIdx.x, r = blockIdx.y, j = threadIdx.x, half = d >> 1;
   // not written by any kernel of this forward: the cache length word, the scales and the biases
@@ -382,6 +385,7 @@ __global__ void fin_qkv_kernel(const float* __restrict__ part, int S, int m, con
     if (bi) { bi_a = bi[hl * d + j]; bi_b = bi[hl * d + j + half]; }
   }
   pdl_wait();
+  if (threadIdx.x == 0) stamp_released(stamp);
   __shared__ float s_rstd;
   // every load of this kernel is issued before the first result is needed
   const int width = (hq + 2 * hkv) * d;
@@ -407,34 +411,40 @@ __global__ void fin_qkv_kernel(const float* __restrict__ part, int S, int m, con
   a = a * rstd * sc_a + bi_a;
   b = b * rstd * sc_b + bi_b;
   if (head < hq) {
-    bf16* o = q + ((size_t)r * hq + head) * d;
-    o[j] = __float2bfloat16_rn(a * c.x - b * c.y);
-    o[j + half] = __float2bfloat16_rn(b * c.x + a * c.y);
+    T* o = q + ((size_t)r * hq + head) * d;
+    o[j] = from_f32<T>(a * c.x - b * c.y);
+    o[j + half] = from_f32<T>(b * c.x + a * c.y);
   } else if (head < hq + hkv) {
     const int hk = head - hq;
-    bf16* o = kc + ((size_t)hk * max_seq + pos0 + r) * d;
-    o[j] = __float2bfloat16_rn(a * c.x - b * c.y);
-    o[j + half] = __float2bfloat16_rn(b * c.x + a * c.y);
+    T* o = kc + ((size_t)hk * max_seq + pos0 + r) * d;
+    o[j] = from_f32<T>(a * c.x - b * c.y);
+    o[j + half] = from_f32<T>(b * c.x + a * c.y);
   } else {
     const int hk = head - hq - hkv;
-    bf16* o = vc + ((size_t)hk * max_seq + pos0 + r) * d;
-    o[j] = __float2bfloat16_rn(a);
-    o[j + half] = __float2bfloat16_rn(b);
+    T* o = vc + ((size_t)hk * max_seq + pos0 + r) * d;
+    o[j] = from_f32<T>(a);
+    o[j + half] = from_f32<T>(b);
   }
+  if (threadIdx.x == 0) stamp_end(stamp);
 }
 void launch_fin_qkv(const float* part, int S, int m, const float* cs, const float* ssq, int nt, int hidden, float eps,
                     const float* bq, const float* bk, const float* bv, const float* sq, const float* sk, const float* sv, void* q, void* kc, void* vc, int pos0, int hq,
-                    int hkv, int d, int max_seq, cudaStream_t st, const int* len_ptr) {
-  launch_pdl(fin_qkv_kernel, dim3(hq + 2 * hkv, m), dim3(d / 2), 0, st, part, S, m, (const float2*)cs, ssq, nt, 1.f / (float)hidden, eps, bq, bk,
-                                                          bv, sq, sk, sv, (bf16*)q, (bf16*)kc, (bf16*)vc, pos0, hq, hkv, d, max_seq, len_ptr);
+                    int hkv, int d, int max_seq, int kv_type, cudaStream_t st, const int* len_ptr, KStamp* stamp) {
+  if (kv_type == KV_F16)
+    launch_pdl(fin_qkv_kernel<__half>, dim3(hq + 2 * hkv, m), dim3(d / 2), 0, st, part, S, m, (const float2*)cs, ssq, nt, 1.f / (float)hidden,
+               eps, bq, bk, bv, sq, sk, sv, (__half*)q, (__half*)kc, (__half*)vc, pos0, hq, hkv, d, max_seq, len_ptr, stamp);
+  else
+    launch_pdl(fin_qkv_kernel<bf16>, dim3(hq + 2 * hkv, m), dim3(d / 2), 0, st, part, S, m, (const float2*)cs, ssq, nt, 1.f / (float)hidden,
+               eps, bq, bk, bv, sq, sk, sv, (bf16*)q, (bf16*)kc, (bf16*)vc, pos0, hq, hkv, d, max_seq, len_ptr, stamp);
 }
 
-// Residual finalisation: h += sum of split-K partials; xg = bf16(h * gain of the next norm); ssq[row][tile] =
-// sum of h^2 over the tile's 128 columns.  grid (nt tiles, m rows), 128 threads.
+// Residual finalisation: h += sum of split-K partials; xg = h * gain of the next norm (stored as `fmt`);
+// ssq[row][tile] = sum of h^2 over the tile's 128 columns.  grid (nt tiles, m rows), 128 threads.
 __global__ void __launch_bounds__(128) fin_resid_kernel(const float* __restrict__ part, int S, int m, int hidden,
                                                         float* __restrict__ h, const float* __restrict__ g,
-                                                        bf16* __restrict__ xg, float* __restrict__ ssq, int nt,
-                                                        const float* __restrict__ scale) {
+                                                        void* __restrict__ xg, size_t lo_off, int fmt, float* __restrict__ ssq, int nt,
+                                                        const float* __restrict__ scale, KStamp* stamp) {
+  if (threadIdx.x == 0) stamp_start(stamp);
   pdl_trigger();
   __shared__ float red[32];
   const int t = blockIdx.x, r = blockIdx.y, c = t * 128 + threadIdx.x;
@@ -442,6 +452,7 @@ __global__ void __launch_bounds__(128) fin_resid_kernel(const float* __restrict_
   const float gc = (c < hidden) ? g[c] : 0.f;
   const float sc = (c < hidden && scale) ? scale[c] : 1.f;
   pdl_wait();
+  if (threadIdx.x == 0) stamp_released(stamp);
   float v = 0.f;
   if (c < hidden) {
     const size_t idx = (size_t)r * hidden + c, sstride = (size_t)m * hidden;
@@ -450,22 +461,24 @@ __global__ void __launch_bounds__(128) fin_resid_kernel(const float* __restrict_
     const float hv = __ldcg(h + idx);
     v = hv + sum_partials_from(part + idx, sstride, 32, S, add_partials(pv, 0.f)) * sc;
     h[idx] = v;
-    xg[idx] = __float2bfloat16_rn(v * gc);
+    store_act(xg, lo_off, idx, v * gc, fmt);
   }
   const float ss = block_sum(v * v, red);
-  if (threadIdx.x == 0) ssq[(size_t)r * nt + t] = ss;
+  if (threadIdx.x == 0) { ssq[(size_t)r * nt + t] = ss; stamp_end(stamp); }
 }
-void launch_fin_resid(const float* part, int S, int m, int hidden, float* h, const float* g, void* xg, float* ssq, int nt,
-                      const float* scale, cudaStream_t st) {
-  launch_pdl(fin_resid_kernel, dim3(nt, m), dim3(128), 0, st, part, S, m, hidden, h, g, (bf16*)xg, ssq, nt, scale);
+void launch_fin_resid(const float* part, int S, int m, int hidden, float* h, const float* g, void* xg, size_t lo_off, int fmt,
+                      float* ssq, int nt, const float* scale, cudaStream_t st, KStamp* stamp) {
+  launch_pdl(fin_resid_kernel, dim3(nt, m), dim3(128), 0, st, part, S, m, hidden, h, g, xg, lo_off, fmt, ssq, nt, scale, stamp);
 }
 
 // Merge the per-warp softmax statistics of the LM-head epilogue into confidence and prediction per row.
 // stats[e * m + row] = (max, sum exp(l - max), argmax id) for e in [0, n_part).  grid m rows, 256 threads.
 __global__ void __launch_bounds__(512) stats_merge_kernel(const float4* __restrict__ stats, int n_part, int m,
-                                                          float* __restrict__ conf, int32_t* __restrict__ pred) {
+                                                          float* __restrict__ conf, int32_t* __restrict__ pred, KStamp* stamp) {
+  if (threadIdx.x == 0) stamp_start(stamp);
   pdl_trigger();
   pdl_wait();
+  if (threadIdx.x == 0) stamp_released(stamp);
   __shared__ float sm_m[16], sm_s[16];
   __shared__ int sm_i[16];
   const int r = blockIdx.x;
@@ -504,10 +517,11 @@ __global__ void __launch_bounds__(512) stats_merge_kernel(const float4* __restri
     for (int k = 1; k < (int)(blockDim.x >> 5); ++k) merge(sm_m[k], sm_s[k], sm_i[k]);
     conf[r] = 1.f / s;
     pred[r] = ix;
+    stamp_end(stamp);
   }
 }
-void launch_stats_merge(const void* stats, int n_part, int m, float* conf, int32_t* pred, cudaStream_t st) {
-  launch_pdl(stats_merge_kernel, dim3(m), dim3(512), 0, st, (const float4*)stats, n_part, m, conf, pred);
+void launch_stats_merge(const void* stats, int n_part, int m, float* conf, int32_t* pred, cudaStream_t st, KStamp* stamp) {
+  launch_pdl(stats_merge_kernel, dim3(m), dim3(512), 0, st, (const float4*)stats, n_part, m, conf, pred, stamp);
 }
 
 // ================================================================================================
@@ -583,7 +597,7 @@ void launch_row_stats(const float* logits, int n, int vocab, int mask_id, float*
 __global__ void select_kernel(const float* __restrict__ conf, const int32_t* __restrict__ pred,
                               int32_t* __restrict__ tokens, uint8_t* __restrict__ masked,
                               uint8_t* __restrict__ unmask, int32_t* __restrict__ info, int n, int rule,
-                              float threshold, int k, int shift) {
+                              float threshold, int k, int shift, cudaGraphConditionalHandle cond, int loop) {
   pdl_trigger();
   pdl_wait();
   __shared__ float c[64];
@@ -616,11 +630,22 @@ __global__ void select_kernel(const float* __restrict__ conf, const int32_t* __r
     unmask[i] = (uint8_t)sel;
     if (sel) { tokens[i] = pred[i - shift]; masked[i] = 0; }
   }
-  if (i == 0) { info[0] = n_sel; info[1] = n_masked - n_sel + stuck; info[2] = info[2] + 1; }
+  if (i == 0) {
+    const int left = n_masked - n_sel + stuck;
+    info[0] = n_sel; info[1] = left; info[2] = info[2] + 1;
+    if (loop) {
+      // body of the on-device decode loop: run another denoise step while masked positions are left.  Every step
+      // reveals at least one position, so the loop ends after at most n steps; the explicit count is a second bound.
+      const int it = info[5] + 1;
+      info[5] = it;
+      cudaGraphSetConditional(cond, (left > 0 && n_sel > 0 && it < n) ? 1u : 0u);
+    }
+  }
 }
 void launch_select(const float* conf, const int32_t* pred, int32_t* tokens, uint8_t* masked, uint8_t* unmask,
-                   int32_t* info, int n, int rule, float threshold, int k, cudaStream_t st, int shift) {
-  select_kernel<<<1, 64, 0, st>>>(conf, pred, tokens, masked, unmask, info, n, rule, threshold, k, shift);
+                   int32_t* info, int n, int rule, float threshold, int k, cudaStream_t st, int shift,
+                   cudaGraphConditionalHandle cond, int loop) {
+  select_kernel<<<1, 64, 0, st>>>(conf, pred, tokens, masked, unmask, info, n, rule, threshold, k, shift, cond, loop);
 }
 
 // Longest accepted prefix of a drafted block d against the causal predictions a (a[j] predicts the token after d[j]):

@@ -4,6 +4,8 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include "common.cuh"
+
 namespace fdk {
 
 // ---- small-M linear: y[m,n] = sum_k x[m,k] w[n,k] (* scale[n]) (+ bias[n]) ---------------------
@@ -20,14 +22,16 @@ struct LinearArgs {
   size_t workspace_bytes;
 };
 size_t linear_workspace_bytes(int m, int n, int k, int dtype);
-// Returns the number of kernels launched, or -1 with *err set.
-int launch_linear(const LinearArgs& a, cudaStream_t st, cudaError_t* err);
 
 // ---- elementwise / reduction kernels -----------------------------------------------------------
-void launch_embed(const void* table, const int32_t* tokens, float* h, int n, int hidden, int dtype, cudaStream_t st);
+// tokens outside [0, vocab) read row 0 and leave ST_BAD_TOKEN in *status
+void launch_embed(const void* table, const int32_t* tokens, float* h, int n, int hidden, int dtype, int vocab, int* status,
+                  cudaStream_t st);
+void launch_bf16_to_f16(const void* in, void* out, size_t n, cudaStream_t st);
 void launch_rows_to_f32(const void* rows, float* h, int n, int hidden, int dtype, cudaStream_t st);
 void launch_rmsnorm(const float* h, const float* g, void* out, int n, int hidden, float eps, int dtype, cudaStream_t st);
-void launch_rope_table(float* cs, int n, int pos0, int head_dim, float theta, cudaStream_t st, const int* len_ptr = nullptr);
+void launch_rope_table(float* cs, int n, int pos0, int head_dim, float theta, cudaStream_t st, const int* len_ptr = nullptr,
+                       KStamp* stamp = nullptr);
 void launch_set_len(int* len_ptr, int value, cudaStream_t st);
 // qkv fp32 [n, (Hq + 2 Hkv) d] -> q (act type) [n, Hq, d] rotated; K (rotated) and V written into the
 // layer's cache planes [Hkv, max_seq, d] at positions pos0 .. pos0 + n - 1.
@@ -36,8 +40,11 @@ void launch_qkv_post(const float* qkv, const float* cs, void* q, void* kc, void*
 void launch_swiglu(const float* gu, void* act, int n, int inter, int dtype, cudaStream_t st);
 void launch_row_stats(const float* logits, int n, int vocab, int mask_id, float* conf, int32_t* pred, cudaStream_t st);
 // Unmask selection + block-state update.  info = {n_unmasked, n_remaining, step_index}.
+// loop = 1: the launch is the last node of a conditional WHILE body; it counts the iteration in info[5] and sets `cond`
+// to "masked positions remain".
 void launch_select(const float* conf, const int32_t* pred, int32_t* tokens, uint8_t* masked, uint8_t* unmask,
-                   int32_t* info, int n, int rule, float threshold, int k, cudaStream_t st, int shift = 0);
+                   int32_t* info, int n, int rule, float threshold, int k, cudaStream_t st, int shift = 0,
+                   cudaGraphConditionalHandle cond = 0, int loop = 0);
 // out[0] = accepted length k, out[1] = a[k - 1] (Alg. 1 "Accept: left-to-right comparison")
 void launch_accept(const int32_t* a, const int32_t* d, int n, int32_t* out, cudaStream_t st);
 void launch_init_block(int32_t* tokens, uint8_t* masked, int32_t* info, const int32_t* init, int n, int mask_id,
@@ -47,7 +54,8 @@ void launch_init_block(int32_t* tokens, uint8_t* masked, int32_t* info, const in
 enum { TC_MODE_PARTIAL = 0, TC_MODE_DIRECT = 1, TC_MODE_SWIGLU = 2, TC_MODE_LOGITS = 3 };
 // Up to three bf16 matrices that share x and K; their outputs sit side by side in one row of width ld.
 struct TcGroup {
-  const void* x; int m, k;
+  const void* x; int m, k;   // bf16 weights: bf16 rows (hi plane); fp8 weights: f16 rows
+  const void* x_lo;          // bf16 weights only, nullable: the rows' low-order bf16 plane (x = hi + lo)
   const void* w[3]; int n[3]; int n_mats;
   const float* scale[3]; const float* bias[3];
   int fp8;   // weights are e4m3 bytes (scale[] holds the per-output-channel factors)
@@ -63,26 +71,30 @@ struct TcOut {
   int mode;
   float* part; size_t part_bytes; int* splits_out;
   float* y; int ld; int accumulate;
-  void* act;
+  void* act; size_t act_lo_off; int act_fmt;   // SWIGLU output, stored as XF_* (lo plane act_lo_off elements on)
   const float* ssq_in; int nt_in; int hidden; float eps;
   void* stats; int mask_id; int write_logits;
-  int* status;   // device word set non-zero if a bounded wait inside the kernel gave up
+  int* status;   // two device words: [0] set non-zero if a bounded wait inside the kernel gave up; [1] read at kernel
+                 // start, non-zero sends every role down its give-up path at once
+  KStamp* stamp; // in-chain timing of the launch, nullable
 };
 bool tc_linear_supported(int m, int n, int k, int dtype);
 // Split-K workspace of a group with m rows, output width ld, `tiles` 128-row weight tiles and depth k.
 size_t tc_workspace_bytes(int m, int ld, int tiles, int k);
 cudaError_t tc_group_launch(const TcGroup& g, const TcOut& o, cudaStream_t st);
 
-// Tensor-core path glue (bf16).  ssq[row][nt] holds per-128-column partial sums of h^2.
-void launch_embed_prep(const void* table, const int32_t* tokens, const void* rows, float* h, void* xg, const float* g,
-                       float* ssq, int nt, int n, int hidden, cudaStream_t st);
+// Tensor-core path glue.  ssq[row][nt] holds per-128-column partial sums of h^2; xg / lo_off / fmt: a GEMM input
+// stored as XF_* (common.cuh).  q, kc, vc of fin_qkv are KV_BF16 or KV_F16 elements (kv_type).
+void launch_embed_prep(const void* table, const int32_t* tokens, const void* rows, float* h, void* xg, size_t lo_off, int fmt,
+                       const float* g, float* ssq, int nt, int n, int hidden, int vocab, int* status, cudaStream_t st,
+                       KStamp* stamp = nullptr);
 void launch_fin_qkv(const float* part, int S, int m, const float* cs, const float* ssq, int nt, int hidden, float eps,
                     const float* bq, const float* bk, const float* bv, const float* sq, const float* sk, const float* sv, void* q,
                     void* kc, void* vc, int pos0, int hq,
-                    int hkv, int d, int max_seq, cudaStream_t st, const int* len_ptr = nullptr);
-void launch_fin_resid(const float* part, int S, int m, int hidden, float* h, const float* g, void* xg, float* ssq, int nt,
-                      const float* scale, cudaStream_t st);
-void launch_stats_merge(const void* stats, int n_part, int m, float* conf, int32_t* pred, cudaStream_t st);
+                    int hkv, int d, int max_seq, int kv_type, cudaStream_t st, const int* len_ptr = nullptr, KStamp* stamp = nullptr);
+void launch_fin_resid(const float* part, int S, int m, int hidden, float* h, const float* g, void* xg, size_t lo_off, int fmt,
+                      float* ssq, int nt, const float* scale, cudaStream_t st, KStamp* stamp = nullptr);
+void launch_stats_merge(const void* stats, int n_part, int m, float* conf, int32_t* pred, cudaStream_t st, KStamp* stamp = nullptr);
 
 // ---- attention -----------------------------------------------------------------------------------
 struct AttnArgs {
@@ -91,10 +103,14 @@ struct AttnArgs {
   const void* vc;
   void* out;       // [n, Hq*d]
   int n, cache_len, max_seq, hq, hkv, d, causal, dtype;
+  int kv_type;          // tensor-core kernel: element type of q, kc, vc (KV_BF16 / KV_F16)
+  int out_fmt;          // tensor-core kernel: storage of `out` (XF_*), lo plane out_lo_off elements on
+  size_t out_lo_off;
   void* workspace;
-  const int* len_ptr;   // nullable: device word holding the cache length (overrides cache_len; bf16 kernel only)
+  const int* len_ptr;   // nullable: device word holding the cache length (overrides cache_len; tensor-core kernel only)
+  int* status;          // nullable: device status words (see TcOut::status)
+  KStamp* stamp;        // nullable: two consecutive entries (attention, chunk merge)
 };
 size_t attention_workspace_bytes(int n, int hq, int hkv, int d);
-int launch_attention(const AttnArgs& a, cudaStream_t st, cudaError_t* err);
 
 }  // namespace fdk

@@ -11,25 +11,14 @@ TOL = {I.F32: dict(logits=1e-4, conf=1e-4), I.BF16: dict(logits=3e-2, conf=5e-3)
 MARGIN = 1e-3
 
 
-def depth_tolerance(shape, logit_std):
-    """Logit tolerance of a deep bf16-activation model.  The CUDA path rounds about eight tensors per layer to bf16
-    (GEMM inputs, q / k / v and the KV cache, attention probabilities and output, the MLP activation), each a relative
-    error of at most 2^-9; on random-init N(0, 0.02) models every layer's increment dominates the residual it is added
-    to, so the errors add in quadrature without damping: sigma = logit_std * 2^-9 * sqrt(8 * layers).  The bound is
-    5 sigma (the maximum is taken over ~150k logits), never below the stated tolerance of the dtype."""
-    sigma = float(logit_std) * 2.0 ** -9 * np.sqrt(8.0 * shape.n_layers)
-    tol = dict(TOL[shape.dtype])
-    tol["logits"] = max(tol["logits"], 5.0 * sigma)
-    return tol
-
-
-def make_pair(shape, seed, max_seq, max_block=64, stream=None, **wkw):
+def make_pair(shape, seed, max_seq, max_block=64, stream=None, kv_dtype=None, **wkw):
     """`stream`: a torch.cuda.Stream for the handle (the library then replays captured CUDA graphs; on the default
-    stream it launches kernel by kernel)."""
+    stream it launches kernel by kernel).  `kv_dtype`: binding.KV_F16 (default) or binding.KV_BF16."""
     from paper_2604_06832_b200 import binding as B
     w = I.make_weights(shape, seed, **wkw)
     oracle = orc.Oracle(shape, I.weights_to_numpy(w))
-    handle = B.Handle(shape, B.weights_to_device(w), max_seq=max_seq, max_block=max_block, stream=stream)
+    handle = B.Handle(shape, B.weights_to_device(w), max_seq=max_seq, max_block=max_block, stream=stream,
+                      kv_dtype=B.KV_F16 if kv_dtype is None else kv_dtype)
     return oracle, handle, w
 
 

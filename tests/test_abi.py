@@ -36,7 +36,7 @@ def test_every_declared_symbol_is_exported_and_bound(lib):
 
 def good_cfg(**kw):
     d = dict(n_layers=1, hidden=64, n_q_heads=2, n_kv_heads=1, head_dim=64, intermediate=128, vocab=100, mask_id=99,
-             rms_eps=1e-6, rope_theta=1e6, tie_embeddings=1, dtype=B.DT_F32, max_seq=64, max_block=8)
+             rms_eps=1e-6, rope_theta=1e6, tie_embeddings=1, dtype=B.DT_F32, max_seq=64, max_block=8, kv_dtype=B.KV_BF16)
     d.update(kw)
     return B.Config(*[d[n] for n, _ in B.Config._fields_])
 
@@ -61,6 +61,7 @@ def fake_weights(n_layers=1, lm_head=None):
     (dict(max_seq=4), B.ERR_INVALID_ARG),
     (dict(rms_eps=0.0), B.ERR_INVALID_ARG),
     (dict(n_layers=0), B.ERR_INVALID_ARG),
+    (dict(kv_dtype=2), B.ERR_INVALID_ARG),
 ])
 def test_create_rejects_bad_config_before_touching_the_device(lib, kw, code):
     w, _keep = fake_weights()
@@ -91,6 +92,10 @@ def test_null_handle_calls_do_not_crash(lib):
     assert lib.fdvlm_reset(None) == B.ERR_INVALID_ARG
     assert lib.fdvlm_commit_block(None, None) == B.ERR_INVALID_ARG
     assert lib.fdvlm_prefill(None, None, 0, None, 0, None) == B.ERR_INVALID_ARG
+    assert lib.fdvlm_synchronize(None) == B.ERR_INVALID_ARG
+    assert lib.fdvlm_debug_poison(None, 1) == B.ERR_INVALID_ARG
+    assert lib.fdvlm_decode_block(None, 4, None, None, None, None) == B.ERR_INVALID_ARG
+    assert lib.fdvlm_profile_read_chain(None, None, 0, None) == B.ERR_INVALID_ARG
     lib.fdvlm_destroy(None)
 
 
@@ -99,9 +104,15 @@ def test_op_argument_checks(lib):
     assert lib.fdvlm_op_linear(0x10, 0x10, None, None, 0x10, 65, 8, 8, B.DT_F32, 0x10, None) == B.ERR_INVALID_ARG
     assert lib.fdvlm_op_linear(0x10, 0x10, None, None, 0x10, 4, 8, 12, B.DT_F32, 0x10, None) == B.ERR_INVALID_ARG
     assert lib.fdvlm_op_linear(0x10, 0x10, None, None, 0x10, 4, 8, 16, B.DT_FP8, 0x10, None) == B.ERR_INVALID_ARG
-    assert lib.fdvlm_op_attention(0x10, 0x10, 0x10, 0x10, 4, 60, 62, 4, 2, 64, 0, B.DT_F32, None, None) == B.ERR_INVALID_ARG
-    assert lib.fdvlm_op_attention(0x10, 0x10, 0x10, 0x10, 4, 0, 62, 4, 3, 64, 0, B.DT_F32, None, None) == B.ERR_INVALID_ARG
-    assert lib.fdvlm_op_linear_workspace_bytes(32, 2048, 2048, B.DT_BF16) >= 0
+    assert lib.fdvlm_op_linear(0x10, 0x10, None, None, 0x10, 4, 8, 16, B.DT_BF16, None, None) == B.ERR_INVALID_ARG   # no workspace
+    assert lib.fdvlm_op_attention(0x10, 0x10, 0x10, 0x10, 4, 60, 62, 4, 2, 64, 0, B.DT_F32, B.KV_BF16, None, None) == B.ERR_INVALID_ARG
+    assert lib.fdvlm_op_attention(0x10, 0x10, 0x10, 0x10, 4, 0, 62, 4, 3, 64, 0, B.DT_F32, B.KV_BF16, None, None) == B.ERR_INVALID_ARG
+    assert lib.fdvlm_op_attention(0x10, 0x10, 0x10, 0x10, 4, 0, 62, 4, 2, 64, 0, B.DT_BF16, 5, 0x10, None) == B.ERR_INVALID_ARG
+    # every workspace starts with the kernels' status words, so it is never empty
+    assert lib.fdvlm_op_linear_workspace_bytes(32, 2048, 2048, B.DT_BF16) >= 256
+    # (with a GPU present the fp8 figure also holds the f16 copy of the rows; without one both are the CUDA-core sizes)
+    assert (lib.fdvlm_op_linear_workspace_bytes(32, 2048, 2048, B.DT_FP8)
+            >= lib.fdvlm_op_linear_workspace_bytes(32, 2048, 2048, B.DT_BF16))
 
 
 def test_no_gpu_means_loud_failure_not_fallback(lib):
