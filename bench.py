@@ -81,6 +81,13 @@ class ClockSampler:
                 "reasons": reasons, "samples": len(sm)}
 
 
+def config_of(wl: I.Workload, block: int, world: int) -> dict:
+    """The workload description both arms print."""
+    return {"workload": wl.name, "block": block, "prefix": wl.n_embeds + wl.n_tokens,
+            "denoise_steps_per_block": schedule(wl, block), "rule": wl.rule,
+            "cache_flush": "inputs (gigabytes of weights per forward) larger than L2", "parallelism": f"replicas x{world}"}
+
+
 def schedule(wl: I.Workload, block: int):
     """Denoise steps per block on a random-init model: top-k gives ceil(B/k) steps; threshold 0.9 never
     fires on near-uniform confidences, so the at-least-one rule gives B steps."""
@@ -90,31 +97,46 @@ def schedule(wl: I.Workload, block: int):
 # ------------------------------------------------------------------------------------------------
 # CPU oracle timing (the reported cpu_baseline, and the whole of --impl reference)
 # ------------------------------------------------------------------------------------------------
-def oracle_sample(wl: I.Workload, block: int, weights_cpu: dict, reps: int = 1):
-    """Time the oracle on a bounded sample: after an (untimed) 32-row prefill, one denoise step and one
-    commit of a block; tokens/s extrapolated with the workload's schedule."""
+def make_oracle_at_prefix(wl: I.Workload, weights_cpu: dict):
+    """The oracle with a cache of the workload's prefix length.  The prefill is outside the metric and would take the
+    oracle minutes at these lengths, so the cache is filled with N(0, 1) values of the right shape instead: the time of
+    a denoise or commit forward depends on the cache's length, not on its contents."""
     import numpy as np
     from oracle import fdvlm_oracle as orc
     shape = wl.shape
     o = orc.Oracle(shape, I.weights_to_numpy(weights_cpu))
-    emb, toks = I.make_prefix(shape, 16, 16, wl.prefix_seed)
-    o.prefill(I.as_numpy_storage(emb), toks.numpy(), want_logits=False)
+    L0 = wl.n_embeds + wl.n_tokens
+    rng = np.random.default_rng(wl.prefix_seed)
+    for l in range(shape.n_layers):
+        o.K[l] = rng.standard_normal((L0, shape.n_kv_heads, shape.head_dim))
+        o.V[l] = rng.standard_normal((L0, shape.n_kv_heads, shape.head_dim))
+    o.cache_len = L0
+    return o
+
+
+def oracle_forward_seconds(o, wl: I.Workload, block: int, commit: bool):
+    """One timed oracle forward of a block at the current cache length: a denoise step, or the causal commit (whose
+    cache growth is undone afterwards so that every sample sees the same length)."""
+    import numpy as np
+    from oracle import fdvlm_oracle as orc
     rule = orc.TOPK if wl.rule == "topk" else orc.THRESHOLD
-    t_steps, t_commits = [], []
-    for _ in range(reps):
-        o.block_begin(block)
+    L0 = o.cache_len
+    o.block_begin(block)
+    if not commit:
         t0 = time.perf_counter()
         o.block_step(rule, wl.threshold, wl.k)
-        t_steps.append(time.perf_counter() - t0)
-        o.block_tokens[:] = np.arange(block) % (shape.vocab - 1)
-        o.masked[:] = False
-        t0 = time.perf_counter()
-        o.commit_block(want_logits=True)
-        t_commits.append(time.perf_counter() - t0)
-    ts, tc = statistics.median(t_steps), statistics.median(t_commits)
-    n_steps = schedule(wl, block)
-    tok_s = block / (n_steps * ts + tc)
-    return tok_s, ts, tc
+        return time.perf_counter() - t0
+    o.block_tokens[:] = np.arange(block) % (wl.shape.vocab - 1)
+    o.masked[:] = False
+    t0 = time.perf_counter()
+    o.commit_block(want_logits=False)
+    dt = time.perf_counter() - t0
+    o.truncate(L0)
+    return dt
+
+
+def oracle_tok_s(wl, block, t_step, t_commit):
+    return block / (schedule(wl, block) * t_step + t_commit)
 
 
 def run_reference(args, wl, block):
@@ -124,23 +146,36 @@ def run_reference(args, wl, block):
     shape = wl.shape
     weights = I.make_weights(shape, wl.weight_seed)
     cores = torch.get_num_threads()
-    vals = []
-    for _ in range(args.warmup):
-        pass   # nothing to warm on the CPU path beyond the first BLAS call inside the first sample
+    o = make_oracle_at_prefix(wl, weights)
+    L0 = o.cache_len
+    n_steps = schedule(wl, block)
+    # A bench step is one block = n_steps denoise forwards + 1 commit forward.  One oracle forward of the 3B shape takes
+    # ~13 s, so each timed "step" of this arm is a bounded sample of the block: ONE denoise forward (the commit forward
+    # is timed once, before the loop); tokens/s extrapolates the block from them.  The loop stops after ~3 minutes and
+    # `steps` reports what was really run.
+    t_commit = oracle_forward_seconds(o, wl, block, commit=True)
     t_all0 = time.perf_counter()
+    for _ in range(max(0, args.warmup)):
+        if time.perf_counter() - t_all0 > 45.0:
+            break
+        oracle_forward_seconds(o, wl, block, commit=False)
+    t_loop0 = time.perf_counter()
+    t_steps = []
     for _ in range(max(1, args.steps)):
-        v, ts, tc = oracle_sample(wl, block, weights)
-        vals.append(v)
-        if time.perf_counter() - t_all0 > 150.0:     # keep the whole arm within a few minutes
+        t_steps.append(oracle_forward_seconds(o, wl, block, commit=False))
+        if time.perf_counter() - t_loop0 > 170.0:
             break
     wall = time.perf_counter() - t_all0
-    value = statistics.median(vals)
-    sample = (f"per step: one denoise forward + one commit forward of a {block}-token block at cache length 32, "
-              f"tokens/s extrapolated over the schedule ({schedule(wl, block)} denoise steps + 1 commit per block)")
+    t_step = statistics.median(t_steps)
+    value = oracle_tok_s(wl, block, t_step, t_commit)
+    sample = (f"each timed step = one denoise forward of a {block}-token block at cache length {L0} (median {t_step:.1f} s over "
+              f"{len(t_steps)} forwards); the commit forward was timed once ({t_commit:.1f} s); tokens/s = {block} / "
+              f"({n_steps} x step + commit); the cache holds N(0,1) values (the prefill is outside the metric)")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "tok/s", "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1000.0 * block / value, "higher_is_better": True,
+            "steps": len(t_steps), "steps_requested": args.steps, "warmup": args.warmup,
+            "ms_per_step": 1000.0 * t_step, "ms_per_block_extrapolated": 1000.0 * block / value, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": wl.name, "block": block},
+            "config": config_of(wl, block, 1),
             "cpu_baseline": {"value": value, "unit": "tok/s", "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": "tok/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "wall_s": wall}
@@ -200,17 +235,12 @@ def run_ours(args, wl, block):
                 handle.commit_block()
                 launches[0] += handle.last_launch_count()
                 return info.step_index
-            handle.block_begin(block)
-            n = 0
-            while True:
-                info = handle.block_step(rule, wl.threshold, wl.k)
-                launches[0] += handle.last_launch_count()
-                n += 1
-                if info.n_remaining == 0:
-                    break
+            # threshold rule: the step count depends on the confidences, so the loop itself runs on the device
+            info = handle.decode_block(block, rule, wl.threshold, wl.k)
+            launches[0] += handle.last_launch_count()
             handle.commit_block()
             launches[0] += handle.last_launch_count()
-            return n
+            return info.step_index
 
         conf_h = torch.empty(block, dtype=torch.float32).pin_memory()
         pred_h = torch.empty(block, dtype=torch.int32).pin_memory()
@@ -250,22 +280,35 @@ def run_ours(args, wl, block):
         one_block_host()
         ms_e2e = timed(one_block_host, K)
 
-        # per-step latency and roofline of the dominant kernel family (projection GEMMs), profiled repeat
-        handle.profile_enable(True)
-        step_ms = []
+        # (1) the projection launches timed one by one with CUDA events (kernels launched singly: no overlap)
+        handle.profile_enable(1)
         handle.block_begin(block)
-        L_step = handle.cache_len()
         for _ in range(n_steps):
-            a, b = ev(), ev()
-            a.record(stream)
             handle.block_step(rule, wl.threshold, wl.k)
-            b.record(stream)
-            stream.synchronize()
-            step_ms.append(a.elapsed_time(b))
         prof = handle.profile_read()
-        handle.profile_enable(False)
-        # unprofiled per-step latency
+        handle.profile_enable(0)
         handle.commit_block()
+        # (2) in-chain timing: the production launch sequence (graph replay, dependent launches), every kernel stamping the
+        # GPU's global timer.  The timeline of a forward is cut at the kernels' end times: kernel i owns the interval
+        # (end of kernel i-1, end of kernel i], so the shares add up to the forward's duration.
+        handle.profile_enable(2)
+        handle.block_begin(block)
+        handle.block_step(rule, wl.threshold, wl.k)        # the stamped graph's first use (capture)
+        chain_us, chain_total, chain_n = {}, [], 0
+        while handle.last_info_remaining() > 0:
+            handle.block_step(rule, wl.threshold, wl.k)
+            recs = handle.profile_read_chain()
+            prev = recs[0]["start_us"]
+            for r in recs:
+                end = max(r["end_us"], prev)
+                chain_us[r["kind"]] = chain_us.get(r["kind"], 0.0) + (end - prev)
+                prev = end
+            chain_total.append(prev - recs[0]["start_us"])
+            chain_n += 1
+        handle.profile_enable(0)
+        handle.commit_block()
+        chain_us = {k_: v / max(chain_n, 1) for k_, v in chain_us.items()}
+        # (3) unprofiled per-step latency
         handle.block_begin(block)
         L_step = handle.cache_len()
         lat = []
@@ -323,37 +366,49 @@ def run_ours(args, wl, block):
     e2e_value = R.whole_job_rate(K * block, world, ms_e2e)
     peak, peak_kind = measured_peaks()
     wbytes = shape.weight_bytes()
-    gemm_ms_per_fwd = prof["ms_linear"] / n_steps
-    gemm_gbs = wbytes / (gemm_ms_per_fwd / 1000.0) / 1e9
-    # DRAM bytes of the same launches, from the ncu captures summarised under profiles/ (dram read + write over
-    # algorithmic bytes of the four layer projections, measured on the 4-layer cut of the shape and scaled by the
-    # weight bytes: traffic grows in proportion).  None for shapes without a capture.
-    ratio = {"cfg2_3b_bf16_p1024_b32_top8": 158.91 / 154.15, "cfg3_3b_bf16_p2048_sweep": 158.91 / 154.15,
-             "cfg4_3b_bf16_p8192_b32_top8": 158.91 / 154.15, "cfg5_7b_fp8_p1024_b32": 240.66 / 233.06}.get(wl.name)
-    traffic = None if ratio is None or block != 32 else wbytes * ratio
-    traffic_note = None if traffic is None else "scaled from the 4-layer ncu capture of the same layer shapes (profiles/)"
-    step_bytes = wbytes + shape.kv_bytes_per_token() * L_step
+    gemm_ms_isolated = prof["ms_linear"] / n_steps
+    gemm_kinds = ("gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "gemm_lm_head")
+    gemm_us_chain = sum(chain_us.get(k_, 0.0) for k_ in gemm_kinds)
+    gemm_gbs = wbytes / (gemm_us_chain * 1e-6) / 1e9
+    kv_bytes = shape.kv_bytes_per_token() * L_step
+    attn_us_chain = chain_us.get("attention", 0.0) + chain_us.get("attn_merge", 0.0)
+    # DRAM bytes of the same launches: dram read + write over algorithmic bytes of the layer projections, from the ncu
+    # capture summarised in profiles/ncu_traffic.json (taken on the 4-layer cut of the shape; traffic grows in
+    # proportion to the weight bytes).  Null when there is no capture of the kernel as it stands.
+    traffic, traffic_note = None, None
+    try:
+        with open(os.path.join(ROOT, "profiles", "ncu_traffic.json")) as f:
+            cap = json.load(f).get("gemm_tc", {}).get(shape.dtype)
+        if cap and block == cap.get("block"):
+            traffic = wbytes * cap["dram_bytes"] / cap["algorithmic_bytes"]
+            traffic_note = cap.get("note")
+    except (OSError, ValueError, KeyError):
+        pass
+    step_bytes = wbytes + kv_bytes
     step_med = statistics.median(lat)
     line = {
         "metric": METRIC, "value": value, "unit": "tok/s", "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms_dev / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": {"f32": "f32", "bf16": "bf16", "fp8": "bf16 x e4m3 weights"}[shape.dtype], "data": "synthetic",
-        "config": {"workload": wl.name, "block": block, "prefix": L0, "denoise_steps_per_block": n_steps,
-                   "rule": wl.rule, "cache_flush": "inputs (6.2 GB of weights per forward) larger than L2",
-                   "parallelism": f"replicas x{world}"},
+        "dtype": {"f32": "f32", "bf16": "bf16", "fp8": "f16 x e4m3 weights"}[shape.dtype], "data": "synthetic",
+        "config": config_of(wl, block, world),
+        "kv_dtype": "bf16" if kv_dtype == B.KV_BF16 else "f16",
         "e2e": {"value": e2e_value, "unit": "tok/s", "h2d_bytes_per_step": block * 4,
-                "d2h_bytes_per_step": n_steps * (block * 13 + 16)},
+                "d2h_bytes_per_step": n_steps * (block * 13 + 32)},
         "gpu_launches": n_launch,
         "clocks": clocks,
+        # dominant kernel: the projection GEMMs.  achieved = every linear weight byte of one forward / the time those
+        # launches own in the production chain (in-chain timing, see above); frac x peak x that time = the bytes.
         "roofline": {"bound": "hbm", "achieved": gemm_gbs, "peak": peak, "unit": "GB/s", "frac": gemm_gbs / peak,
                      "traffic": traffic, "traffic_note": traffic_note, "peak_kind": peak_kind,
-                     "kernel": "gemm_tc_kernel: all projection launches of one forward (timed one by one with CUDA events, "
-                               "i.e. without the overlap of the live chain)",
-                     "algorithmic_bytes_per_forward": wbytes, "ms_per_forward": gemm_ms_per_fwd,
-                     # the same bytes over the whole live step (every kernel of the forward, chained and overlapped as in
-                     # production): a lower bound of what the projection launches reach inside the chain
-                     "live_step_lower_bound": {"achieved": wbytes / (step_med / 1000.0) / 1e9,
-                                               "frac": wbytes / (step_med / 1000.0) / 1e9 / peak}},
+                     "kernel": "gemm_tc_kernel: all projection launches of one denoise forward, in-chain",
+                     "algorithmic_bytes_per_forward": wbytes, "in_chain_ms_per_forward": gemm_us_chain / 1000.0,
+                     "forward_ms_in_chain_timing": statistics.median(chain_total) / 1000.0 if chain_total else None,
+                     "isolated": {"ms_per_forward": gemm_ms_isolated, "achieved": wbytes / (gemm_ms_isolated / 1000.0) / 1e9,
+                                  "note": "the same launches timed one by one with CUDA events, without the chain's overlap"}},
+        "attention": {"kernel": "attn_mma_kernel + attn_combine_kernel, in-chain", "kv_bytes_per_forward": kv_bytes,
+                      "in_chain_ms_per_forward": attn_us_chain / 1000.0,
+                      "achieved_gbs": kv_bytes / (attn_us_chain * 1e-6) / 1e9 if attn_us_chain > 0 else None},
+        "chain_us_per_forward": {k_: round(v, 2) for k_, v in sorted(chain_us.items())},
         "step": {"latency_ms_median": step_med, "latency_ms_all": lat, "cache_len": L_step, "bytes": step_bytes,
                  "gbs": step_bytes / (step_med / 1000.0) / 1e9, "frac_of_peak": step_bytes / (step_med / 1000.0) / 1e9 / peak,
                  "frac_of_8tbs": step_bytes / (step_med / 1000.0) / 1e9 / 8000.0},
@@ -363,10 +418,14 @@ def run_ours(args, wl, block):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         wcpu = {k: (v.cpu() if isinstance(v, torch.Tensor) else v) for k, v in weights.items() if k != "layers"}
         wcpu["layers"] = [{k: (v.cpu() if isinstance(v, torch.Tensor) else v) for k, v in lw.items()} for lw in weights["layers"]]
-        v, ts, tc = oracle_sample(wl, block, wcpu)
-        line["cpu_baseline"] = {"value": v, "unit": "tok/s", "cores": torch.get_num_threads(), "kind": "oracle",
+        o = make_oracle_at_prefix(wl, wcpu)
+        ts = oracle_forward_seconds(o, wl, block, commit=False)
+        tc = oracle_forward_seconds(o, wl, block, commit=True)
+        line["cpu_baseline"] = {"value": oracle_tok_s(wl, block, ts, tc), "unit": "tok/s", "cores": torch.get_num_threads(),
+                                "kind": "oracle",
                                 "sample": f"one denoise forward ({ts:.1f} s) + one commit forward ({tc:.1f} s) of a {block}-token block "
-                                          f"at cache length 32, extrapolated over {n_steps} denoise steps + 1 commit per block"}
+                                          f"at cache length {o.cache_len} (cache filled with N(0,1) values: the prefill is outside the "
+                                          f"metric), extrapolated over {n_steps} denoise steps + 1 commit per block"}
     handle.close()
     if R.prints_result(rank):
         print(json.dumps(line), flush=True)

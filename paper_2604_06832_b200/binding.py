@@ -216,7 +216,12 @@ class Handle:
         p, info = StepParams(rule, threshold, k, pred_shift), StepInfo()
         self._check(lib().fdvlm_block_step(self._h, C.byref(p), _ptr(logits), _ptr(conf), _ptr(pred), _ptr(unmask),
                                            _ptr(block_tokens), C.byref(info)))
+        self._remaining = info.n_remaining
         return info
+
+    def last_info_remaining(self) -> int:
+        """n_remaining reported by the last block_step of this wrapper."""
+        return getattr(self, "_remaining", 0)
 
     def block_step_host(self, rule: int, threshold: float = 0.9, k: int = 8, conf=None, pred=None, unmask=None,
                         block_tokens=None, pred_shift: int = 0) -> StepInfo:

@@ -53,7 +53,7 @@ __global__ void __launch_bounds__(128) attn_combine_kernel(const float* __restri
                        threadIdx.x & 31);
   }
   __syncthreads();
-  if (threadIdx.x == 0) stamp_end(stamp);
+  if (threadIdx.x == 0) stamp_end(stamp, true);
 }
 
 // ---- host side -------------------------------------------------------------------------------------

@@ -99,10 +99,23 @@ __device__ __forceinline__ unsigned long long global_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-// each called by ONE thread of a CTA
-__device__ __forceinline__ void stamp_start(KStamp* s) { if (s) atomicMin(&s->start, global_ns()); }
-__device__ __forceinline__ void stamp_released(KStamp* s) { if (s) atomicMin(&s->released, global_ns()); }
-__device__ __forceinline__ void stamp_end(KStamp* s) { if (s) atomicMin(&s->end_inv, ~global_ns()); }
+// Each called by ONE thread of a CTA.  A CTA that can see it would not lower the minimum skips the atomic (hundreds of
+// CTAs updating one word would stretch the small kernels they are meant to time); `sampled` end stamps, for kernels of
+// many short equal CTAs, come from every eighth CTA and the last one only.
+__device__ __forceinline__ void stamp_min(unsigned long long* p, unsigned long long t) {
+  if (t < *reinterpret_cast<volatile unsigned long long*>(p)) atomicMin(p, t);
+}
+__device__ __forceinline__ void stamp_start(KStamp* s) { if (s) stamp_min(&s->start, global_ns()); }
+__device__ __forceinline__ void stamp_released(KStamp* s) { if (s) stamp_min(&s->released, global_ns()); }
+__device__ __forceinline__ void stamp_end(KStamp* s, bool sampled = false) {
+  if (!s) return;
+  if (sampled) {
+    const unsigned id = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z);
+    const unsigned total = gridDim.x * gridDim.y * gridDim.z;
+    if ((id & 7u) != 0 && id != total - 1) return;
+  }
+  atomicMin(&s->end_inv, ~global_ns());
+}
 
 enum { MODE_BIDIR = 0, MODE_CAUSAL = 1 };
 enum { DT_F32 = 0, DT_BF16 = 1, DT_FP8 = 2 };

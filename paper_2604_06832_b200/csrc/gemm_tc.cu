@@ -8,8 +8,9 @@
 // buffers, so the epilogue of one work item overlaps the mainloop of the next); four epilogue warps
 // read the accumulators with tcgen05.ld.  CTAs are persistent over a static round-robin list of
 // work items (tile, K-split).  bf16 weights: the activations arrive as two bf16 planes, hi = bf16(v) and
-// lo = bf16(v - hi); every streamed weight tile is multiplied by both (two MMAs into the same accumulator), so the
-// activation side of the product carries ~16 significant bits at no extra HBM traffic.  FP8-E4M3 weights take the
+// lo = bf16(v - hi); both land side by side in the stage and form ONE MMA operand of twice the rows, so every streamed
+// weight tile is read from shared memory once and multiplied by both; the epilogue adds the two halves of the
+// accumulator.  The activation side of the product thus carries ~16 significant bits at no extra HBM traffic.  FP8-E4M3 weights take the
 // same road with half the bytes: the byte tile lands in the stage, four converter warps widen it exactly to f16
 // (one cvt per pair) into a swizzled buffer of its own, and the MMA (f16 x f16, activations stored as f16) reads
 // that buffer; the per-channel scales are applied by the epilogues.
@@ -137,7 +138,10 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
   volatile int* abort_flag = (volatile int*)(sm + L::BAR_OFF + 8 * (2 * TC_STAGES + 8) + 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  constexpr int TMEM_COLS = (2 * M_PAD <= 32) ? 32 : ((2 * M_PAD <= 64) ? 64 : 128);
+  // two accumulator buffers; bf16 weights: each holds the hi-plane product in columns [0, M_PAD) and the lo-plane
+  // product in [M_PAD, 2 M_PAD)
+  constexpr int ACC_COLS = FP8 ? M_PAD : 2 * M_PAD;
+  constexpr int TMEM_COLS = (2 * ACC_COLS <= 32) ? 32 : ((2 * ACC_COLS <= 64) ? 64 : ((2 * ACC_COLS <= 128) ? 128 : 256));
 
   // fp8 launches in which no CTA has a second work item: the epilogue warps, idle until the accumulator is complete,
   // widen half of every weight tile beside the four converter warps
@@ -267,8 +271,8 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
   } else if (warp == 1) {
     // ------------------------------------------------ MMA issuer --------------------------------------------------
     if (lane == 0) {
-      const uint32_t idesc = FP8 ? umma_idesc_f16(M_PAD) : umma_idesc_bf16(M_PAD);
       const bool two_planes = !FP8 && p.has_lo;
+      const uint32_t idesc = FP8 ? umma_idesc_f16(M_PAD) : umma_idesc_bf16(two_planes ? 2 * M_PAD : M_PAD);
       int stage = 0, cbuf = 0;
       uint32_t phase = 0, cphase = 0;
       int local = 0;
@@ -279,7 +283,7 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
         const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * M_PAD);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * ACC_COLS);
         const int kb0 = split * p.kb_per_split;
         const int kb1 = min(p.kblocks, kb0 + p.kb_per_split);
         for (int kb = kb0; kb < kb1; ++kb) {
@@ -292,11 +296,6 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
 #pragma unroll
           for (int kk = 0; kk < TC_BK / 16; ++kk)
             umma_bf16(d_tmem, adesc + 2u * kk, bdesc + 2u * kk, idesc, (kb > kb0 || kk > 0) ? 1u : 0u);
-          if (two_planes) {     // the same weight tile against the activations' low-order plane
-            const uint64_t ldesc = umma_desc_sw128(a_addr + L::W_BYTES + L::B_BYTES);
-#pragma unroll
-            for (int kk = 0; kk < TC_BK / 16; ++kk) umma_bf16(d_tmem, adesc + 2u * kk, ldesc + 2u * kk, idesc, 1u);
-          }
           umma_commit(empty_bar(stage));
           if (FP8) {
             umma_commit(cempty_bar(cbuf));
@@ -341,9 +340,19 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       float v[M_PAD];
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * M_PAD);
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * ACC_COLS);
 #pragma unroll
       for (int c = 0; c < M_PAD; c += 16) tmem_ld16(taddr + c, v + c);
+      if (!FP8 && p.has_lo) {      // the low-order plane's product sits M_PAD columns further on
+#pragma unroll
+        for (int c = 0; c < M_PAD; c += 16) {
+          float lo[16];
+          tmem_ld16(taddr + M_PAD + c, lo);
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+          for (int i = 0; i < 16; ++i) v[c + i] += lo[i];
+        }
+      }
       asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();

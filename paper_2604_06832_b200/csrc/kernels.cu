@@ -425,7 +425,7 @@ __global__ void fin_qkv_kernel(const float* __restrict__ part, int S, int m, con
     o[j] = from_f32<T>(a);
     o[j + half] = from_f32<T>(b);
   }
-  if (threadIdx.x == 0) stamp_end(stamp);
+  if (threadIdx.x == 0) stamp_end(stamp, true);
 }
 void launch_fin_qkv(const float* part, int S, int m, const float* cs, const float* ssq, int nt, int hidden, float eps,
                     const float* bq, const float* bk, const float* bv, const float* sq, const float* sk, const float* sv, void* q, void* kc, void* vc, int pos0, int hq,
@@ -464,7 +464,7 @@ __global__ void __launch_bounds__(128) fin_resid_kernel(const float* __restrict_
     store_act(xg, lo_off, idx, v * gc, fmt);
   }
   const float ss = block_sum(v * v, red);
-  if (threadIdx.x == 0) { ssq[(size_t)r * nt + t] = ss; stamp_end(stamp); }
+  if (threadIdx.x == 0) { ssq[(size_t)r * nt + t] = ss; stamp_end(stamp, true); }
 }
 void launch_fin_resid(const float* part, int S, int m, int hidden, float* h, const float* g, void* xg, size_t lo_off, int fmt,
                       float* ssq, int nt, const float* scale, cudaStream_t st, KStamp* stamp) {
