@@ -13,7 +13,9 @@ Pinned by tests that do not call back into this file's own formulas: B=1 == caus
 chunked prefill + commit == one dense causal pass, cached path == dense brute-force mask,
 dependency probes, selection closed forms, softmax identities, GQA == MHA with repeated
 K/V weights, RoPE shift invariance, RMSNorm / SwiGLU closed forms, hand-checkable
-zero-layer logits, and an independent torch restatement of attention.
+zero-layer logits, an independent torch restatement of attention, a hand-worked e4m3 matrix
+with per-row scales, and the untied FP8 LM head recomputed row by row; planted errors (a rotation
+sign, a scale on the wrong axis, an ignored head or head scale) must make those pins fail.
 Parity unpinned: absolute logit values of the random-init models (the paper prints no
 worked numerical example of a denoise step).
 """

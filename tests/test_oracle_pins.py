@@ -367,12 +367,160 @@ def test_fp32_oracle_close_to_fp64_oracle():
     assert np.abs(outs[0] - outs[1]).max() < 1e-5
 
 
-# ---- planted mistakes must be caught (a transposed operand, a wrong rotation sign) ------------------
-def test_pins_detect_planted_rope_sign_error(monkeypatch):
-    good = orc.rope
+# ---- FP8 storage with per-output-channel scales, and the untied LM head -----------------------------
+def _hand_e4m3():
+    """A 2 x 3 e4m3 matrix written out code by code (sign | 4 exponent bits, bias 7 | 3 mantissa bits) with one scale per
+    ROW (= output channel), and its value worked by hand."""
+    codes = np.array([[0x38, 0x40, 0xB8],        #  1.0   2.0   -1.0
+                      [0x3C, 0x30, 0x7E]],       #  1.5   0.5   448 (largest finite)
+                     dtype=np.uint8)
+    scales = np.array([0.5, 3.0], dtype=np.float32)
+    value = [[0.5, 1.0, -0.5], [4.5, 1.5, 1344.0]]
+    return codes, scales, value
 
-    def bad(x, pos, theta):
-        return good(x, -np.asarray(pos), theta)
-    monkeypatch.setattr(orc, "rope", bad)
-    v = np.array([[[1.0, 0.0]]])
-    assert not np.allclose(orc.rope(v, np.array([1]), 1e6)[0, 0], [math.cos(1.0), math.sin(1.0)])
+
+def test_fp8_weight_with_row_scales_by_hand():
+    codes, scales, value = _hand_e4m3()
+    o = orc.Oracle(MICRO, {"layers": [{"wq": codes, "s_q": scales}]})
+    w = o._lin(0, "wq")
+    assert w.shape == (2, 3)
+    for r in range(2):
+        for c in range(3):
+            assert w[r, c] == value[r][c], (r, c, w[r, c])
+    # orientation in a projection: [out, in], so a one-hot input picks a COLUMN of the matrix
+    assert np.array_equal(np.array([0.0, 1.0, 0.0]) @ w.T, [1.0, 1.5])
+    # a matrix without scales is taken as stored
+    assert np.array_equal(orc.Oracle(MICRO, {"layers": [{"wq": codes}]})._lin(0, "wq"), [[1.0, 2.0, -1.0], [1.5, 0.5, 448.0]])
+
+
+FP8_MICRO = MICRO.with_(dtype=I.FP8, tie_embeddings=False)
+
+
+def _untied_logits_by_hand(o, w, h):
+    """RMSNorm(h; g_final) . (e4m3(lm_head) * s_lm_head[row])^T with plain Python loops and torch's own e4m3 cast."""
+    shape = o.s
+    table = w["lm_head"].view(torch.float8_e4m3fn).to(torch.float64).numpy()
+    s_head = w["s_lm_head"].double().numpy()
+    g = w["g_final"].double().numpy()
+    out = np.zeros((h.shape[0], shape.vocab))
+    for r in range(h.shape[0]):
+        ms = sum(float(v) ** 2 for v in h[r]) / shape.hidden
+        a = [float(h[r, c]) / math.sqrt(ms + shape.rms_eps) * g[c] for c in range(shape.hidden)]
+        for v in range(shape.vocab):
+            out[r, v] = sum(a[c] * table[v, c] * s_head[v] for c in range(shape.hidden))
+    return out
+
+
+def test_untied_fp8_lm_head_row_by_row():
+    o, w = make(FP8_MICRO, seed=5, final_gain=1.7)
+    assert w["lm_head"] is not None and w["lm_head"].dtype == torch.uint8 and w["s_lm_head"].shape == (FP8_MICRO.vocab,)
+    # the scales must differ from row to row for the test to see a wrong axis
+    assert len(set(np.round(w["s_lm_head"].numpy(), 9).tolist())) > FP8_MICRO.vocab // 2
+    h = np.random.default_rng(1).standard_normal((3, FP8_MICRO.hidden))
+    got = o.logits_of(h)
+    want = _untied_logits_by_hand(o, w, h)
+    assert np.abs(got - want).max() < 1e-12
+    # and the embedding table plays no part in an untied head
+    o.w["embed"] = np.zeros_like(o.w["embed"])
+    assert np.array_equal(o.logits_of(h), got)
+
+
+def test_fp8_micro_model_layer_matmuls_use_row_scales():
+    """A whole forward of the FP8 micro model against the torch restatement fed with explicitly de-quantised weights
+    (value = e4m3 code * scale of its output row), so every projection's scale handling is covered."""
+    o, w = make(FP8_MICRO, seed=6)
+    deq = {"embed": w["embed"].double(), "g_final": w["g_final"].double(),
+           "lm_head": w["lm_head"].view(torch.float8_e4m3fn).double() * w["s_lm_head"].double()[:, None], "layers": []}
+    for lw in w["layers"]:
+        d = {}
+        for name, sname in (("wq", "s_q"), ("wk", "s_k"), ("wv", "s_v"), ("wo", "s_o"), ("w_gate", "s_gate"), ("w_up", "s_up"),
+                            ("w_down", "s_down")):
+            d[name] = lw[name].view(torch.float8_e4m3fn).double() * lw[sname].double()[:, None]
+        deq["layers"].append(d)
+    s = FP8_MICRO
+    toks = torch.tensor([3, 9, 27, 5, 11])
+    h = deq["embed"][toks]
+    T = len(toks)
+    pos = torch.arange(T, dtype=torch.float64)
+    half = s.head_dim // 2
+    inv = s.rope_theta ** (-torch.arange(half, dtype=torch.float64) * 2 / s.head_dim)
+    cos, sin = torch.cos(pos[:, None] * inv), torch.sin(pos[:, None] * inv)
+
+    def rot(x):
+        x1, x2 = x[..., :half], x[..., half:]
+        return torch.cat([x1 * cos[:, None] - x2 * sin[:, None], x2 * cos[:, None] + x1 * sin[:, None]], -1)
+
+    def norm(x):
+        return x / torch.sqrt((x * x).mean(-1, keepdim=True) + s.rms_eps)
+    for d in deq["layers"]:
+        a = norm(h)
+        q = rot((a @ d["wq"].T).view(T, s.n_q_heads, s.head_dim))
+        k = rot((a @ d["wk"].T).view(T, s.n_kv_heads, s.head_dim))
+        v = (a @ d["wv"].T).view(T, s.n_kv_heads, s.head_dim)
+        rep = s.n_q_heads // s.n_kv_heads
+        att = torch.nn.functional.scaled_dot_product_attention(q.transpose(0, 1), k.repeat_interleave(rep, 1).transpose(0, 1),
+                                                               v.repeat_interleave(rep, 1).transpose(0, 1), is_causal=True)
+        h = h + att.transpose(0, 1).reshape(T, -1) @ d["wo"].T
+        m = norm(h)
+        h = h + (torch.nn.functional.silu(m @ d["w_gate"].T) * (m @ d["w_up"].T)) @ d["w_down"].T
+    want = (norm(h) * deq["g_final"]) @ deq["lm_head"].T
+    got = o.prefill(None, toks.numpy())
+    assert np.abs(got - want[-1].numpy()).max() < 1e-10
+
+
+# ---- planted mistakes must be caught: each plants one plausible error in the oracle and requires a pin above to FAIL ----
+def _must_fail(pin, *args):
+    try:
+        pin(*args)
+    except AssertionError:
+        return
+    raise AssertionError(f"{pin.__name__} did not notice the planted error")
+
+
+def test_planted_rope_sign_error_fails_the_hand_rotation_pin(monkeypatch):
+    good = orc.rope
+    monkeypatch.setattr(orc, "rope", lambda x, pos, theta: good(x, -np.asarray(pos), theta))
+    _must_fail(test_rope_position_zero_identity_and_hand_rotation)
+
+
+def test_planted_scale_on_the_wrong_axis_fails_the_fp8_pins(monkeypatch):
+    def bad_lin(self, layer, name):
+        lw = self.w["layers"][layer]
+        w = orc.to_f64(lw[name])
+        sc = lw.get({"wq": "s_q", "wk": "s_k", "wv": "s_v", "wo": "s_o", "w_gate": "s_gate", "w_up": "s_up", "w_down": "s_down"}[name])
+        if sc is not None:
+            n = min(w.shape)
+            w = w.copy()
+            w[:n, :n] = w[:n, :n] * orc.to_f64(sc)[None, :n]          # per INPUT column instead of per output row
+        return w
+    monkeypatch.setattr(orc.Oracle, "_lin", bad_lin)
+    _must_fail(test_fp8_weight_with_row_scales_by_hand)
+    _must_fail(test_fp8_micro_model_layer_matmuls_use_row_scales)
+
+
+def test_planted_ignored_lm_head_fails_the_untied_pin(monkeypatch):
+    good = orc.Oracle.logits_of
+
+    def bad(self, h, chunk=16384):
+        saved = self.w.get("lm_head")
+        self.w["lm_head"] = None                                     # falls back to the embedding table
+        try:
+            return good(self, h, chunk)
+        finally:
+            self.w["lm_head"] = saved
+    monkeypatch.setattr(orc.Oracle, "logits_of", bad)
+    _must_fail(test_untied_fp8_lm_head_row_by_row)
+
+
+def test_planted_ignored_head_scale_fails_the_untied_pin(monkeypatch):
+    good = orc.Oracle.logits_of
+
+    def bad(self, h, chunk=16384):
+        saved = self.w.get("s_lm_head")
+        self.w["s_lm_head"] = None
+        try:
+            return good(self, h, chunk)
+        finally:
+            self.w["s_lm_head"] = saved
+    monkeypatch.setattr(orc.Oracle, "logits_of", bad)
+    _must_fail(test_untied_fp8_lm_head_row_by_row)
