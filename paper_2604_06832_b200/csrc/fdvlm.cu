@@ -424,6 +424,7 @@ static int build_loop_graph(fdvlm_t* h, int B, const fdvlm_step_params* p, bool 
   h->loop_exec = exec;
   h->loop_n = B; h->loop_rule = (int)p->rule; h->loop_k = p->k; h->loop_shift = p->pred_shift; h->loop_threshold = p->threshold;
   h->loop_body_launches = body_launches;
+  h->loop_long = attention_long_cache(h->cache_len + B) ? 1 : 0;
   return FDVLM_OK;
 }
 
@@ -438,8 +439,9 @@ extern "C" int fdvlm_decode_block(fdvlm_t* h, int block_size, const int32_t* ini
   if (rc) return rc;
   h->launches = 0;
   if (h->n_remaining > 0) {
+    const int long_cache = attention_long_cache(h->cache_len + block_size) ? 1 : 0;
     const bool have = h->loop_exec && h->loop_n == block_size && h->loop_rule == (int)p->rule && h->loop_k == p->k &&
-                      h->loop_shift == p->pred_shift && h->loop_threshold == p->threshold;
+                      h->loop_shift == p->pred_shift && h->loop_threshold == p->threshold && h->loop_long == long_cache;
     if (!have) {
       rc = build_loop_graph(h, block_size, p, true);
       if (rc) rc = build_loop_graph(h, block_size, p, false);
@@ -673,7 +675,7 @@ extern "C" int fdvlm_op_attention(const void* q, const void* k_cache, const void
   if (kv_dtype != FDVLM_KV_BF16 && kv_dtype != FDVLM_KV_F16) return FDVLM_ERR_INVALID_ARG;
   AttnArgs a;
   memset(&a, 0, sizeof(a));
-  a.kv_type = (int)kv_dtype; a.out_fmt = kv_dtype == FDVLM_KV_F16 ? XF_F16 : XF_BF16;
+  a.kv_type = (int)kv_dtype; a.out_fmt = kv_dtype == FDVLM_KV_F16 ? XF_F16 : XF_BF16; a.long_cache = -1;
   a.q = q; a.kc = k_cache; a.vc = v_cache; a.out = out; a.n = n_rows; a.cache_len = cache_len; a.max_seq = max_seq;
   a.hq = n_q_heads; a.hkv = n_kv_heads; a.d = head_dim; a.causal = causal ? 1 : 0; a.dtype = (int)dtype; a.workspace = workspace;
   cudaError_t e;

@@ -117,7 +117,7 @@ static int forward_rows_simt(fdvlm_t* h, int n, int mode, int logits_rows) {
     memset(&at, 0, sizeof(at));
     at.q = h->q; at.kc = kv_ptr(h, l, 0); at.vc = kv_ptr(h, l, 1); at.out = h->ao; at.n = n; at.cache_len = h->cache_len;
     at.max_seq = c.max_seq; at.hq = c.n_q_heads; at.hkv = c.n_kv_heads; at.d = d; at.causal = (mode == MODE_CAUSAL);
-    at.dtype = dt; at.workspace = h->ws; at.kv_type = KV_BF16; at.out_fmt = XF_BF16;
+    at.dtype = dt; at.workspace = h->ws; at.kv_type = KV_BF16; at.out_fmt = XF_BF16; at.long_cache = -1;
     prof_begin(h, 1);
     int r = launch_attention(at, h->st, &e);
     prof_end(h);
@@ -160,7 +160,8 @@ static int forward_rows_simt(fdvlm_t* h, int n, int mode, int logits_rows) {
 //            [down GEMM -> partials] [sum + residual + gain + ssq]
 // head:      [LM-head GEMM, folded final norm, logits + softmax statistics epilogue] [statistics merge]
 // stamped: every launch gets the next record of h->stamps (in-chain timing, fdvlm_profile_enable(h, 2)).
-static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int want_logits, const int* len_ptr, bool stamped) {
+static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int want_logits, const int* len_ptr, bool stamped,
+                           int long_cache = -1) {
   const fdvlm_config& c = h->cfg;
   const int H = c.hidden, I = c.intermediate, d = c.head_dim, nt = h->nt;
   const int NQ = c.n_q_heads * d, NKV = c.n_kv_heads * d, NQKV = NQ + 2 * NKV;
@@ -215,6 +216,7 @@ static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int wan
     at.max_seq = c.max_seq; at.hq = c.n_q_heads; at.hkv = c.n_kv_heads; at.d = d; at.causal = (mode == MODE_CAUSAL);
     at.dtype = h->dt; at.workspace = h->ws; at.kv_type = h->kv_type; at.out_fmt = h->xfmt; at.out_lo_off = h->ao_lo;
     at.status = h->info + 3;
+    at.long_cache = long_cache;
     at.stamp = stamp(FDVLM_K_ATTENTION);
     if (at.stamp && !stamp(FDVLM_K_ATTN_MERGE)) at.stamp = nullptr;     // the launcher uses two consecutive records
     prof_begin(h, 1);
@@ -274,11 +276,13 @@ static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int wan
 // edges are kept.
 static int forward_rows_graph(fdvlm_t* h, int n, int mode, int logits_rows, int want_logits) {
   const int stamped = (h->prof_on == 2) ? 1 : 0;
+  const int long_cache = attention_long_cache(h->cache_len + n) ? 1 : 0;
   launch_set_len(h->dev_len, h->cache_len, h->st);
   h->launches++;
   if (stamped) CU(h, cudaMemsetAsync(h->stamps, 0xFF, sizeof(KStamp) * FDVLM_MAX_STAMPS, h->st));
   for (auto& g : h->graphs) {
-    if (g.n == n && g.mode == mode && g.logits_rows == logits_rows && g.want_logits == want_logits && g.stamped == stamped) {
+    if (g.n == n && g.mode == mode && g.logits_rows == logits_rows && g.want_logits == want_logits && g.stamped == stamped &&
+        g.long_cache == long_cache) {
       if (stamped) {      // the records' kinds are those of the capture: replay the bookkeeping only
         h->stamp_kind = g.kinds;
         h->stamp_used = (int)g.kinds.size();
@@ -290,13 +294,13 @@ static int forward_rows_graph(fdvlm_t* h, int n, int mode, int logits_rows, int 
   }
   const int before = h->launches;
   CU(h, cudaStreamBeginCapture(h->st, cudaStreamCaptureModeThreadLocal));
-  const int rc = forward_rows_tc(h, n, mode, logits_rows, want_logits, h->dev_len, stamped != 0);
+  const int rc = forward_rows_tc(h, n, mode, logits_rows, want_logits, h->dev_len, stamped != 0, long_cache);
   cudaGraph_t graph = nullptr;
   cudaError_t e = cudaStreamEndCapture(h->st, &graph);
   if (rc != FDVLM_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
   if (e != cudaSuccess) return fail(h, FDVLM_ERR_CUDA, "graph capture: %s", cudaGetErrorString(e));
   fdvlm::FwdGraph g;
-  g.n = n; g.mode = mode; g.logits_rows = logits_rows; g.want_logits = want_logits; g.stamped = stamped;
+  g.n = n; g.mode = mode; g.logits_rows = logits_rows; g.want_logits = want_logits; g.stamped = stamped; g.long_cache = long_cache;
   g.launches = h->launches - before; g.exec = nullptr;
   if (stamped) g.kinds = h->stamp_kind;
   e = cudaGraphInstantiate(&g.exec, graph, 0);
@@ -310,7 +314,7 @@ static int forward_rows_graph(fdvlm_t* h, int n, int mode, int logits_rows, int 
 // The kernels of one tensor-core forward enqueued on the handle's stream, cache length taken from the device word:
 // what a caller that is itself capturing the stream (the on-device decode loop) records.
 int forward_rows_enqueue(fdvlm_t* h, int n, int mode, int logits_rows, int want_logits) {
-  return forward_rows_tc(h, n, mode, logits_rows, want_logits, h->dev_len, false);
+  return forward_rows_tc(h, n, mode, logits_rows, want_logits, h->dev_len, false, attention_long_cache(h->cache_len + n) ? 1 : 0);
 }
 
 int forward_rows(fdvlm_t* h, int n, int mode, int logits_rows, int want_logits) {

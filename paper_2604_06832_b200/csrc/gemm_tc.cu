@@ -152,8 +152,7 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
     for (int c = 0; c < TC_NCONV; ++c) { mbar_init(cfull_bar(c), helpers ? 8 : 4); mbar_init(cempty_bar(c), 1); }
     for (int pr = 0; pr < 2; ++pr) { mbar_init(exw_bar(pr), 2); mbar_init(exr_bar(pr), 2); }
     stamp_start(p.stamp);
-    // status[1] is written by the host only (never by a kernel of the chain), so it may be read before the wait
-    *abort_flag = (p.status && *reinterpret_cast<const volatile int*>(p.status + 1) != 0) ? 1 : 0;
+    *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -165,7 +164,8 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
-  const bool poisoned = *abort_flag != 0;   // every role then leaves by its give-up path without issuing anything
+  // Dependents may start only now that this CTA holds its tensor memory: a successor CTA that allocated first and then
+  // waited for this grid could otherwise keep it from ever getting any.
   pdl_trigger();
 
   const int total_tiles = p.tile_begin[p.n_mats];
@@ -175,7 +175,6 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
   auto convert_all = [&](int cvt_tid) -> bool {
     int stage = 0, cbuf = 0;
     uint32_t phase = 0, cphase = 0;
-    if (poisoned) return false;
     for (int it = blockIdx.x; it < n_items; it += gridDim.x) {
       const int split = it / total_tiles;
       const int kb0 = split * kbps;
@@ -200,6 +199,11 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
     // ------------------------------------------------ TMA producer ------------------------------------------------
     if (lane == 0) {
       const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
+      // The host-set test hook (status[1]; written by the host only, never by a kernel of the chain, so it may be read
+      // before the wait): the producer issues nothing and raises the abort flag, which every other role's first wait
+      // sees -- all leave by the path a timed-out wait takes.  Only this thread pays for the read.
+      const bool poisoned = p.status && *reinterpret_cast<const volatile int*>(p.status + 1) != 0;
+      if (poisoned) *abort_flag = 1;
       int stage = 0;
       uint32_t phase = 0;
       uint32_t armed = 0;           // bit s: full[s] armed and not yet known complete
@@ -222,7 +226,12 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
         }
         const int kb0 = split * p.kb_per_split;
         const int kb1 = min(p.kblocks, kb0 + p.kb_per_split);
-        for (int kb = kb0; kb < kb1; ++kb) {
+        // Every CTA walks its k-blocks from a different starting point (and wraps): the activation tile of a k-block
+        // is the same few L2 lines for all CTAs, and in lockstep they would all ask for them at the same moment.
+        const int nkb = kb1 - kb0;
+        const int rot = (int)((blockIdx.x * 7u) % (unsigned)nkb);
+        for (int j = 0; j < nkb; ++j) {
+          const int kb = kb0 + ((j + rot) >= nkb ? j + rot - nkb : j + rot);
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t a_dst = base + stage * L::STAGE_BYTES;
           mbar_expect_tx(full_bar(stage), stage_tx);
@@ -276,7 +285,7 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
       int stage = 0, cbuf = 0;
       uint32_t phase = 0, cphase = 0;
       int local = 0;
-      bool ok = !poisoned;
+      bool ok = true;
       for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++local) {
         const int split = it / total_tiles;
         const int acc = local & 1;
@@ -316,7 +325,7 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
     // ------------------------------------------------ epilogue warps ----------------------------------------------
     const int q = warp & 3;  // TMEM lane quarter this warp may read
     int local = 0;
-    bool ok = !poisoned;
+    bool ok = true;
     if (helpers) ok = convert_all(128 + (int)threadIdx.x - 64);
     pdl_wait();   // the epilogue reads the predecessor's row statistics and overwrites buffers it may still be reading
     // folded RMSNorm: lane l keeps the factor of rows l and l + 32; broadcast by shuffle where needed
@@ -490,8 +499,7 @@ static EncodeTiledFn encode_fn() {
 // 2-D row-major [rows, cols] tensor, box {64 columns, box_rows}, zero OOB fill.  16-bit elements (kind 0 = bf16,
 // 2 = f16): 128-byte swizzle (rows of the box are 128 bytes); e4m3 bytes (kind 1): no swizzle (rows of 64 bytes,
 // widened by the converter warps).
-enum { TM_BF16 = 0, TM_E4M3 = 1, TM_F16 = 2 };
-static bool make_tmap(CUtensorMap* tm, const void* ptr, int rows, int cols, int box_rows, int kind = TM_BF16) {
+bool make_tmap(CUtensorMap* tm, const void* ptr, int rows, int cols, int box_rows, int kind) {
   typedef std::tuple<const void*, int, int, int, int> Key;
   static std::map<Key, CUtensorMap> cache;
   static std::mutex mu;

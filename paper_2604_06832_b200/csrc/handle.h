@@ -26,11 +26,11 @@ struct fdvlm {
   char* slab;      // one allocation behind every device buffer below except the KV cache
   int32_t* dev_len;   // device copy of cache_len, read by the captured forward graphs
   int use_graphs;     // tensor-core path: replay one captured CUDA graph per (rows, mode, logits mode)
-  struct FwdGraph { int n, mode, logits_rows, want_logits, stamped, launches; cudaGraphExec_t exec; std::vector<int> kinds; };
+  struct FwdGraph { int n, mode, logits_rows, want_logits, stamped, long_cache, launches; cudaGraphExec_t exec; std::vector<int> kinds; };
   std::vector<FwdGraph> graphs;
   // on-device decode loop (fdvlm_decode_block): a graph whose conditional WHILE node repeats the denoise step
   cudaGraphExec_t loop_exec;
-  int loop_n, loop_rule, loop_k, loop_shift, loop_body_launches;
+  int loop_n, loop_rule, loop_k, loop_shift, loop_long, loop_body_launches;
   float loop_threshold;
   // device buffers (R = max_block rows)
   char* kv;        // [n_layers][2][Hkv][max_seq][d]

@@ -1,5 +1,6 @@
 // Launchers of the fdvlm kernels (host-callable; all asynchronous on `st`).
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stddef.h>
 #include <stdint.h>
@@ -78,6 +79,11 @@ struct TcOut {
                  // start, non-zero sends every role down its give-up path at once
   KStamp* stamp; // in-chain timing of the launch, nullable
 };
+// Tensor map of a 2-D row-major [rows, cols] tensor with box {64 columns, box_rows}, zero fill outside the tensor
+// (cached per argument set).  kind TM_BF16 / TM_F16: 16-bit elements, 128-byte swizzle; TM_E4M3: bytes, no swizzle.
+// False when the driver entry point is missing or the encode fails.
+enum { TM_BF16 = 0, TM_E4M3 = 1, TM_F16 = 2 };
+bool make_tmap(CUtensorMap* tm, const void* ptr, int rows, int cols, int box_rows, int kind = TM_BF16);
 bool tc_linear_supported(int m, int n, int k, int dtype);
 // Split-K workspace of a group with m rows, output width ld, `tiles` 128-row weight tiles and depth k.
 size_t tc_workspace_bytes(int m, int ld, int tiles, int k);
@@ -106,11 +112,14 @@ struct AttnArgs {
   int kv_type;          // tensor-core kernel: element type of q, kc, vc (KV_BF16 / KV_F16)
   int out_fmt;          // tensor-core kernel: storage of `out` (XF_*), lo plane out_lo_off elements on
   size_t out_lo_off;
+  int long_cache;       // tensor-core kernel: -1 pick the CTA shape from cache_len; 0 / 1 the short- / long-cache shape
+                        // (a captured launch serves every later length of its class)
   void* workspace;
   const int* len_ptr;   // nullable: device word holding the cache length (overrides cache_len; tensor-core kernel only)
   int* status;          // nullable: device status words (see TcOut::status)
   KStamp* stamp;        // nullable: two consecutive entries (attention, chunk merge)
 };
 size_t attention_workspace_bytes(int n, int hq, int hkv, int d);
+bool attention_long_cache(int keys);   // whether the tensor-core kernel takes its long-cache shape for this many keys
 
 }  // namespace fdk
