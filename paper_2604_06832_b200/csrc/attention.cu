@@ -12,19 +12,12 @@
 // byte crosses from L2 half as often and the whole chunk is in flight from the start).
 // Every mbarrier wait is bounded; a wait that gives up records ST_ATTENTION in the status word and the CTA drains its
 // copies in flight and returns.
+#include "attn_plan.cuh"
 #include "kernels.h"
 #include "tc_ptx.cuh"
 
 namespace fdk {
 
-constexpr int AT_KEYS = 64;    // keys per shared-memory tile
-constexpr float LOG2E = 1.4426950408889634f;
-
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
@@ -62,16 +55,6 @@ __device__ __forceinline__ uint32_t swz_q(int row, int chunk) {
 // chunks XOR-swizzled by the key's row (the 128-byte swizzle of the tensor map)
 __device__ __forceinline__ uint32_t swz_kv(int row, int chunk) {
   return (uint32_t)((chunk >> 3) * (AT_KEYS * 128) + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
-}
-
-// Split of T keys into chunks of whole 64-key tiles, at most `bound` chunks (the same on host and device, so a launch
-// whose grid was sized for `bound` can take the sequence length from device memory).
-__host__ __device__ inline void attn_chunking(int T, int bound, int* chunk_keys, int* n_chunks) {
-  const int tiles = (T + AT_KEYS - 1) / AT_KEYS;
-  int want = bound < tiles ? bound : tiles;
-  if (want < 1) want = 1;
-  *chunk_keys = ((tiles + want - 1) / want) * AT_KEYS;
-  *n_chunks = (T + *chunk_keys - 1) / *chunk_keys;
 }
 
 template <int D, int ROWS>
@@ -409,6 +392,19 @@ __global__ void __launch_bounds__(128) attn_combine_kernel(const float* __restri
 }
 
 // ---- host side -------------------------------------------------------------------------------------
+// The chunk merge that follows either attention kernel.  grid_x: the chunk slots the partials were laid out for.
+cudaError_t launch_attn_combine(const float* part_o, const float2* part_ml, const AttnArgs& a, int n_chunks, int grid_x,
+                                KStamp* stamp, cudaStream_t st) {
+  cudaError_t e;
+  if (a.d == 128)
+    e = launch_pdl(attn_combine_kernel<128>, dim3((a.n * a.hq + 3) / 4), dim3(128), 0, st, part_o, part_ml, a.out, a.out_lo_off, a.out_fmt,
+                   a.n, a.hq, n_chunks, a.len_ptr, grid_x, stamp);
+  else
+    e = launch_pdl(attn_combine_kernel<64>, dim3((a.n * a.hq + 3) / 4), dim3(128), 0, st, part_o, part_ml, a.out, a.out_lo_off, a.out_fmt,
+                   a.n, a.hq, n_chunks, a.len_ptr, grid_x, stamp);
+  return e != cudaSuccess ? e : cudaGetLastError();
+}
+
 // CTAs of 128 rows once the keys make more than this many tiles per 64-row CTA (all SMs busy either way)
 constexpr int AT_LONG_KEYS = 3072;
 
@@ -476,10 +472,7 @@ static cudaError_t attn_launch_t(const AttnArgs& a, const AttnPlan& pl, cudaStre
   dim3 grid(grid_x, pl.groups, a.hkv);
   e = launch_pdl(attn_mma_kernel<D, E, ROWS>, grid, dim3(S::THREADS), (size_t)S::TOTAL, st, p);
   if (e != cudaSuccess) return e;
-  e = launch_pdl(attn_combine_kernel<D>, dim3((a.n * a.hq + 3) / 4), dim3(128), 0, st, (const float*)p.part_o, (const float2*)p.part_ml,
-                 a.out, a.out_lo_off, a.out_fmt, a.n, a.hq, pl.n_chunks, a.len_ptr, grid_x, a.stamp ? a.stamp + 1 : nullptr);
-  if (e != cudaSuccess) return e;
-  return cudaGetLastError();
+  return launch_attn_combine(p.part_o, p.part_ml, a, pl.n_chunks, grid_x, a.stamp ? a.stamp + 1 : nullptr, st);
 }
 
 template <int D, typename E>
@@ -491,8 +484,8 @@ bool attention_long_cache(int keys) { return keys > AT_LONG_KEYS; }
 
 int launch_attention_mma(const AttnArgs& a, cudaStream_t st, cudaError_t* err) {
   const bool long_cache = a.long_cache >= 0 ? a.long_cache != 0 : attention_long_cache(a.cache_len + a.n);
-  const AttnPlan pl = attn_plan(a.n, a.cache_len + a.n, a.hq, a.hkv, long_cache);
   if (!a.workspace) { *err = cudaErrorInvalidValue; return -1; }
+  const AttnPlan pl = attn_plan(a.n, a.cache_len + a.n, a.hq, a.hkv, long_cache);
   if (a.kv_type == KV_F16) *err = (a.d == 128) ? attn_launch_r<128, __half>(a, pl, st) : attn_launch_r<64, __half>(a, pl, st);
   else *err = (a.d == 128) ? attn_launch_r<128, bf16>(a, pl, st) : attn_launch_r<64, bf16>(a, pl, st);
   return *err == cudaSuccess ? 2 : -1;
