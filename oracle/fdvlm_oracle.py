@@ -63,6 +63,36 @@ def decode_e4m3(bits: np.ndarray) -> np.ndarray:
     return _E4M3[bits]
 
 
+def round_e4m3(v: np.ndarray) -> np.ndarray:
+    """Nearest OCP e4m3fn value of every element (ties to the even mantissa), saturating at +-448.
+
+    The format has 3 mantissa bits, normal exponents 2^-6 .. 2^8 and subnormals in steps of 2^-9, so the spacing at
+    |v| in [2^e, 2^(e+1)) is 2^(e-3) with e clamped to >= -6.  Input and the rounding decision are float32 (the type
+    in which the quantised path forms the value it rounds); the result is returned exactly, as float64."""
+    v = np.asarray(v, dtype=np.float32)
+    a = np.abs(v)
+    _, ex = np.frexp(a)                                  # a = m * 2^ex, m in [0.5, 1)
+    e = np.clip(ex.astype(np.int32) - 1, -6, 8)
+    quantum = np.ldexp(np.float32(1.0), e - 3).astype(np.float32)
+    q = np.rint(a / quantum) * quantum                   # power-of-two scaling: exact; rint rounds half to even
+    q = np.minimum(q, np.float32(448.0))
+    return np.copysign(q, v).astype(np.float64)
+
+
+def quantize_rows_e4m3(a: np.ndarray) -> np.ndarray:
+    """Per-token (per-row) dynamic FP8 quantisation of an activation matrix, returned de-quantised.
+
+    scale_r = max_k |a_rk| / 448 (1 for an all-zero row), code = e4m3(a / scale_r), value = code * scale_r: the
+    activation half of the W8A8 setting of Sec. 3.4 "System integration" / Sec. 4.5 (the smoothing of SmoothQuant is a
+    per-channel rescaling folded into the preceding norm gain and the weights offline, so nothing of it is left at run
+    time).  The row maximum, the scale, the quotient and the rounding are taken in float32."""
+    a32 = np.asarray(a, dtype=np.float32)
+    amax = np.max(np.abs(a32), axis=-1, keepdims=True)
+    scale = np.where(amax > 0, amax / np.float32(448.0), np.float32(1.0)).astype(np.float32)
+    codes = round_e4m3(a32 / scale)
+    return codes * scale.astype(np.float64)
+
+
 def to_f64(a: np.ndarray) -> np.ndarray:
     """Exact value of a storage array: float32/float64 as is, uint16 = bf16 bits, uint8 = e4m3 bits."""
     if a.dtype == np.uint16:
@@ -173,11 +203,17 @@ class Oracle:
     bq bk bv, g_attn, g_mlp.
     """
 
-    def __init__(self, shape, weights, ftype=np.float64):
+    def __init__(self, shape, weights, ftype=np.float64, act_fp8: bool = False):
+        """act_fp8: the input rows of the four layer projections (QKV, O, gate/up, down) pass through
+        quantize_rows_e4m3 -- W8A8 when the weights are FP8 as well.  The LM head keeps unquantised inputs."""
         self.s = shape
         self.w = weights
         self.ft = ftype
+        self.act_fp8 = act_fp8
         self.reset()
+
+    def _act(self, a: np.ndarray) -> np.ndarray:
+        return quantize_rows_e4m3(a).astype(self.ft) if self.act_fp8 else a
 
     # -- state ---------------------------------------------------------------------------------
     def reset(self):
@@ -227,7 +263,7 @@ class Oracle:
         h = np.array(x, dtype=self.ft, copy=True)
         for l in range(s.n_layers):
             lw = self.w["layers"][l]
-            a = rmsnorm(h, self._vec(lw["g_attn"]), s.rms_eps)
+            a = self._act(rmsnorm(h, self._vec(lw["g_attn"]), s.rms_eps))
             q = a @ self._lin(l, "wq").T
             k = a @ self._lin(l, "wk").T
             v = a @ self._lin(l, "wv").T
@@ -240,10 +276,10 @@ class Oracle:
             v = v.reshape(n, s.n_kv_heads, s.head_dim)
             k_all = np.concatenate([self.K[l], k], axis=0)
             v_all = np.concatenate([self.V[l], v], axis=0)
-            o = attend(q, k_all, v_all, allowed).reshape(n, s.n_q_heads * s.head_dim)
+            o = self._act(attend(q, k_all, v_all, allowed).reshape(n, s.n_q_heads * s.head_dim))
             h = h + o @ self._lin(l, "wo").T
-            m = rmsnorm(h, self._vec(lw["g_mlp"]), s.rms_eps)
-            act = silu(m @ self._lin(l, "w_gate").T) * (m @ self._lin(l, "w_up").T)
+            m = self._act(rmsnorm(h, self._vec(lw["g_mlp"]), s.rms_eps))
+            act = self._act(silu(m @ self._lin(l, "w_gate").T) * (m @ self._lin(l, "w_up").T))
             h = h + act @ self._lin(l, "w_down").T
             if update_cache:
                 self.K[l], self.V[l] = k_all, v_all

@@ -126,7 +126,7 @@ __global__ void __launch_bounds__(AtSmem<D, ROWS>::THREADS, ROWS == 64 ? 2 : 1) 
   if (warp == NW) {
     // ------------------------------------------------ TMA producer ------------------------------------------------
     if (lane == 0) {
-      const uint64_t pol = policy_evict_first();
+      const uint64_t pol = policy_evict_last();     // the cache is read again by the other head groups and by the next step
       // The host-set test hook (status[1], never written by a kernel): the producer issues nothing and raises the
       // abort flag, so every wait of the compute warps gives up.  Only this thread pays for the read, off the
       // critical path of the others.

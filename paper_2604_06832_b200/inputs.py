@@ -98,6 +98,8 @@ WORKLOADS: Dict[str, Workload] = {
     # prefix.  About 0.75 GB (bf16) of weights per forward -- larger than L2, small enough for a counter capture.
     "prof_3b_bf16_4layers": Workload("prof_3b_bf16_4layers", QWEN3B.with_(n_layers=4, vocab=32768, mask_id=32767), 1, 16,
                                      96, 32, 64, (32,), "topk"),
+    "prof_3b_bf16_4layers_p8192": Workload("prof_3b_bf16_4layers_p8192", QWEN3B.with_(n_layers=4, vocab=32768, mask_id=32767), 1, 18,
+                                           7168, 1024, 64, (32,), "topk"),
     "prof_7b_fp8_4layers": Workload("prof_7b_fp8_4layers", QWEN7B_FP8.with_(n_layers=4, vocab=32768, mask_id=32767), 5, 17,
                                     96, 32, 64, (32,), "topk"),
 }
