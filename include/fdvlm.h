@@ -59,7 +59,13 @@ typedef enum {
 typedef enum {
   FDVLM_F32 = 0,
   FDVLM_BF16 = 1,
-  FDVLM_W_FP8E4M3 = 2 /* OCP e4m3fn bytes + fp32 per-output-channel scale: w = e4m3(byte) * scale[out] */
+  FDVLM_W_FP8E4M3 = 2, /* OCP e4m3fn bytes + fp32 per-output-channel scale: w = e4m3(byte) * scale[out] */
+  /* W8A8 (Sec. 3.4 "System integration", Sec. 4.5): weights as FDVLM_W_FP8E4M3, and the input rows of the four layer
+   * projections (QKV, O, gate/up, down) quantised per token to e4m3 -- scale = max|row| / 448 over the row as stored
+   * (f16), code = e4m3(x / scale), float32 quotient, round to nearest even, saturating -- so that those GEMMs run
+   * e4m3 x e4m3 on the tensor cores.  The LM head keeps 16-bit input rows.  Needs shapes the tensor-core kernels
+   * take (FDVLM_ERR_UNSUPPORTED otherwise).  Of the single operators below only fdvlm_op_linear takes this value. */
+  FDVLM_W8A8_FP8E4M3 = 3
 } fdvlm_dtype;
 
 /* Element type of the KV cache (and of q, and of the attention probabilities in the P.V product) for the bf16 /
@@ -261,7 +267,10 @@ const char *fdvlm_last_error(const fdvlm_t *h);
  * The call is asynchronous; fdvlm_op_linear_status(workspace, stream) waits for the stream and returns
  * FDVLM_ERR_TIMEOUT if a bounded wait inside the kernels of the LAST call on that workspace gave up (y is then
  * undefined), else FDVLM_OK.  workspace = NULL asks about the built-in scratch of fdvlm_op_linear_static on the
- * current device. */
+ * current device.
+ * dtype = FDVLM_W8A8_FP8E4M3: w and scale as for fp8 weights; the bf16 rows of x are first stored as f16 (saturating)
+ * and each row is then quantised to e4m3 with its own scale max|row| / 448 inside the GEMM kernel, which multiplies
+ * e4m3 by e4m3; FDVLM_ERR_UNSUPPORTED where the tensor-core kernel does not take the shape (k not a multiple of 16). */
 int fdvlm_op_linear(const void *x, const void *w, const float *scale, const float *bias, float *y,
                     int m, int n, int k, fdvlm_dtype dtype, void *workspace, void *cuda_stream);
 size_t fdvlm_op_linear_workspace_bytes(int m, int n, int k, fdvlm_dtype dtype);

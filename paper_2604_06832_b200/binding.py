@@ -20,12 +20,12 @@ LIB_PATH = os.path.join(_HERE, "libfdvlm.so")
 
 FDVLM_OK = 0
 ERR_INVALID_ARG, ERR_STATE, ERR_CAPACITY, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_OOM = -1, -2, -3, -4, -5, -6, -7
-DT_F32, DT_BF16, DT_FP8 = 0, 1, 2
+DT_F32, DT_BF16, DT_FP8, DT_W8A8 = 0, 1, 2, 3
 KV_BF16, KV_F16 = 0, 1
 RULE_THRESHOLD, RULE_TOPK = 0, 1
 KERNEL_KINDS = ("rope_table", "gemm_qkv", "fin_qkv", "attention", "attn_merge", "gemm_o", "fin_resid", "gemm_gate_up",
                 "gemm_down", "gemm_lm_head", "stats_merge")
-_DTYPE_CODE = {_in.F32: DT_F32, _in.BF16: DT_BF16, _in.FP8: DT_FP8}
+_DTYPE_CODE = {_in.F32: DT_F32, _in.BF16: DT_BF16, _in.FP8: DT_FP8, _in.W8A8: DT_W8A8}
 
 
 class Config(C.Structure):

@@ -313,7 +313,7 @@ __global__ void __launch_bounds__(AtSmem<D, ROWS>::THREADS, ROWS == 64 ? 2 : 1) 
 // The result is stored as `fmt` (XF_*) at element offset out_idx of `out`.
 template <int D>
 __device__ __forceinline__ void attn_merge_warp(const float* att_o, const float2* att_ml, void* out, size_t out_idx, size_t lo_off,
-                                                int fmt, size_t slot0, int n_chunks, int lane) {
+                                                int fmt, size_t slot0, int n_chunks, int lane, float* amax_out = nullptr) {
   constexpr int VPL = D / 32;
   constexpr int CB = 16;     // chunks whose partial outputs are in flight together
   // The statistics and the first CB partial outputs are requested together: one L2 round trip for up to 16 chunks.
@@ -366,13 +366,21 @@ __device__ __forceinline__ void attn_merge_warp(const float* att_o, const float2
   const float inv = 1.f / den;
 #pragma unroll
   for (int i = 0; i < VPL; ++i) store_act(out, lo_off, out_idx + lane * VPL + i, acc[i] * inv, fmt);
+  if (amax_out) {     // W8A8: the O projection quantises this row; its maximum as stored (f16) over this head
+    float am = 0.f;
+#pragma unroll
+    for (int i = 0; i < VPL; ++i) am = fmaxf(am, fabsf(__half2float(__ushort_as_half(f16_bits_sat(acc[i] * inv)))));
+    am = warp_max(am);
+    if (lane == 0) *amax_out = am;
+  }
 }
 
 // out[i][head] = sum_c w_c O_c / sum_c w_c l_c, w_c = 2^(m_c - max_c m_c): one warp per (row, head), four per CTA
 template <int D>
 __global__ void __launch_bounds__(128) attn_combine_kernel(const float* __restrict__ part_o, const float2* __restrict__ part_ml,
                                                           void* __restrict__ out, size_t lo_off, int fmt, int n, int hq, int n_chunks,
-                                                          const int* __restrict__ len_ptr, int bound, KStamp* stamp) {
+                                                          const int* __restrict__ len_ptr, int bound, float* __restrict__ amax_out,
+                                                          KStamp* stamp) {
   if (threadIdx.x == 0) stamp_start(stamp);
   pdl_trigger();
   if (len_ptr) {
@@ -385,7 +393,7 @@ __global__ void __launch_bounds__(128) attn_combine_kernel(const float* __restri
   if (p < n * hq) {
     const int i = p / hq, head = p % hq;
     attn_merge_warp<D>(part_o, part_ml, out, ((size_t)i * hq + head) * D, lo_off, fmt, ((size_t)head * n + i) * n_chunks, n_chunks,
-                       threadIdx.x & 31);
+                       threadIdx.x & 31, amax_out ? amax_out + (size_t)i * hq + head : nullptr);
   }
   __syncthreads();
   if (threadIdx.x == 0) stamp_end(stamp, true);
@@ -398,10 +406,10 @@ cudaError_t launch_attn_combine(const float* part_o, const float2* part_ml, cons
   cudaError_t e;
   if (a.d == 128)
     e = launch_pdl(attn_combine_kernel<128>, dim3((a.n * a.hq + 3) / 4), dim3(128), 0, st, part_o, part_ml, a.out, a.out_lo_off, a.out_fmt,
-                   a.n, a.hq, n_chunks, a.len_ptr, grid_x, stamp);
+                   a.n, a.hq, n_chunks, a.len_ptr, grid_x, a.amax_out, stamp);
   else
     e = launch_pdl(attn_combine_kernel<64>, dim3((a.n * a.hq + 3) / 4), dim3(128), 0, st, part_o, part_ml, a.out, a.out_lo_off, a.out_fmt,
-                   a.n, a.hq, n_chunks, a.len_ptr, grid_x, stamp);
+                   a.n, a.hq, n_chunks, a.len_ptr, grid_x, a.amax_out, stamp);
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 

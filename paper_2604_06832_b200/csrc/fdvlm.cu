@@ -13,7 +13,7 @@ static int check_config(const fdvlm_config* c) {
     return fail(nullptr, FDVLM_ERR_INVALID_ARG, "config: non-positive dimension");
   if (c->head_dim != 64 && c->head_dim != 128) return fail(nullptr, FDVLM_ERR_UNSUPPORTED, "head_dim must be 64 or 128");
   if (c->n_q_heads % c->n_kv_heads) return fail(nullptr, FDVLM_ERR_INVALID_ARG, "n_q_heads not a multiple of n_kv_heads");
-  if (c->dtype != FDVLM_F32 && c->dtype != FDVLM_BF16 && c->dtype != FDVLM_W_FP8E4M3)
+  if (c->dtype != FDVLM_F32 && c->dtype != FDVLM_BF16 && c->dtype != FDVLM_W_FP8E4M3 && c->dtype != FDVLM_W8A8_FP8E4M3)
     return fail(nullptr, FDVLM_ERR_INVALID_ARG, "unknown dtype %d", (int)c->dtype);
   int mult = c->dtype == FDVLM_F32 ? 8 : 16;
   if (c->hidden % mult || c->intermediate % mult)
@@ -52,7 +52,8 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
   if (!w->embed || !w->g_final || !w->layers) return fail(nullptr, FDVLM_ERR_INVALID_ARG, "weights: NULL embed / g_final / layers");
   if (cfg->tie_embeddings ? (w->lm_head != nullptr) : (w->lm_head == nullptr))
     return fail(nullptr, FDVLM_ERR_INVALID_ARG, "lm_head must be NULL exactly when tie_embeddings is set");
-  if (cfg->dtype == FDVLM_W_FP8E4M3 && !cfg->tie_embeddings && !w->s_lm_head)
+  const bool w8 = cfg->dtype == FDVLM_W_FP8E4M3 || cfg->dtype == FDVLM_W8A8_FP8E4M3;
+  if (w8 && !cfg->tie_embeddings && !w->s_lm_head)
     return fail(nullptr, FDVLM_ERR_INVALID_ARG, "fp8 lm_head needs s_lm_head");
   for (int l = 0; l < cfg->n_layers; ++l) {
     const fdvlm_layer_weights& lw = w->layers[l];
@@ -60,7 +61,7 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
       return fail(nullptr, FDVLM_ERR_INVALID_ARG, "layer %d: NULL weight", l);
     int nb = (lw.bq != nullptr) + (lw.bk != nullptr) + (lw.bv != nullptr);
     if (nb != 0 && nb != 3) return fail(nullptr, FDVLM_ERR_INVALID_ARG, "layer %d: biases must be all NULL or all set", l);
-    if (cfg->dtype == FDVLM_W_FP8E4M3 && (!lw.s_q || !lw.s_k || !lw.s_v || !lw.s_o || !lw.s_gate || !lw.s_up || !lw.s_down))
+    if (w8 && (!lw.s_q || !lw.s_k || !lw.s_v || !lw.s_o || !lw.s_gate || !lw.s_up || !lw.s_down))
       return fail(nullptr, FDVLM_ERR_INVALID_ARG, "layer %d: fp8 weights need all scales", l);
   }
   int ndev = 0;
@@ -74,7 +75,8 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
   h->w = *w;
   h->w.layers = h->layers.data();
   h->st = (cudaStream_t)cuda_stream;
-  h->dt = (int)cfg->dtype;
+  h->act8 = cfg->dtype == FDVLM_W8A8_FP8E4M3 ? 1 : 0;       // W8A8 = the fp8-weight path with quantised projection inputs
+  h->dt = h->act8 ? DT_FP8 : (int)cfg->dtype;
   h->act_sz = cfg->dtype == FDVLM_F32 ? 4 : 2;
   h->err[0] = 0;
   h->cache_len = h->block_size = h->n_remaining = h->step_index = h->block_open = 0;
@@ -82,6 +84,7 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
   h->prof_on = 0;
   h->prof_used = 0;
   h->kv = nullptr; h->h = nullptr; h->a = h->ao = h->act = h->q = nullptr; h->y = nullptr; h->cs = nullptr; h->ssq = nullptr;
+  h->amax_a = h->amax_ao = h->amax_act = nullptr;
   h->stats = nullptr; h->logits = nullptr; h->conf = nullptr; h->pred = nullptr; h->unmask = nullptr; h->blk_tokens = nullptr;
   h->blk_masked = nullptr; h->info = nullptr; h->init_stage = nullptr; h->ws = nullptr; h->info_host = nullptr;
   h->host_stage = nullptr;
@@ -96,6 +99,7 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
   const int R = cfg->max_block, H = cfg->hidden, I = cfg->intermediate, d = cfg->head_dim;
   const int NQ = cfg->n_q_heads * d, NKV = cfg->n_kv_heads * d, NQKV = NQ + 2 * NKV;
   h->nt = (H + 127) / 128;
+  h->n_gu = 2 * ((I + 63) / 64);
   size_t ws = 0;
   const int shapes[][2] = {{NQ, H}, {NKV, H}, {H, NQ}, {I, H}, {H, I}, {cfg->vocab, H}};
   for (auto& s : shapes) { size_t b = linear_workspace_bytes(R, s[0], s[1], h->dt); if (b > ws) ws = b; }
@@ -103,6 +107,10 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
   if (wa > ws) ws = wa;
   h->use_tc = (h->dt == DT_BF16 || h->dt == DT_FP8) && tc_linear_supported(R, NQ, H, h->dt) && tc_linear_supported(R, H, I, h->dt);
   h->kv_type = (int)cfg->kv_dtype;
+  if (h->act8 && !h->use_tc) {
+    delete h;
+    return fail(nullptr, FDVLM_ERR_UNSUPPORTED, "W8A8 needs shapes the tensor-core kernels take");
+  }
   if (!h->use_tc && h->dt != DT_F32 && h->kv_type != KV_BF16) {
     delete h;
     return fail(nullptr, FDVLM_ERR_UNSUPPORTED, "an f16 KV cache needs shapes the tensor-core kernels take");
@@ -131,6 +139,9 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
       {(void**)&h->blk_masked, 64},
       {(void**)&h->init_stage, 64 * 4},
       {(void**)&h->ssq, (size_t)R * h->nt * 4},
+      {(void**)&h->amax_a, h->act8 ? (size_t)R * h->nt * 4 : 16},
+      {(void**)&h->amax_ao, h->act8 ? (size_t)R * cfg->n_q_heads * 4 : 16},
+      {(void**)&h->amax_act, h->act8 ? (size_t)R * h->n_gu * 4 : 16},
       {(void**)&h->cs, (size_t)R * d * 4},
       {(void**)&h->stamps, h->use_tc ? sizeof(KStamp) * FDVLM_MAX_STAMPS : 16},
       {(void**)&h->h, (size_t)R * H * 4},
@@ -649,15 +660,16 @@ extern "C" size_t fdvlm_op_linear_workspace_bytes(int m, int n, int k, fdvlm_dty
 extern "C" int fdvlm_op_linear(const void* x, const void* w, const float* scale, const float* bias, float* y, int m,
                                int n, int k, fdvlm_dtype dtype, void* workspace, void* cuda_stream) {
   if (!x || !w || !y || m < 1 || m > 64 || n < 1 || k < 8 || (k % 8)) return FDVLM_ERR_INVALID_ARG;
-  if (dtype != FDVLM_F32 && dtype != FDVLM_BF16 && dtype != FDVLM_W_FP8E4M3) return FDVLM_ERR_INVALID_ARG;
-  if (dtype == FDVLM_W_FP8E4M3 && !scale) return FDVLM_ERR_INVALID_ARG;
+  if (dtype != FDVLM_F32 && dtype != FDVLM_BF16 && dtype != FDVLM_W_FP8E4M3 && dtype != FDVLM_W8A8_FP8E4M3) return FDVLM_ERR_INVALID_ARG;
+  if ((dtype == FDVLM_W_FP8E4M3 || dtype == FDVLM_W8A8_FP8E4M3) && !scale) return FDVLM_ERR_INVALID_ARG;
   LinearArgs a;
   a.x = x; a.w = w; a.scale = scale; a.bias = bias; a.y = y; a.m = m; a.n = n; a.k = k; a.ldy = n; a.accumulate = 0;
   a.dtype = (int)dtype; a.workspace = workspace; a.workspace_bytes = linear_workspace_bytes(m, n, k, (int)dtype);
   if (!workspace) return FDVLM_ERR_INVALID_ARG;
   cudaError_t e;
   int r = launch_linear(a, (cudaStream_t)cuda_stream, &e);
-  return r < 0 ? FDVLM_ERR_CUDA : FDVLM_OK;
+  if (r < 0) return e == cudaErrorNotSupported ? FDVLM_ERR_UNSUPPORTED : FDVLM_ERR_CUDA;
+  return FDVLM_OK;
 }
 
 extern "C" size_t fdvlm_op_attention_workspace_bytes(int n_rows, int n_q_heads, int n_kv_heads, int head_dim) {

@@ -11,19 +11,21 @@ int launch_attention_simt(const AttnArgs& a, cudaStream_t st, cudaError_t* err);
 size_t attention_mma_workspace_bytes(int n, int hq, int hkv, int d);
 int launch_attention_mma(const AttnArgs& a, cudaStream_t st, cudaError_t* err);
 void launch_splitk_epilogue(const float* part, int S, int m, int n, const float* scale, const float* bias, float* y, int ldy,
-                            int accumulate, cudaStream_t st);
+                            int accumulate, cudaStream_t st, const float* row_amax = nullptr);
 
 thread_local char g_create_error[512] = "";
 
 // Stand-alone projection.  The caller's workspace starts with OP_HEAD bytes for the two status words (see
-// TcOut::status; cleared here on the stream), then -- fp8 weights only -- an f16 copy of the bf16 rows, then the
-// split-K partial sums.
+// TcOut::status; cleared here on the stream), then -- fp8 weights only -- an f16 copy of the bf16 rows (W8A8: followed
+// by one 256-byte-rounded array of per-row maxima), then the split-K partial sums.
+static size_t op_amax_bytes(int m, int dtype) { return dtype == DT_A8 ? (((size_t)m * 4 + 255) / 256) * 256 : 0; }
 static size_t op_x16_bytes(int m, int k, int dtype) {
-  return dtype == DT_FP8 ? (((size_t)m * k * 2 + 255) / 256) * 256 : 0;
+  return (dtype == DT_FP8 || dtype == DT_A8) ? (((size_t)m * k * 2 + 255) / 256) * 256 + op_amax_bytes(m, dtype) : 0;
 }
 size_t linear_workspace_bytes(int m, int n, int k, int dtype) {
-  size_t a = simt_workspace_bytes(m, n, k);
-  size_t b = tc_linear_supported(m, n, k, dtype) ? tc_workspace_bytes(m, n, (n + 127) / 128, k) + op_x16_bytes(m, k, dtype) : 0;
+  const int wdt = dtype == DT_A8 ? DT_FP8 : dtype;
+  size_t a = dtype == DT_A8 ? 0 : simt_workspace_bytes(m, n, k);
+  size_t b = tc_linear_supported(m, n, k, wdt) ? tc_workspace_bytes(m, n, (n + 127) / 128, k) + op_x16_bytes(m, k, dtype) : 0;
   return OP_HEAD + (a > b ? a : b);
 }
 
@@ -36,15 +38,24 @@ int launch_linear(const LinearArgs& a, cudaStream_t st, cudaError_t* err) {
   LinearArgs b = a;
   b.workspace = (char*)a.workspace + OP_HEAD;
   b.workspace_bytes = a.workspace_bytes - OP_HEAD;
-  if (!tc_linear_supported(a.m, a.n, a.k, a.dtype)) return launch_linear_simt(b, st, err);
+  const bool a8 = a.dtype == DT_A8;
+  if (!tc_linear_supported(a.m, a.n, a.k, a8 ? DT_FP8 : a.dtype)) {
+    if (a8) { *err = cudaErrorNotSupported; return -1; }      // the quantising projection exists on the tensor cores only
+    return launch_linear_simt(b, st, err);
+  }
   TcGroup g;
   memset(&g, 0, sizeof(g));
   g.x = a.x; g.m = a.m; g.k = a.k; g.w[0] = a.w; g.n[0] = a.n; g.n_mats = 1;
-  g.fp8 = (a.dtype == DT_FP8);
+  g.fp8 = (a.dtype == DT_FP8 || a8); g.a8 = a8;
   const size_t x16 = op_x16_bytes(a.m, a.k, a.dtype);
   if (b.workspace_bytes < x16) { *err = cudaErrorInvalidValue; return -1; }
+  float* row_amax = a8 ? (float*)((char*)b.workspace + x16 - op_amax_bytes(a.m, a.dtype)) : nullptr;
   int launched = 2;
-  if (g.fp8) {     // the fp8 GEMM multiplies f16 by f16
+  if (a8) {        // f16 rows and each row's maximum: the kernel quantises the rows to e4m3 itself
+    launch_bf16_rows_to_f16_amax(a.x, b.workspace, a.m, a.k, row_amax, st);
+    g.x = b.workspace;
+    ++launched;
+  } else if (g.fp8) {     // the fp8 GEMM multiplies f16 by f16
     launch_bf16_to_f16(a.x, b.workspace, (size_t)a.m * a.k, st);
     g.x = b.workspace;
     ++launched;
@@ -55,9 +66,10 @@ int launch_linear(const LinearArgs& a, cudaStream_t st, cudaError_t* err) {
   memset(&o, 0, sizeof(o));
   o.mode = TC_MODE_PARTIAL; o.part = part; o.part_bytes = b.workspace_bytes - x16; o.splits_out = &splits;
   o.ld = a.n; o.status = (int*)a.workspace;
+  o.amax_in = row_amax; o.n_amax_in = 1;
   *err = tc_group_launch(g, o, st);
   if (*err != cudaSuccess) return -1;
-  launch_splitk_epilogue(part, splits, a.m, a.n, a.scale, a.bias, a.y, a.ldy, a.accumulate, st);
+  launch_splitk_epilogue(part, splits, a.m, a.n, a.scale, a.bias, a.y, a.ldy, a.accumulate, st, row_amax);
   *err = cudaGetLastError();
   return *err == cudaSuccess ? launched : -1;
 }
@@ -73,7 +85,8 @@ int stage_rows(fdvlm_t* h, int row0, int n, const int32_t* tokens, const void* e
   const int edt = h->dt == DT_F32 ? DT_F32 : DT_BF16;
   if (h->use_tc) {
     launch_embed_prep(h->w.embed, tokens, embeds, h->h + (size_t)row0 * H, (char*)h->a + (size_t)row0 * H * 2, h->a_lo, h->xfmt,
-                      h->layers[0].g_attn, h->ssq + (size_t)row0 * h->nt, h->nt, n, H, h->cfg.vocab, h->info + 3, h->st);
+                      h->layers[0].g_attn, h->ssq + (size_t)row0 * h->nt, h->nt, n, H, h->cfg.vocab, h->info + 3, h->st, nullptr,
+                      h->act8 ? h->amax_a + (size_t)row0 * h->nt : nullptr);
   } else if (tokens) {
     launch_embed(h->w.embed, tokens, h->h + (size_t)row0 * H, n, H, edt, h->cfg.vocab, h->info + 3, h->st);
   } else {
@@ -174,6 +187,8 @@ static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int wan
     return h->stamps + h->stamp_used++;
   };
   const bool fp8 = (h->dt == DT_FP8);
+  const bool a8 = h->act8 != 0;                      // W8A8: the four layer projections quantise their input rows
+  const int n_gu = h->n_gu;
   // a GEMM input buffer: hi (or only) plane, and its lo plane when the format has one
   auto group = [&](const void* x, size_t lo_off, size_t row0_elems, int m, int k, int nm, const void* w0, int n0, const void* w1, int n1,
                    const void* w2, int n2) {
@@ -182,7 +197,7 @@ static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int wan
     g.x = (const char*)x + row0_elems * 2; g.m = m; g.k = k; g.n_mats = nm;
     g.x_lo = (h->xfmt == XF_BF16X2) ? (const char*)x + (lo_off + row0_elems) * 2 : nullptr;
     g.w[0] = w0; g.n[0] = n0; g.w[1] = w1; g.n[1] = n1; g.w[2] = w2; g.n[2] = n2;
-    g.fp8 = fp8;
+    g.fp8 = fp8; g.a8 = a8;
     return g;
   };
   auto out = [&](int tc_mode, int kind) {
@@ -205,10 +220,12 @@ static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int wan
     int S = 0;
     TcOut o = out(TC_MODE_PARTIAL, FDVLM_K_GEMM_QKV);
     o.ld = NQKV; o.splits_out = &S;
+    o.amax_in = a8 ? h->amax_a : nullptr; o.n_amax_in = nt;
     if (!gemm(group(h->a, h->a_lo, 0, n, H, 3, lw.wq, NQ, lw.wk, NKV, lw.wv, NKV), o))
       return fail(h, FDVLM_ERR_CUDA, "qkv projection launch: %s", cudaGetErrorString(e));
     launch_fin_qkv(part, S, n, h->cs, h->ssq, nt, H, c.rms_eps, lw.bq, lw.bk, lw.bv, lw.s_q, lw.s_k, lw.s_v, h->q, kv_ptr(h, l, 0), kv_ptr(h, l, 1),
-                   h->cache_len, c.n_q_heads, c.n_kv_heads, d, c.max_seq, h->kv_type, h->st, len_ptr, stamp(FDVLM_K_FIN_QKV));
+                   h->cache_len, c.n_q_heads, c.n_kv_heads, d, c.max_seq, h->kv_type, h->st, len_ptr, stamp(FDVLM_K_FIN_QKV),
+                   a8 ? h->amax_a : nullptr);
     AttnArgs at;
     memset(&at, 0, sizeof(at));
     at.len_ptr = len_ptr;
@@ -216,6 +233,7 @@ static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int wan
     at.max_seq = c.max_seq; at.hq = c.n_q_heads; at.hkv = c.n_kv_heads; at.d = d; at.causal = (mode == MODE_CAUSAL);
     at.dtype = h->dt; at.workspace = h->ws; at.kv_type = h->kv_type; at.out_fmt = h->xfmt; at.out_lo_off = h->ao_lo;
     at.status = h->info + 3;
+    at.amax_out = a8 ? h->amax_ao : nullptr;
     at.long_cache = long_cache;
     at.stamp = stamp(FDVLM_K_ATTENTION);
     if (at.stamp && !stamp(FDVLM_K_ATTN_MERGE)) at.stamp = nullptr;     // the launcher uses two consecutive records
@@ -226,25 +244,29 @@ static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int wan
     h->launches += r + 1;
     o = out(TC_MODE_PARTIAL, FDVLM_K_GEMM_O);
     o.ld = H; o.splits_out = &S;
+    o.amax_in = a8 ? h->amax_ao : nullptr; o.n_amax_in = c.n_q_heads;
     if (!gemm(group(h->ao, h->ao_lo, 0, n, NQ, 1, lw.wo, H, nullptr, 0, nullptr, 0), o))
       return fail(h, FDVLM_ERR_CUDA, "o projection launch: %s", cudaGetErrorString(e));
-    launch_fin_resid(part, S, n, H, h->h, lw.g_mlp, h->a, h->a_lo, h->xfmt, h->ssq, nt, lw.s_o, h->st, stamp(FDVLM_K_FIN_RESID));
+    launch_fin_resid(part, S, n, H, h->h, lw.g_mlp, h->a, h->a_lo, h->xfmt, h->ssq, nt, lw.s_o, h->st, stamp(FDVLM_K_FIN_RESID),
+                     a8 ? h->amax_ao : nullptr, c.n_q_heads, a8 ? h->amax_a : nullptr);
     o = out(TC_MODE_SWIGLU, FDVLM_K_GEMM_GATE_UP);
     o.act = h->act; o.act_lo_off = h->act_lo; o.act_fmt = h->xfmt;
     o.ssq_in = h->ssq; o.nt_in = nt; o.hidden = H; o.eps = c.rms_eps;
+    o.amax_in = a8 ? h->amax_a : nullptr; o.n_amax_in = nt; o.amax_out = a8 ? h->amax_act : nullptr; o.n_amax_out = n_gu;
     TcGroup gu = group(h->a, h->a_lo, 0, n, H, 2, lw.w_gate, I, lw.w_up, I, nullptr, 0);
     gu.scale[0] = lw.s_gate; gu.scale[1] = lw.s_up;
     if (!gemm(gu, o))
       return fail(h, FDVLM_ERR_CUDA, "gate/up projection launch: %s", cudaGetErrorString(e));
     o = out(TC_MODE_PARTIAL, FDVLM_K_GEMM_DOWN);
     o.ld = H; o.splits_out = &S;
+    o.amax_in = a8 ? h->amax_act : nullptr; o.n_amax_in = n_gu;
     if (!gemm(group(h->act, h->act_lo, 0, n, I, 1, lw.w_down, H, nullptr, 0, nullptr, 0), o))
       return fail(h, FDVLM_ERR_CUDA, "down projection launch: %s", cudaGetErrorString(e));
     // the last layer feeds the LM head, whose table (a tied bf16 embedding under fp8 layer weights) may want another format
     const bool last = (l + 1 == c.n_layers);
     const float* g_next = last ? h->w.g_final : h->layers[l + 1].g_attn;
     launch_fin_resid(part, S, n, H, h->h, g_next, h->a, h->a_lo, last ? h->head_fmt : h->xfmt, h->ssq, nt, lw.s_down, h->st,
-                     stamp(FDVLM_K_FIN_RESID));
+                     stamp(FDVLM_K_FIN_RESID), a8 ? h->amax_act : nullptr, n_gu, (a8 && !last) ? h->amax_a : nullptr);
     h->launches += 2;
   }
   if (logits_rows > 0) {
@@ -257,6 +279,7 @@ static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int wan
     o.stats = h->stats; o.mask_id = c.mask_id;
     TcGroup lm = group(h->a, h->a_lo, (size_t)first * H, m, H, 1, table, c.vocab, nullptr, 0, nullptr, 0);
     lm.fp8 = (h->head_fmt == XF_F16);
+    lm.a8 = 0;                                       // the LM head keeps 16-bit input rows
     lm.x_lo = (h->head_fmt == XF_BF16X2) ? (const char*)h->a + (h->a_lo + (size_t)first * H) * 2 : nullptr;
     if (!c.tie_embeddings) lm.scale[0] = h->w.s_lm_head;
     if (!gemm(lm, o))

@@ -64,23 +64,38 @@ struct TcParams {
   int* status;          // device words: [0] set non-zero when a wait timed out; [1] read at start: non-zero makes
                         // every role take its give-up path at once (a host-set test hook for that path)
   KStamp* stamp;        // in-chain timing of this launch (null: off)
+  // TC_KIND_A8: amax_in[row][n_amax_in] = partial maxima of |x[row]| left by the producer of x; the row's quantisation
+  // scale is their maximum / 448.  SWIGLU mode also leaves amax_out[row][n_amax_out] (two per 64-feature tile) for the
+  // consumer of `act`.
+  const float* amax_in; int n_amax_in;
+  float* amax_out; int n_amax_out;
 };
 
-template <int M_PAD, bool FP8>
+// Operand kinds of the kernel:
+//   TC_KIND_BF16: bf16 weights x bf16 hi/lo activation planes
+//   TC_KIND_FP8 : e4m3 weights widened to f16 by converter warps x f16 activations
+//   TC_KIND_A8  : e4m3 weights x activations quantised to e4m3 per row inside the kernel (W8A8, Sec. 3.4 "System
+//                 integration"); a k-block is 128 elements, the byte tile of the weights is the MMA operand as it lands
+enum { TC_KIND_BF16 = 0, TC_KIND_FP8 = 1, TC_KIND_A8 = 2 };
+
+template <int M_PAD, int KIND>
 struct TcSmem {
-  static constexpr int STAGES = FP8 ? 6 : (M_PAD <= 32 ? 4 : 3);       // two CTAs per SM must fit
+  static constexpr bool FP8 = KIND == TC_KIND_FP8, A8 = KIND == TC_KIND_A8;
+  static constexpr int STAGES = FP8 ? 6 : (M_PAD <= 32 ? 4 : 3);       // two CTAs per SM must fit (A8, M_PAD > 32: one)
+  static constexpr int KB_ELEMS = A8 ? 2 * TC_BK : TC_BK;              // k per stage
   static constexpr int W_BYTES = FP8 ? TC_BM * TC_BK : TC_A_BYTES;     // weight tile as it is streamed
-  static constexpr int W_ROW = FP8 ? TC_BK : TC_BK * 2;                // bytes per weight row in the stage
-  static constexpr int B_BYTES = M_PAD * TC_BK * 2;                    // one activation plane
-  static constexpr int X_PLANES = FP8 ? 1 : 2;                         // f16, or bf16 hi + lo
+  static constexpr int B_BYTES = M_PAD * TC_BK * 2;                    // one activation plane (A8: one 64-k half, f16)
+  static constexpr int X_PLANES = FP8 ? 1 : 2;                         // f16; bf16 hi + lo; A8: two 64-k halves
   static constexpr int STAGE_BYTES = W_BYTES + X_PLANES * B_BYTES;
-  static constexpr int CONV_OFF = STAGES * STAGE_BYTES;                // bf16 tiles made by the converters
-  static constexpr int EX_OFF = CONV_OFF + (FP8 ? TC_NCONV * TC_A_BYTES : 0);   // SwiGLU epilogue: gate/up exchange
-  static constexpr int EX_ROWS = FP8 ? 16 : 32;                         // rows that pass through it per round
+  static constexpr int CONV_OFF = STAGES * STAGE_BYTES;                // tiles made by the converters
+  static constexpr int CONV_BYTES = FP8 ? TC_A_BYTES : (A8 ? M_PAD * 128 : 0);   // f16 weight tile / e4m3 activation tile
+  static constexpr int EX_OFF = CONV_OFF + TC_NCONV * CONV_BYTES;      // SwiGLU epilogue: gate/up exchange
+  static constexpr int EX_ROWS = KIND != TC_KIND_BF16 ? 16 : 32;       // rows that pass through it per round
   static constexpr int EX_ROUNDS = (M_PAD + EX_ROWS - 1) / EX_ROWS;
   static constexpr int EX_BYTES = (M_PAD / EX_ROUNDS) * 256;
   static constexpr int BAR_OFF = EX_OFF + EX_BYTES;
-  static constexpr int TOTAL = BAR_OFF + 256 + 1024;  // barriers + alignment slack
+  static constexpr int ROWSC_OFF = BAR_OFF + 256;                      // A8: the rows' quantisation scales (64 floats)
+  static constexpr int TOTAL = ROWSC_OFF + 256 + 1024;  // + alignment slack
 };
 
 // sixteen e4m3 bytes -> sixteen f16 (exact: every e4m3 value, subnormals included, is an f16 value)
@@ -115,10 +130,45 @@ __device__ __forceinline__ void convert_pieces(const uint8_t* src, uint32_t dst,
   }
 }
 
-template <int M_PAD, bool FP8>
-__global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_kernel(const __grid_constant__ TcParams p) {
+// Quantise NP 16-byte pieces (tid, tid + stride, ...) of the activation tile of one stage -- two 128-byte-swizzled f16
+// halves of 64 k each -- into the 128-byte-swizzled e4m3 tile [M_PAD rows][128 k] the MMA reads: code = e4m3(x / scale
+// of the row), float32 quotient, round to nearest even, saturating.
+template <int M_PAD, int NP>
+__device__ __forceinline__ void quantize_pieces(const uint8_t* x_tile, uint32_t dst, const volatile float* row_scale, int tid, int stride) {
+#pragma unroll
+  for (int i = 0; i < NP; ++i) {
+    const int piece = tid + stride * i;
+    if (piece >= M_PAD * 8) break;
+    const int r = piece >> 3, j = piece & 7;                 // row, 16-byte piece (16 k) of the output row
+    const uint8_t* half = x_tile + (j >> 2) * (M_PAD * 128) + r * 128;
+    const int c0 = 2 * (j & 3);
+    const uint4 a = *reinterpret_cast<const uint4*>(half + ((c0 ^ (r & 7)) << 4));
+    const uint4 b = *reinterpret_cast<const uint4*>(half + (((c0 + 1) ^ (r & 7)) << 4));
+    const float sc = row_scale[r];
+    const uint32_t in[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    uint32_t out[4];
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      unsigned short pair[2];
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const __half2 hv = *reinterpret_cast<const __half2*>(&in[2 * w + h]);
+        const float x0 = __fdiv_rn(__low2float(hv), sc), x1 = __fdiv_rn(__high2float(hv), sc);
+        asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(pair[h]) : "f"(x1), "f"(x0));   // first source -> upper byte
+      }
+      out[w] = (uint32_t)pair[0] | ((uint32_t)pair[1] << 16);
+    }
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + r * 128 + ((j ^ (r & 7)) << 4)), "r"(out[0]), "r"(out[1]), "r"(out[2]), "r"(out[3]) : "memory");
+  }
+}
+
+template <int M_PAD, int KIND>
+__global__ void __launch_bounds__(KIND != TC_KIND_BF16 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_kernel(const __grid_constant__ TcParams p) {
   extern __shared__ uint8_t smem_raw[];
-  using L = TcSmem<M_PAD, FP8>;
+  using L = TcSmem<M_PAD, KIND>;
+  constexpr bool A8 = KIND == TC_KIND_A8;
+  constexpr bool FP8 = KIND != TC_KIND_BF16;       // a converter stage sits between the ring and the MMA
+  constexpr bool WIDEN = KIND == TC_KIND_FP8;      // ... which widens the weight tile (A8: quantises the activation tile)
   constexpr int TC_STAGES = L::STAGES;
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
@@ -136,6 +186,7 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
   auto exr_bar = [&](int pr) { return bar0 + 8u * (2 * TC_STAGES + 12 + pr); };
   volatile uint32_t* tmem_slot = (volatile uint32_t*)(sm + L::BAR_OFF + 8 * (2 * TC_STAGES + 8));
   volatile int* abort_flag = (volatile int*)(sm + L::BAR_OFF + 8 * (2 * TC_STAGES + 8) + 8);
+  volatile float* row_scale = reinterpret_cast<volatile float*>(sm + L::ROWSC_OFF);   // A8 only
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // two accumulator buffers; bf16 weights: each holds the hi-plane product in columns [0, M_PAD) and the lo-plane
@@ -145,7 +196,7 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
 
   // fp8 launches in which no CTA has a second work item: the epilogue warps, idle until the accumulator is complete,
   // widen half of every weight tile beside the four converter warps
-  const bool helpers = FP8 && p.tile_begin[p.n_mats] * p.splits <= (int)gridDim.x;
+  const bool helpers = WIDEN && p.tile_begin[p.n_mats] * p.splits <= (int)gridDim.x;
   if (threadIdx.x == 0) {
     for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
@@ -182,8 +233,9 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
       for (int kb = kb0; kb < kb1; ++kb) {
         if (!mbar_wait(full_bar(stage), phase, abort_flag) || !mbar_wait(cempty_bar(cbuf), cphase ^ 1u, abort_flag)) return false;
         const uint8_t* src = sm + stage * L::STAGE_BYTES;
-        const uint32_t dst = base + L::CONV_OFF + cbuf * TC_A_BYTES;
-        if (helpers) convert_pieces<2>(src, dst, cvt_tid, 256);
+        const uint32_t dst = base + L::CONV_OFF + cbuf * L::CONV_BYTES;
+        if (A8) quantize_pieces<M_PAD, (M_PAD * 8 + 127) / 128>(src + L::W_BYTES, dst, row_scale, cvt_tid, 128);
+        else if (helpers) convert_pieces<2>(src, dst, cvt_tid, 256);
         else convert_pieces<4>(src, dst, cvt_tid, 128);
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> the MMA's async-proxy reads
         __syncwarp();
@@ -211,10 +263,11 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
       bool ok = !poisoned;
       bool waited = false;
       int n_pend = 0, pend_stage[TC_STAGES], pend_kb[TC_STAGES];
-      const uint32_t stage_tx = L::W_BYTES + (p.has_lo ? 2 : 1) * L::B_BYTES;
+      const uint32_t stage_tx = L::W_BYTES + ((A8 || p.has_lo) ? 2 : 1) * L::B_BYTES;
       auto load_x = [&](int st_, int kb_) {
         const uint32_t dst = base + st_ * L::STAGE_BYTES + L::W_BYTES;
-        tma_load_2d(dst, &p.tm_x, full_bar(st_), kb_ * TC_BK, 0, pol_x);
+        tma_load_2d(dst, &p.tm_x, full_bar(st_), kb_ * L::KB_ELEMS, 0, pol_x);
+        if (A8) tma_load_2d(dst + L::B_BYTES, &p.tm_x, full_bar(st_), kb_ * L::KB_ELEMS + TC_BK, 0, pol_x);   // second 64 k
         if (!FP8 && p.has_lo) tma_load_2d(dst + L::B_BYTES, &p.tm_xl, full_bar(st_), kb_ * TC_BK, 0, pol_x);
       };
       for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
@@ -239,11 +292,11 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
           armed_parity = (armed_parity & ~(1u << stage)) | (phase << stage);
           if (p.mode == TC_MODE_SWIGLU) {
             // 64 features per tile: their gate rows fill TMEM lanes 0..63, their up rows lanes 64..127
-            tma_load_2d(a_dst, &p.tm_w[0], full_bar(stage), kb * TC_BK, tile * 64, pol_w);
-            tma_load_2d(a_dst + L::W_BYTES / 2, &p.tm_w[1], full_bar(stage), kb * TC_BK, tile * 64, pol_w);
+            tma_load_2d(a_dst, &p.tm_w[0], full_bar(stage), kb * L::KB_ELEMS, tile * 64, pol_w);
+            tma_load_2d(a_dst + L::W_BYTES / 2, &p.tm_w[1], full_bar(stage), kb * L::KB_ELEMS, tile * 64, pol_w);
           } else {
-            tma_load_2d(a_dst, &p.tm_w[mi], full_bar(stage), kb * TC_BK, r0, pol_w);
-            tma_load_2d(a_dst + L::W_BYTES / 2, &p.tm_w[mi], full_bar(stage), kb * TC_BK, r0 + 64, pol_w);
+            tma_load_2d(a_dst, &p.tm_w[mi], full_bar(stage), kb * L::KB_ELEMS, r0, pol_w);
+            tma_load_2d(a_dst + L::W_BYTES / 2, &p.tm_w[mi], full_bar(stage), kb * L::KB_ELEMS, r0 + 64, pol_w);
           }
           // The weights do not depend on the predecessor kernel: the first ring of weight loads is issued before waiting
           // for it; the activation tiles of those stages follow once it has completed.
@@ -281,7 +334,7 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
     // ------------------------------------------------ MMA issuer --------------------------------------------------
     if (lane == 0) {
       const bool two_planes = !FP8 && p.has_lo;
-      const uint32_t idesc = FP8 ? umma_idesc_f16(M_PAD) : umma_idesc_bf16(two_planes ? 2 * M_PAD : M_PAD);
+      const uint32_t idesc = A8 ? umma_idesc_e4m3(M_PAD) : (FP8 ? umma_idesc_f16(M_PAD) : umma_idesc_bf16(two_planes ? 2 * M_PAD : M_PAD));
       int stage = 0, cbuf = 0;
       uint32_t phase = 0, cphase = 0;
       int local = 0;
@@ -296,15 +349,25 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
         const int kb0 = split * p.kb_per_split;
         const int kb1 = min(p.kblocks, kb0 + p.kb_per_split);
         for (int kb = kb0; kb < kb1; ++kb) {
-          // fp8: the converters have waited for the stage and left the widened tile in buffer cbuf
+          // fp8: the converters have waited for the stage and left their tile in buffer cbuf (the widened weights; A8:
+          // the quantised activations, the weight bytes being read from the stage itself, whose barrier this thread
+          // then observes too)
           if (!mbar_wait(FP8 ? cfull_bar(cbuf) : full_bar(stage), FP8 ? cphase : phase, abort_flag)) { ok = false; break; }
+          if (A8 && !mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t a_addr = base + stage * L::STAGE_BYTES;
-          const uint64_t adesc = umma_desc_sw128(FP8 ? base + L::CONV_OFF + cbuf * TC_A_BYTES : a_addr);
-          const uint64_t bdesc = umma_desc_sw128(a_addr + L::W_BYTES);
+          const uint32_t c_addr = base + L::CONV_OFF + cbuf * L::CONV_BYTES;
+          const uint64_t adesc = umma_desc_sw128(WIDEN ? c_addr : a_addr);
+          const uint64_t bdesc = umma_desc_sw128(A8 ? c_addr : a_addr + L::W_BYTES);
+          if (A8) {
 #pragma unroll
-          for (int kk = 0; kk < TC_BK / 16; ++kk)
-            umma_bf16(d_tmem, adesc + 2u * kk, bdesc + 2u * kk, idesc, (kb > kb0 || kk > 0) ? 1u : 0u);
+            for (int kk = 0; kk < 4; ++kk)      // 32 bytes of k per instruction
+              umma_f8(d_tmem, adesc + 2u * kk, bdesc + 2u * kk, idesc, (kb > kb0 || kk > 0) ? 1u : 0u);
+          } else {
+#pragma unroll
+            for (int kk = 0; kk < TC_BK / 16; ++kk)
+              umma_bf16(d_tmem, adesc + 2u * kk, bdesc + 2u * kk, idesc, (kb > kb0 || kk > 0) ? 1u : 0u);
+          }
           umma_commit(empty_bar(stage));
           if (FP8) {
             umma_commit(cempty_bar(cbuf));
@@ -317,9 +380,20 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
       if (!ok) atomicCAS(p.status, 0, TC_ERR_MMA);
     }
   } else if (FP8 && warp >= 6) {
-    // ------------------------------------------------ e4m3 -> bf16 converters ---------------------------------------
-    // 128 threads (256 with the epilogue warps helping): thread t widens the 16-byte pieces t, t + 128 (256), ... of
-    // each 8 KB byte tile
+    // ------------------------------------------------ converters -----------------------------------------------------
+    // TC_KIND_FP8: 128 threads (256 with the epilogue warps helping): thread t widens the 16-byte pieces t, t + 128
+    // (256), ... of each 8 KB byte tile.  TC_KIND_A8: the same threads quantise the activation tile; first they form
+    // every row's scale = max of the producer's partial maxima / 448 (two threads per row; 1 for an all-zero row).
+    if (A8) {
+      const int t = (int)threadIdx.x - 192, r = t >> 1;
+      pdl_wait();                      // the partial maxima are the predecessor's
+      float mx = 0.f;
+      if (r < p.m && p.amax_in)
+        for (int i = (t & 1); i < p.n_amax_in; i += 2) mx = fmaxf(mx, __ldcg(p.amax_in + (size_t)r * p.n_amax_in + i));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      if ((t & 1) == 0) row_scale[r] = mx > 0.f ? __fdiv_rn(mx, 448.f) : 1.f;
+      asm volatile("bar.sync 2, 128;" ::: "memory");
+    }
     if (!convert_all(threadIdx.x - 192) && threadIdx.x == 192) atomicCAS(p.status, 0, TC_ERR_MMA);
   } else {
     // ------------------------------------------------ epilogue warps ----------------------------------------------
@@ -348,6 +422,12 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
       const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
       if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag)) { ok = false; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      if (A8 && local == 0) {
+        // the converters left every row's quantisation scale in shared memory before the first tile they made; the
+        // accumulator holds sums of code products, so the scale multiplies the folded norm factor
+        rs0 *= row_scale[lane];
+        rs1 *= row_scale[lane + 32];
+      }
       float v[M_PAD];
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * ACC_COLS);
 #pragma unroll
@@ -403,7 +483,14 @@ __global__ void __launch_bounds__(FP8 ? TC_THREADS_FP8 : TC_THREADS, 1) gemm_tc_
             const float mine = side ? v[hi] * sc * rs_hi : v[lo] * sc * rs_lo;
             const float g = side ? other : mine, u = side ? mine : other;
             const int row = side ? hi : lo;
-            if (live && row < p.m) store_act(p.act, p.act_lo_off, (size_t)row * p.inter + col, g / (1.f + __expf(-g)) * u, p.act_fmt);
+            const float val = g / (1.f + __expf(-g)) * u;
+            if (live && row < p.m) store_act(p.act, p.act_lo_off, (size_t)row * p.inter + col, val, p.act_fmt);
+            if (A8 && p.amax_out) {
+              // partial maximum of |act| as stored (f16) over this warp's 32 features, for the consumer's quantiser
+              float am = (live && row < p.m) ? fabsf(__half2float(__ushort_as_half(f16_bits_sat(val)))) : 0.f;
+              am = warp_max(am);
+              if (lane == 0 && row < p.m) p.amax_out[(size_t)row * p.n_amax_out + tile * 2 + pr] = am;
+            }
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(exr_bar(pr));
@@ -496,15 +583,16 @@ static EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// 2-D row-major [rows, cols] tensor, box {64 columns, box_rows}, zero OOB fill.  16-bit elements (kind 0 = bf16,
-// 2 = f16): 128-byte swizzle (rows of the box are 128 bytes); e4m3 bytes (kind 1): no swizzle (rows of 64 bytes,
-// widened by the converter warps).
+// 2-D row-major [rows, cols] tensor, box {64 columns, box_rows}, zero OOB fill.  16-bit elements (TM_BF16, TM_F16):
+// 128-byte swizzle (rows of the box are 128 bytes); e4m3 bytes: TM_E4M3 no swizzle (rows of 64 bytes, widened by the
+// converter warps), TM_E4M3_128 a box of 128 columns with the 128-byte swizzle (the tile is an MMA operand as it lands).
 bool make_tmap(CUtensorMap* tm, const void* ptr, int rows, int cols, int box_rows, int kind) {
   typedef std::tuple<const void*, int, int, int, int> Key;
   static std::map<Key, CUtensorMap> cache;
   static std::mutex mu;
   std::lock_guard<std::mutex> lock(mu);
-  const bool fp8 = kind == TM_E4M3;
+  const bool fp8 = kind == TM_E4M3 || kind == TM_E4M3_128;
+  const bool wide = kind == TM_E4M3_128;
   Key key(ptr, rows, cols, box_rows, kind);
   auto it = cache.find(key);
   if (it != cache.end()) { *tm = it->second; return true; }
@@ -512,11 +600,11 @@ bool make_tmap(CUtensorMap* tm, const void* ptr, int rows, int cols, int box_row
   if (!fn) return false;
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)cols * (fp8 ? 1 : 2)};
-  cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows};
+  cuuint32_t box[2] = {(cuuint32_t)(wide ? 2 * TC_BK : TC_BK), (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
   const CUtensorMapDataType dt = fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : (kind == TM_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16);
   CUresult r = fn(tm, dt, 2, const_cast<void*>(ptr), dims, strides,
-                  box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, fp8 ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
+                  box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, (fp8 && !wide) ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return false;
   if (cache.size() > 4096) cache.clear();
@@ -565,15 +653,16 @@ size_t tc_workspace_bytes(int m, int ld, int tiles, int k) {
   return (size_t)s * m * ld * sizeof(float);
 }
 
-template <int M_PAD, bool FP8>
+template <int M_PAD, int KIND>
 static cudaError_t tc_launch_t(const TcParams& p, int grid, cudaStream_t st) {
   static bool attr_set[MAX_DEVICES] = {};
-  cudaError_t e = ensure_dynamic_smem(gemm_tc_kernel<M_PAD, FP8>, TcSmem<M_PAD, FP8>::TOTAL, attr_set);
+  cudaError_t e = ensure_dynamic_smem(gemm_tc_kernel<M_PAD, KIND>, TcSmem<M_PAD, KIND>::TOTAL, attr_set);
   if (e != cudaSuccess) return e;
-  return launch_pdl(gemm_tc_kernel<M_PAD, FP8>, dim3(grid), dim3(FP8 ? TC_THREADS_FP8 : TC_THREADS), (size_t)TcSmem<M_PAD, FP8>::TOTAL, st, p);
+  return launch_pdl(gemm_tc_kernel<M_PAD, KIND>, dim3(grid), dim3(KIND != TC_KIND_BF16 ? TC_THREADS_FP8 : TC_THREADS),
+                    (size_t)TcSmem<M_PAD, KIND>::TOTAL, st, p);
 }
 
-template <bool FP8>
+template <int FP8>
 static cudaError_t tc_launch_f(const TcParams& p, cudaStream_t st) {
   const int items = p.tile_begin[p.n_mats] * p.splits;
   const int grid = items < 2 * sm_count() ? items : 2 * sm_count();
@@ -596,12 +685,15 @@ cudaError_t tc_group_launch(const TcGroup& g, const TcOut& o, cudaStream_t st) {
   const int mode = o.mode;
   const int mp = pad_m(g.m);
   const int xkind = g.fp8 ? TM_F16 : TM_BF16;     // fp8 weights are widened to f16 and meet f16 activations
+  const bool a8 = g.fp8 && g.a8;                  // ... unless the kernel quantises the activations to e4m3 itself
+  if (a8 && (mode == TC_MODE_DIRECT || mode == TC_MODE_LOGITS)) return cudaErrorInvalidValue;
+  if (a8 && (!o.amax_in || o.n_amax_in < 1)) return cudaErrorInvalidValue;
   if (!make_tmap(&p.tm_x, g.x, g.m, g.k, mp, xkind)) return cudaErrorInvalidValue;
   p.has_lo = (!g.fp8 && g.x_lo) ? 1 : 0;
   if (p.has_lo && !make_tmap(&p.tm_xl, g.x_lo, g.m, g.k, mp, xkind)) return cudaErrorInvalidValue;
   int tiles = 0, col = 0;
   for (int i = 0; i < g.n_mats; ++i) {
-    if (!make_tmap(&p.tm_w[i], g.w[i], g.n[i], g.k, 64, g.fp8 ? TM_E4M3 : TM_BF16)) return cudaErrorInvalidValue;
+    if (!make_tmap(&p.tm_w[i], g.w[i], g.n[i], g.k, 64, a8 ? TM_E4M3_128 : (g.fp8 ? TM_E4M3 : TM_BF16))) return cudaErrorInvalidValue;
     p.n_out[i] = g.n[i];
     p.tile_begin[i] = tiles;
     p.out_col[i] = col;
@@ -611,8 +703,9 @@ cudaError_t tc_group_launch(const TcGroup& g, const TcOut& o, cudaStream_t st) {
     col += g.n[i];
   }
   p.n_mats = g.n_mats;
-  p.kblocks = ceil_div(g.k, TC_BK);
+  p.kblocks = ceil_div(g.k, a8 ? 2 * TC_BK : TC_BK);
   p.m = g.m;
+  p.amax_in = o.amax_in; p.n_amax_in = o.n_amax_in; p.amax_out = o.amax_out; p.n_amax_out = o.n_amax_out;
   p.mode = mode;
   p.status = o.status;
   p.stamp = o.stamp;
@@ -633,7 +726,7 @@ cudaError_t tc_group_launch(const TcGroup& g, const TcOut& o, cudaStream_t st) {
     if (mode == TC_MODE_LOGITS && (g.n_mats != 1 || !o.stats)) return cudaErrorInvalidValue;
   }
   if (o.splits_out) *o.splits_out = p.splits;
-  return g.fp8 ? tc_launch_f<true>(p, st) : tc_launch_f<false>(p, st);
+  return a8 ? tc_launch_f<TC_KIND_A8>(p, st) : (g.fp8 ? tc_launch_f<TC_KIND_FP8>(p, st) : tc_launch_f<TC_KIND_BF16>(p, st));
 }
 
 }  // namespace fdk

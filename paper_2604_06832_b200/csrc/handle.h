@@ -18,6 +18,7 @@ struct fdvlm {
   int device;
   int dt;          // DT_*
   size_t act_sz;   // bytes per activation / KV element
+  int act8;        // W8A8: the four layer projections quantise their input rows to e4m3 (weights e4m3 as for DT_FP8)
   int use_tc;      // bf16 / fp8 weights: tcgen05 + TMA GEMMs, tensor-core attention, folded norms
   int kv_type;     // tensor-core path: element type of q and the KV cache (KV_BF16 / KV_F16)
   int xfmt;        // tensor-core path: storage of the GEMM inputs a / ao / act (XF_BF16X2 for bf16 weights, XF_F16 for fp8)
@@ -42,6 +43,9 @@ struct fdvlm {
   float* y;        // [R, max((Hq+2Hkv)d, 2I)] fp32 GEMM output (CUDA-core path)
   float* cs;       // [R, d/2] float2 rotary table
   float* ssq;      // [R, nt] partial sums of h^2 per 128 columns (tensor-core path)
+  // W8A8: partial maxima of |value as stored| of the rows of a [R, nt], ao [R, Hq], act [R, n_gu = 2 ceil(I / 64)]
+  float* amax_a; float* amax_ao; float* amax_act;
+  int n_gu;
   void* stats;     // [ceil(V/128)*4][R] float4 softmax statistics of the LM-head epilogue
   float* logits;   // [R, V]
   float* conf;     // [R]

@@ -116,7 +116,7 @@ linear_simt_kernel(const XT* __restrict__ x, const WT* __restrict__ w, float* __
 // y[r, n] = (accumulate ? y : 0) + (sum_s part[s][r][n]) * scale[n] + bias[n]; fixed summation order.
 __global__ void splitk_epilogue_kernel(const float* __restrict__ part, int S, int m, int N,
                                        const float* __restrict__ scale, const float* __restrict__ bias,
-                                       float* __restrict__ y, int ldy, int accumulate) {
+                                       float* __restrict__ y, int ldy, int accumulate, const float* __restrict__ row_amax) {
   pdl_trigger();
   pdl_wait();
   size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -126,15 +126,16 @@ __global__ void splitk_epilogue_kernel(const float* __restrict__ part, int S, in
   float s = 0.f;
   for (int i = 0; i < S; ++i) s += part[(size_t)i * total + idx];
   if (scale) s *= scale[n];
+  if (row_amax) s *= row_amax[r] > 0.f ? __fdiv_rn(row_amax[r], 448.f) : 1.f;   // sums of e4m3 code products: the row's scale
   if (bias) s += bias[n];
   float* o = y + (size_t)r * ldy + n;
   *o = accumulate ? (*o + s) : s;
 }
 
 void launch_splitk_epilogue(const float* part, int S, int m, int n, const float* scale, const float* bias, float* y, int ldy,
-                            int accumulate, cudaStream_t st) {
+                            int accumulate, cudaStream_t st, const float* row_amax) {
   size_t total = (size_t)m * n;
-  splitk_epilogue_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(part, S, m, n, scale, bias, y, ldy, accumulate);
+  splitk_epilogue_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(part, S, m, n, scale, bias, y, ldy, accumulate, row_amax);
 }
 
 static void simt_plan(int m, int n, int k, int* bm, int* splits, int* kps) {
@@ -178,7 +179,7 @@ int launch_linear_simt(const LinearArgs& a, cudaStream_t st, cudaError_t* err) {
   else simt_dispatch<fp8e4m3, bf16>(a, bm, grid, part, kps, st);
   size_t total = (size_t)a.m * a.n;
   splitk_epilogue_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(part, s, a.m, a.n, a.scale, a.bias, a.y,
-                                                                         a.ldy, a.accumulate);
+                                                                         a.ldy, a.accumulate, nullptr);
   *err = cudaGetLastError();
   return *err == cudaSuccess ? 2 : -1;
 }
@@ -299,10 +300,16 @@ void launch_qkv_post(const float* qkv, const float* cs, void* q, void* kc, void*
 // input (XF_* storage: bf16 hi + lo planes, or f16) and per-128-column partial sums of h^2 (ssq[row][nt]); the
 // consumer's epilogue multiplies by rsqrt(sum(ssq) / hidden + eps).  All sums run in a fixed order => deterministic.
 // ================================================================================================
+// W8A8 (Sec. 3.4 "System integration"): a projection input row is quantised to e4m3 with the scale max|row| / 448, the
+// maximum taken over the values as stored (f16).  Producers leave partial maxima; consumers of code-product sums
+// multiply by the scale.
+__device__ __forceinline__ float abs_as_f16(float v) { return fabsf(__half2float(__ushort_as_half(f16_bits_sat(v)))); }
+__device__ __forceinline__ float scale_of_amax(float amax) { return amax > 0.f ? __fdiv_rn(amax, 448.f) : 1.f; }
+
 __global__ void embed_prep_kernel(const bf16* __restrict__ table, const int32_t* __restrict__ tokens,
                                   const bf16* __restrict__ rows, float* __restrict__ h, void* __restrict__ xg,
                                   size_t lo_off, int fmt, const float* __restrict__ g, float* __restrict__ ssq, int nt,
-                                  int hidden, int vocab, int* status, KStamp* stamp) {
+                                  int hidden, int vocab, int* status, float* __restrict__ amax, KStamp* stamp) {
   if (threadIdx.x == 0) stamp_start(stamp);
   pdl_trigger();
   pdl_wait();
@@ -310,21 +317,28 @@ __global__ void embed_prep_kernel(const bf16* __restrict__ table, const int32_t*
   __shared__ float red[32];
   const int r = blockIdx.x;
   const bf16* src = tokens ? table + (size_t)checked_token(tokens, r, vocab, status) * hidden : rows + (size_t)r * hidden;
-  float ss = 0.f;
+  float ss = 0.f, am = 0.f;
   for (int c = threadIdx.x; c < hidden; c += blockDim.x) {
     const float v = __bfloat162float(src[c]);
     h[(size_t)r * hidden + c] = v;
     store_act(xg, lo_off, (size_t)r * hidden + c, v * g[c], fmt);
     ss = fmaf(v, v, ss);
+    am = fmaxf(am, abs_as_f16(v * g[c]));
   }
   ss = block_sum(ss, red);
   for (int t = threadIdx.x; t < nt; t += blockDim.x) ssq[(size_t)r * nt + t] = (t == 0) ? ss : 0.f;
+  if (amax) {      // same layout as ssq: the whole row's maximum in slot 0
+    __syncthreads();
+    am = block_max(am, red);
+    for (int t = threadIdx.x; t < nt; t += blockDim.x) amax[(size_t)r * nt + t] = (t == 0) ? am : 0.f;
+  }
   if (threadIdx.x == 0) stamp_end(stamp);
 }
 void launch_embed_prep(const void* table, const int32_t* tokens, const void* rows, float* h, void* xg, size_t lo_off, int fmt,
-                       const float* g, float* ssq, int nt, int n, int hidden, int vocab, int* status, cudaStream_t st, KStamp* stamp) {
+                       const float* g, float* ssq, int nt, int n, int hidden, int vocab, int* status, cudaStream_t st, KStamp* stamp,
+                       float* amax) {
   embed_prep_kernel<<<n, 256, 0, st>>>((const bf16*)table, tokens, (const bf16*)rows, h, xg, lo_off, fmt, g, ssq, nt, hidden, vocab,
-                                       status, stamp);
+                                       status, amax, stamp);
 }
 
 // bf16 rows -> f16 rows (saturating), for the operator-level entry points whose callers hand bf16 activations to an
@@ -335,6 +349,24 @@ __global__ void bf16_to_f16_kernel(const bf16* __restrict__ in, unsigned short* 
 }
 void launch_bf16_to_f16(const void* in, void* out, size_t n, cudaStream_t st) {
   bf16_to_f16_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>((const bf16*)in, (unsigned short*)out, n);
+}
+// The same with one block per row, which also leaves amax[row] = max |f16 value| of the row: what the quantising
+// projection takes its per-row scale from.
+__global__ void bf16_rows_to_f16_amax_kernel(const bf16* __restrict__ in, unsigned short* __restrict__ out, int k,
+                                             float* __restrict__ amax) {
+  __shared__ float red[32];
+  const size_t base = (size_t)blockIdx.x * k;
+  float am = 0.f;
+  for (int c = threadIdx.x; c < k; c += blockDim.x) {
+    const unsigned short b = f16_bits_sat(__bfloat162float(in[base + c]));
+    out[base + c] = b;
+    am = fmaxf(am, fabsf(__half2float(__ushort_as_half(b))));
+  }
+  am = block_max(am, red);
+  if (threadIdx.x == 0) amax[blockIdx.x] = am;
+}
+void launch_bf16_rows_to_f16_amax(const void* in, void* out, int m, int k, float* amax, cudaStream_t st) {
+  bf16_rows_to_f16_amax_kernel<<<m, 256, 0, st>>>((const bf16*)in, (unsigned short*)out, k, amax);
 }
 
 // Sum of S split-K partials p[i * stride].  These kernels are a handful of dependent L2 round trips long, so every
@@ -370,7 +402,8 @@ __global__ void fin_qkv_kernel(const float* __restrict__ part, int S, int m, con
                                const float* __restrict__ bq, const float* __restrict__ bk, const float* __restrict__ bv,
                                const float* __restrict__ sq, const float* __restrict__ sk, const float* __restrict__ sv,
                                T* __restrict__ q, T* __restrict__ kc, T* __restrict__ vc, int pos0, int hq, int hkv,
-                               int d, int max_seq, const int* __restrict__ len_ptr, KStamp* stamp) {
+                               int d, int max_seq, const int* __restrict__ len_ptr, const float* __restrict__ amax_in,
+                               KStamp* stamp) {
   if (threadIdx.x == 0) stamp_start(stamp);
   pdl_trigger();
   const int head = blockIdx.x, r = blockIdx.y, j = threadIdx.x, half = d >> 1;
@@ -391,9 +424,12 @@ __global__ void fin_qkv_kernel(const float* __restrict__ part, int S, int m, con
   const int width = (hq + 2 * hkv) * d;
   const size_t sstride = (size_t)m * width;
   const float* pa = part + (size_t)r * width + head * d + j;
-  float ssq_v = 0.f;
-  if (threadIdx.x < 32)
+  float ssq_v = 0.f, am = 0.f;
+  if (threadIdx.x < 32) {
     for (int t = threadIdx.x; t < nt; t += 32) ssq_v += __ldcg(ssq + (size_t)r * nt + t);
+    if (amax_in)     // W8A8: the partial sums are sums of code products; the row's scale joins the norm factor
+      for (int t = threadIdx.x; t < nt; t += 32) am = fmaxf(am, __ldcg(amax_in + (size_t)r * nt + t));
+  }
   const float2 c = (head < hq + hkv) ? __ldcg(&cs[r * half + j]) : make_float2(1.f, 0.f);
   Partials<16> va, vb;
   issue_partials(va, pa, sstride, 0, S);
@@ -401,7 +437,8 @@ __global__ void fin_qkv_kernel(const float* __restrict__ part, int S, int m, con
   if (threadIdx.x < 32) {
     // fixed order: lanes hold disjoint strided subsets, combined by the butterfly below
     const float t = warp_sum(ssq_v);
-    if (threadIdx.x == 0) s_rstd = rsqrtf(t * inv_h + eps);
+    am = warp_max(am);
+    if (threadIdx.x == 0) s_rstd = rsqrtf(t * inv_h + eps) * (amax_in ? scale_of_amax(am) : 1.f);
   }
   float a = add_partials(va, 0.f), b = add_partials(vb, 0.f);
   a = sum_partials_from(pa, sstride, 16, S, a);
@@ -429,13 +466,13 @@ __global__ void fin_qkv_kernel(const float* __restrict__ part, int S, int m, con
 }
 void launch_fin_qkv(const float* part, int S, int m, const float* cs, const float* ssq, int nt, int hidden, float eps,
                     const float* bq, const float* bk, const float* bv, const float* sq, const float* sk, const float* sv, void* q, void* kc, void* vc, int pos0, int hq,
-                    int hkv, int d, int max_seq, int kv_type, cudaStream_t st, const int* len_ptr, KStamp* stamp) {
+                    int hkv, int d, int max_seq, int kv_type, cudaStream_t st, const int* len_ptr, KStamp* stamp, const float* amax_in) {
   if (kv_type == KV_F16)
     launch_pdl(fin_qkv_kernel<__half>, dim3(hq + 2 * hkv, m), dim3(d / 2), 0, st, part, S, m, (const float2*)cs, ssq, nt, 1.f / (float)hidden,
-               eps, bq, bk, bv, sq, sk, sv, (__half*)q, (__half*)kc, (__half*)vc, pos0, hq, hkv, d, max_seq, len_ptr, stamp);
+               eps, bq, bk, bv, sq, sk, sv, (__half*)q, (__half*)kc, (__half*)vc, pos0, hq, hkv, d, max_seq, len_ptr, amax_in, stamp);
   else
     launch_pdl(fin_qkv_kernel<bf16>, dim3(hq + 2 * hkv, m), dim3(d / 2), 0, st, part, S, m, (const float2*)cs, ssq, nt, 1.f / (float)hidden,
-               eps, bq, bk, bv, sq, sk, sv, (bf16*)q, (bf16*)kc, (bf16*)vc, pos0, hq, hkv, d, max_seq, len_ptr, stamp);
+               eps, bq, bk, bv, sq, sk, sv, (bf16*)q, (bf16*)kc, (bf16*)vc, pos0, hq, hkv, d, max_seq, len_ptr, amax_in, stamp);
 }
 
 // Residual finalisation: h += sum of split-K partials; xg = h * gain of the next norm (stored as `fmt`);
@@ -443,16 +480,23 @@ void launch_fin_qkv(const float* part, int S, int m, const float* cs, const floa
 __global__ void __launch_bounds__(128) fin_resid_kernel(const float* __restrict__ part, int S, int m, int hidden,
                                                         float* __restrict__ h, const float* __restrict__ g,
                                                         void* __restrict__ xg, size_t lo_off, int fmt, float* __restrict__ ssq, int nt,
-                                                        const float* __restrict__ scale, KStamp* stamp) {
+                                                        const float* __restrict__ scale, const float* __restrict__ amax_in,
+                                                        int n_amax_in, float* __restrict__ amax_out, KStamp* stamp) {
   if (threadIdx.x == 0) stamp_start(stamp);
   pdl_trigger();
   __shared__ float red[32];
   const int t = blockIdx.x, r = blockIdx.y, c = t * 128 + threadIdx.x;
   // weights (gain, scale) do not depend on the predecessor
   const float gc = (c < hidden) ? g[c] : 0.f;
-  const float sc = (c < hidden && scale) ? scale[c] : 1.f;
+  float sc = (c < hidden && scale) ? scale[c] : 1.f;
   pdl_wait();
   if (threadIdx.x == 0) stamp_released(stamp);
+  if (amax_in) {   // W8A8: the partial sums are sums of code products of a row quantised with the scale max / 448
+    float am = 0.f;
+    for (int i = threadIdx.x; i < n_amax_in; i += 128) am = fmaxf(am, __ldcg(amax_in + (size_t)r * n_amax_in + i));
+    sc *= scale_of_amax(block_max(am, red));
+    __syncthreads();
+  }
   float v = 0.f;
   if (c < hidden) {
     const size_t idx = (size_t)r * hidden + c, sstride = (size_t)m * hidden;
@@ -464,11 +508,18 @@ __global__ void __launch_bounds__(128) fin_resid_kernel(const float* __restrict_
     store_act(xg, lo_off, idx, v * gc, fmt);
   }
   const float ss = block_sum(v * v, red);
+  if (amax_out) {  // the next projection's quantiser: partial maximum of the stored xg over this tile
+    __syncthreads();
+    const float am = block_max(c < hidden ? abs_as_f16(v * gc) : 0.f, red);
+    if (threadIdx.x == 0) amax_out[(size_t)r * nt + t] = am;
+  }
   if (threadIdx.x == 0) { ssq[(size_t)r * nt + t] = ss; stamp_end(stamp, true); }
 }
 void launch_fin_resid(const float* part, int S, int m, int hidden, float* h, const float* g, void* xg, size_t lo_off, int fmt,
-                      float* ssq, int nt, const float* scale, cudaStream_t st, KStamp* stamp) {
-  launch_pdl(fin_resid_kernel, dim3(nt, m), dim3(128), 0, st, part, S, m, hidden, h, g, xg, lo_off, fmt, ssq, nt, scale, stamp);
+                      float* ssq, int nt, const float* scale, cudaStream_t st, KStamp* stamp, const float* amax_in, int n_amax_in,
+                      float* amax_out) {
+  launch_pdl(fin_resid_kernel, dim3(nt, m), dim3(128), 0, st, part, S, m, hidden, h, g, xg, lo_off, fmt, ssq, nt, scale, amax_in,
+             n_amax_in, amax_out, stamp);
 }
 
 // Merge the per-warp softmax statistics of the LM-head epilogue into confidence and prediction per row.

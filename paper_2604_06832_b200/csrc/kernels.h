@@ -29,6 +29,8 @@ size_t linear_workspace_bytes(int m, int n, int k, int dtype);
 void launch_embed(const void* table, const int32_t* tokens, float* h, int n, int hidden, int dtype, int vocab, int* status,
                   cudaStream_t st);
 void launch_bf16_to_f16(const void* in, void* out, size_t n, cudaStream_t st);
+// the same row by row, leaving amax[row] = max |f16 value| of the row
+void launch_bf16_rows_to_f16_amax(const void* in, void* out, int m, int k, float* amax, cudaStream_t st);
 void launch_rows_to_f32(const void* rows, float* h, int n, int hidden, int dtype, cudaStream_t st);
 void launch_rmsnorm(const float* h, const float* g, void* out, int n, int hidden, float eps, int dtype, cudaStream_t st);
 void launch_rope_table(float* cs, int n, int pos0, int head_dim, float theta, cudaStream_t st, const int* len_ptr = nullptr,
@@ -60,6 +62,7 @@ struct TcGroup {
   const void* w[3]; int n[3]; int n_mats;
   const float* scale[3]; const float* bias[3];
   int fp8;   // weights are e4m3 bytes (scale[] holds the per-output-channel factors)
+  int a8;    // with fp8: the kernel quantises the f16 rows to e4m3, one scale per row (W8A8); PARTIAL and SWIGLU only
 };
 // What the GEMM leaves behind.
 //   PARTIAL: part[split][m][ld] = split-K partial sums (*splits_out of them) for the caller's reduce kernel
@@ -78,11 +81,16 @@ struct TcOut {
   int* status;   // two device words: [0] set non-zero if a bounded wait inside the kernel gave up; [1] read at kernel
                  // start, non-zero sends every role down its give-up path at once
   KStamp* stamp; // in-chain timing of the launch, nullable
+  // a8 groups: amax_in[row][n_amax_in] = partial maxima of |x[row]| (as stored) left by whoever wrote x; the accumulators
+  // are sums of code products, so PARTIAL output still lacks the row's scale max / 448 (the reduce kernel applies it) while
+  // SWIGLU applies it itself and leaves amax_out[row][n_amax_out] (two partial maxima per 64-feature tile) of `act`.
+  const float* amax_in; int n_amax_in;
+  float* amax_out; int n_amax_out;
 };
 // Tensor map of a 2-D row-major [rows, cols] tensor with box {64 columns, box_rows}, zero fill outside the tensor
-// (cached per argument set).  kind TM_BF16 / TM_F16: 16-bit elements, 128-byte swizzle; TM_E4M3: bytes, no swizzle.
-// False when the driver entry point is missing or the encode fails.
-enum { TM_BF16 = 0, TM_E4M3 = 1, TM_F16 = 2 };
+// (cached per argument set).  kind TM_BF16 / TM_F16: 16-bit elements, 128-byte swizzle; TM_E4M3: bytes, no swizzle;
+// TM_E4M3_128: bytes, box of 128 columns, 128-byte swizzle.  False when the driver entry point is missing or the encode fails.
+enum { TM_BF16 = 0, TM_E4M3 = 1, TM_F16 = 2, TM_E4M3_128 = 3 };
 bool make_tmap(CUtensorMap* tm, const void* ptr, int rows, int cols, int box_rows, int kind = TM_BF16);
 bool tc_linear_supported(int m, int n, int k, int dtype);
 // Split-K workspace of a group with m rows, output width ld, `tiles` 128-row weight tiles and depth k.
@@ -93,13 +101,15 @@ cudaError_t tc_group_launch(const TcGroup& g, const TcOut& o, cudaStream_t st);
 // stored as XF_* (common.cuh).  q, kc, vc of fin_qkv are KV_BF16 or KV_F16 elements (kv_type).
 void launch_embed_prep(const void* table, const int32_t* tokens, const void* rows, float* h, void* xg, size_t lo_off, int fmt,
                        const float* g, float* ssq, int nt, int n, int hidden, int vocab, int* status, cudaStream_t st,
-                       KStamp* stamp = nullptr);
+                       KStamp* stamp = nullptr, float* amax = nullptr);
 void launch_fin_qkv(const float* part, int S, int m, const float* cs, const float* ssq, int nt, int hidden, float eps,
                     const float* bq, const float* bk, const float* bv, const float* sq, const float* sk, const float* sv, void* q,
                     void* kc, void* vc, int pos0, int hq,
-                    int hkv, int d, int max_seq, int kv_type, cudaStream_t st, const int* len_ptr = nullptr, KStamp* stamp = nullptr);
+                    int hkv, int d, int max_seq, int kv_type, cudaStream_t st, const int* len_ptr = nullptr, KStamp* stamp = nullptr,
+                    const float* amax_in = nullptr);
 void launch_fin_resid(const float* part, int S, int m, int hidden, float* h, const float* g, void* xg, size_t lo_off, int fmt,
-                      float* ssq, int nt, const float* scale, cudaStream_t st, KStamp* stamp = nullptr);
+                      float* ssq, int nt, const float* scale, cudaStream_t st, KStamp* stamp = nullptr,
+                      const float* amax_in = nullptr, int n_amax_in = 0, float* amax_out = nullptr);
 void launch_stats_merge(const void* stats, int n_part, int m, float* conf, int32_t* pred, cudaStream_t st, KStamp* stamp = nullptr);
 
 // ---- attention -----------------------------------------------------------------------------------
@@ -117,6 +127,7 @@ struct AttnArgs {
   void* workspace;
   const int* len_ptr;   // nullable: device word holding the cache length (overrides cache_len; tensor-core kernel only)
   int* status;          // nullable: device status words (see TcOut::status)
+  float* amax_out;      // nullable (tensor-core kernel): [n][hq] maxima of |out| as stored, per row and head
   KStamp* stamp;        // nullable: two consecutive entries (attention, chunk merge)
 };
 size_t attention_workspace_bytes(int n, int hq, int hkv, int d);

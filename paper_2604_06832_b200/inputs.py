@@ -20,6 +20,7 @@ from typing import Dict, List, Optional
 import torch
 
 F32, BF16, FP8 = "f32", "bf16", "fp8"
+W8A8 = "w8a8"      # weights stored as for FP8; the CUDA path also quantises the layer projections' input rows
 E4M3_MAX = 448.0
 
 
@@ -56,7 +57,7 @@ class ModelShape:
         return self.n_layers * per_layer + self.vocab * self.hidden
 
     def weight_bytes(self) -> int:
-        esz = {F32: 4, BF16: 2, FP8: 1}[self.dtype]
+        esz = {F32: 4, BF16: 2, FP8: 1, W8A8: 1}[self.dtype]
         return self.linear_elements() * esz
 
     def kv_bytes_per_token(self) -> int:
@@ -126,7 +127,7 @@ def quantize_e4m3_rows(w: torch.Tensor):
 
 
 def _store_linear(w: torch.Tensor, dtype: str):
-    if dtype == FP8:
+    if dtype in (FP8, W8A8):
         return quantize_e4m3_rows(w)
     return w.to(_storage_dtype(dtype)), None
 
@@ -143,7 +144,7 @@ def linear_dims(shape: ModelShape) -> Dict[str, tuple]:
 
 
 def make_weights(shape: ModelShape, seed: int, *, qkv_bias: bool = False, final_gain: float = 1.0,
-                 std: float = 0.02, device: str = "cpu") -> dict:
+                 std: float = 0.02, device: str = "cpu", gain_spread: float = 0.0) -> dict:
     """All model weights as CPU tensors in storage dtype.
 
     Layout of the returned dict: 'embed' [vocab, hidden] (fp32 for an fp32 model, else bf16; never
@@ -153,6 +154,8 @@ def make_weights(shape: ModelShape, seed: int, *, qkv_bias: bool = False, final_
     The draw order is fixed: embed, (lm_head), then per layer q, k, v, o, gate, up, down, (biases).
     `device` selects where the generator runs (the CPU stream is the one the parity tests use; a CUDA
     generator gives a different, equally seeded stream and is used by the bench for speed).
+    `gain_spread` > 0 replaces the all-ones norm gains by 1 + gain_spread * U(-1, 1), drawn after everything else (so
+    the other tensors do not change with it).
     """
     gen = torch.Generator(device=device).manual_seed(seed)
     H = shape.hidden
@@ -177,6 +180,11 @@ def make_weights(shape: ModelShape, seed: int, *, qkv_bias: bool = False, final_
         lw["g_mlp"] = torch.ones(H, dtype=torch.float32, device=device)
         layers.append(lw)
     out["layers"] = layers
+    if gain_spread > 0.0:
+        draw = lambda: 1.0 + gain_spread * (2.0 * torch.rand(H, generator=gen, dtype=torch.float32, device=device) - 1.0)
+        for lw in layers:
+            lw["g_attn"], lw["g_mlp"] = draw(), draw()
+        out["g_final"] = out["g_final"] * draw()
     return out
 
 
