@@ -104,7 +104,7 @@ def make_oracle_at_prefix(wl: I.Workload, weights_cpu: dict):
     import numpy as np
     from oracle import fdvlm_oracle as orc
     shape = wl.shape
-    o = orc.Oracle(shape, I.weights_to_numpy(weights_cpu))
+    o = orc.Oracle(shape, I.weights_to_numpy(weights_cpu), act_fp8=(shape.dtype == I.W8A8))
     L0 = wl.n_embeds + wl.n_tokens
     rng = np.random.default_rng(wl.prefix_seed)
     for l in range(shape.n_layers):
@@ -211,7 +211,7 @@ def run_ours(args, wl, block):
     weights = I.make_weights(shape, wl.weight_seed, device="cuda")
     stream = torch.cuda.Stream()
     # the 7B configuration prescribes a bf16 KV cache; the others leave the cache's element type open
-    kv_dtype = B.KV_BF16 if shape.dtype == I.FP8 else B.KV_F16
+    kv_dtype = B.KV_BF16 if shape.dtype in (I.FP8, I.W8A8) else B.KV_F16
     handle = B.Handle(shape, weights, max_seq=max_seq, max_block=max(block, 32), stream=stream, kv_dtype=kv_dtype)
     emb, toks = I.make_prefix(shape, wl.n_embeds, wl.n_tokens, wl.prefix_seed)
     emb_d, toks_d = emb.cuda(), toks.cuda()
@@ -408,7 +408,7 @@ def run_ours(args, wl, block):
     line = {
         "metric": METRIC, "value": value, "unit": "tok/s", "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms_dev / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": {"f32": "f32", "bf16": "bf16", "fp8": "f16 x e4m3 weights"}[shape.dtype], "data": "synthetic",
+        "dtype": {"f32": "f32", "bf16": "bf16", "fp8": "f16 x e4m3 weights", "w8a8": "e4m3 x e4m3 (per-token activation scales)"}[shape.dtype], "data": "synthetic",
         "config": config_of(wl, block, world),
         "kv_dtype": "bf16" if kv_dtype == B.KV_BF16 else "f16",
         "e2e": {"value": e2e_value, "unit": "tok/s", "h2d_bytes_per_step": block * 4,

@@ -99,7 +99,6 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
   const int R = cfg->max_block, H = cfg->hidden, I = cfg->intermediate, d = cfg->head_dim;
   const int NQ = cfg->n_q_heads * d, NKV = cfg->n_kv_heads * d, NQKV = NQ + 2 * NKV;
   h->nt = (H + 127) / 128;
-  h->n_gu = 2 * ((I + 63) / 64);
   size_t ws = 0;
   const int shapes[][2] = {{NQ, H}, {NKV, H}, {H, NQ}, {I, H}, {H, I}, {cfg->vocab, H}};
   for (auto& s : shapes) { size_t b = linear_workspace_bytes(R, s[0], s[1], h->dt); if (b > ws) ws = b; }
@@ -141,7 +140,7 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
       {(void**)&h->ssq, (size_t)R * h->nt * 4},
       {(void**)&h->amax_a, h->act8 ? (size_t)R * h->nt * 4 : 16},
       {(void**)&h->amax_ao, h->act8 ? (size_t)R * cfg->n_q_heads * 4 : 16},
-      {(void**)&h->amax_act, h->act8 ? (size_t)R * h->n_gu * 4 : 16},
+      {(void**)&h->amax_act, h->act8 ? (size_t)R * 4 : 16},
       {(void**)&h->cs, (size_t)R * d * 4},
       {(void**)&h->stamps, h->use_tc ? sizeof(KStamp) * FDVLM_MAX_STAMPS : 16},
       {(void**)&h->h, (size_t)R * H * 4},

@@ -188,7 +188,6 @@ static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int wan
   };
   const bool fp8 = (h->dt == DT_FP8);
   const bool a8 = h->act8 != 0;                      // W8A8: the four layer projections quantise their input rows
-  const int n_gu = h->n_gu;
   // a GEMM input buffer: hi (or only) plane, and its lo plane when the format has one
   auto group = [&](const void* x, size_t lo_off, size_t row0_elems, int m, int k, int nm, const void* w0, int n0, const void* w1, int n1,
                    const void* w2, int n2) {
@@ -225,7 +224,7 @@ static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int wan
       return fail(h, FDVLM_ERR_CUDA, "qkv projection launch: %s", cudaGetErrorString(e));
     launch_fin_qkv(part, S, n, h->cs, h->ssq, nt, H, c.rms_eps, lw.bq, lw.bk, lw.bv, lw.s_q, lw.s_k, lw.s_v, h->q, kv_ptr(h, l, 0), kv_ptr(h, l, 1),
                    h->cache_len, c.n_q_heads, c.n_kv_heads, d, c.max_seq, h->kv_type, h->st, len_ptr, stamp(FDVLM_K_FIN_QKV),
-                   a8 ? h->amax_a : nullptr);
+                   a8 ? h->amax_a : nullptr, a8 ? h->amax_act : nullptr);
     AttnArgs at;
     memset(&at, 0, sizeof(at));
     at.len_ptr = len_ptr;
@@ -252,21 +251,21 @@ static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int wan
     o = out(TC_MODE_SWIGLU, FDVLM_K_GEMM_GATE_UP);
     o.act = h->act; o.act_lo_off = h->act_lo; o.act_fmt = h->xfmt;
     o.ssq_in = h->ssq; o.nt_in = nt; o.hidden = H; o.eps = c.rms_eps;
-    o.amax_in = a8 ? h->amax_a : nullptr; o.n_amax_in = nt; o.amax_out = a8 ? h->amax_act : nullptr; o.n_amax_out = n_gu;
+    o.amax_in = a8 ? h->amax_a : nullptr; o.n_amax_in = nt; o.amax_out = a8 ? h->amax_act : nullptr;
     TcGroup gu = group(h->a, h->a_lo, 0, n, H, 2, lw.w_gate, I, lw.w_up, I, nullptr, 0);
     gu.scale[0] = lw.s_gate; gu.scale[1] = lw.s_up;
     if (!gemm(gu, o))
       return fail(h, FDVLM_ERR_CUDA, "gate/up projection launch: %s", cudaGetErrorString(e));
     o = out(TC_MODE_PARTIAL, FDVLM_K_GEMM_DOWN);
     o.ld = H; o.splits_out = &S;
-    o.amax_in = a8 ? h->amax_act : nullptr; o.n_amax_in = n_gu;
+    o.amax_in = a8 ? h->amax_act : nullptr; o.n_amax_in = 1;
     if (!gemm(group(h->act, h->act_lo, 0, n, I, 1, lw.w_down, H, nullptr, 0, nullptr, 0), o))
       return fail(h, FDVLM_ERR_CUDA, "down projection launch: %s", cudaGetErrorString(e));
     // the last layer feeds the LM head, whose table (a tied bf16 embedding under fp8 layer weights) may want another format
     const bool last = (l + 1 == c.n_layers);
     const float* g_next = last ? h->w.g_final : h->layers[l + 1].g_attn;
     launch_fin_resid(part, S, n, H, h->h, g_next, h->a, h->a_lo, last ? h->head_fmt : h->xfmt, h->ssq, nt, lw.s_down, h->st,
-                     stamp(FDVLM_K_FIN_RESID), a8 ? h->amax_act : nullptr, n_gu, (a8 && !last) ? h->amax_a : nullptr);
+                     stamp(FDVLM_K_FIN_RESID), a8 ? h->amax_act : nullptr, 1, (a8 && !last) ? h->amax_a : nullptr);
     h->launches += 2;
   }
   if (logits_rows > 0) {

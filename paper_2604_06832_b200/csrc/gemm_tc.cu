@@ -65,10 +65,10 @@ struct TcParams {
                         // every role take its give-up path at once (a host-set test hook for that path)
   KStamp* stamp;        // in-chain timing of this launch (null: off)
   // TC_KIND_A8: amax_in[row][n_amax_in] = partial maxima of |x[row]| left by the producer of x; the row's quantisation
-  // scale is their maximum / 448.  SWIGLU mode also leaves amax_out[row][n_amax_out] (two per 64-feature tile) for the
-  // consumer of `act`.
+  // scale is their maximum / 448.  SWIGLU mode also raises amax_out[row] (atomic maximum; zero before the launch) to
+  // the maximum of |act[row]| as stored, for the consumer of `act`.
   const float* amax_in; int n_amax_in;
-  float* amax_out; int n_amax_out;
+  float* amax_out;
 };
 
 // Operand kinds of the kernel:
@@ -94,8 +94,8 @@ struct TcSmem {
   static constexpr int EX_ROUNDS = (M_PAD + EX_ROWS - 1) / EX_ROWS;
   static constexpr int EX_BYTES = (M_PAD / EX_ROUNDS) * 256;
   static constexpr int BAR_OFF = EX_OFF + EX_BYTES;
-  static constexpr int ROWSC_OFF = BAR_OFF + 256;                      // A8: the rows' quantisation scales (64 floats)
-  static constexpr int TOTAL = ROWSC_OFF + 256 + 1024;  // + alignment slack
+  static constexpr int ROWSC_OFF = BAR_OFF + 256;                      // A8: the rows' quantisation scales and their reciprocals
+  static constexpr int TOTAL = ROWSC_OFF + 512 + 1024;  // + alignment slack
 };
 
 // sixteen e4m3 bytes -> sixteen f16 (exact: every e4m3 value, subnormals included, is an f16 value)
@@ -132,9 +132,12 @@ __device__ __forceinline__ void convert_pieces(const uint8_t* src, uint32_t dst,
 
 // Quantise NP 16-byte pieces (tid, tid + stride, ...) of the activation tile of one stage -- two 128-byte-swizzled f16
 // halves of 64 k each -- into the 128-byte-swizzled e4m3 tile [M_PAD rows][128 k] the MMA reads: code = e4m3(x / scale
-// of the row), float32 quotient, round to nearest even, saturating.
+// of the row), float32 quotient, round to nearest even, saturating.  The quotient is formed without the division
+// routine: with y = RN(1 / scale), q0 = RN(x y) and the exact remainder r = x - q0 scale (one FMA), RN(q0 + r y) is the
+// correctly rounded x / scale (Markstein's correction step; no operand here is zero, infinite or subnormal except
+// x = 0, which gives 0 either way).
 template <int M_PAD, int NP>
-__device__ __forceinline__ void quantize_pieces(const uint8_t* x_tile, uint32_t dst, const volatile float* row_scale, int tid, int stride) {
+__device__ __forceinline__ void quantize_pieces(const uint8_t* x_tile, uint32_t dst, const volatile float2* row_scale, int tid, int stride) {
 #pragma unroll
   for (int i = 0; i < NP; ++i) {
     const int piece = tid + stride * i;
@@ -144,7 +147,7 @@ __device__ __forceinline__ void quantize_pieces(const uint8_t* x_tile, uint32_t 
     const int c0 = 2 * (j & 3);
     const uint4 a = *reinterpret_cast<const uint4*>(half + ((c0 ^ (r & 7)) << 4));
     const uint4 b = *reinterpret_cast<const uint4*>(half + (((c0 + 1) ^ (r & 7)) << 4));
-    const float sc = row_scale[r];
+    const float sc = row_scale[r].x, rinv = row_scale[r].y;
     const uint32_t in[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
     uint32_t out[4];
 #pragma unroll
@@ -153,7 +156,9 @@ __device__ __forceinline__ void quantize_pieces(const uint8_t* x_tile, uint32_t 
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         const __half2 hv = *reinterpret_cast<const __half2*>(&in[2 * w + h]);
-        const float x0 = __fdiv_rn(__low2float(hv), sc), x1 = __fdiv_rn(__high2float(hv), sc);
+        const float a0 = __low2float(hv), a1 = __high2float(hv);
+        const float q0 = a0 * rinv, q1 = a1 * rinv;
+        const float x0 = fmaf(fmaf(-q0, sc, a0), rinv, q0), x1 = fmaf(fmaf(-q1, sc, a1), rinv, q1);
         asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(pair[h]) : "f"(x1), "f"(x0));   // first source -> upper byte
       }
       out[w] = (uint32_t)pair[0] | ((uint32_t)pair[1] << 16);
@@ -186,7 +191,7 @@ __global__ void __launch_bounds__(KIND != TC_KIND_BF16 ? TC_THREADS_FP8 : TC_THR
   auto exr_bar = [&](int pr) { return bar0 + 8u * (2 * TC_STAGES + 12 + pr); };
   volatile uint32_t* tmem_slot = (volatile uint32_t*)(sm + L::BAR_OFF + 8 * (2 * TC_STAGES + 8));
   volatile int* abort_flag = (volatile int*)(sm + L::BAR_OFF + 8 * (2 * TC_STAGES + 8) + 8);
-  volatile float* row_scale = reinterpret_cast<volatile float*>(sm + L::ROWSC_OFF);   // A8 only
+  volatile float2* row_scale = reinterpret_cast<volatile float2*>(sm + L::ROWSC_OFF);   // A8 only: (scale, RN(1 / scale))
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // two accumulator buffers; bf16 weights: each holds the hi-plane product in columns [0, M_PAD) and the lo-plane
@@ -388,10 +393,23 @@ __global__ void __launch_bounds__(KIND != TC_KIND_BF16 ? TC_THREADS_FP8 : TC_THR
       const int t = (int)threadIdx.x - 192, r = t >> 1;
       pdl_wait();                      // the partial maxima are the predecessor's
       float mx = 0.f;
-      if (r < p.m && p.amax_in)
-        for (int i = (t & 1); i < p.n_amax_in; i += 2) mx = fmaxf(mx, __ldcg(p.amax_in + (size_t)r * p.n_amax_in + i));
+      if (r < p.m && p.amax_in) {
+        // sixteen loads in flight per thread: the usual counts (a few dozen partial maxima) cost one round trip
+        const float* src = p.amax_in + (size_t)r * p.n_amax_in;
+        for (int i0 = (t & 1); i0 < p.n_amax_in; i0 += 32) {
+          float v[16];
+#pragma unroll
+          for (int u = 0; u < 16; ++u) v[u] = (i0 + 2 * u < p.n_amax_in) ? __ldcg(src + i0 + 2 * u) : 0.f;
+#pragma unroll
+          for (int u = 0; u < 16; ++u) mx = fmaxf(mx, v[u]);
+        }
+      }
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-      if ((t & 1) == 0) row_scale[r] = mx > 0.f ? __fdiv_rn(mx, 448.f) : 1.f;
+      if ((t & 1) == 0) {
+        const float sc = mx > 0.f ? __fdiv_rn(mx, 448.f) : 1.f;
+        row_scale[r].x = sc;
+        row_scale[r].y = __frcp_rn(sc);
+      }
       asm volatile("bar.sync 2, 128;" ::: "memory");
     }
     if (!convert_all(threadIdx.x - 192) && threadIdx.x == 192) atomicCAS(p.status, 0, TC_ERR_MMA);
@@ -425,8 +443,8 @@ __global__ void __launch_bounds__(KIND != TC_KIND_BF16 ? TC_THREADS_FP8 : TC_THR
       if (A8 && local == 0) {
         // the converters left every row's quantisation scale in shared memory before the first tile they made; the
         // accumulator holds sums of code products, so the scale multiplies the folded norm factor
-        rs0 *= row_scale[lane];
-        rs1 *= row_scale[lane + 32];
+        rs0 *= row_scale[lane].x;
+        rs1 *= row_scale[lane + 32].x;
       }
       float v[M_PAD];
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * ACC_COLS);
@@ -486,10 +504,11 @@ __global__ void __launch_bounds__(KIND != TC_KIND_BF16 ? TC_THREADS_FP8 : TC_THR
             const float val = g / (1.f + __expf(-g)) * u;
             if (live && row < p.m) store_act(p.act, p.act_lo_off, (size_t)row * p.inter + col, val, p.act_fmt);
             if (A8 && p.amax_out) {
-              // partial maximum of |act| as stored (f16) over this warp's 32 features, for the consumer's quantiser
+              // maximum of |act| as stored (f16) over this warp's 32 features, for the consumer's quantiser; values
+              // are non-negative, so their bit patterns order like integers (and the result does not depend on order)
               float am = (live && row < p.m) ? fabsf(__half2float(__ushort_as_half(f16_bits_sat(val)))) : 0.f;
               am = warp_max(am);
-              if (lane == 0 && row < p.m) p.amax_out[(size_t)row * p.n_amax_out + tile * 2 + pr] = am;
+              if (lane == 0 && row < p.m && am > 0.f) atomicMax(reinterpret_cast<int*>(p.amax_out) + row, __float_as_int(am));
             }
           }
           __syncwarp();
@@ -705,7 +724,7 @@ cudaError_t tc_group_launch(const TcGroup& g, const TcOut& o, cudaStream_t st) {
   p.n_mats = g.n_mats;
   p.kblocks = ceil_div(g.k, a8 ? 2 * TC_BK : TC_BK);
   p.m = g.m;
-  p.amax_in = o.amax_in; p.n_amax_in = o.n_amax_in; p.amax_out = o.amax_out; p.n_amax_out = o.n_amax_out;
+  p.amax_in = o.amax_in; p.n_amax_in = o.n_amax_in; p.amax_out = o.amax_out;
   p.mode = mode;
   p.status = o.status;
   p.stamp = o.stamp;

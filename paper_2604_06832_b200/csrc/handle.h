@@ -43,9 +43,9 @@ struct fdvlm {
   float* y;        // [R, max((Hq+2Hkv)d, 2I)] fp32 GEMM output (CUDA-core path)
   float* cs;       // [R, d/2] float2 rotary table
   float* ssq;      // [R, nt] partial sums of h^2 per 128 columns (tensor-core path)
-  // W8A8: partial maxima of |value as stored| of the rows of a [R, nt], ao [R, Hq], act [R, n_gu = 2 ceil(I / 64)]
+  // W8A8: maxima of |value as stored| of the rows of a ([R, nt] partial maxima), ao ([R, Hq] partial maxima) and
+  // act ([R], raised atomically by the gate/up epilogue, zeroed by the QKV finalisation of the same layer)
   float* amax_a; float* amax_ao; float* amax_act;
-  int n_gu;
   void* stats;     // [ceil(V/128)*4][R] float4 softmax statistics of the LM-head epilogue
   float* logits;   // [R, V]
   float* conf;     // [R]

@@ -403,7 +403,7 @@ __global__ void fin_qkv_kernel(const float* __restrict__ part, int S, int m, con
                                const float* __restrict__ sq, const float* __restrict__ sk, const float* __restrict__ sv,
                                T* __restrict__ q, T* __restrict__ kc, T* __restrict__ vc, int pos0, int hq, int hkv,
                                int d, int max_seq, const int* __restrict__ len_ptr, const float* __restrict__ amax_in,
-                               KStamp* stamp) {
+                               float* __restrict__ amax_zero, KStamp* stamp) {
   if (threadIdx.x == 0) stamp_start(stamp);
   pdl_trigger();
   const int head = blockIdx.x, r = blockIdx.y, j = threadIdx.x, half = d >> 1;
@@ -420,6 +420,9 @@ __global__ void fin_qkv_kernel(const float* __restrict__ part, int S, int m, con
   pdl_wait();
   if (threadIdx.x == 0) stamp_released(stamp);
   __shared__ float s_rstd;
+  // W8A8: the row's slot of the running maximum that this layer's gate/up epilogue raises; its last readers (the
+  // previous layer's down projection) are long done, its next writers start after this kernel
+  if (amax_zero && head == 0 && threadIdx.x == 0) amax_zero[r] = 0.f;
   // every load of this kernel is issued before the first result is needed
   const int width = (hq + 2 * hkv) * d;
   const size_t sstride = (size_t)m * width;
@@ -466,13 +469,14 @@ __global__ void fin_qkv_kernel(const float* __restrict__ part, int S, int m, con
 }
 void launch_fin_qkv(const float* part, int S, int m, const float* cs, const float* ssq, int nt, int hidden, float eps,
                     const float* bq, const float* bk, const float* bv, const float* sq, const float* sk, const float* sv, void* q, void* kc, void* vc, int pos0, int hq,
-                    int hkv, int d, int max_seq, int kv_type, cudaStream_t st, const int* len_ptr, KStamp* stamp, const float* amax_in) {
+                    int hkv, int d, int max_seq, int kv_type, cudaStream_t st, const int* len_ptr, KStamp* stamp, const float* amax_in,
+                    float* amax_zero) {
   if (kv_type == KV_F16)
     launch_pdl(fin_qkv_kernel<__half>, dim3(hq + 2 * hkv, m), dim3(d / 2), 0, st, part, S, m, (const float2*)cs, ssq, nt, 1.f / (float)hidden,
-               eps, bq, bk, bv, sq, sk, sv, (__half*)q, (__half*)kc, (__half*)vc, pos0, hq, hkv, d, max_seq, len_ptr, amax_in, stamp);
+               eps, bq, bk, bv, sq, sk, sv, (__half*)q, (__half*)kc, (__half*)vc, pos0, hq, hkv, d, max_seq, len_ptr, amax_in, amax_zero, stamp);
   else
     launch_pdl(fin_qkv_kernel<bf16>, dim3(hq + 2 * hkv, m), dim3(d / 2), 0, st, part, S, m, (const float2*)cs, ssq, nt, 1.f / (float)hidden,
-               eps, bq, bk, bv, sq, sk, sv, (bf16*)q, (bf16*)kc, (bf16*)vc, pos0, hq, hkv, d, max_seq, len_ptr, amax_in, stamp);
+               eps, bq, bk, bv, sq, sk, sv, (bf16*)q, (bf16*)kc, (bf16*)vc, pos0, hq, hkv, d, max_seq, len_ptr, amax_in, amax_zero, stamp);
 }
 
 // Residual finalisation: h += sum of split-K partials; xg = h * gain of the next norm (stored as `fmt`);
@@ -491,29 +495,41 @@ __global__ void __launch_bounds__(128) fin_resid_kernel(const float* __restrict_
   float sc = (c < hidden && scale) ? scale[c] : 1.f;
   pdl_wait();
   if (threadIdx.x == 0) stamp_released(stamp);
-  if (amax_in) {   // W8A8: the partial sums are sums of code products of a row quantised with the scale max / 448
-    float am = 0.f;
-    for (int i = threadIdx.x; i < n_amax_in; i += 128) am = fmaxf(am, __ldcg(amax_in + (size_t)r * n_amax_in + i));
-    sc *= scale_of_amax(block_max(am, red));
-    __syncthreads();
+  // W8A8: the partial sums are sums of code products of a row quantised with the scale max / 448; the maxima are
+  // asked for first and reduced only after the other loads are on their way
+  float am_in = 0.f;
+  if (amax_in) {
+    if (n_amax_in == 1) am_in = __ldcg(amax_in + r);
+    else for (int i = threadIdx.x; i < n_amax_in; i += 128) am_in = fmaxf(am_in, __ldcg(amax_in + (size_t)r * n_amax_in + i));
   }
   float v = 0.f;
+  Partials<32> pv;
+  float hv = 0.f;
+  const size_t idx = (size_t)r * hidden + c, sstride = (size_t)m * hidden;
   if (c < hidden) {
-    const size_t idx = (size_t)r * hidden + c, sstride = (size_t)m * hidden;
-    Partials<32> pv;
     issue_partials(pv, part + idx, sstride, 0, S);
-    const float hv = __ldcg(h + idx);
+    hv = __ldcg(h + idx);
+  }
+  if (amax_in) sc *= scale_of_amax(n_amax_in == 1 ? am_in : block_max(am_in, red));
+  if (c < hidden) {
     v = hv + sum_partials_from(part + idx, sstride, 32, S, add_partials(pv, 0.f)) * sc;
     h[idx] = v;
     store_act(xg, lo_off, idx, v * gc, fmt);
   }
-  const float ss = block_sum(v * v, red);
-  if (amax_out) {  // the next projection's quantiser: partial maximum of the stored xg over this tile
+  // one pass for the tile's sum of squares and (W8A8: the next projection's quantiser) the maximum of the stored xg
+  __shared__ float red_s[4], red_m[4];
+  {
+    const float ws = warp_sum(v * v);
+    const float wm = amax_out ? warp_max(c < hidden ? abs_as_f16(v * gc) : 0.f) : 0.f;
     __syncthreads();
-    const float am = block_max(c < hidden ? abs_as_f16(v * gc) : 0.f, red);
-    if (threadIdx.x == 0) amax_out[(size_t)r * nt + t] = am;
+    if ((threadIdx.x & 31) == 0) { red_s[threadIdx.x >> 5] = ws; red_m[threadIdx.x >> 5] = wm; }
+    __syncthreads();
   }
-  if (threadIdx.x == 0) { ssq[(size_t)r * nt + t] = ss; stamp_end(stamp, true); }
+  if (threadIdx.x == 0) {
+    ssq[(size_t)r * nt + t] = (red_s[0] + red_s[2]) + (red_s[1] + red_s[3]);
+    if (amax_out) amax_out[(size_t)r * nt + t] = fmaxf(fmaxf(red_m[0], red_m[1]), fmaxf(red_m[2], red_m[3]));
+    stamp_end(stamp, true);
+  }
 }
 void launch_fin_resid(const float* part, int S, int m, int hidden, float* h, const float* g, void* xg, size_t lo_off, int fmt,
                       float* ssq, int nt, const float* scale, cudaStream_t st, KStamp* stamp, const float* amax_in, int n_amax_in,

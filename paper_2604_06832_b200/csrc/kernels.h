@@ -83,9 +83,9 @@ struct TcOut {
   KStamp* stamp; // in-chain timing of the launch, nullable
   // a8 groups: amax_in[row][n_amax_in] = partial maxima of |x[row]| (as stored) left by whoever wrote x; the accumulators
   // are sums of code products, so PARTIAL output still lacks the row's scale max / 448 (the reduce kernel applies it) while
-  // SWIGLU applies it itself and leaves amax_out[row][n_amax_out] (two partial maxima per 64-feature tile) of `act`.
+  // SWIGLU applies it itself and raises amax_out[row] (atomic maximum: zero before the launch) to max |act[row]|.
   const float* amax_in; int n_amax_in;
-  float* amax_out; int n_amax_out;
+  float* amax_out;
 };
 // Tensor map of a 2-D row-major [rows, cols] tensor with box {64 columns, box_rows}, zero fill outside the tensor
 // (cached per argument set).  kind TM_BF16 / TM_F16: 16-bit elements, 128-byte swizzle; TM_E4M3: bytes, no swizzle;
@@ -106,7 +106,7 @@ void launch_fin_qkv(const float* part, int S, int m, const float* cs, const floa
                     const float* bq, const float* bk, const float* bv, const float* sq, const float* sk, const float* sv, void* q,
                     void* kc, void* vc, int pos0, int hq,
                     int hkv, int d, int max_seq, int kv_type, cudaStream_t st, const int* len_ptr = nullptr, KStamp* stamp = nullptr,
-                    const float* amax_in = nullptr);
+                    const float* amax_in = nullptr, float* amax_zero = nullptr);
 void launch_fin_resid(const float* part, int S, int m, int hidden, float* h, const float* g, void* xg, size_t lo_off, int fmt,
                       float* ssq, int nt, const float* scale, cudaStream_t st, KStamp* stamp = nullptr,
                       const float* amax_in = nullptr, int n_amax_in = 0, float* amax_out = nullptr);

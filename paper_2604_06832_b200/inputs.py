@@ -95,6 +95,8 @@ WORKLOADS: Dict[str, Workload] = {
     "cfg3_3b_bf16_p2048_sweep": Workload("cfg3_3b_bf16_p2048_sweep", QWEN3B, 1, 13, 1536, 512, 256, (4, 8, 16, 32, 64), "threshold"),
     "cfg4_3b_bf16_p8192_b32_top8": Workload("cfg4_3b_bf16_p8192_b32_top8", QWEN3B, 1, 14, 7168, 1024, 512, (32,), "topk"),
     "cfg5_7b_fp8_p1024_b32": Workload("cfg5_7b_fp8_p1024_b32", QWEN7B_FP8, 5, 15, 768, 256, 256, (32,), "threshold"),
+    # the 7B shape with the layer projections' inputs quantised per token as well (Sec. 3.4 "System integration")
+    "w8a8_7b_p1024_b32": Workload("w8a8_7b_p1024_b32", QWEN7B_FP8.with_(dtype=W8A8), 5, 15, 768, 256, 256, (32,), "threshold"),
     # Profiler-sized cuts of the 3B / 7B shapes: same per-layer matrices, 4 layers and a 32768-row LM head, short
     # prefix.  About 0.75 GB (bf16) of weights per forward -- larger than L2, small enough for a counter capture.
     "prof_3b_bf16_4layers": Workload("prof_3b_bf16_4layers", QWEN3B.with_(n_layers=4, vocab=32768, mask_id=32767), 1, 16,
