@@ -105,6 +105,8 @@ WORKLOADS: Dict[str, Workload] = {
                                            7168, 1024, 64, (32,), "topk"),
     "prof_7b_fp8_4layers": Workload("prof_7b_fp8_4layers", QWEN7B_FP8.with_(n_layers=4, vocab=32768, mask_id=32767), 5, 17,
                                     96, 32, 64, (32,), "topk"),
+    "prof_7b_w8a8_4layers": Workload("prof_7b_w8a8_4layers", QWEN7B_FP8.with_(n_layers=4, vocab=32768, mask_id=32767, dtype=W8A8), 5, 17,
+                                     96, 32, 64, (32,), "topk"),
 }
 
 
