@@ -251,15 +251,30 @@ class Oracle:
         A_ij = 1) or rows j <= i in CAUSAL mode (Alg. 1 verify mask, A_ij = 1[i >= j]; M_C2C).
         The cache is appended with the new rows' post-rotary K and V only if update_cache
         (Alg. 1: draft = "no cache update", verify/prefill = "update cache")."""
+        n = x.shape[0]
+        L = self.cache_len
+        if mode == CAUSAL:
+            among = np.tril(np.ones((n, n), dtype=bool))
+        elif mode == BIDIR:
+            among = np.ones((n, n), dtype=bool)
+        else:
+            raise ValueError(mode)
+        h, k_new, v_new = self.forward_rows_masked(x, among, np.arange(L, L + n))
+        if update_cache:
+            self.append_cache(k_new, v_new, np.arange(n))
+        return h
+
+    def forward_rows_masked(self, x: np.ndarray, among: np.ndarray, pos: np.ndarray):
+        """n new rows against the cache under an explicit mask among themselves: row i reads every cached key and the
+        new rows j with among[i, j]; pos[i] is row i's position id (rotary).  The cache is not touched.
+        Returns (final hidden states, per-layer post-rotary K of the new rows, per-layer V)."""
         s = self.s
         n = x.shape[0]
         L = self.cache_len
-        pos = np.arange(L, L + n)
         allowed = np.ones((n, L + n), dtype=bool)
-        if mode == CAUSAL:
-            allowed[:, L:] = np.tril(np.ones((n, n), dtype=bool))
-        elif mode != BIDIR:
-            raise ValueError(mode)
+        allowed[:, L:] = among
+        pos = np.asarray(pos)
+        k_new, v_new = [], []
         h = np.array(x, dtype=self.ft, copy=True)
         for l in range(s.n_layers):
             lw = self.w["layers"][l]
@@ -281,11 +296,17 @@ class Oracle:
             m = self._act(rmsnorm(h, self._vec(lw["g_mlp"]), s.rms_eps))
             act = self._act(silu(m @ self._lin(l, "w_gate").T) * (m @ self._lin(l, "w_up").T))
             h = h + act @ self._lin(l, "w_down").T
-            if update_cache:
-                self.K[l], self.V[l] = k_all, v_all
-        if update_cache:
-            self.cache_len = L + n
-        return h
+            k_new.append(k)
+            v_new.append(v)
+        return h, k_new, v_new
+
+    def append_cache(self, k_new, v_new, rows):
+        """The cache gains, in the order given, the K / V of `rows` of a forward_rows_masked result."""
+        rows = np.asarray(rows, dtype=np.int64)
+        for l in range(self.s.n_layers):
+            self.K[l] = np.concatenate([self.K[l], k_new[l][rows]], axis=0)
+            self.V[l] = np.concatenate([self.V[l], v_new[l][rows]], axis=0)
+        self.cache_len += len(rows)
 
     def logits_of(self, h: np.ndarray, chunk: int = 16384) -> np.ndarray:
         """RMSNorm(h; g_final) E_out^T, E_out = the embedding table when tied."""
@@ -432,6 +453,40 @@ class Oracle:
         self.truncate(L0 + k)
         return dict(draft=d, a=a, accepted=k, new_tokens=a[:k].copy(), next_token=int(a[k - 1]))
 
+    # -- quadratic self-speculative decoding (Appendix B, Alg. 2) -------------------------------------
+    def quad_first_draft(self, block_size: int, last_logits: np.ndarray) -> np.ndarray:
+        """Alg. 2 step 1 in cached form.  The prompt is in the cache (its rows ran causally, as the step-1 mask
+        prescribes for them) and `last_logits` is its last row's output; B mask tokens follow, each reading the whole
+        prompt and every mask token.  d_i = argmax h_{L-1+i}: d_0 comes from the prompt's last row, d_1 .. d_{B-1}
+        from the first B-1 mask rows.  The cache keeps the prompt only.  Argmax excludes the mask token."""
+        B = block_size
+        d0 = confidence(np.asarray(last_logits)[None, :], self.s.mask_id)[0][0]
+        x = self.embed_tokens(np.full(B, self.s.mask_id, dtype=np.int64))
+        h = self.forward_rows(x, BIDIR, update_cache=False)
+        pred = confidence(self.logits_of(h), self.s.mask_id)[0]
+        return np.concatenate([[d0], pred[:B - 1]]).astype(np.int64)
+
+    def quad_step(self, d, chain: bool = False):
+        """One iteration of Alg. 2's verify + propose loop on the draft block d (B tokens; the cache holds the prompt and
+        the s tokens accepted so far, cache_len = L + s).
+
+        Input q = B groups [d_i, M^B]; position ids cache_len + i + j for entry j of group i; mask = quad_mask; one
+        forward, no cache update; P_{i,j} = argmax (mask token excluded) of entry j of group i; acceptance and the next
+        draft by quad_accept; the cache gains the K / V of the first tokens of groups 0 .. k-1 (of the forward's
+        entries only every (B+1)-th belongs to a draft token, and of those only the accepted ones are part of the
+        sequence).  Returns dict(logits [B(B+1), vocab] in the order of q, P [B, B+1], accepted, new_tokens,
+        next_draft)."""
+        d = np.asarray(d, dtype=np.int64)
+        B = len(d)
+        q = quad_input(d, self.s.mask_id)
+        pos = quad_positions(self.cache_len, B)
+        h, k_new, v_new = self.forward_rows_masked(self.embed_tokens(q), quad_mask(B, chain), pos)
+        logits = self.logits_of(h)
+        P = confidence(logits, self.s.mask_id)[0].reshape(B, B + 1)
+        k, d_next = quad_accept(P, d)
+        self.append_cache(k_new, v_new, np.arange(k) * (B + 1))
+        return dict(logits=logits, P=P, accepted=k, new_tokens=d[:k].copy(), next_draft=d_next)
+
     # -- brute force: no cache, explicit [T, T] mask ----------------------------------------------
     def forward_dense(self, x: np.ndarray, allowed: np.ndarray, positions=None) -> np.ndarray:
         """Logits of T rows recomputed from scratch under an explicit boolean mask allowed[i, j]
@@ -496,3 +551,56 @@ def draft_mask(L: int, B: int) -> np.ndarray:
 
 def causal_mask(T: int) -> np.ndarray:
     return np.tril(np.ones((T, T), dtype=bool))
+
+
+# -- Appendix B, Alg. 2 ("Quadratic Speculative Block-Causal Decoding") ---------------------------------------------
+def quad_input(d, mask_id: int) -> np.ndarray:
+    """q = [d_0, M^B, d_1, M^B, ..., d_{B-1}, M^B]: B groups of B+1 tokens, group i = the draft token d_i followed
+    by B mask tokens.  Entry j of group i has index i (B+1) + j."""
+    B = len(d)
+    q = np.full(B * (B + 1), mask_id, dtype=np.int64)
+    q[::B + 1] = np.asarray(d, dtype=np.int64)
+    return q
+
+
+def quad_positions(s_abs: int, B: int) -> np.ndarray:
+    """Position ids: group i covers [s+i, s+i+1, ..., s+i+B] ("if accepted up to d_i, generate the next B tokens");
+    s_abs = the absolute position of d_0, i.e. prompt length + accepted tokens."""
+    return np.array([s_abs + i + j for i in range(B) for j in range(B + 1)], dtype=np.int64)
+
+
+def quad_mask(B: int, chain: bool = False) -> np.ndarray:
+    """Boolean [B(B+1), B(B+1)] mask among the entries of q (rule (a), "all tokens attend to the entire KV cache",
+    is outside this matrix):
+      (b) the first token of group i reads the first tokens of groups <= i;
+      (c) a non-first token of group i reads every token of group i;
+      (d) nothing else: no attention across groups for non-first tokens.
+    chain=True is the other reading of (d) (non-first tokens are not READ across groups): a non-first token of group i
+    also reads the first tokens of groups < i, the draft tokens its position ids assume accepted."""
+    n = B * (B + 1)
+    m = np.zeros((n, n), dtype=bool)
+    for i in range(B):
+        first = i * (B + 1)
+        for i2 in range(i + 1):
+            m[first, i2 * (B + 1)] = True                       # (b)
+        for j in range(1, B + 1):
+            m[first + j, first:first + B + 1] = True            # (c)
+            if chain:
+                for i2 in range(i):
+                    m[first + j, i2 * (B + 1)] = True
+    return m
+
+
+def quad_accept(P, d):
+    """Alg. 2's verify loop: k = 1, next draft = P_{0,1:B}; while k < B and P_{k-1,0} = d_k: next draft = P_{k,1:B},
+    k += 1.  (P_{i,0}, the first token of group i, is the autoregressive prediction for the position after d_i;
+    P_{i,1..B} are the mask tokens' own predictions for the B positions after d_i.)  Returns (k, next draft)."""
+    P = np.asarray(P)
+    B = len(d)
+    k = 1
+    d_next = P[0, 1:B + 1].copy()
+    while k < B and P[k - 1, 0] == d[k]:
+        d_next = P[k, 1:B + 1].copy()
+        k += 1
+    return k, d_next
+
