@@ -216,6 +216,35 @@ typedef struct { int accepted; int32_t next_token; int cache_len; } fdvlm_spec_i
 int fdvlm_spec_block(fdvlm_t *h, int block_size, int32_t seed_token, int32_t *draft_tokens,
                      int32_t *verify_pred, fdvlm_spec_info *info);
 
+/* ---- quadratic self-speculative decoding (Appendix B, Alg. 2 and the paragraph "Quadratic speculative decoding") ----
+ * One forward verifies a draft block d_0 .. d_{B-1} and proposes the next one.  Its input is B groups [d_i, MASK x B];
+ * entry j of group i has position id cache_len + i + j; every entry reads the whole cache; (b) the first token of group
+ * i reads the first tokens of groups <= i; (c) a mask token of group i reads every entry of group i; (d) nothing else.
+ * chain != 0 takes the other reading of (d): a mask token of group i also reads the first tokens of groups < i.
+ * P_{i,0} = argmax of group i's first token (the autoregressive prediction for the position after d_i), P_{i,j} = argmax
+ * of its j-th mask token (mask_id excluded throughout).  Verify loop: k = 1; while k < B and P_{k-1,0} = d_k: k += 1.
+ * d_0 .. d_{k-1} join the sequence, their K / V join the cache (cache_len += k) and P_{k-1,1..B} is the next draft.
+ * ROW ORDER of this library (row_pred, logits): rows 0 .. B-1 are the first tokens d_0 .. d_{B-1}, row B + i B + (j-1) is
+ * mask token j of group i -- the paper lists the groups one after the other; with the first tokens in front, "keep every
+ * (B+1)-th K / V entry" is the first k staging rows of the cache and nothing is moved.
+ * The forward has B (B + 1) rows: B (B + 1) <= min(max_block, 64), i.e. B <= 7.
+ *
+ * fdvlm_quad_begin: Alg. 2 step 1 in cached form.  The prompt is in the cache (fdvlm_prefill); first_token is the token
+ *   its last row predicts (argmax of last_logits, mask_id excluded) = d_0; B mask tokens are run in one denoise pass and
+ *   the first B-1 of them give d_1 .. d_{B-1} (row i-1 predicts d_i).  The cache is unchanged.  draft: device int32 [B],
+ *   nullable.  Synchronous.  Errors: STATE inside an open block; CAPACITY as above or past max_seq; INVALID_ARG.
+ * fdvlm_quad_set_draft: overwrite the current draft (device int32 [B]); lets a test replay another implementation's.
+ * fdvlm_quad_step: one iteration of the loop.  accepted_tokens device int32 [B] (entries >= accepted are -1), next_draft
+ *   device int32 [B], row_pred device int32 [B (B+1)], logits device fp32 [B (B+1), vocab] -- all nullable, in the row
+ *   order above; info HOST, required.  Always synchronous (the accepted length decides the cache length).
+ * fdvlm_quad_end: leave the mode (the cache keeps what was accepted). */
+typedef struct { int accepted; int cache_len; } fdvlm_quad_info;
+int fdvlm_quad_begin(fdvlm_t *h, int block_size, int32_t first_token, int chain, int32_t *draft);
+int fdvlm_quad_set_draft(fdvlm_t *h, const int32_t *draft);
+int fdvlm_quad_step(fdvlm_t *h, int32_t *accepted_tokens, int32_t *next_draft, int32_t *row_pred, float *logits,
+                    fdvlm_quad_info *info);
+int fdvlm_quad_end(fdvlm_t *h);
+
 /* Committed positions, or a negative status for a NULL handle. */
 int fdvlm_cache_len(const fdvlm_t *h);
 

@@ -64,6 +64,10 @@ class SpecInfo(C.Structure):
     _fields_ = [("accepted", C.c_int), ("next_token", C.c_int32), ("cache_len", C.c_int)]
 
 
+class QuadInfo(C.Structure):
+    _fields_ = [("accepted", C.c_int), ("cache_len", C.c_int)]
+
+
 EXPORTS = {
     "fdvlm_create": (C.c_int, [C.POINTER(Config), C.POINTER(Weights), C.c_void_p, C.POINTER(C.c_void_p)]),
     "fdvlm_destroy": (None, [C.c_void_p]),
@@ -86,6 +90,10 @@ EXPORTS = {
     "fdvlm_commit_block_verify": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "fdvlm_truncate": (C.c_int, [C.c_void_p, C.c_int]),
     "fdvlm_spec_block": (C.c_int, [C.c_void_p, C.c_int, C.c_int32, C.c_void_p, C.c_void_p, C.POINTER(SpecInfo)]),
+    "fdvlm_quad_begin": (C.c_int, [C.c_void_p, C.c_int, C.c_int32, C.c_int, C.c_void_p]),
+    "fdvlm_quad_set_draft": (C.c_int, [C.c_void_p, C.c_void_p]),
+    "fdvlm_quad_step": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(QuadInfo)]),
+    "fdvlm_quad_end": (C.c_int, [C.c_void_p]),
     "fdvlm_cache_len": (C.c_int, [C.c_void_p]),
     "fdvlm_cache_read": (C.c_int, [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p]),
     "fdvlm_last_launch_count": (C.c_int, [C.c_void_p]),
@@ -256,6 +264,22 @@ class Handle:
         self._check(lib().fdvlm_spec_block(self._h, block_size, seed_token, _ptr(draft_tokens), _ptr(verify_pred),
                                            C.byref(info)))
         return info
+
+    def quad_begin(self, block_size: int, first_token: int, chain: bool = False, draft: Optional[torch.Tensor] = None):
+        self._check(lib().fdvlm_quad_begin(self._h, block_size, first_token, int(chain), _ptr(draft)))
+
+    def quad_set_draft(self, draft: torch.Tensor):
+        self._check(lib().fdvlm_quad_set_draft(self._h, _ptr(draft)))
+
+    def quad_step(self, accepted_tokens: Optional[torch.Tensor] = None, next_draft: Optional[torch.Tensor] = None,
+                  row_pred: Optional[torch.Tensor] = None, logits: Optional[torch.Tensor] = None) -> QuadInfo:
+        info = QuadInfo()
+        self._check(lib().fdvlm_quad_step(self._h, _ptr(accepted_tokens), _ptr(next_draft), _ptr(row_pred), _ptr(logits),
+                                          C.byref(info)))
+        return info
+
+    def quad_end(self):
+        self._check(lib().fdvlm_quad_end(self._h))
 
     def cache_len(self) -> int:
         return lib().fdvlm_cache_len(self._h)

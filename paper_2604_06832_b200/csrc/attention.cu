@@ -75,6 +75,7 @@ struct AttnParams {
   float2* part_ml;            // [Hq][n][chunks]
   int n, L, max_seq, hq, hkv, qh, chunk_keys, n_chunks, causal;
   const int* len_ptr;         // nullable: the cache length is read from device memory and the chunking derived from it
+  const unsigned long long* row_mask;   // nullable: bit r' of word r = row r reads row r' of this forward (AttnArgs::row_mask)
   int* status;                // nullable: status words (see TcOut::status)
   KStamp* stamp;
 };
@@ -187,6 +188,12 @@ __global__ void __launch_bounds__(AtSmem<D, ROWS>::THREADS, ROWS == 64 ? 2 : 1) 
     const int lim_lo = (r_lo < m_valid) ? (p.causal ? L + (r_lo % n) + 1 : T) : 0;
     const int lim_hi = (r_hi < m_valid) ? (p.causal ? L + (r_hi % n) + 1 : T) : 0;
     const float sl2 = rsqrtf((float)D) * LOG2E;       // scores kept in the log2 domain
+    // explicit mask among the forward's own rows (keys L .. L+n-1); set up by the host before the chain, not by a kernel of it
+    unsigned long long msk_lo = ~0ull, msk_hi = ~0ull;
+    if (p.row_mask) {
+      if (r_lo < m_valid) msk_lo = p.row_mask[r_lo % n];
+      if (r_hi < m_valid) msk_hi = p.row_mask[r_hi % n];
+    }
 
     uint32_t qf[D / 16][4];
 #pragma unroll
@@ -240,6 +247,12 @@ __global__ void __launch_bounds__(AtSmem<D, ROWS>::THREADS, ROWS == 64 ? 2 : 1) 
           s[nt][1] = (j + 1 < lim_lo) ? s[nt][1] * sl2 : -INFINITY;
           s[nt][2] = (j < lim_hi) ? s[nt][2] * sl2 : -INFINITY;
           s[nt][3] = (j + 1 < lim_hi) ? s[nt][3] * sl2 : -INFINITY;
+          if (p.row_mask && j0 + AT_KEYS > L) {              // uniform over the warp: this tile holds rows of the forward
+            if (j >= L && !((msk_lo >> ((j - L) & 63)) & 1ull)) s[nt][0] = -INFINITY;
+            if (j + 1 >= L && !((msk_lo >> ((j + 1 - L) & 63)) & 1ull)) s[nt][1] = -INFINITY;
+            if (j >= L && !((msk_hi >> ((j - L) & 63)) & 1ull)) s[nt][2] = -INFINITY;
+            if (j + 1 >= L && !((msk_hi >> ((j + 1 - L) & 63)) & 1ull)) s[nt][3] = -INFINITY;
+          }
           mx_lo = fmaxf(mx_lo, fmaxf(s[nt][0], s[nt][1]));
           mx_hi = fmaxf(mx_hi, fmaxf(s[nt][2], s[nt][3]));
         }
@@ -473,7 +486,7 @@ static cudaError_t attn_launch_t(const AttnArgs& a, const AttnPlan& pl, cudaStre
   p.part_o = (float*)a.workspace;
   p.part_ml = (float2*)((char*)a.workspace + ((slots * D * 4 + 255) / 256) * 256);
   p.n = a.n; p.L = a.cache_len; p.max_seq = a.max_seq; p.hq = a.hq; p.hkv = a.hkv; p.qh = pl.qh;
-  p.chunk_keys = pl.chunk_keys; p.n_chunks = pl.n_chunks; p.causal = a.causal; p.len_ptr = a.len_ptr; p.status = a.status; p.stamp = a.stamp;
+  p.chunk_keys = pl.chunk_keys; p.n_chunks = pl.n_chunks; p.causal = a.row_mask ? 0 : a.causal; p.row_mask = a.row_mask; p.len_ptr = a.len_ptr; p.status = a.status; p.stamp = a.stamp;
   static bool attr_set[MAX_DEVICES] = {};
   cudaError_t e = ensure_dynamic_smem(attn_mma_kernel<D, E, ROWS>, S::TOTAL, attr_set);
   if (e != cudaSuccess) return e;

@@ -117,7 +117,7 @@ __device__ __forceinline__ void stamp_end(KStamp* s, bool sampled = false) {
   atomicMin(&s->end_inv, ~global_ns());
 }
 
-enum { MODE_BIDIR = 0, MODE_CAUSAL = 1 };
+enum { MODE_BIDIR = 0, MODE_CAUSAL = 1, MODE_MASKED = 2 };   // MASKED: per-row bit masks among the rows + per-row position ids
 enum { DT_F32 = 0, DT_BF16 = 1, DT_FP8 = 2, DT_A8 = 3 };   // DT_A8: fp8 weights and per-row fp8 inputs (stand-alone projection only)
 // Element type of q and the KV cache on the tensor-core path.
 enum { KV_BF16 = 0, KV_F16 = 1 };

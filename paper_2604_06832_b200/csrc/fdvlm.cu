@@ -94,6 +94,7 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
   h->stamps = nullptr;
   h->stamp_used = 0;
   h->loop_exec = nullptr;
+  h->q_d = nullptr; h->q_mask = nullptr; h->q_pos_off = nullptr; h->quad_B = 0;
   cudaGetDevice(&h->device);
 
   const int R = cfg->max_block, H = cfg->hidden, I = cfg->intermediate, d = cfg->head_dim;
@@ -137,6 +138,9 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
       {(void**)&h->blk_tokens, 64 * 4},
       {(void**)&h->blk_masked, 64},
       {(void**)&h->init_stage, 64 * 4},
+      {(void**)&h->q_d, 64 * 4},
+      {(void**)&h->q_mask, 64 * 8},
+      {(void**)&h->q_pos_off, 64 * 4},
       {(void**)&h->ssq, (size_t)R * h->nt * 4},
       {(void**)&h->amax_a, h->act8 ? (size_t)R * h->nt * 4 : 16},
       {(void**)&h->amax_ao, h->act8 ? (size_t)R * cfg->n_q_heads * 4 : 16},
@@ -191,6 +195,7 @@ extern "C" int fdvlm_reset(fdvlm_t* h) {
   if (!h) return FDVLM_ERR_INVALID_ARG;
   h->cache_len = 0;
   h->block_open = 0;
+  h->quad_B = 0;
   h->block_size = h->n_remaining = h->step_index = 0;
   return FDVLM_OK;
 }
@@ -581,6 +586,85 @@ extern "C" int fdvlm_spec_block(fdvlm_t* h, int block_size, int32_t seed_token, 
   info->accepted = k;
   info->next_token = ((const int32_t*)h->host_stage)[1];
   info->cache_len = h->cache_len;
+  return FDVLM_OK;
+}
+
+// ---- quadratic self-speculative decoding (Appendix B, Alg. 2) --------------------------------------------------------
+extern "C" int fdvlm_quad_begin(fdvlm_t* h, int block_size, int32_t first_token, int chain, int32_t* draft) {
+  if (!h) return FDVLM_ERR_INVALID_ARG;
+  const int B = block_size;
+  if (B < 1) return fail(h, FDVLM_ERR_INVALID_ARG, "block_size must be positive");
+  if (first_token < 0 || first_token >= h->cfg.vocab || first_token == h->cfg.mask_id)
+    return fail(h, FDVLM_ERR_INVALID_ARG, "first token %d is not a vocabulary token", (int)first_token);
+  if (B * (B + 1) > h->cfg.max_block || B * (B + 1) > 64)
+    return fail(h, FDVLM_ERR_CAPACITY, "quadratic decoding runs B (B + 1) = %d rows per forward; max_block is %d (and at most 64)",
+                B * (B + 1), h->cfg.max_block);
+  if (h->block_open) return fail(h, FDVLM_ERR_STATE, "a block is open");
+  if (h->cache_len + B * (B + 1) > h->cfg.max_seq)
+    return fail(h, FDVLM_ERR_CAPACITY, "quad: %d + %d exceed max_seq %d", h->cache_len, B * (B + 1), h->cfg.max_seq);
+  // step 1: B mask tokens after the prompt, one denoise pass; the cache keeps the prompt only
+  h->launches = 0;
+  launch_init_block(h->blk_tokens, h->blk_masked, h->info, nullptr, B, h->cfg.mask_id, 0, h->st);
+  int rc = stage_rows(h, 0, B, h->blk_tokens, nullptr);
+  if (rc) return rc;
+  rc = forward_rows(h, B, MODE_BIDIR, B, 0);
+  if (rc) return rc;
+  launch_quad_first_draft(h->pred, first_token, B, h->q_d, h->st);
+  launch_quad_layout(B, chain ? 1 : 0, h->q_mask, h->q_pos_off, h->st);
+  h->launches += 3;
+  CU(h, cudaGetLastError());
+  if (draft) CU(h, cudaMemcpyAsync(draft, h->q_d, (size_t)B * 4, cudaMemcpyDeviceToDevice, h->st));
+  rc = sync_info(h);
+  if (rc) return rc;
+  h->quad_B = B;
+  return FDVLM_OK;
+}
+
+extern "C" int fdvlm_quad_set_draft(fdvlm_t* h, const int32_t* draft) {
+  if (!h || !draft) return FDVLM_ERR_INVALID_ARG;
+  if (!h->quad_B) return fail(h, FDVLM_ERR_STATE, "no quadratic decode is open");
+  CU(h, cudaMemcpyAsync(h->q_d, draft, (size_t)h->quad_B * 4, cudaMemcpyDeviceToDevice, h->st));
+  return FDVLM_OK;
+}
+
+extern "C" int fdvlm_quad_step(fdvlm_t* h, int32_t* accepted_tokens, int32_t* next_draft, int32_t* row_pred, float* logits,
+                               fdvlm_quad_info* info) {
+  if (!h) return FDVLM_ERR_INVALID_ARG;
+  if (!info) return fail(h, FDVLM_ERR_INVALID_ARG, "quad_step needs the host info struct");
+  if (!h->quad_B) return fail(h, FDVLM_ERR_STATE, "no quadratic decode is open");
+  if (h->block_open) return fail(h, FDVLM_ERR_STATE, "a block is open");
+  const int B = h->quad_B, n = B * (B + 1), L0 = h->cache_len;
+  if (L0 + n > h->cfg.max_seq) return fail(h, FDVLM_ERR_CAPACITY, "quad: %d + %d exceed max_seq %d", L0, n, h->cfg.max_seq);
+  h->launches = 0;
+  launch_quad_build(h->q_d, B, h->cfg.mask_id, h->blk_tokens, h->blk_masked, h->st);
+  int rc = stage_rows(h, 0, n, h->blk_tokens, nullptr);
+  if (rc) return rc;
+  rc = forward_rows(h, n, MODE_MASKED, n, logits != nullptr);
+  if (rc) return rc;
+  const cudaMemcpyKind DD = cudaMemcpyDeviceToDevice;
+  if (logits) CU(h, cudaMemcpyAsync(logits, h->logits, (size_t)n * h->cfg.vocab * 4, DD, h->st));
+  if (row_pred) CU(h, cudaMemcpyAsync(row_pred, h->pred, (size_t)n * 4, DD, h->st));
+  // verify loop on the device; the accepted tokens land in init_stage[8 ..], the count in init_stage[0]
+  launch_quad_accept(h->pred, h->q_d, B, h->init_stage + 8, h->init_stage, h->st);
+  h->launches += 2;
+  CU(h, cudaGetLastError());
+  if (accepted_tokens) CU(h, cudaMemcpyAsync(accepted_tokens, h->init_stage + 8, (size_t)B * 4, DD, h->st));
+  if (next_draft) CU(h, cudaMemcpyAsync(next_draft, h->q_d, (size_t)B * 4, DD, h->st));
+  CU(h, cudaMemcpyAsync(h->host_stage, h->init_stage, 4, cudaMemcpyDeviceToHost, h->st));
+  rc = sync_info(h);              // synchronises, and reports a timed-out device wait
+  if (rc) return rc;
+  const int k = ((const int32_t*)h->host_stage)[0];
+  if (k < 1 || k > B) return fail(h, FDVLM_ERR_CUDA, "verify kernel returned %d", k);
+  // the first tokens are the first rows of the forward: the K / V of d_0 .. d_{k-1} already sit at cache rows L0 .. L0+k-1
+  h->cache_len = L0 + k;
+  info->accepted = k;
+  info->cache_len = h->cache_len;
+  return FDVLM_OK;
+}
+
+extern "C" int fdvlm_quad_end(fdvlm_t* h) {
+  if (!h) return FDVLM_ERR_INVALID_ARG;
+  h->quad_B = 0;
   return FDVLM_OK;
 }
 

@@ -116,7 +116,7 @@ static int forward_rows_simt(fdvlm_t* h, int n, int mode, int logits_rows) {
     return 0;
   };
   const int dt = h->dt;
-  launch_rope_table(h->cs, n, h->cache_len, d, c.rope_theta, h->st);
+  launch_rope_table(h->cs, n, h->cache_len, d, c.rope_theta, h->st, nullptr, nullptr, mode == MODE_MASKED ? h->q_pos_off : nullptr);
   h->launches++;
   for (int l = 0; l < c.n_layers; ++l) {
     const fdvlm_layer_weights& lw = h->layers[l];
@@ -130,6 +130,7 @@ static int forward_rows_simt(fdvlm_t* h, int n, int mode, int logits_rows) {
     memset(&at, 0, sizeof(at));
     at.q = h->q; at.kc = kv_ptr(h, l, 0); at.vc = kv_ptr(h, l, 1); at.out = h->ao; at.n = n; at.cache_len = h->cache_len;
     at.max_seq = c.max_seq; at.hq = c.n_q_heads; at.hkv = c.n_kv_heads; at.d = d; at.causal = (mode == MODE_CAUSAL);
+    at.row_mask = (mode == MODE_MASKED) ? h->q_mask : nullptr;
     at.dtype = dt; at.workspace = h->ws; at.kv_type = KV_BF16; at.out_fmt = XF_BF16; at.long_cache = -1;
     prof_begin(h, 1);
     int r = launch_attention(at, h->st, &e);
@@ -212,7 +213,8 @@ static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int wan
     h->launches++;
     return e == cudaSuccess;
   };
-  launch_rope_table(h->cs, n, h->cache_len, d, c.rope_theta, h->st, len_ptr, stamp(FDVLM_K_ROPE_TABLE));
+  launch_rope_table(h->cs, n, h->cache_len, d, c.rope_theta, h->st, len_ptr, stamp(FDVLM_K_ROPE_TABLE),
+                    mode == MODE_MASKED ? h->q_pos_off : nullptr);
   h->launches++;
   for (int l = 0; l < c.n_layers; ++l) {
     const fdvlm_layer_weights& lw = h->layers[l];
@@ -230,6 +232,7 @@ static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int wan
     at.len_ptr = len_ptr;
     at.q = h->q; at.kc = kv_ptr(h, l, 0); at.vc = kv_ptr(h, l, 1); at.out = h->ao; at.n = n; at.cache_len = h->cache_len;
     at.max_seq = c.max_seq; at.hq = c.n_q_heads; at.hkv = c.n_kv_heads; at.d = d; at.causal = (mode == MODE_CAUSAL);
+    at.row_mask = (mode == MODE_MASKED) ? h->q_mask : nullptr;
     at.dtype = h->dt; at.workspace = h->ws; at.kv_type = h->kv_type; at.out_fmt = h->xfmt; at.out_lo_off = h->ao_lo;
     at.status = h->info + 3;
     at.amax_out = a8 ? h->amax_ao : nullptr;

@@ -56,6 +56,12 @@ struct fdvlm {
   int32_t* info;   // {n_unmasked, n_remaining, step_index, device status, poison (host-set test hook),
                    //  iterations of the on-device decode loop, 2 spare}
   int32_t* init_stage;  // [64] device staging of host-given block tokens
+  // quadratic self-speculative decoding (Appendix B, Alg. 2): the draft block, and the row masks / position offsets of
+  // its B (B + 1)-row forward (MODE_MASKED), written once per fdvlm_quad_begin
+  int32_t* q_d;                 // [64] d_0 .. d_{B-1}
+  unsigned long long* q_mask;   // [64]
+  int* q_pos_off;               // [64]
+  int quad_B;                   // 0: no quadratic decode open
   void* ws;        // GEMM split-K / attention split-KV workspace
   size_t ws_bytes;
   int32_t* info_host;  // pinned

@@ -240,8 +240,10 @@ __global__ void set_len_kernel(int* len_ptr, int value) {
 }
 void launch_set_len(int* len_ptr, int value, cudaStream_t st) { set_len_kernel<<<1, 1, 0, st>>>(len_ptr, value); }
 
+// cs[r][j] = (cos, sin) of position(r) * theta^(-j / half); position(r) = pos0 + r, or pos0 + pos_off[r] when the rows
+// carry their own position ids (Appendix B, Alg. 2: group i of the quadratic input covers positions s+i .. s+i+B)
 __global__ void rope_table_kernel(float2* __restrict__ cs, int n, int pos0, int half, double theta, const int* __restrict__ len_ptr,
-                                  KStamp* stamp) {
+                                  const int* __restrict__ pos_off, KStamp* stamp) {
   if (threadIdx.x == 0) stamp_start(stamp);
   pdl_trigger();
   pdl_wait();
@@ -251,13 +253,15 @@ __global__ void rope_table_kernel(float2* __restrict__ cs, int n, int pos0, int 
   if (idx >= n * half) return;
   int r = idx / half, j = idx % half;
   double inv = pow(theta, -(double)j / (double)half);
-  double ang = (double)(pos0 + r) * inv, s, c;
+  double ang = (double)(pos0 + (pos_off ? pos_off[r] : r)) * inv, s, c;
   sincos(ang, &s, &c);
   cs[idx] = make_float2((float)c, (float)s);
 }
-void launch_rope_table(float* cs, int n, int pos0, int head_dim, float theta, cudaStream_t st, const int* len_ptr, KStamp* stamp) {
+void launch_rope_table(float* cs, int n, int pos0, int head_dim, float theta, cudaStream_t st, const int* len_ptr, KStamp* stamp,
+                       const int* pos_off) {
   int half = head_dim / 2, total = n * half;
-  launch_pdl(rope_table_kernel, dim3((total + 127) / 128), dim3(128), 0, st, (float2*)cs, n, pos0, half, (double)theta, len_ptr, stamp);
+  launch_pdl(rope_table_kernel, dim3((total + 127) / 128), dim3(128), 0, st, (float2*)cs, n, pos0, half, (double)theta, len_ptr, pos_off,
+             stamp);
 }
 
 // rotate-half pairing (j, j + d/2); q -> q buffer, k -> cache K plane, v -> cache V plane
@@ -730,6 +734,78 @@ void launch_accept(const int32_t* a, const int32_t* d, int n, int32_t* out, cuda
   accept_kernel<<<1, 64, 0, st>>>(a, d, n, out);
 }
 
+// ---- quadratic self-speculative decoding (Appendix B, Alg. 2) --------------------------------------------------------
+// Row order of the B (B + 1) rows of one forward: rows 0 .. B-1 are the draft tokens d_0 .. d_{B-1} (the first tokens of
+// the groups), row B + i B + (j - 1) is mask token j (1 <= j <= B) of group i.  With the first tokens in front, the rows
+// whose K / V outlive the forward ("keep every (B+1)-th entry", and of those the accepted ones) are the first k staging
+// rows of the cache.
+//   pos_off[r]: position id minus the position of d_0: i for a first token, i + j for a mask token
+//   mask[r]   : bit r' = row r reads row r'.  (b) first token i reads first tokens <= i; (c) a mask token of group i reads
+//               its group's first token and all its mask tokens; (d) nothing else -- chain != 0: also the first tokens of
+//               the groups before i.
+__global__ void quad_layout_kernel(int B, int chain, unsigned long long* __restrict__ mask, int* __restrict__ pos_off) {
+  const int r = threadIdx.x, n = B * (B + 1);
+  if (r >= n) return;
+  if (r < B) {
+    mask[r] = (2ull << r) - 1ull;                              // bits 0 .. r
+    pos_off[r] = r;
+  } else {
+    const int i = (r - B) / B, j = (r - B) % B + 1;
+    const unsigned long long group = ((B == 64 ? 0ull : (1ull << B)) - 1ull) << (B + i * B);   // its B mask rows
+    unsigned long long m = group | (1ull << i);
+    if (chain) m |= (1ull << i) - 1ull;
+    mask[r] = m;
+    pos_off[r] = i + j;
+  }
+}
+void launch_quad_layout(int B, int chain, unsigned long long* mask, int* pos_off, cudaStream_t st) {
+  quad_layout_kernel<<<1, 64, 0, st>>>(B, chain, mask, pos_off);
+}
+// tokens of the rows above from the draft d
+__global__ void quad_build_kernel(const int32_t* __restrict__ d, int B, int mask_id, int32_t* __restrict__ tokens,
+                                  uint8_t* __restrict__ masked) {
+  const int r = threadIdx.x;
+  if (r >= B * (B + 1)) return;
+  tokens[r] = r < B ? d[r] : mask_id;
+  masked[r] = r >= B;
+}
+void launch_quad_build(const int32_t* d, int B, int mask_id, int32_t* tokens, uint8_t* masked, cudaStream_t st) {
+  quad_build_kernel<<<1, 64, 0, st>>>(d, B, mask_id, tokens, masked);
+}
+// Alg. 2 step 1: d_0 = the token the prompt's last row predicts, d_i = prediction of mask row i - 1 (shift by one)
+__global__ void quad_first_draft_kernel(const int32_t* __restrict__ pred, int32_t first, int B, int32_t* __restrict__ d) {
+  const int i = threadIdx.x;
+  if (i < B) d[i] = i == 0 ? first : pred[i - 1];
+}
+void launch_quad_first_draft(const int32_t* pred, int32_t first, int B, int32_t* d, cudaStream_t st) {
+  quad_first_draft_kernel<<<1, 64, 0, st>>>(pred, first, B, d);
+}
+// Alg. 2's verify loop on the predictions of one forward (P_{i,0} = pred[i], P_{i,j} = pred[B + i B + j - 1]):
+// k = 1; while k < B and P_{k-1,0} = d_k: k += 1.  accepted[0 .. k) = d_0 .. d_{k-1}; d <- P_{k-1,1..B}; out = {k}.
+__global__ void quad_accept_kernel(const int32_t* __restrict__ pred, int32_t* __restrict__ d, int B, int32_t* __restrict__ accepted,
+                                   int32_t* __restrict__ out) {
+  __shared__ int k_s;
+  __shared__ int32_t old_d[64];
+  const int t = threadIdx.x;
+  if (t < B) old_d[t] = d[t];
+  __syncthreads();
+  if (t == 0) {
+    int k = 1;
+    while (k < B && pred[k - 1] == old_d[k]) ++k;
+    k_s = k;
+    out[0] = k;
+  }
+  __syncthreads();
+  const int k = k_s;
+  if (t < B) {
+    if (accepted) accepted[t] = t < k ? old_d[t] : -1;
+    d[t] = pred[B + (k - 1) * B + t];
+  }
+}
+void launch_quad_accept(const int32_t* pred, int32_t* d, int B, int32_t* accepted, int32_t* out, cudaStream_t st) {
+  quad_accept_kernel<<<1, 64, 0, st>>>(pred, d, B, accepted, out);
+}
+
 __global__ void init_block_kernel(int32_t* tokens, uint8_t* masked, int32_t* info, const int32_t* init, int n, int mask_id,
                                   int step) {
   int i = threadIdx.x;
@@ -751,7 +827,8 @@ void launch_init_block(int32_t* tokens, uint8_t* masked, int32_t* info, const in
 template <typename AT>
 __global__ void __launch_bounds__(128) attn_simt_kernel(const AT* __restrict__ q, const AT* __restrict__ kc,
                                                         const AT* __restrict__ vc, AT* __restrict__ out, int n,
-                                                        int L, int max_seq, int hq, int hkv, int d, int causal) {
+                                                        int L, int max_seq, int hq, int hkv, int d, int causal,
+                                                        const unsigned long long* __restrict__ row_mask) {
   extern __shared__ float smem[];
   float* qs = smem;          // [d]
   float* red = smem + d;     // [32]
@@ -773,6 +850,8 @@ __global__ void __launch_bounds__(128) attn_simt_kernel(const AT* __restrict__ q
     float p = 0.f;
     for (int e = 0; e < epl; ++e) p = fmaf(qs[lane * epl + e], to_f32(kr[e]), p);
     p = warp_sum(p);
+    // explicit mask among the n rows: bit r' of row_mask[r] = row r reads row r' (the cache is always read)
+    if (row_mask && j >= L && !((row_mask[r] >> (j - L)) & 1ull)) p = -INFINITY;
     if (lane == 0) sc[j] = p;
   }
   __syncthreads();
@@ -802,12 +881,12 @@ int launch_attention_simt(const AttnArgs& a, cudaStream_t st, cudaError_t* err) 
     if (smem > 48 * 1024) *err = cudaFuncSetAttribute(attn_simt_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (*err != cudaSuccess) return -1;
     attn_simt_kernel<float><<<grid, 128, smem, st>>>((const float*)a.q, (const float*)a.kc, (const float*)a.vc,
-                                                     (float*)a.out, a.n, a.cache_len, a.max_seq, a.hq, a.hkv, a.d, a.causal);
+                                                     (float*)a.out, a.n, a.cache_len, a.max_seq, a.hq, a.hkv, a.d, a.causal, a.row_mask);
   } else {
     if (smem > 48 * 1024) *err = cudaFuncSetAttribute(attn_simt_kernel<bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (*err != cudaSuccess) return -1;
     attn_simt_kernel<bf16><<<grid, 128, smem, st>>>((const bf16*)a.q, (const bf16*)a.kc, (const bf16*)a.vc, (bf16*)a.out,
-                                                    a.n, a.cache_len, a.max_seq, a.hq, a.hkv, a.d, a.causal);
+                                                    a.n, a.cache_len, a.max_seq, a.hq, a.hkv, a.d, a.causal, a.row_mask);
   }
   *err = cudaGetLastError();
   return *err == cudaSuccess ? 1 : -1;

@@ -34,7 +34,12 @@ void launch_bf16_rows_to_f16_amax(const void* in, void* out, int m, int k, float
 void launch_rows_to_f32(const void* rows, float* h, int n, int hidden, int dtype, cudaStream_t st);
 void launch_rmsnorm(const float* h, const float* g, void* out, int n, int hidden, float eps, int dtype, cudaStream_t st);
 void launch_rope_table(float* cs, int n, int pos0, int head_dim, float theta, cudaStream_t st, const int* len_ptr = nullptr,
-                       KStamp* stamp = nullptr);
+                       KStamp* stamp = nullptr, const int* pos_off = nullptr);
+// quadratic self-speculative decoding (Appendix B, Alg. 2): row layout, input tokens, first draft, verify loop
+void launch_quad_layout(int B, int chain, unsigned long long* mask, int* pos_off, cudaStream_t st);
+void launch_quad_build(const int32_t* d, int B, int mask_id, int32_t* tokens, uint8_t* masked, cudaStream_t st);
+void launch_quad_first_draft(const int32_t* pred, int32_t first, int B, int32_t* d, cudaStream_t st);
+void launch_quad_accept(const int32_t* pred, int32_t* d, int B, int32_t* accepted, int32_t* out, cudaStream_t st);
 void launch_set_len(int* len_ptr, int value, cudaStream_t st);
 // qkv fp32 [n, (Hq + 2 Hkv) d] -> q (act type) [n, Hq, d] rotated; K (rotated) and V written into the
 // layer's cache planes [Hkv, max_seq, d] at positions pos0 .. pos0 + n - 1.
@@ -122,6 +127,8 @@ struct AttnArgs {
   int kv_type;          // tensor-core kernel: element type of q, kc, vc (KV_BF16 / KV_F16)
   int out_fmt;          // tensor-core kernel: storage of `out` (XF_*), lo plane out_lo_off elements on
   size_t out_lo_off;
+  const unsigned long long* row_mask;   // nullable, n <= 64 words: bit r' of word r = row r reads row r' of this forward
+                                        // (the cached keys are always read); overrides `causal`
   int long_cache;       // tensor-core kernel: -1 pick the CTA shape from cache_len; 0 / 1 the short- / long-cache shape
                         // (a captured launch serves every later length of its class)
   void* workspace;
