@@ -188,12 +188,6 @@ __global__ void __launch_bounds__(AtSmem<D, ROWS>::THREADS, ROWS == 64 ? 2 : 1) 
     const int lim_lo = (r_lo < m_valid) ? (p.causal ? L + (r_lo % n) + 1 : T) : 0;
     const int lim_hi = (r_hi < m_valid) ? (p.causal ? L + (r_hi % n) + 1 : T) : 0;
     const float sl2 = rsqrtf((float)D) * LOG2E;       // scores kept in the log2 domain
-    // explicit mask among the forward's own rows (keys L .. L+n-1); set up by the host before the chain, not by a kernel of it
-    unsigned long long msk_lo = ~0ull, msk_hi = ~0ull;
-    if (p.row_mask) {
-      if (r_lo < m_valid) msk_lo = p.row_mask[r_lo % n];
-      if (r_hi < m_valid) msk_hi = p.row_mask[r_hi % n];
-    }
 
     uint32_t qf[D / 16][4];
 #pragma unroll
@@ -238,6 +232,21 @@ __global__ void __launch_bounds__(AtSmem<D, ROWS>::THREADS, ROWS == 64 ? 2 : 1) 
             mma_16816<E>(s[2 * np + 1], qf[kk], b2, b3);
           }
         }
+        // explicit mask among the forward's own rows (keys L .. L+n-1; the words are set up before the chain, not by a
+        // kernel of it).  Only the last tile or two hold such keys, so the words are fetched there and kept out of the
+        // main loop's registers.
+        if (p.row_mask && j0 + AT_KEYS > L) {                // uniform over the warp
+          const unsigned long long msk_lo = (r_lo < m_valid) ? p.row_mask[r_lo % n] : 0ull;
+          const unsigned long long msk_hi = (r_hi < m_valid) ? p.row_mask[r_hi % n] : 0ull;
+#pragma unroll
+          for (int nt = 0; nt < AT_KEYS / 8; ++nt) {
+            const int j = j0 + nt * 8 + tq * 2;
+            if (j >= L && !((msk_lo >> ((j - L) & 63)) & 1ull)) s[nt][0] = -INFINITY;
+            if (j + 1 >= L && !((msk_lo >> ((j + 1 - L) & 63)) & 1ull)) s[nt][1] = -INFINITY;
+            if (j >= L && !((msk_hi >> ((j - L) & 63)) & 1ull)) s[nt][2] = -INFINITY;
+            if (j + 1 >= L && !((msk_hi >> ((j + 1 - L) & 63)) & 1ull)) s[nt][3] = -INFINITY;
+          }
+        }
         // mask + running max
         float mx_lo = -INFINITY, mx_hi = -INFINITY;
 #pragma unroll
@@ -247,12 +256,6 @@ __global__ void __launch_bounds__(AtSmem<D, ROWS>::THREADS, ROWS == 64 ? 2 : 1) 
           s[nt][1] = (j + 1 < lim_lo) ? s[nt][1] * sl2 : -INFINITY;
           s[nt][2] = (j < lim_hi) ? s[nt][2] * sl2 : -INFINITY;
           s[nt][3] = (j + 1 < lim_hi) ? s[nt][3] * sl2 : -INFINITY;
-          if (p.row_mask && j0 + AT_KEYS > L) {              // uniform over the warp: this tile holds rows of the forward
-            if (j >= L && !((msk_lo >> ((j - L) & 63)) & 1ull)) s[nt][0] = -INFINITY;
-            if (j + 1 >= L && !((msk_lo >> ((j + 1 - L) & 63)) & 1ull)) s[nt][1] = -INFINITY;
-            if (j >= L && !((msk_hi >> ((j - L) & 63)) & 1ull)) s[nt][2] = -INFINITY;
-            if (j + 1 >= L && !((msk_hi >> ((j + 1 - L) & 63)) & 1ull)) s[nt][3] = -INFINITY;
-          }
           mx_lo = fmaxf(mx_lo, fmaxf(s[nt][0], s[nt][1]));
           mx_hi = fmaxf(mx_hi, fmaxf(s[nt][2], s[nt][3]));
         }
