@@ -127,3 +127,34 @@ def test_w8a8_model_is_as_close_to_the_oracle_as_rounding_allows(shape, B_, L_e,
         effect = np.abs(ref - unq).reshape(L, -1).max(axis=1)
         assert np.median(per_row) <= 0.25 * np.median(effect), (np.median(per_row), np.median(effect))
         assert _rms(got - ref) <= 0.35 * _rms(ref - unq), (_rms(got - ref), _rms(ref - unq))
+
+
+def test_w8a8_give_up_path_and_recovery():
+    """The quantising GEMM kind under the poison flag: every role (the converter warps included) leaves by the branch a
+    timed-out wait takes, the call reports FDVLM_ERR_TIMEOUT, and after the flag is cleared the handle computes, bit for
+    bit, what it computed before (the path is deterministic)."""
+    b = B()
+    w = I.make_weights(SMALL, 7, gain_spread=0.5)
+    st = torch.cuda.Stream()
+    h = b.Handle(SMALL, b.weights_to_device(w), max_seq=128, max_block=64, stream=st)
+    emb, toks = I.make_prefix(SMALL, 10, 14, 3)
+    lg = [torch.empty(16, SMALL.vocab, dtype=torch.float32, device="cuda") for _ in range(2)]
+    with torch.cuda.stream(st):
+        h.prefill(emb.cuda(), toks.cuda())
+        h.block_begin(16)
+        h.block_step(b.RULE_TOPK, 0.0, 4, logits=lg[0])
+        h.synchronize()
+        h.reset()
+        h.debug_poison(True)
+        h.prefill(emb.cuda(), toks.cuda())
+        with pytest.raises(b.FdvlmError) as e:
+            h.synchronize()
+        assert e.value.code == b.ERR_TIMEOUT
+        h.debug_poison(False)
+        h.reset()
+        h.prefill(emb.cuda(), toks.cuda())
+        h.block_begin(16)
+        h.block_step(b.RULE_TOPK, 0.0, 4, logits=lg[1])
+        h.synchronize()
+    assert torch.equal(lg[0], lg[1])
+    h.close()
