@@ -186,8 +186,9 @@ def test_small_bf16_peaked_discrete_parity():
     emb, toks = I.make_prefix(SMALL_BF16, 20, 20, 4)
     oracle.prefill(I.as_numpy_storage(emb), toks.numpy(), want_logits=False)
     handle.prefill(*upload_prefix(emb, toks))
-    stats = replay_decode(oracle, handle, SMALL_BF16, 32, orc.THRESHOLD, 0.9, n_blocks=1, tol=dict(logits=0.5, conf=5e-2, gap=1.0))
-    assert stats.get("rows_sure", 0) > 0
+    stats = replay_decode(oracle, handle, SMALL_BF16, 32, orc.THRESHOLD, 0.9, n_blocks=1, tol=dict(gap=2 * TOL[I.BF16]["logits"], **TOL[I.BF16]))     # the stated bf16 bounds, although the final gain is 16
+    print("peaked small bf16:", stats)
+    assert stats.get("rows_sure", 0) > 100 and stats.get("steps_clear", 0) > 0
     handle.close()
 
 
