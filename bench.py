@@ -212,7 +212,10 @@ def run_ours(args, wl, block):
     stream = torch.cuda.Stream()
     # the 7B configuration prescribes a bf16 KV cache; the others leave the cache's element type open
     kv_dtype = B.KV_BF16 if shape.dtype in (I.FP8, I.W8A8) else B.KV_F16
-    handle = B.Handle(shape, weights, max_seq=max_seq, max_block=max(block, 32), stream=stream, kv_dtype=kv_dtype)
+    # top-k schedules: the commit of block t rides in the forward of block t+1's first step (one forward over 2 x block rows)
+    fused_commit = wl.rule == "topk" and 2 * block <= 64
+    handle = B.Handle(shape, weights, max_seq=max_seq, max_block=max(2 * block if fused_commit else block, 32), stream=stream,
+                      kv_dtype=kv_dtype)
     emb, toks = I.make_prefix(shape, wl.n_embeds, wl.n_tokens, wl.prefix_seed)
     emb_d, toks_d = emb.cuda(), toks.cuda()
     rule = B.RULE_TOPK if wl.rule == "topk" else B.RULE_THRESHOLD
@@ -229,9 +232,22 @@ def run_ours(args, wl, block):
         prefill_ms = t0.elapsed_time(t1)
 
         launches = [0]
+        open_block = [False]          # fused_commit: the block decoded by the previous call, not yet committed
+
+        def close_open_block():
+            if open_block[0]:
+                handle.commit_block()
+                open_block[0] = False
 
         def one_block_device():
-            if wl.rule == "topk":      # fixed schedule: every step enqueued without a host round trip in between
+            if fused_commit:
+                # fixed schedule, every step enqueued without a host round trip in between; the previous call's block is
+                # committed by this call's first forward.  Per call: one block committed, one block decoded.
+                info = handle.commit_decode_block_topk(block, wl.k)
+                launches[0] += handle.last_launch_count()
+                open_block[0] = True
+                return info.step_index
+            if wl.rule == "topk":
                 info = handle.decode_block_topk(block, wl.k)
                 launches[0] += handle.last_launch_count()
                 handle.commit_block()
@@ -263,6 +279,17 @@ def run_ours(args, wl, block):
         init_h = torch.full((block,), shape.mask_id, dtype=torch.int32).pin_memory()
 
         def one_block_host():
+            if fused_commit:
+                if open_block[0]:
+                    info = handle.commit_begin_step_host(block, rule, wl.threshold, wl.k, next_init_tokens=init_h, conf=conf_h,
+                                                         pred=pred_h, unmask=um_h, block_tokens=tok_h)
+                else:
+                    handle.block_begin_host(block, init_h)
+                    info = handle.block_step_host(rule, wl.threshold, wl.k, conf=conf_h, pred=pred_h, unmask=um_h, block_tokens=tok_h)
+                while info.n_remaining:
+                    info = handle.block_step_host(rule, wl.threshold, wl.k, conf=conf_h, pred=pred_h, unmask=um_h, block_tokens=tok_h)
+                open_block[0] = True
+                return
             handle.block_begin_host(block, init_h)
             while True:
                 info = handle.block_step_host(rule, wl.threshold, wl.k, conf=conf_h, pred=pred_h, unmask=um_h, block_tokens=tok_h)
@@ -293,6 +320,7 @@ def run_ours(args, wl, block):
         # end to end: host buffers through the C ABI (H2D of the block's init tokens, D2H of every step's results)
         one_block_host()
         ms_e2e = timed(one_block_host, K)
+        close_open_block()
 
         # (1) the projection launches timed one by one with CUDA events (kernels launched singly: no overlap)
         handle.profile_enable(1)
@@ -431,6 +459,9 @@ def run_ours(args, wl, block):
         "dtype": {"f32": "f32", "bf16": "bf16", "fp8": "f16 x e4m3 weights", "w8a8": "e4m3 x e4m3 (per-token activation scales)"}[shape.dtype], "data": "synthetic",
         "config": config_of(wl, block, world),
         "kv_dtype": "bf16" if kv_dtype == B.KV_BF16 else "f16",
+        # per block: n denoise steps + one causal commit; with fused_commit the commit of block t and the first step of
+        # block t+1 are one forward over 2 x block rows (same results, every weight byte streamed once for both)
+        "forwards_per_block": (n_steps if fused_commit else n_steps + 1), "fused_commit": fused_commit,
         "e2e": {"value": e2e_value, "unit": "tok/s", "h2d_bytes_per_step": block * 4,
                 "d2h_bytes_per_step": n_steps * (block * 13 + 32)},
         "gpu_launches": n_launch,

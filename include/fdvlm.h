@@ -197,6 +197,28 @@ int fdvlm_commit_block(fdvlm_t *h, float *next_logits);
  * next_logits device fp32 [vocab]; all nullable. */
 int fdvlm_commit_block_verify(fdvlm_t *h, int32_t *row_pred, float *row_conf, float *next_logits);
 
+/* fdvlm_commit_block, fdvlm_block_begin and the first fdvlm_block_step of the next block as ONE forward over
+ * B_finished + B_next rows (Sec. 3.3: clean context is causal, M_C2C; a noisy block reads the clean context before it,
+ * M_N2C, and itself bidirectionally, M_N2N -- the same three masks in one pass): the finished rows run causally among
+ * themselves and their K / V land at the positions they are committed to; the next block's rows read the cache, the
+ * finished rows and one another.  Results are those of the three calls made one after the other (same arithmetic on
+ * other tile shapes); every weight byte is streamed once instead of twice.  Needs B_finished + B_next <=
+ * min(max_block, 64) (FDVLM_ERR_CAPACITY otherwise: use the three calls).
+ *   next_logits   device fp32 [vocab], nullable: logits of the finished block's last row, as from fdvlm_commit_block
+ *   next_init_tokens, p, logits .. info: as for fdvlm_block_begin / fdvlm_block_step, for the next block
+ * The _host variant takes and returns host buffers like fdvlm_block_begin_host / fdvlm_block_step_host.
+ * Errors: STATE if no block is open or masked positions remain in it; otherwise as the three calls. */
+int fdvlm_commit_begin_step(fdvlm_t *h, float *next_logits, int next_block_size, const int32_t *next_init_tokens,
+                            const fdvlm_step_params *p, float *logits, float *conf, int32_t *pred, uint8_t *unmask,
+                            int32_t *block_tokens, fdvlm_step_info *info);
+int fdvlm_commit_begin_step_host(fdvlm_t *h, int next_block_size, const int32_t *next_init_tokens_host,
+                                 const fdvlm_step_params *p, float *conf_host, int32_t *pred_host, uint8_t *unmask_host,
+                                 int32_t *block_tokens_host, fdvlm_step_info *info);
+/* fdvlm_decode_block_topk that first commits the open, fully revealed block, if there is one, in the same forward as the
+ * new block's first step (as above); with no block open it is fdvlm_decode_block_topk. */
+int fdvlm_commit_decode_block_topk(fdvlm_t *h, int block_size, const int32_t *init_tokens, int k, int pred_shift,
+                                   int32_t *block_tokens, fdvlm_step_info *info);
+
 /* Drop committed positions from the end of the cache: cache_len = new_len (Alg. 1 "Crop").  The dropped K/V rows
  * are simply overwritten by later commits.  Errors: STATE inside an open block; INVALID_ARG unless
  * 0 <= new_len <= cache_len. */

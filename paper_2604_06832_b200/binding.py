@@ -86,6 +86,11 @@ EXPORTS = {
                                         C.c_void_p, C.POINTER(StepInfo)]),
     "fdvlm_block_set_tokens": (C.c_int, [C.c_void_p, C.c_void_p]),
     "fdvlm_decode_block_topk": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.POINTER(StepInfo)]),
+    "fdvlm_commit_decode_block_topk": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.POINTER(StepInfo)]),
+    "fdvlm_commit_begin_step": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.POINTER(StepParams), C.c_void_p, C.c_void_p,
+                                          C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(StepInfo)]),
+    "fdvlm_commit_begin_step_host": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.POINTER(StepParams), C.c_void_p, C.c_void_p,
+                                               C.c_void_p, C.c_void_p, C.POINTER(StepInfo)]),
     "fdvlm_commit_block": (C.c_int, [C.c_void_p, C.c_void_p]),
     "fdvlm_commit_block_verify": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "fdvlm_truncate": (C.c_int, [C.c_void_p, C.c_int]),
@@ -236,6 +241,30 @@ class Handle:
         p, info = StepParams(rule, threshold, k, pred_shift), StepInfo()
         self._check(lib().fdvlm_block_step_host(self._h, C.byref(p), _ptr(conf), _ptr(pred), _ptr(unmask),
                                                 _ptr(block_tokens), C.byref(info)))
+        return info
+
+    def commit_begin_step(self, next_block_size: int, rule: int, threshold: float = 0.9, k: int = 8, next_logits=None,
+                          next_init_tokens=None, logits=None, conf=None, pred=None, unmask=None, block_tokens=None,
+                          pred_shift: int = 0) -> StepInfo:
+        p, info = StepParams(rule, threshold, k, pred_shift), StepInfo()
+        self._check(lib().fdvlm_commit_begin_step(self._h, _ptr(next_logits), next_block_size, _ptr(next_init_tokens), C.byref(p),
+                                                  _ptr(logits), _ptr(conf), _ptr(pred), _ptr(unmask), _ptr(block_tokens),
+                                                  C.byref(info)))
+        self._remaining = info.n_remaining
+        return info
+
+    def commit_begin_step_host(self, next_block_size: int, rule: int, threshold: float = 0.9, k: int = 8, next_init_tokens=None,
+                               conf=None, pred=None, unmask=None, block_tokens=None, pred_shift: int = 0) -> StepInfo:
+        p, info = StepParams(rule, threshold, k, pred_shift), StepInfo()
+        self._check(lib().fdvlm_commit_begin_step_host(self._h, next_block_size, _ptr(next_init_tokens), C.byref(p), _ptr(conf),
+                                                       _ptr(pred), _ptr(unmask), _ptr(block_tokens), C.byref(info)))
+        return info
+
+    def commit_decode_block_topk(self, block_size: int, k: int, init_tokens: Optional[torch.Tensor] = None, pred_shift: int = 0,
+                                 block_tokens: Optional[torch.Tensor] = None) -> StepInfo:
+        info = StepInfo()
+        self._check(lib().fdvlm_commit_decode_block_topk(self._h, block_size, _ptr(init_tokens), k, pred_shift,
+                                                         _ptr(block_tokens), C.byref(info)))
         return info
 
     def decode_block_topk(self, block_size: int, k: int, init_tokens: Optional[torch.Tensor] = None, pred_shift: int = 0,

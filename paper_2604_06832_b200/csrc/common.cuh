@@ -117,7 +117,9 @@ __device__ __forceinline__ void stamp_end(KStamp* s, bool sampled = false) {
   atomicMin(&s->end_inv, ~global_ns());
 }
 
-enum { MODE_BIDIR = 0, MODE_CAUSAL = 1, MODE_MASKED = 2 };   // MASKED: per-row bit masks among the rows + per-row position ids
+// MASKED: per-row bit masks among the rows + per-row position ids (Appendix B, Alg. 2).  FUSED: the causal commit of a
+// finished block and the first denoise step of the next block as one forward (per-row bit masks, natural positions).
+enum { MODE_BIDIR = 0, MODE_CAUSAL = 1, MODE_MASKED = 2, MODE_FUSED = 3 };
 enum { DT_F32 = 0, DT_BF16 = 1, DT_FP8 = 2, DT_A8 = 3 };   // DT_A8: fp8 weights and per-row fp8 inputs (stand-alone projection only)
 // Element type of q and the KV cache on the tensor-core path.
 enum { KV_BF16 = 0, KV_F16 = 1 };

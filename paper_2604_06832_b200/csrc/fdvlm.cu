@@ -95,6 +95,7 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
   h->stamp_used = 0;
   h->loop_exec = nullptr;
   h->q_d = nullptr; h->q_mask = nullptr; h->q_pos_off = nullptr; h->quad_B = 0;
+  h->f_rows = nullptr; h->f_mask = nullptr;
   cudaGetDevice(&h->device);
 
   const int R = cfg->max_block, H = cfg->hidden, I = cfg->intermediate, d = cfg->head_dim;
@@ -141,6 +142,8 @@ extern "C" int fdvlm_create(const fdvlm_config* cfg, const fdvlm_weights* w, voi
       {(void**)&h->q_d, 64 * 4},
       {(void**)&h->q_mask, 64 * 8},
       {(void**)&h->q_pos_off, 64 * 4},
+      {(void**)&h->f_rows, 64 * 4},
+      {(void**)&h->f_mask, 64 * 8},
       {(void**)&h->ssq, (size_t)R * h->nt * 4},
       {(void**)&h->amax_a, h->act8 ? (size_t)R * h->nt * 4 : 16},
       {(void**)&h->amax_ao, h->act8 ? (size_t)R * cfg->n_q_heads * 4 : 16},
@@ -532,6 +535,121 @@ extern "C" int fdvlm_commit_block_verify(fdvlm_t* h, int32_t* row_pred, float* r
   if (row_pred) CU(h, cudaMemcpyAsync(row_pred, h->pred, (size_t)B * 4, DD, h->st));
   if (row_conf) CU(h, cudaMemcpyAsync(row_conf, h->conf, (size_t)B * 4, DD, h->st));
   if (next_logits) CU(h, cudaMemcpyAsync(next_logits, h->logits + (size_t)(B - 1) * h->cfg.vocab, (size_t)h->cfg.vocab * 4, DD, h->st));
+  return FDVLM_OK;
+}
+
+// ---- commit of the finished block + first denoise step of the next block as ONE forward ---------------------------------
+// Rows [finished block ; next block]: the finished rows run causally among themselves and their K / V are staged at the
+// positions they are committed to; the next block's rows read them, the cache and one another.  Every weight byte is
+// streamed once instead of twice.
+static int commit_step_core(fdvlm_t* h, int Bn, const int32_t* init_dev, const fdvlm_step_params* p, int want_logits) {
+  if (!h) return FDVLM_ERR_INVALID_ARG;
+  int prc = check_step_params(h, p);
+  if (prc) return prc;
+  if (!h->block_open) return fail(h, FDVLM_ERR_STATE, "commit without an open block");
+  if (h->n_remaining != 0) return fail(h, FDVLM_ERR_STATE, "commit with %d masked positions left", h->n_remaining);
+  const int Bc = h->block_size, n = Bc + Bn;
+  if (Bn < 1) return fail(h, FDVLM_ERR_INVALID_ARG, "block_size must be positive");
+  if (n > h->cfg.max_block || n > 64)
+    return fail(h, FDVLM_ERR_CAPACITY, "commit + step in one forward needs %d + %d rows; max_block is %d (and at most 64)", Bc, Bn,
+                h->cfg.max_block);
+  if (h->cache_len + n > h->cfg.max_seq)
+    return fail(h, FDVLM_ERR_CAPACITY, "block: %d + %d exceed max_seq %d", h->cache_len, n, h->cfg.max_seq);
+  h->launches = 0;
+  launch_fuse_begin(h->blk_tokens, h->blk_masked, Bc, init_dev, Bn, h->cfg.mask_id, h->f_rows, h->f_mask, h->info, h->st);
+  CU(h, cudaGetLastError());
+  if (init_dev) {                  // the masked count of the given tokens
+    int rc = sync_info(h);
+    if (rc) return rc;
+  } else {
+    h->n_remaining = Bn;
+  }
+  int rc = stage_rows(h, 0, n, h->f_rows, nullptr);
+  if (rc) return rc;
+  rc = forward_rows(h, n, MODE_FUSED, n, want_logits);
+  if (rc) return rc;
+  launch_select(h->conf + Bc, h->pred + Bc, h->blk_tokens, h->blk_masked, h->unmask, h->info, Bn, (int)p->rule, p->threshold, p->k,
+                h->st, p->pred_shift);
+  h->launches += 2;
+  CU(h, cudaGetLastError());
+  h->cache_len += Bc;
+  h->block_size = Bn;
+  h->block_open = 1;
+  h->step_index = 1;
+  return FDVLM_OK;
+}
+
+extern "C" int fdvlm_commit_begin_step(fdvlm_t* h, float* next_logits, int next_block_size, const int32_t* next_init_tokens,
+                                       const fdvlm_step_params* p, float* logits, float* conf, int32_t* pred, uint8_t* unmask,
+                                       int32_t* block_tokens, fdvlm_step_info* info) {
+  if (!h) return FDVLM_ERR_INVALID_ARG;
+  const int Bc = h->block_size, B = next_block_size;
+  int rc = commit_step_core(h, B, next_init_tokens, p, (logits != nullptr || next_logits != nullptr) ? 1 : 0);
+  if (rc) return rc;
+  const size_t V = (size_t)h->cfg.vocab;
+  const cudaMemcpyKind DD = cudaMemcpyDeviceToDevice;
+  if (next_logits) CU(h, cudaMemcpyAsync(next_logits, h->logits + (size_t)(Bc - 1) * V, V * 4, DD, h->st));
+  if (logits) CU(h, cudaMemcpyAsync(logits, h->logits + (size_t)Bc * V, (size_t)B * V * 4, DD, h->st));
+  if (conf) CU(h, cudaMemcpyAsync(conf, h->conf + Bc, (size_t)B * 4, DD, h->st));
+  if (pred) CU(h, cudaMemcpyAsync(pred, h->pred + Bc, (size_t)B * 4, DD, h->st));
+  if (unmask) CU(h, cudaMemcpyAsync(unmask, h->unmask, (size_t)B, DD, h->st));
+  if (block_tokens) CU(h, cudaMemcpyAsync(block_tokens, h->blk_tokens, (size_t)B * 4, DD, h->st));
+  return finish_info(h, info);
+}
+
+extern "C" int fdvlm_commit_begin_step_host(fdvlm_t* h, int next_block_size, const int32_t* next_init_tokens_host,
+                                            const fdvlm_step_params* p, float* conf_host, int32_t* pred_host,
+                                            uint8_t* unmask_host, int32_t* block_tokens_host, fdvlm_step_info* info) {
+  if (!h) return FDVLM_ERR_INVALID_ARG;
+  const int Bc = h->block_size, B = next_block_size;
+  if (B < 1 || B > 64) return fail(h, FDVLM_ERR_INVALID_ARG, "block_size out of range");
+  const int32_t* init_dev = nullptr;
+  if (next_init_tokens_host) {
+    memcpy(h->host_stage, next_init_tokens_host, (size_t)B * 4);
+    CU(h, cudaMemcpyAsync(h->init_stage, h->host_stage, (size_t)B * 4, cudaMemcpyHostToDevice, h->st));
+    init_dev = h->init_stage;
+  }
+  int rc = commit_step_core(h, B, init_dev, p, 0);
+  if (rc) return rc;
+  char* s = h->host_stage;  // [conf 256 | pred 256 | tokens 256 | unmask 64]
+  const cudaMemcpyKind DH = cudaMemcpyDeviceToHost;
+  if (conf_host) CU(h, cudaMemcpyAsync(s, h->conf + Bc, (size_t)B * 4, DH, h->st));
+  if (pred_host) CU(h, cudaMemcpyAsync(s + 256, h->pred + Bc, (size_t)B * 4, DH, h->st));
+  if (block_tokens_host) CU(h, cudaMemcpyAsync(s + 512, h->blk_tokens, (size_t)B * 4, DH, h->st));
+  if (unmask_host) CU(h, cudaMemcpyAsync(s + 768, h->unmask, (size_t)B, DH, h->st));
+  rc = finish_info(h, info);
+  if (rc) return rc;
+  if (conf_host) memcpy(conf_host, s, (size_t)B * 4);
+  if (pred_host) memcpy(pred_host, s + 256, (size_t)B * 4);
+  if (block_tokens_host) memcpy(block_tokens_host, s + 512, (size_t)B * 4);
+  if (unmask_host) memcpy(unmask_host, s + 768, (size_t)B);
+  return FDVLM_OK;
+}
+
+extern "C" int fdvlm_commit_decode_block_topk(fdvlm_t* h, int block_size, const int32_t* init_tokens, int k, int pred_shift,
+                                              int32_t* block_tokens, fdvlm_step_info* info) {
+  if (!h) return FDVLM_ERR_INVALID_ARG;
+  if (!h->block_open) return fdvlm_decode_block_topk(h, block_size, init_tokens, k, pred_shift, block_tokens, info);
+  if (!info) return fail(h, FDVLM_ERR_INVALID_ARG, "commit_decode_block_topk needs the host info struct");
+  if (k < 1) return fail(h, FDVLM_ERR_INVALID_ARG, "top-k needs k >= 1");
+  fdvlm_step_params p;
+  p.rule = FDVLM_RULE_TOPK; p.threshold = 0.f; p.k = k; p.pred_shift = pred_shift;
+  int rc = commit_step_core(h, block_size, init_tokens, &p, 0);
+  if (rc) return rc;
+  const int steps = (h->n_remaining + k - 1) / k;      // of which the first has just run
+  int launches = h->launches;
+  for (int s = 1; s < steps; ++s) {
+    h->n_remaining = 1;            // the device keeps the true count; the host checks it once, below
+    rc = step_core(h, &p, 0);
+    if (rc) return rc;
+    launches += h->launches;
+  }
+  h->launches = launches;
+  if (block_tokens) CU(h, cudaMemcpyAsync(block_tokens, h->blk_tokens, (size_t)block_size * 4, cudaMemcpyDeviceToDevice, h->st));
+  rc = sync_info(h);
+  if (rc) return rc;
+  info->n_unmasked = h->info_host[0]; info->n_remaining = h->info_host[1]; info->step_index = h->info_host[2];
+  if (h->n_remaining != 0) return fail(h, FDVLM_ERR_STATE, "%d masked positions left after %d top-%d steps", h->n_remaining, steps, k);
   return FDVLM_OK;
 }
 

@@ -130,7 +130,7 @@ static int forward_rows_simt(fdvlm_t* h, int n, int mode, int logits_rows) {
     memset(&at, 0, sizeof(at));
     at.q = h->q; at.kc = kv_ptr(h, l, 0); at.vc = kv_ptr(h, l, 1); at.out = h->ao; at.n = n; at.cache_len = h->cache_len;
     at.max_seq = c.max_seq; at.hq = c.n_q_heads; at.hkv = c.n_kv_heads; at.d = d; at.causal = (mode == MODE_CAUSAL);
-    at.row_mask = (mode == MODE_MASKED) ? h->q_mask : nullptr;
+    at.row_mask = (mode == MODE_MASKED) ? h->q_mask : (mode == MODE_FUSED ? h->f_mask : nullptr);
     at.dtype = dt; at.workspace = h->ws; at.kv_type = KV_BF16; at.out_fmt = XF_BF16; at.long_cache = -1;
     prof_begin(h, 1);
     int r = launch_attention(at, h->st, &e);
@@ -232,7 +232,7 @@ static int forward_rows_tc(fdvlm_t* h, int n, int mode, int logits_rows, int wan
     at.len_ptr = len_ptr;
     at.q = h->q; at.kc = kv_ptr(h, l, 0); at.vc = kv_ptr(h, l, 1); at.out = h->ao; at.n = n; at.cache_len = h->cache_len;
     at.max_seq = c.max_seq; at.hq = c.n_q_heads; at.hkv = c.n_kv_heads; at.d = d; at.causal = (mode == MODE_CAUSAL);
-    at.row_mask = (mode == MODE_MASKED) ? h->q_mask : nullptr;
+    at.row_mask = (mode == MODE_MASKED) ? h->q_mask : (mode == MODE_FUSED ? h->f_mask : nullptr);
     at.dtype = h->dt; at.workspace = h->ws; at.kv_type = h->kv_type; at.out_fmt = h->xfmt; at.out_lo_off = h->ao_lo;
     at.status = h->info + 3;
     at.amax_out = a8 ? h->amax_ao : nullptr;

@@ -62,6 +62,9 @@ struct fdvlm {
   unsigned long long* q_mask;   // [64]
   int* q_pos_off;               // [64]
   int quad_B;                   // 0: no quadratic decode open
+  // commit + first step of the next block as one forward (MODE_FUSED): its rows' tokens and row masks
+  int32_t* f_rows;              // [64]
+  unsigned long long* f_mask;   // [64]
   void* ws;        // GEMM split-K / attention split-KV workspace
   size_t ws_bytes;
   int32_t* info_host;  // pinned

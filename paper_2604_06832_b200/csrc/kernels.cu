@@ -806,6 +806,32 @@ void launch_quad_accept(const int32_t* pred, int32_t* d, int B, int32_t* accepte
   quad_accept_kernel<<<1, 64, 0, st>>>(pred, d, B, accepted, out);
 }
 
+// Commit of the finished block (Bc rows) and opening of the next one (Bn rows) for ONE forward over Bc + Bn rows:
+// rows = [finished tokens ; next block's initial tokens]; mask: a finished row reads the finished rows up to itself
+// (Alg. 1 verify mask), a row of the next block reads every row (the committed block is part of its context, its own
+// block is bidirectional); the block state becomes the next block's.
+__global__ void fuse_begin_kernel(int32_t* __restrict__ blk_tokens, uint8_t* __restrict__ blk_masked, int Bc,
+                                  const int32_t* __restrict__ init, int Bn, int mask_id, int32_t* __restrict__ rows,
+                                  unsigned long long* __restrict__ mask, int32_t* __restrict__ info) {
+  __shared__ int32_t nxt[64];
+  const int i = threadIdx.x, n = Bc + Bn;
+  const int32_t old = i < Bc ? blk_tokens[i] : 0;
+  nxt[i] = (i < Bn && init) ? init[i] : mask_id;
+  __syncthreads();
+  if (i < n) {
+    rows[i] = i < Bc ? old : nxt[i - Bc];
+    mask[i] = i < Bc ? (2ull << i) - 1ull : (n == 64 ? ~0ull : (1ull << n) - 1ull);
+  }
+  const int m = (i < Bn) && (nxt[i] == mask_id);
+  if (i < Bn) { blk_tokens[i] = nxt[i]; blk_masked[i] = (uint8_t)m; }
+  const int cnt = __syncthreads_count(m);
+  if (i == 0) { info[0] = 0; info[1] = cnt; info[2] = 0; }
+}
+void launch_fuse_begin(int32_t* blk_tokens, uint8_t* blk_masked, int Bc, const int32_t* init, int Bn, int mask_id, int32_t* rows,
+                       unsigned long long* mask, int32_t* info, cudaStream_t st) {
+  fuse_begin_kernel<<<1, 64, 0, st>>>(blk_tokens, blk_masked, Bc, init, Bn, mask_id, rows, mask, info);
+}
+
 __global__ void init_block_kernel(int32_t* tokens, uint8_t* masked, int32_t* info, const int32_t* init, int n, int mask_id,
                                   int step) {
   int i = threadIdx.x;

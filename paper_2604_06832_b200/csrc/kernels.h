@@ -36,6 +36,9 @@ void launch_rmsnorm(const float* h, const float* g, void* out, int n, int hidden
 void launch_rope_table(float* cs, int n, int pos0, int head_dim, float theta, cudaStream_t st, const int* len_ptr = nullptr,
                        KStamp* stamp = nullptr, const int* pos_off = nullptr);
 // quadratic self-speculative decoding (Appendix B, Alg. 2): row layout, input tokens, first draft, verify loop
+// commit of the finished block + opening of the next one as one forward: rows, row masks, block state
+void launch_fuse_begin(int32_t* blk_tokens, uint8_t* blk_masked, int Bc, const int32_t* init, int Bn, int mask_id, int32_t* rows,
+                       unsigned long long* mask, int32_t* info, cudaStream_t st);
 void launch_quad_layout(int B, int chain, unsigned long long* mask, int* pos_off, cudaStream_t st);
 void launch_quad_build(const int32_t* d, int B, int mask_id, int32_t* tokens, uint8_t* masked, cudaStream_t st);
 void launch_quad_first_draft(const int32_t* pred, int32_t first, int B, int32_t* d, cudaStream_t st);
