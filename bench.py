@@ -213,7 +213,7 @@ def run_ours(args, wl, block):
     # the 7B configuration prescribes a bf16 KV cache; the others leave the cache's element type open
     kv_dtype = B.KV_BF16 if shape.dtype in (I.FP8, I.W8A8) else B.KV_F16
     # top-k schedules: the commit of block t rides in the forward of block t+1's first step (one forward over 2 x block rows)
-    fused_commit = wl.rule == "topk" and 2 * block <= 64
+    fused_commit = 2 * block <= 64
     handle = B.Handle(shape, weights, max_seq=max_seq, max_block=max(2 * block if fused_commit else block, 32), stream=stream,
                       kv_dtype=kv_dtype)
     emb, toks = I.make_prefix(shape, wl.n_embeds, wl.n_tokens, wl.prefix_seed)
@@ -240,13 +240,18 @@ def run_ours(args, wl, block):
                 open_block[0] = False
 
         def one_block_device():
-            if fused_commit:
-                # fixed schedule, every step enqueued without a host round trip in between; the previous call's block is
-                # committed by this call's first forward.  Per call: one block committed, one block decoded.
-                info = handle.commit_decode_block_topk(block, wl.k)
+            if fused_commit and (wl.rule == "topk" or device_loop):
+                # no host round trip between the steps (top-k: fixed schedule enqueued back to back; threshold: the loop
+                # runs on the device); the previous call's block is committed by this call's first forward.  Per call: one
+                # block committed, one block decoded.
+                if wl.rule == "topk":
+                    info = handle.commit_decode_block_topk(block, wl.k)
+                else:
+                    info = handle.commit_decode_block(block, rule, wl.threshold, wl.k)
                 launches[0] += handle.last_launch_count()
                 open_block[0] = True
                 return info.step_index
+            close_open_block()
             if wl.rule == "topk":
                 info = handle.decode_block_topk(block, wl.k)
                 launches[0] += handle.last_launch_count()

@@ -218,6 +218,11 @@ int fdvlm_commit_begin_step_host(fdvlm_t *h, int next_block_size, const int32_t 
  * new block's first step (as above); with no block open it is fdvlm_decode_block_topk. */
 int fdvlm_commit_decode_block_topk(fdvlm_t *h, int block_size, const int32_t *init_tokens, int k, int pred_shift,
                                    int32_t *block_tokens, fdvlm_step_info *info);
+/* The same for fdvlm_decode_block (either rule, loop on the device): the open, fully revealed block is committed in the
+ * forward of the new block's first step; the host reads the masked count once after that step (it decides whether the
+ * on-device loop runs at all), then once at the end. */
+int fdvlm_commit_decode_block(fdvlm_t *h, int block_size, const int32_t *init_tokens, const fdvlm_step_params *p,
+                              int32_t *block_tokens, fdvlm_step_info *info);
 
 /* Drop committed positions from the end of the cache: cache_len = new_len (Alg. 1 "Crop").  The dropped K/V rows
  * are simply overwritten by later commits.  Errors: STATE inside an open block; INVALID_ARG unless

@@ -87,6 +87,7 @@ EXPORTS = {
     "fdvlm_block_set_tokens": (C.c_int, [C.c_void_p, C.c_void_p]),
     "fdvlm_decode_block_topk": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.POINTER(StepInfo)]),
     "fdvlm_commit_decode_block_topk": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.POINTER(StepInfo)]),
+    "fdvlm_commit_decode_block": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.POINTER(StepParams), C.c_void_p, C.POINTER(StepInfo)]),
     "fdvlm_commit_begin_step": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.POINTER(StepParams), C.c_void_p, C.c_void_p,
                                           C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(StepInfo)]),
     "fdvlm_commit_begin_step_host": (C.c_int, [C.c_void_p, C.c_int, C.c_void_p, C.POINTER(StepParams), C.c_void_p, C.c_void_p,
@@ -258,6 +259,14 @@ class Handle:
         p, info = StepParams(rule, threshold, k, pred_shift), StepInfo()
         self._check(lib().fdvlm_commit_begin_step_host(self._h, next_block_size, _ptr(next_init_tokens), C.byref(p), _ptr(conf),
                                                        _ptr(pred), _ptr(unmask), _ptr(block_tokens), C.byref(info)))
+        return info
+
+    def commit_decode_block(self, block_size: int, rule: int, threshold: float = 0.9, k: int = 8,
+                            init_tokens: Optional[torch.Tensor] = None, pred_shift: int = 0,
+                            block_tokens: Optional[torch.Tensor] = None) -> StepInfo:
+        p, info = StepParams(rule, threshold, k, pred_shift), StepInfo()
+        self._check(lib().fdvlm_commit_decode_block(self._h, block_size, _ptr(init_tokens), C.byref(p), _ptr(block_tokens),
+                                                    C.byref(info)))
         return info
 
     def commit_decode_block_topk(self, block_size: int, k: int, init_tokens: Optional[torch.Tensor] = None, pred_shift: int = 0,

@@ -397,6 +397,9 @@ extern "C" int fdvlm_decode_block_topk(fdvlm_t* h, int block_size, const int32_t
 // of the block's tokens, the forward, the selection); the selection kernel sets the loop condition on the device.
 // Built once per (block size, step parameters) and kept.  Dependent-launch edges are tried first; if the runtime
 // refuses them inside a conditional body the kernels are recorded with ordinary edges.
+static int decode_loop_rest(fdvlm_t* h, int block_size, const fdvlm_step_params* p, int32_t* block_tokens, fdvlm_step_info* info,
+                            int steps_done);
+
 static int build_loop_graph(fdvlm_t* h, int B, const fdvlm_step_params* p, bool with_pdl) {
   cudaGraph_t g = nullptr;
   CU(h, cudaGraphCreate(&g, 0));
@@ -456,6 +459,14 @@ extern "C" int fdvlm_decode_block(fdvlm_t* h, int block_size, const int32_t* ini
   rc = fdvlm_block_begin(h, block_size, init_tokens);      // (reads the masked count back when tokens are given)
   if (rc) return rc;
   h->launches = 0;
+  return decode_loop_rest(h, block_size, p, block_tokens, info, 0);
+}
+
+// The on-device loop over the open block's remaining denoise steps; steps_done of them have already run.
+static int decode_loop_rest(fdvlm_t* h, int block_size, const fdvlm_step_params* p, int32_t* block_tokens, fdvlm_step_info* info,
+                            int steps_done) {
+  int rc = FDVLM_OK;
+  const int first_launches = h->launches;
   if (h->n_remaining > 0) {
     const int long_cache = attention_long_cache(h->cache_len + block_size) ? 1 : 0;
     const bool have = h->loop_exec && h->loop_n == block_size && h->loop_rule == (int)p->rule && h->loop_k == p->k &&
@@ -466,19 +477,38 @@ extern "C" int fdvlm_decode_block(fdvlm_t* h, int block_size, const int32_t* ini
       if (rc) return rc;
     }
     launch_set_len(h->dev_len, h->cache_len, h->st);
-    CU(h, cudaMemsetAsync(h->info + 5, 0, 4, h->st));
+    CU(h, cudaMemcpyAsync(h->info + 5, &steps_done, 4, cudaMemcpyHostToDevice, h->st));
     CU(h, cudaGraphLaunch(h->loop_exec, h->st));
+  } else {
+    CU(h, cudaMemcpyAsync(h->info + 5, &steps_done, 4, cudaMemcpyHostToDevice, h->st));
   }
   if (block_tokens) CU(h, cudaMemcpyAsync(block_tokens, h->blk_tokens, (size_t)block_size * 4, cudaMemcpyDeviceToDevice, h->st));
   rc = sync_info(h);
   if (rc) return rc;
   info->n_unmasked = h->info_host[0]; info->n_remaining = h->info_host[1]; info->step_index = h->info_host[2];
   h->step_index = h->info_host[2];
-  h->launches = 1 + h->info_host[5] * h->loop_body_launches;
+  h->launches = first_launches + 1 + (h->info_host[5] - steps_done) * h->loop_body_launches;
   if (h->n_remaining != 0)
     return fail(h, FDVLM_ERR_STATE, "%d masked positions left after %d steps (a masked position 0 under pred_shift = 1 cannot be revealed)",
                 h->n_remaining, h->info_host[5]);
   return FDVLM_OK;
+}
+
+static int commit_step_core(fdvlm_t* h, int Bn, const int32_t* init_dev, const fdvlm_step_params* p, int want_logits);
+
+extern "C" int fdvlm_commit_decode_block(fdvlm_t* h, int block_size, const int32_t* init_tokens, const fdvlm_step_params* p,
+                                         int32_t* block_tokens, fdvlm_step_info* info) {
+  if (!h) return FDVLM_ERR_INVALID_ARG;
+  if (!h->block_open) return fdvlm_decode_block(h, block_size, init_tokens, p, block_tokens, info);
+  if (!info) return fail(h, FDVLM_ERR_INVALID_ARG, "commit_decode_block needs the host info struct");
+  int rc = check_step_params(h, p);
+  if (rc) return rc;
+  if (!h->use_graphs) return fail(h, FDVLM_ERR_UNSUPPORTED, "decode_block needs the tensor-core path on a non-default stream");
+  rc = commit_step_core(h, block_size, init_tokens, p, 0);      // the finished block's commit + this block's first step
+  if (rc) return rc;
+  rc = sync_info(h);                                            // what the first step left masked decides whether the loop runs
+  if (rc) return rc;
+  return decode_loop_rest(h, block_size, p, block_tokens, info, 1);
 }
 
 extern "C" int fdvlm_block_step_host(fdvlm_t* h, const fdvlm_step_params* p, float* conf_host, int32_t* pred_host,

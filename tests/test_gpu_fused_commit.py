@@ -77,33 +77,42 @@ def test_commit_begin_step_equals_the_three_calls(shape, stream, Bc, Bn, rule, k
     handle.close()
 
 
-def test_commit_decode_chain_matches_block_by_block_decoding_on_a_peaked_model():
-    # top-k schedule over three blocks: [decode, commit] x 3 against [decode, then commit fused into the next decode] x 3.
-    # The two ways run the same arithmetic on other tile shapes, so tokens are compared only where the separate path's
-    # top-k decisions are clear of the confidence tolerance.
+@pytest.mark.parametrize("rule,tau,k", [(orc.TOPK, 0.0, 4), (orc.THRESHOLD, 0.6, 0)])
+def test_commit_decode_chain_matches_block_by_block_decoding_on_a_peaked_model(rule, tau, k):
+    # three blocks: [steps, commit] x 3 against [commit fused into the next block's first step, remaining steps] x 3 (top-k:
+    # fdvlm_commit_decode_block_topk; threshold: fdvlm_commit_decode_block, loop on the device).  The two ways run the same
+    # arithmetic on other tile shapes, so tokens are compared only while the separate path's decisions are not near-ties.
     b = B_()
-    shape, Bsz, k = SMALL_BF16, 16, 4
+    shape, Bsz = SMALL_BF16, 16
+    rule_code = b.RULE_TOPK if rule == orc.TOPK else b.RULE_THRESHOLD
     sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
     _, ha, w = make_pair(shape, 33, max_seq=256, max_block=64, stream=sa, final_gain=16.0)
     hb = b.Handle(shape, b.weights_to_device(w), max_seq=256, max_block=64, stream=sb)
     emb, toks = I.make_prefix(shape, 10, 20, 5)
-    blocks_a, blocks_b, clear = [], [], []
+    blocks_a, blocks_b, steps_a, steps_b, clear = [], [], [], [], []
     with torch.cuda.stream(sa):
         ha.prefill(*upload_prefix(emb, toks))
         for _ in range(3):
             ha.block_begin(Bsz)
-            ok = True
+            ok, n = True, 0
             conf = torch.empty(Bsz, dtype=torch.float32, device="cuda")
             tok = torch.empty(Bsz, dtype=torch.int32, device="cuda")
             masked = np.ones(Bsz, dtype=bool)
-            for _s in range(Bsz // k):
+            while masked.any():
                 um = torch.empty(Bsz, dtype=torch.uint8, device="cuda")
-                ha.block_step(b.RULE_TOPK, 0.0, k, conf=conf, unmask=um, block_tokens=tok)
+                ha.block_step(rule_code, tau, k, conf=conf, unmask=um, block_tokens=tok)
+                n += 1
                 c = np.sort(conf.cpu().numpy()[masked])[::-1]
-                if len(c) > k and c[k - 1] - c[k] <= 1e-4:          # (the two ways differ by ~1e-6 in confidence)
-                    ok = False
+                if rule == orc.TOPK:
+                    near = len(c) > k and c[k - 1] - c[k] <= 1e-5
+                else:
+                    near = np.any(np.abs(c - tau) <= 1e-5) or (c[0] <= tau and len(c) > 1 and c[0] - c[1] <= 1e-5)
+                if near:
+                    print("near-tie at step", n, "sorted confidences", c[:6])
+                ok = ok and not near                                # (the two ways differ by ~1e-6 in confidence)
                 masked &= ~um.cpu().numpy().astype(bool)
             blocks_a.append(tok.cpu().numpy().copy())
+            steps_a.append(n)
             clear.append(ok)
             ha.commit_block()
     with torch.cuda.stream(sb):
@@ -111,17 +120,21 @@ def test_commit_decode_chain_matches_block_by_block_decoding_on_a_peaked_model()
         L0 = hb.cache_len()
         for i in range(3):
             tok = torch.empty(Bsz, dtype=torch.int32, device="cuda")
-            info = hb.commit_decode_block_topk(Bsz, k, block_tokens=tok)
-            assert info.n_remaining == 0 and info.step_index == Bsz // k
+            if rule == orc.TOPK:
+                info = hb.commit_decode_block_topk(Bsz, k, block_tokens=tok)
+            else:
+                info = hb.commit_decode_block(Bsz, rule_code, tau, k, block_tokens=tok)
+            assert info.n_remaining == 0 and 1 <= info.step_index <= Bsz
             assert hb.cache_len() == L0 + i * Bsz                 # the previous block went in with this call
             blocks_b.append(tok.cpu().numpy().copy())
+            steps_b.append(info.step_index)
         hb.commit_block()
         assert hb.cache_len() == L0 + 3 * Bsz == ha.cache_len()
-    assert any(clear)
-    for a_, b_, ok in zip(blocks_a, blocks_b, clear):
+    assert clear[0]
+    for a_, b_, na, nb, ok in zip(blocks_a, blocks_b, steps_a, steps_b, clear):
         if not ok:
             break                                                   # later blocks start from a different context
-        assert np.array_equal(a_, b_)
+        assert np.array_equal(a_, b_) and na == nb
     ha.close()
     hb.close()
 
