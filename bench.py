@@ -232,6 +232,7 @@ def run_ours(args, wl, block):
         prefill_ms = t0.elapsed_time(t1)
 
         launches = [0]
+        fused_device = fused_commit and (wl.rule == "topk" or device_loop)    # (the stepwise exact path commits separately)
         open_block = [False]          # fused_commit: the block decoded by the previous call, not yet committed
 
         def close_open_block():
@@ -240,7 +241,7 @@ def run_ours(args, wl, block):
                 open_block[0] = False
 
         def one_block_device():
-            if fused_commit and (wl.rule == "topk" or device_loop):
+            if fused_device:
                 # no host round trip between the steps (top-k: fixed schedule enqueued back to back; threshold: the loop
                 # runs on the device); the previous call's block is committed by this call's first forward.  Per call: one
                 # block committed, one block decoded.
@@ -466,7 +467,8 @@ def run_ours(args, wl, block):
         "kv_dtype": "bf16" if kv_dtype == B.KV_BF16 else "f16",
         # per block: n denoise steps + one causal commit; with fused_commit the commit of block t and the first step of
         # block t+1 are one forward over 2 x block rows (same results, every weight byte streamed once for both)
-        "forwards_per_block": (n_steps if fused_commit else n_steps + 1), "fused_commit": fused_commit,
+        "forwards_per_block": (n_steps if fused_device else n_steps + 1), "fused_commit": fused_device,
+        "e2e_fused_commit": fused_commit,
         "e2e": {"value": e2e_value, "unit": "tok/s", "h2d_bytes_per_step": block * 4,
                 "d2h_bytes_per_step": n_steps * (block * 13 + 32)},
         "gpu_launches": n_launch,
