@@ -459,6 +459,24 @@ def run_ours(args, wl, block):
         pass
     step_bytes = wbytes + kv_bytes
     step_med = statistics.median(lat)
+    lat_sorted = sorted(lat)
+    pct = lambda q: lat_sorted[min(len(lat_sorted) - 1, max(0, int(round(q * (len(lat_sorted) - 1)))))]
+    # a second denominator beside the copy bandwidth: what a plain read-only streaming kernel of the library reaches on this
+    # GPU, on a 2 GiB buffer (larger than L2), median of 5 after 3 warm-up launches
+    with torch.cuda.stream(stream):
+        rbuf = torch.empty(2 << 30, dtype=torch.uint8, device="cuda")
+        rsink = torch.zeros(1, dtype=torch.int32, device="cuda")
+        rt = []
+        for i in range(8):
+            a, b = ev(), ev()
+            a.record(stream)
+            B.util_stream_read(rbuf, rsink, stream)
+            b.record(stream)
+            stream.synchronize()
+            if i >= 3:
+                rt.append(a.elapsed_time(b))
+        read_peak = rbuf.numel() / (statistics.median(rt) / 1000.0) / 1e9
+        del rbuf
     line = {
         "metric": METRIC, "value": value, "unit": "tok/s", "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms_dev / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -486,9 +504,11 @@ def run_ours(args, wl, block):
                       "in_chain_ms_per_forward": attn_us_chain / 1000.0,
                       "achieved_gbs": kv_bytes / (attn_us_chain * 1e-6) / 1e9 if attn_us_chain > 0 else None},
         "chain_us_per_forward": {k_: round(v, 2) for k_, v in sorted(chain_us.items())},
-        "step": {"latency_ms_median": step_med, "latency_ms_all": lat, "cache_len": L_step, "bytes": step_bytes,
+        "step": {"latency_ms_median": step_med, "latency_ms_p10": pct(0.1), "latency_ms_p90": pct(0.9), "latency_ms_all": lat,
+                 "cache_len": L_step, "bytes": step_bytes,
                  "gbs": step_bytes / (step_med / 1000.0) / 1e9, "frac_of_peak": step_bytes / (step_med / 1000.0) / 1e9 / peak,
-                 "frac_of_8tbs": step_bytes / (step_med / 1000.0) / 1e9 / 8000.0},
+                 "frac_of_8tbs": step_bytes / (step_med / 1000.0) / 1e9 / 8000.0,
+                 "read_only_stream_gbs": read_peak, "frac_of_read_only_stream": step_bytes / (step_med / 1000.0) / 1e9 / read_peak},
         "prefill_ms": prefill_ms,
         "modes": modes,
     }

@@ -312,6 +312,14 @@ int fdvlm_debug_poison(fdvlm_t *h, int on);
  * With h = NULL returns the message of the last failed fdvlm_create on this thread. */
 const char *fdvlm_last_error(const fdvlm_t *h);
 
+/* ---- a yardstick for measurement (the paper has no counterpart) ---------------------------------------- */
+
+/* Read `bytes` bytes of device memory once, with a plain streaming kernel of this library (16-byte loads, 8 CTAs per SM,
+ * nothing written but one 4-byte word at device_sink that the kernel may increment): timed by the caller with CUDA events
+ * on a buffer larger than L2, it gives the read-only bandwidth a kernel can reach on this GPU, a second denominator
+ * beside the copy bandwidth.  device_buf 16-byte aligned.  Asynchronous on cuda_stream. */
+int fdvlm_util_stream_read(const void *device_buf, size_t bytes, void *device_sink, void *cuda_stream);
+
 /* ---- single operators of the path, for kernel-level tests and timing -------------------------------- */
 
 /* y[m, n] = sum_k x[m, k] * w[n, k] (* scale[n]) (+ bias[n]): the small-M weight-streaming GEMM that

@@ -95,6 +95,7 @@ EXPORTS = {
     "fdvlm_commit_block": (C.c_int, [C.c_void_p, C.c_void_p]),
     "fdvlm_commit_block_verify": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "fdvlm_truncate": (C.c_int, [C.c_void_p, C.c_int]),
+    "fdvlm_util_stream_read": (C.c_int, [C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]),
     "fdvlm_spec_block": (C.c_int, [C.c_void_p, C.c_int, C.c_int32, C.c_void_p, C.c_void_p, C.POINTER(SpecInfo)]),
     "fdvlm_quad_begin": (C.c_int, [C.c_void_p, C.c_int, C.c_int32, C.c_int, C.c_void_p]),
     "fdvlm_quad_set_draft": (C.c_int, [C.c_void_p, C.c_void_p]),
@@ -344,6 +345,12 @@ class Handle:
         ml, ma, nl, na = C.c_double(), C.c_double(), C.c_int(), C.c_int()
         self._check(lib().fdvlm_profile_read(self._h, C.byref(ml), C.byref(nl), C.byref(ma), C.byref(na)))
         return dict(ms_linear=ml.value, n_linear=nl.value, ms_attention=ma.value, n_attention=na.value)
+
+
+def util_stream_read(buf: torch.Tensor, sink: torch.Tensor, stream: Optional[torch.cuda.Stream] = None):
+    rc = lib().fdvlm_util_stream_read(_ptr(buf), buf.numel() * buf.element_size(), _ptr(sink), _stream_ptr(stream))
+    if rc != FDVLM_OK:
+        raise FdvlmError(rc, "fdvlm_util_stream_read")
 
 
 def op_linear(x: torch.Tensor, w: torch.Tensor, scale=None, bias=None, dtype: int = DT_BF16,

@@ -882,6 +882,16 @@ extern "C" int fdvlm_profile_read(fdvlm_t* h, double* ms_linear, int* n_linear, 
   return FDVLM_OK;
 }
 
+// ---- measurement yardstick ------------------------------------------------------------------------------
+extern "C" int fdvlm_util_stream_read(const void* device_buf, size_t bytes, void* device_sink, void* cuda_stream) {
+  if (!device_buf || !device_sink || bytes < 16 || ((uintptr_t)device_buf & 15)) return FDVLM_ERR_INVALID_ARG;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return FDVLM_ERR_CUDA;
+  launch_stream_read(device_buf, bytes, (unsigned*)device_sink, sms * 8, (cudaStream_t)cuda_stream);
+  return cudaGetLastError() == cudaSuccess ? FDVLM_OK : FDVLM_ERR_CUDA;
+}
+
 // ---- single operators ---------------------------------------------------------------------------------
 extern "C" size_t fdvlm_op_linear_workspace_bytes(int m, int n, int k, fdvlm_dtype dtype) {
   if (m < 1 || n < 1 || k < 1) return 0;

@@ -734,6 +734,27 @@ void launch_accept(const int32_t* a, const int32_t* d, int n, int32_t* out, cuda
   accept_kernel<<<1, 64, 0, st>>>(a, d, n, out);
 }
 
+// Read-only streaming of a buffer: every CTA walks its share with 16-byte loads, eight in flight per thread, and folds
+// what it reads into one word (so that the loads cannot be dropped).  A yardstick for the read bandwidth a kernel of this
+// library can reach at all; no part of the decoding path.
+__global__ void __launch_bounds__(256) stream_read_kernel(const uint4* __restrict__ buf, size_t n16, unsigned* __restrict__ sink) {
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  unsigned acc = 0;
+  for (; i + 7 * stride < n16; i += 8 * stride) {
+    uint4 v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) v[u] = __ldcs(buf + i + u * stride);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) acc ^= v[u].x ^ v[u].y ^ v[u].z ^ v[u].w;
+  }
+  for (; i < n16; i += stride) { const uint4 v = __ldcs(buf + i); acc ^= v.x ^ v.y ^ v.z ^ v.w; }
+  if (acc == 0x9e3779b9u) atomicAdd(sink, 1u);     // practically never: keeps the loads alive without a store per thread
+}
+void launch_stream_read(const void* buf, size_t bytes, unsigned* sink, int ctas, cudaStream_t st) {
+  stream_read_kernel<<<ctas, 256, 0, st>>>((const uint4*)buf, bytes / 16, sink);
+}
+
 // ---- quadratic self-speculative decoding (Appendix B, Alg. 2) --------------------------------------------------------
 // Row order of the B (B + 1) rows of one forward: rows 0 .. B-1 are the draft tokens d_0 .. d_{B-1} (the first tokens of
 // the groups), row B + i B + (j - 1) is mask token j (1 <= j <= B) of group i.  With the first tokens in front, the rows

@@ -36,6 +36,8 @@ void launch_rmsnorm(const float* h, const float* g, void* out, int n, int hidden
 void launch_rope_table(float* cs, int n, int pos0, int head_dim, float theta, cudaStream_t st, const int* len_ptr = nullptr,
                        KStamp* stamp = nullptr, const int* pos_off = nullptr);
 // quadratic self-speculative decoding (Appendix B, Alg. 2): row layout, input tokens, first draft, verify loop
+// read-only streaming yardstick (see the kernel)
+void launch_stream_read(const void* buf, size_t bytes, unsigned* sink, int ctas, cudaStream_t st);
 // commit of the finished block + opening of the next one as one forward: rows, row masks, block state
 void launch_fuse_begin(int32_t* blk_tokens, uint8_t* blk_masked, int Bc, const int32_t* init, int Bn, int mask_id, int32_t* rows,
                        unsigned long long* mask, int32_t* info, cudaStream_t st);
