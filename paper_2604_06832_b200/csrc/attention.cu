@@ -331,8 +331,8 @@ template <int D>
 __device__ __forceinline__ void attn_merge_warp(const float* att_o, const float2* att_ml, void* out, size_t out_idx, size_t lo_off,
                                                 int fmt, size_t slot0, int n_chunks, int lane, float* amax_out = nullptr) {
   constexpr int VPL = D / 32;
-  constexpr int CB = 16;     // chunks whose partial outputs are in flight together
-  // The statistics and the first CB partial outputs are requested together: one L2 round trip for up to 16 chunks.
+  constexpr int CB = 32;     // chunks whose partial outputs are in flight together
+  // The statistics and the first CB partial outputs are requested together: one L2 round trip for up to 32 chunks.
   float2 ml0 = make_float2(-INFINITY, 0.f);
   if (lane < n_chunks) ml0 = __ldcg(&att_ml[slot0 + lane]);
   float ov[CB][VPL];
