@@ -168,3 +168,23 @@ def test_attention_at_the_long_prefix_length():
             out = B().op_attention(q.cuda(), kc.cuda(), vc.cuda(), L, bool(causal), dtype=B().DT_BF16)
             torch.cuda.synchronize()
             assert np.abs(out.double().cpu().numpy() - ref).max() <= bound
+
+
+# ---- the fused commit, Alg. 2's masked forward and the W8A8 projection at the real layer widths -------------------
+@pytest.mark.parametrize("shape", [CUT_3B, I.QWEN7B_FP8.with_(n_layers=4)], ids=["3b-bf16-cut", "7b-fp8-cut"])
+def test_fused_commit_at_full_width(shape):
+    from test_gpu_fused_commit import fused_case
+    fused_case(shape, True, 32, 32, orc.TOPK, 8)          # the 64-row forward the bench's top-k workloads run
+
+
+def test_quadratic_decoding_at_full_width():
+    from test_gpu_quad import run_iterations
+    stats = run_iterations(CUT_3B, 7, False, n_iter=1, stream=True)      # 56 rows, the largest block one forward takes
+    print("quadratic, 3B-width cut:", stats)
+
+
+@pytest.mark.parametrize("n,k", [(3584 + 2 * 512, 3584), (3584, 18944), (2 * 18944, 3584)], ids=["qkv", "down", "gate-up"])
+def test_w8a8_projection_at_the_7b_shapes(n, k):
+    from test_gpu_w8a8 import test_op_linear_w8a8_quantises_like_the_oracle as case
+    case(32, n, k)
+

@@ -27,6 +27,10 @@ def B_():
 @pytest.mark.parametrize("Bc,Bn,rule,k", [(16, 16, orc.TOPK, 4), (32, 32, orc.TOPK, 8), (8, 24, orc.THRESHOLD, 0), (5, 3, orc.TOPK, 2),
                                           (1, 1, orc.THRESHOLD, 0)])
 def test_commit_begin_step_equals_the_three_calls(shape, stream, Bc, Bn, rule, k):
+    fused_case(shape, stream, Bc, Bn, rule, k)
+
+
+def fused_case(shape, stream, Bc, Bn, rule, k):
     b = B_()
     tol = TOL[shape.dtype]
     st = torch.cuda.Stream() if stream else None
