@@ -177,6 +177,13 @@ def test_fused_commit_at_full_width(shape):
     fused_case(shape, True, 32, 32, orc.TOPK, 8)          # the 64-row forward the bench's top-k workloads run
 
 
+def test_fused_commit_at_full_depth_is_the_forward_the_bench_times():
+    # cfg2's model, all 36 layers: the 64-row forward (commit of one block + first top-8 step of the next) at the stated bounds
+    from test_gpu_fused_commit import fused_case
+    wl = I.WORKLOADS["cfg2_3b_bf16_p1024_b32_top8"]
+    fused_case(wl.shape, True, 32, 32, orc.TOPK, 8, weight_seed=wl.weight_seed)
+
+
 def test_quadratic_decoding_at_full_width():
     from test_gpu_quad import run_iterations
     stats = run_iterations(CUT_3B, 7, False, n_iter=1, stream=True)      # 56 rows, the largest block one forward takes

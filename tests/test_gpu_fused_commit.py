@@ -30,11 +30,11 @@ def test_commit_begin_step_equals_the_three_calls(shape, stream, Bc, Bn, rule, k
     fused_case(shape, stream, Bc, Bn, rule, k)
 
 
-def fused_case(shape, stream, Bc, Bn, rule, k):
+def fused_case(shape, stream, Bc, Bn, rule, k, weight_seed=21):
     b = B_()
     tol = TOL[shape.dtype]
     st = torch.cuda.Stream() if stream else None
-    oracle, handle, _ = make_pair(shape, 21, max_seq=256, max_block=64, stream=st)
+    oracle, handle, _ = make_pair(shape, weight_seed, max_seq=256, max_block=64, stream=st)
     emb, toks = I.make_prefix(shape, 12, 15, 6)
     oracle.prefill(I.as_numpy_storage(emb), toks.numpy(), want_logits=False)
     final = I.random_tokens(shape, Bc, 9)
