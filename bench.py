@@ -213,7 +213,7 @@ def run_ours(args, wl, block):
     # the 7B configuration prescribes a bf16 KV cache; the others leave the cache's element type open
     kv_dtype = B.KV_BF16 if shape.dtype in (I.FP8, I.W8A8) else B.KV_F16
     # top-k schedules: the commit of block t rides in the forward of block t+1's first step (one forward over 2 x block rows)
-    fused_commit = 2 * block <= 64
+    fused_commit = 2 * block <= 64 and not args.separate_commit
     handle = B.Handle(shape, weights, max_seq=max_seq, max_block=max(2 * block if fused_commit else block, 32), stream=stream,
                       kv_dtype=kv_dtype)
     emb, toks = I.make_prefix(shape, wl.n_embeds, wl.n_tokens, wl.prefix_seed)
@@ -540,6 +540,8 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(I.WORKLOADS))
     ap.add_argument("--block", type=int, default=0, help="block size (default: the workload's last listed size)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--separate-commit", action="store_true",
+                    help="commit every block by a forward of its own instead of inside the next block's first step")
     args = ap.parse_args()
     wl = I.WORKLOADS[args.workload]
     block = args.block or (32 if 32 in wl.block_sizes else wl.block_sizes[-1])
