@@ -14,6 +14,11 @@
  *   fdvlm_commit_block  causal forward of the finished block WITH cache update (Alg. 1 verify step;
  *                       Sec. 3.3 M_C2C: clean context is token-causal)
  *
+ * and, built from the same forward: the decode loops without host round trips (fdvlm_decode_block_topk,
+ * fdvlm_decode_block), the commit fused into the next block's first step (fdvlm_commit_begin_step,
+ * fdvlm_commit_decode_block(_topk)), linear and quadratic self-speculative decoding (fdvlm_spec_block, Alg. 1;
+ * fdvlm_quad_begin / fdvlm_quad_step, Alg. 2), W8A8 (FDVLM_W8A8_FP8E4M3), and the single operators.
+ *
  * Conventions
  *   - All `device` pointers are CUDA device memory of the handle's GPU; `host` pointers are ordinary
  *     host memory.  No pointer is retained beyond a call except the weight pointers given to
