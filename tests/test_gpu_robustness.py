@@ -213,3 +213,15 @@ def test_two_handles_on_two_streams_in_one_process():
     assert st1["steps"] == st2["steps"] == 2
     h1.close()
     h2.close()
+
+
+def test_stream_read_yardstick_runs_and_rejects_bad_arguments():
+    b = B()
+    buf = torch.zeros(64 << 20, dtype=torch.uint8, device="cuda")
+    sink = torch.zeros(1, dtype=torch.int32, device="cuda")
+    b.util_stream_read(buf, sink)
+    torch.cuda.synchronize()
+    assert int(sink.item()) == 0                                   # all-zero data never folds to the magic word
+    with pytest.raises(b.FdvlmError):
+        b.util_stream_read(buf[1:], sink)                          # not 16-byte aligned
+    assert b.lib().fdvlm_util_stream_read(None, 1024, sink.data_ptr(), None) == b.ERR_INVALID_ARG
